@@ -1,0 +1,184 @@
+/*
+ * flashloop.h -- C ABI of the B200 (sm_100a) FlashLoop loop-r prefill library.
+ *
+ * The library implements one step of "FlashLoop: Fast and Memory-Efficient Looped Transformers via
+ * Lazy Updates": the prefill of loop r > 1 of one layer, i.e.
+ *   (1) cross-loop token scoring and top-k token selection        (Section 4.1, Appendix D.1, Eq. 5)
+ *   (2) column-sparse attention replacement                       (Section 4.2, Appendix D.2, Eq. 6-7)
+ *   (3) quantization of the cross-loop K/V residuals              (Section 4.3, Appendix D.3, Eq. 8)
+ *   (4) dequantize-and-add reconstruction of K/V inside attention (Section 4.3 "at read time", App. G)
+ * plus the dense source loop that produces the statistics loop 2 starts from (Eq. 2, Eq. 6 with m_C = 1).
+ *
+ * Conventions
+ *  - Plain C. Every pointer is a DEVICE pointer unless its comment says "host". All device buffers are
+ *    owned by the caller, must be 16-byte aligned, and must stay valid until the stream has run the call.
+ *  - Every call validates its arguments on the host, enqueues its kernels on `stream` (a cudaStream_t
+ *    passed as void*) and returns without synchronising. Return value: FL_OK or a negative fl_status.
+ *    Nothing is launched when an argument is rejected.
+ *  - No call allocates device memory except fl_create (one fixed workspace, freed by fl_destroy).
+ *  - Results are deterministic: the same inputs give bit-identical outputs.
+ *  - Row-major tensors; [n, H, dh] means n rows of H heads of dh elements, dh fastest.
+ *    "storage type" is fl_shape.dtype: FL_BF16 (2 bytes) or FL_F32 (4 bytes).
+ *  - Notation: L tokens, H heads, dh head dimension, d = H*dh, A^(r) active-token set of loop r,
+ *    nb = ceil(L / q_block) query blocks of q_block consecutive token positions,
+ *    S[h,b] the key columns selected for head h and block b, T_i = { j in S[h, block(i)] : j <= i }.
+ *    G^(r) is the hidden state entering loop r (the paper's H^(r-1)).
+ */
+#ifndef FLASHLOOP_H_
+#define FLASHLOOP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define FL_API __attribute__((visibility("default")))
+#else
+#define FL_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  FL_OK = 0,
+  FL_ERR_INVALID_ARG = -1, /* null / misaligned pointer, size out of range, inconsistent store */
+  FL_ERR_UNSUPPORTED = -2, /* a valid request this build has no kernel for (e.g. head_dim 96) */
+  FL_ERR_WORKSPACE = -3,   /* problem larger than the context workspace allows */
+  FL_ERR_CUDA = -4,        /* a CUDA runtime call failed (launch error, wrong device, ...) */
+  FL_ERR_TIMEOUT = -5      /* reported through the device status word: a bounded wait ran out */
+} fl_status;
+
+enum { FL_BF16 = 0, FL_F32 = 1 };
+#define FL_MAX_LOOPS 32 /* residual streams per store: loops 2 .. FL_MAX_LOOPS+1 */
+
+/* Opaque context: device ordinal, SM count, one small workspace. Not thread-safe per context. */
+typedef struct fl_ctx fl_ctx;
+FL_API int fl_create(fl_ctx** out /* host */, int device);
+FL_API int fl_destroy(fl_ctx* ctx);
+FL_API const char* fl_status_string(int status); /* host string, static storage */
+FL_API int fl_version(void);
+
+/* Fixed per model / configuration. */
+typedef struct {
+  int32_t L;        /* tokens in the prompt, >= 1 */
+  int32_t n_heads;  /* H >= 1 */
+  int32_t head_dim; /* dh in {64, 128} */
+  int32_t dtype;    /* FL_BF16 or FL_F32: storage type of hidden states, Q, K, V, O and the K/V base */
+  int32_t q_block;  /* query-block width in token positions, >= 1 (1 = the per-position rule of Eq. 6) */
+  int32_t bits;     /* residual code width: 2, 4, 8, or 16 = codec off (rows stored in storage type) */
+  int32_t group;    /* codec group: consecutive head_dim elements sharing scale and offset;
+                       one of 8, 16, 32, 64, 128 and a divisor of head_dim */
+  float eps;        /* Eq. 5 epsilon (added to the norm, not to its square) */
+  float sm_scale;   /* logit scale, normally 1/sqrt(head_dim) */
+} fl_shape;
+
+/* One loop's residual payload for K or for V (Eq. 8: only active rows carry payload).
+ * Row t belongs to token position active_idx[t] of that loop; slot_of_pos inverts the map.
+ *   bits in {2,4,8}: codes [n_rows, H, dh*bits/8] bytes, little-endian inside a byte (element
+ *                    (8/bits)*t+u occupies bits [u*bits, (u+1)*bits) of byte t);
+ *                    scale, zero [n_rows, H, dh/group] IEEE fp16 bit patterns;
+ *                    value = code * scale + zero (one binary32 rounding).
+ *   bits == 16     : codes [n_rows, H, dh] in storage type holds the loop's rows themselves;
+ *                    scale and zero are ignored (may be NULL). */
+typedef struct {
+  void* codes;
+  uint16_t* scale;
+  uint16_t* zero;
+  const int32_t* slot_of_pos; /* [L]: row of this stream holding the position, or -1 */
+  int32_t n_rows;
+  int32_t reserved_;
+} fl_kv_stream;
+
+/* Per-layer K/V store: loop-1 base (storage type, all L rows) plus one residual stream per later loop.
+ * k_res[r-2] / v_res[r-2] hold loop r. Reconstruction (Eq. 4 / Eq. 8), in binary32 and in loop order:
+ *   Xhat^(r)_i = ((base_i + D_2) + D_3) + ... over the loops <= r in which position i was active. */
+typedef struct {
+  void* k_base;
+  void* v_base; /* [L, H, dh] */
+  fl_kv_stream k_res[FL_MAX_LOOPS];
+  fl_kv_stream v_res[FL_MAX_LOOPS];
+  int32_t n_streams; /* streams filled so far: loops 2 .. n_streams+1 */
+  int32_t reserved_;
+} fl_kv_store; /* host struct holding device pointers */
+
+/* Stage 1 -- Eq. 5. Scores the candidate rows and keeps the top k.
+ *   s_i = ||G^(r)_i - G^(r-1)_i||_2 / (||G^(r)_i||_2 + eps), accumulated in binary32 over d = H*dh;
+ *   A^(r) = the min(k, n_cand) candidates with the largest s, ties to the lowest position.
+ * h_prev, h_cur : [L, d] storage type.  cand: ascending positions [n_cand], or NULL for all L rows
+ * (then n_cand must equal L).  Outputs: scores f32 [n_cand] (aligned with cand), active_idx int32
+ * [min(k, n_cand)] ascending, slot_of_pos int32 [L] (rank in active_idx, or -1).
+ * Inputs must be finite. Errors: null pointers, k < 1, n_cand < 1 or > L, loop_r < 2. */
+FL_API int fl_select_tokens(fl_ctx* ctx, const fl_shape* shape, int loop_r, const void* h_prev, const void* h_cur,
+                     const int32_t* cand, int32_t n_cand, int32_t k, float* scores, int32_t* active_idx,
+                     int32_t* slot_of_pos, int32_t* status, void* stream);
+
+/* Active-row execution (Appendix G, "sparse execution over active tokens"):
+ * gather: dst[t, :] = src[idx[t], :];  scatter: dst[idx[t], :] = src[t, :], other rows untouched.
+ * row_bytes must be a positive multiple of 16; idx ascending without repeats; n >= 0. */
+FL_API int fl_gather_rows(fl_ctx* ctx, const void* src, const int32_t* idx, int32_t n, int64_t row_bytes, void* dst,
+                   void* stream);
+FL_API int fl_scatter_update(fl_ctx* ctx, const void* src, const int32_t* idx, int32_t n, int64_t row_bytes,
+                      void* dst, void* stream);
+
+/* Stage 3 -- Eq. 8 with the quantizer of Appendix E (asymmetric, group-wise, min/max).
+ * For each active row i = active_idx[t], X in {K, V}, head, group of `group` elements, in binary32:
+ *   delta = X^(r)_i - Xhat^(r-1)_i            (Xhat^(r-1) rebuilt from base + streams of loops < r)
+ *   zero  = fp16 round-down(min delta);  range = max delta - zero
+ *   scale = range == 0 ? 0 : fp16 round-up(range / (2^bits - 1))
+ *   code  = scale == 0 ? 0 : clamp(round-half-even((delta - zero) / scale), 0, 2^bits - 1)
+ * and writes stream r (store->k_res[loop_r-2], v_res[loop_r-2]; codes/scale/zero pre-allocated by the
+ * caller for n_rows == n_active, slot_of_pos already filled for loop r). |delta| must stay below 65504.
+ * k_new, v_new: [n_active, H, dh] storage type. store is a host struct; store->n_streams must be
+ * >= loop_r - 1 (the stream being written counts). Errors: loop_r < 2 or > FL_MAX_LOOPS+1, bad bits or
+ * group, null buffers, n_rows mismatch. n_active == 0 is a no-op. */
+FL_API int fl_quant_kv_residual(fl_ctx* ctx, const fl_shape* shape, int loop_r, const void* k_new, const void* v_new,
+                         const int32_t* active_idx, int32_t n_active, const fl_kv_store* store,
+                         int32_t* status, void* stream);
+
+/* Dense source loop -- Eq. 2 for all L rows, causal, plus what loop 2 needs (Eq. 6 with m_C = 1):
+ *   o [L, H, dh] storage type;  lse f32 [H, L] = log sum_{j<=i} exp(sm_scale q_i.k_j);
+ *   col_scores f32 [H, nb, L]: col_scores[h,b,j] = sum_{i in block b, i >= j} p_ij for j <= last row of
+ *   block b (entries beyond are not written). lse and col_scores may be NULL (col_scores needs lse). */
+FL_API int fl_dense_loop_attention(fl_ctx* ctx, const fl_shape* shape, const void* q, const void* k, const void* v,
+                            void* o, float* lse, float* col_scores, int32_t* status, void* stream);
+
+/* Eq. 6: per (head, block) S = TopK_c over the candidate columns, ties to the lowest column.
+ *   cand_cols == NULL : dense source. col_scores is [H, nb, L]; block b's candidates are columns
+ *                       0 .. min(L, (b+1)*q_block)-1.
+ *   cand_cols != NULL : sparse source. cand_cols int32 [H, nb, n_cand] ascending with cand_cnt[H, nb] valid
+ *                       entries each; col_scores is [H, nb, n_cand], aligned with cand_cols.
+ * Outputs: col_idx int32 [H, nb, c] ascending, padded with -1; col_cnt int32 [H, nb] = min(c, candidates).
+ * n_cand is the row stride of the candidate arrays (L for a dense source). */
+FL_API int fl_select_columns(fl_ctx* ctx, const fl_shape* shape, const float* col_scores, const int32_t* cand_cols,
+                      const int32_t* cand_cnt, int32_t n_cand, int32_t c, int32_t* col_idx, int32_t* col_cnt,
+                      int32_t* status, void* stream);
+
+/* Stages 2 + 4 -- Eq. 7 (equivalently Eq. 3) over K/V reconstructed inside the kernel.
+ * For head h, active row t (position i = active_idx[t], block b), T_i = { j in col_idx[h,b,:] : j <= i }:
+ *   p_old_j = exp(sm_scale q_old_t . Khat^(r-1)_j - lse_prev[h,i])       previous loop's probabilities
+ *   m_i     = sum_{T_i} p_old_j                                          cached global mass
+ *   p_new_j = m_i softmax_{T_i}(sm_scale q_new_t . Khat^(r)_j)
+ *   o_out_t = o_prev_t - sum p_old_j Vhat^(r-1)_j + sum p_new_j Vhat^(r)_j
+ *   lse_out[h,i] = logsumexp_{T_i}(sm_scale q_new_t . Khat^(r)_j) - log m_i
+ *   col_scores_next[h,b,u] = sum over the block's active rows of p_new for column col_idx[h,b,u]
+ * Rows with empty T_i keep o and lse. Khat^(r-1) uses streams of loops < r, Khat^(r) adds loop r
+ * (store->n_streams >= loop_r - 1). q_new, q_old, o_prev, o_out: [n_active, H, dh] storage type;
+ * lse_prev, lse_out: f32 [H, L] indexed by position (only active rows are read / written).
+ * o_out may alias o_prev and lse_out may alias lse_prev. col_scores_next f32 [H, nb, c] or NULL. */
+FL_API int fl_loop_attention(fl_ctx* ctx, const fl_shape* shape, int loop_r, const void* q_new, const void* q_old,
+                      const int32_t* active_idx, int32_t n_active, const fl_kv_store* store,
+                      const int32_t* col_idx, const int32_t* col_cnt, int32_t c, const float* lse_prev,
+                      float* lse_out, const void* o_prev, void* o_out, float* col_scores_next,
+                      int32_t* status, void* stream);
+
+/* KV-cache accounting (Section 1's 48 GiB example; Section 4.3): bytes held for one layer by this store
+ * after n_loops loops, and by a dense looped cache of n_loops loops. Host-only, no device access.
+ * share_layers = number of layers sharing each loop's slot map and index list (>= 1). */
+FL_API int fl_kv_store_bytes(const fl_shape* shape, const fl_kv_store* store, int n_loops, int share_layers,
+                      int64_t* flashloop_bytes /* host */, int64_t* dense_bytes /* host */);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FLASHLOOP_H_ */

@@ -279,7 +279,10 @@ def sparse_loop_attention(q_new, khat_new, vhat_new, vhat_old, o_prev, active, c
     p_old_cache : {(h,b): (rows, P)} with P[t, u] = p^(r-1) of query rows[t], column S[h,b][u]
                   (zero where the column is not causal); rows must contain the block's active rows.
     Returns dict: O [n,H,dh] fp64, mass {(h,b): m_i per active row}, probs {(h,b): (rows, P_new)},
-                  col_scores {(h,b): sum over rows of P_new, per column of S}.
+                  col_scores {(h,b): sum over rows of P_new, per column of S},
+                  lse [H, n] fp64: the one-number summary of each row's cached probabilities,
+                  p_new_ij = exp(logit_ij - lse_i), i.e. logsumexp_{T_i}(logits) - log m_i (NaN where
+                  T_i is empty).  The oracle itself never reads it; tests use it to feed a GPU stage.
     """
     q_new = np.asarray(q_new)
     active = np.asarray(active, dtype=np.int64)
@@ -288,6 +291,7 @@ def sparse_loop_attention(q_new, khat_new, vhat_new, vhat_old, o_prev, active, c
     nb = n_blocks(L, q_block)
     O = np.array(o_prev, dtype=F64, copy=True)
     mass, probs, scores = {}, {}, {}
+    lse = np.full((H, n), np.nan, dtype=F64)
     heads = range(H) if head_list is None else head_list
     blk = active // q_block
     for h in heads:
@@ -319,7 +323,9 @@ def sparse_loop_attention(q_new, khat_new, vhat_new, vhat_old, o_prev, active, c
             mass[(h, b)] = m
             probs[(h, b)] = (rows, P_new)
             scores[(h, b)] = P_new.sum(axis=0)
-    return {"O": O, "mass": mass, "probs": probs, "col_scores": scores}
+            with np.errstate(divide="ignore", invalid="ignore"):
+                lse[h, t_idx] = np.where(has, mx + np.log(np.where(den > 0, den, 1.0)) - np.log(m), np.nan)
+    return {"O": O, "mass": mass, "probs": probs, "col_scores": scores, "lse": lse}
 
 
 def old_term_local_softmax(q_old, khat_old, vhat_old, rows, S, m, sm_scale, head):
@@ -423,14 +429,16 @@ class LayerOracle:
             act = active_sets[r - 2]
             khat_new, k_pay = residual_update(np.asarray(K[r - 1])[act], khat, act, self.bits, self.group)
             vhat_new, v_pay = residual_update(np.asarray(V[r - 1])[act], vhat, act, self.bits, self.group)
-            res = sparse_loop_attention(np.asarray(Q[r - 1])[act], khat_new, vhat_new, vhat, o_full[act],
+            o_prev_rows = o_full[act]
+            res = sparse_loop_attention(np.asarray(Q[r - 1])[act], khat_new, vhat_new, vhat, o_prev_rows,
                                         act, col_sets, cache, self.sm_scale, self.q_block,
                                         head_list=self.head_list)
             o_full = o_full.copy()
             o_full[act] = res["O"]
             rec = {"r": r, "active": act, "col_sets": dict(col_sets), "k_payload": k_pay, "v_payload": v_pay,
                    "khat": khat_new, "vhat": vhat_new, "khat_old": khat, "vhat_old": vhat,
-                   "O_rows": res["O"], "O_full": o_full, "mass": res["mass"], "p_old": cache,
+                   "O_rows": res["O"], "O_full": o_full, "O_prev_rows": o_prev_rows, "lse_rows": res["lse"],
+                   "mass": res["mass"], "p_old": cache,
                    "p_new": res["probs"], "col_scores_next": res["col_scores"]}
             out["loops"].append(rec)
             # prepare loop r+1: prune within S with the next budget, keep the matching probabilities

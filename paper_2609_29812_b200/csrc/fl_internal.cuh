@@ -1,0 +1,155 @@
+// Internal declarations shared by the kernels of libflashloop (never installed).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "flashloop.h"
+
+struct fl_ctx {
+  int device;
+  int sm_count;
+  int max_smem_optin;
+  void* workspace;
+  size_t workspace_bytes;
+};
+
+#define FL_CHECK_CUDA(expr)                    \
+  do {                                         \
+    cudaError_t e__ = (expr);                  \
+    if (e__ != cudaSuccess) return FL_ERR_CUDA; \
+  } while (0)
+
+#define FL_REQUIRE(cond)                     \
+  do {                                       \
+    if (!(cond)) return FL_ERR_INVALID_ARG;  \
+  } while (0)
+
+static inline bool fl_aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Host-side checks every entry point shares. Returns FL_OK, FL_ERR_INVALID_ARG or FL_ERR_UNSUPPORTED.
+int fl_check_shape(const fl_shape* s);
+int fl_check_store(const fl_shape* s, const fl_kv_store* st, int n_streams_needed);
+int fl_launch_status();  // maps cudaGetLastError() to a status
+
+static inline int fl_elem_bytes(const fl_shape* s) { return s->dtype == FL_F32 ? 4 : 2; }
+static inline int fl_n_blocks(const fl_shape* s) { return (s->L + s->q_block - 1) / s->q_block; }
+
+// ---------------------------------------------------------------------------------------------
+// Device view of one side (K or V) of a store: base rows and the residual streams in loop order.
+// ---------------------------------------------------------------------------------------------
+struct DevStream {
+  const uint8_t* codes;
+  const __half* scale;
+  const __half* zero;
+  const int32_t* slot;
+};
+struct DevSide {
+  const void* base;
+  DevStream s[FL_MAX_LOOPS];
+};
+
+static inline void fl_dev_side(const fl_kv_store* st, bool is_k, DevSide* out) {
+  out->base = is_k ? st->k_base : st->v_base;
+  for (int i = 0; i < FL_MAX_LOOPS; ++i) {
+    const fl_kv_stream& s = is_k ? st->k_res[i] : st->v_res[i];
+    out->s[i].codes = static_cast<const uint8_t*>(s.codes);
+    out->s[i].scale = reinterpret_cast<const __half*>(s.scale);
+    out->s[i].zero = reinterpret_cast<const __half*>(s.zero);
+    out->s[i].slot = s.slot_of_pos;
+  }
+}
+
+#ifdef __CUDACC__
+// ---- 8-element vector access in storage type ---------------------------------------------------
+template <typename T>
+__device__ __forceinline__ void load8(const T* p, float (&v)[8]);
+template <>
+__device__ __forceinline__ void load8<__nv_bfloat16>(const __nv_bfloat16* p, float (&v)[8]) {
+  uint4 raw = *reinterpret_cast<const uint4*>(p);
+  const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&raw);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    float2 f = __bfloat1622float2(h[i]);
+    v[2 * i] = f.x;
+    v[2 * i + 1] = f.y;
+  }
+}
+template <>
+__device__ __forceinline__ void load8<float>(const float* p, float (&v)[8]) {
+  float4 a = *reinterpret_cast<const float4*>(p);
+  float4 b = *reinterpret_cast<const float4*>(p + 4);
+  v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+  v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+}
+template <typename T>
+__device__ __forceinline__ void store8(T* p, const float (&v)[8]);
+template <>
+__device__ __forceinline__ void store8<__nv_bfloat16>(__nv_bfloat16* p, const float (&v)[8]) {
+  uint4 raw;
+  __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&raw);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) h[i] = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+  *reinterpret_cast<uint4*>(p) = raw;
+}
+template <>
+__device__ __forceinline__ void store8<float>(float* p, const float (&v)[8]) {
+  *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]);
+  *reinterpret_cast<float4*>(p + 4) = make_float4(v[4], v[5], v[6], v[7]);
+}
+
+// Extract the 8 codes of one lane (8 consecutive elements) from the packed stream row.
+// `off8` is the element offset inside the row (multiple of 8).
+template <int BITS>
+__device__ __forceinline__ void load_codes8(const uint8_t* row_codes, int off8, uint32_t (&c)[8]) {
+  if (BITS == 8) {
+    uint2 raw = *reinterpret_cast<const uint2*>(row_codes + off8);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      c[i] = (raw.x >> (8 * i)) & 0xFFu;
+      c[4 + i] = (raw.y >> (8 * i)) & 0xFFu;
+    }
+  } else if (BITS == 4) {
+    uint32_t raw = *reinterpret_cast<const uint32_t*>(row_codes + off8 / 2);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) c[i] = (raw >> (4 * i)) & 0xFu;
+  } else {  // 2 bits
+    uint32_t raw = *reinterpret_cast<const uint16_t*>(row_codes + off8 / 4);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) c[i] = (raw >> (2 * i)) & 0x3u;
+  }
+}
+
+// Add one residual stream's contribution to 8 consecutive elements of position `pos` (Eq. 8):
+// x <- x + D(code) in binary32 (or x <- stored row when the codec is off). Returns false when the
+// position carries no payload in this stream. `elem` = h*dh + e0 is the element offset inside a row of
+// d elements (multiple of 8).
+template <typename T, int BITS>
+__device__ __forceinline__ bool apply_stream8(const DevStream& st, int pos, int elem, int d, int group,
+                                              float (&x)[8]) {
+  const int slot = __ldg(st.slot + pos);
+  if (slot < 0) return false;
+  if (BITS == 16) {
+    load8<T>(reinterpret_cast<const T*>(st.codes) + (size_t)slot * d + elem, x);
+  } else {
+    uint32_t c[8];
+    load_codes8<BITS>(st.codes + (size_t)slot * (d * BITS / 8), elem, c);
+    const size_t gi = (size_t)slot * (d / group) + elem / group;
+    const float sc = __half2float(st.scale[gi]);
+    const float zr = __half2float(st.zero[gi]);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) x[i] = __fadd_rn(x[i], __fmaf_rn((float)c[i], sc, zr));
+  }
+  return true;
+}
+
+// Reconstruct 8 consecutive elements of Xhat after the first n_use residual streams
+// (Eq. 8 chain in binary32, loop order): x = ((base + D_2) + D_3) + ...
+template <typename T, int BITS>
+__device__ __forceinline__ void recon8(const DevSide& side, int n_use, int pos, int elem, int d, int group,
+                                       float (&x)[8]) {
+  load8<T>(static_cast<const T*>(side.base) + (size_t)pos * d + elem, x);
+  for (int s = 0; s < n_use; ++s) apply_stream8<T, BITS>(side.s[s], pos, elem, d, group, x);
+}
+#endif  // __CUDACC__

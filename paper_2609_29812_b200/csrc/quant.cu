@@ -1,0 +1,133 @@
+// Stage 3: residual quantization of the active rows' K and V (Eq. 8 with the asymmetric group-wise
+// min/max quantizer of Appendix E). HBM-bound: each thread owns 8 consecutive elements (one 16-byte
+// load in bf16), group min/max by sub-warp shuffles, codes packed and stored coalesced.
+#include "fl_internal.cuh"
+
+namespace {
+
+struct QuantArgs {
+  DevSide k, v;                 // base + earlier streams (read), in loop order
+  const void* k_new;            // [n, H, dh]
+  const void* v_new;
+  const int32_t* active_idx;    // [n]
+  uint8_t* k_codes; __half* k_scale; __half* k_zero;   // stream being written
+  uint8_t* v_codes; __half* v_scale; __half* v_zero;
+  int n_prev;                   // residual streams already in the chain (loop_r - 2)
+  int d, group;
+};
+
+template <typename T, int BITS>
+__global__ void __launch_bounds__(256) quant_residual_kernel(const __grid_constant__ QuantArgs a) {
+  const int t = blockIdx.x;                 // active row
+  const bool is_v = blockIdx.y != 0;
+  const DevSide& side = is_v ? a.v : a.k;
+  const T* x_new = static_cast<const T*>(is_v ? a.v_new : a.k_new) + (size_t)t * a.d;
+  uint8_t* codes = is_v ? a.v_codes : a.k_codes;
+  __half* scale = is_v ? a.v_scale : a.k_scale;
+  __half* zero = is_v ? a.v_zero : a.k_zero;
+  const int pos = __ldg(a.active_idx + t);
+  const int lanes_per_group = a.group >> 3;  // 1, 2, 4, 8 or 16
+
+  for (int elem = threadIdx.x * 8; elem < a.d; elem += blockDim.x * 8) {
+    float xn[8], xh[8];
+    load8<T>(x_new + elem, xn);
+    recon8<T, BITS>(side, a.n_prev, pos, elem, a.d, a.group, xh);
+    if (BITS == 16) {  // codec off: the stream keeps the row itself
+      store8<T>(reinterpret_cast<T*>(codes) + (size_t)t * a.d + elem, xn);
+      continue;
+    }
+    float dl[8];
+    float mn, mx;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) dl[i] = __fsub_rn(xn[i], xh[i]);
+    mn = mx = dl[0];
+#pragma unroll
+    for (int i = 1; i < 8; ++i) { mn = fminf(mn, dl[i]); mx = fmaxf(mx, dl[i]); }
+    // every lane of the warp is here: the host only launches row widths for which all threads of the
+    // block run the same number of iterations (d % 256 == 0, and d % 2048 == 0 beyond 2048)
+    for (int o = 1; o < lanes_per_group; o <<= 1) {
+      mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    }
+    const __half zh = __float2half_rd(mn);
+    const float zf = __half2float(zh);
+    const float range = __fsub_rn(mx, zf);
+    const float qmax = (float)((1 << BITS) - 1);
+    const __half sh = range == 0.f ? __float2half_rn(0.f) : __float2half_ru(__fdiv_rn(range, qmax));
+    const float sf = __half2float(sh);
+    uint32_t packed_lo = 0, packed_hi = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      uint32_t c = 0;
+      if (sf != 0.f) {
+        float q = __fdiv_rn(__fsub_rn(dl[i], zf), sf);
+        q = fminf(fmaxf(rintf(q), 0.f), qmax);
+        c = (uint32_t)q;
+      }
+      if (BITS == 8) {
+        if (i < 4) packed_lo |= c << (8 * i); else packed_hi |= c << (8 * (i - 4));
+      } else {
+        packed_lo |= c << (BITS * i);
+      }
+    }
+    uint8_t* row = codes + (size_t)t * (a.d * BITS / 8);
+    if (BITS == 8) *reinterpret_cast<uint2*>(row + elem) = make_uint2(packed_lo, packed_hi);
+    else if (BITS == 4) *reinterpret_cast<uint32_t*>(row + elem / 2) = packed_lo;
+    else *reinterpret_cast<uint16_t*>(row + elem / 4) = (uint16_t)packed_lo;
+    if (((elem >> 3) & (lanes_per_group - 1)) == 0) {
+      const size_t gi = (size_t)t * (a.d / a.group) + elem / a.group;
+      scale[gi] = sh;
+      zero[gi] = zh;
+    }
+  }
+}
+
+template <typename T>
+int launch_quant(const fl_shape* s, const QuantArgs& a, int n_active, cudaStream_t st) {
+  const int threads = a.d / 8 < 256 ? a.d / 8 : 256;
+  dim3 grid(n_active, 2);
+  switch (s->bits) {
+    case 2: quant_residual_kernel<T, 2><<<grid, threads, 0, st>>>(a); break;
+    case 4: quant_residual_kernel<T, 4><<<grid, threads, 0, st>>>(a); break;
+    case 8: quant_residual_kernel<T, 8><<<grid, threads, 0, st>>>(a); break;
+    default: quant_residual_kernel<T, 16><<<grid, threads, 0, st>>>(a); break;
+  }
+  return fl_launch_status();
+}
+
+}  // namespace
+
+extern "C" int fl_quant_kv_residual(fl_ctx* ctx, const fl_shape* shape, int loop_r, const void* k_new,
+                                    const void* v_new, const int32_t* active_idx, int32_t n_active,
+                                    const fl_kv_store* store, int32_t* status, void* stream) {
+  (void)status;
+  FL_REQUIRE(ctx != nullptr);
+  int rc = fl_check_shape(shape);
+  if (rc != FL_OK) return rc;
+  FL_REQUIRE(loop_r >= 2 && loop_r <= FL_MAX_LOOPS + 1);
+  FL_REQUIRE(n_active >= 0 && n_active <= shape->L);
+  rc = fl_check_store(shape, store, loop_r - 1);
+  if (rc != FL_OK) return rc;
+  const fl_kv_stream& ks = store->k_res[loop_r - 2];
+  const fl_kv_stream& vs = store->v_res[loop_r - 2];
+  FL_REQUIRE(ks.n_rows == n_active && vs.n_rows == n_active);
+  if (n_active == 0) return FL_OK;
+  FL_REQUIRE(k_new != nullptr && v_new != nullptr && active_idx != nullptr);
+  FL_REQUIRE(fl_aligned16(k_new) && fl_aligned16(v_new));
+  const int d = shape->n_heads * shape->head_dim;
+  // whole warps must enter or leave the element loop together (sub-warp shuffles inside)
+  if (d % 256 != 0 || (d > 2048 && d % 2048 != 0)) return FL_ERR_UNSUPPORTED;
+
+  QuantArgs a;
+  fl_dev_side(store, true, &a.k);
+  fl_dev_side(store, false, &a.v);
+  a.k_new = k_new; a.v_new = v_new; a.active_idx = active_idx;
+  a.k_codes = static_cast<uint8_t*>(ks.codes); a.k_scale = reinterpret_cast<__half*>(ks.scale);
+  a.k_zero = reinterpret_cast<__half*>(ks.zero);
+  a.v_codes = static_cast<uint8_t*>(vs.codes); a.v_scale = reinterpret_cast<__half*>(vs.scale);
+  a.v_zero = reinterpret_cast<__half*>(vs.zero);
+  a.n_prev = loop_r - 2; a.d = d; a.group = shape->group;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  return shape->dtype == FL_F32 ? launch_quant<float>(shape, a, n_active, st)
+                                : launch_quant<__nv_bfloat16>(shape, a, n_active, st);
+}

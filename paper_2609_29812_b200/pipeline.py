@@ -1,0 +1,160 @@
+"""Call-order harness for one layer: allocates device buffers with PyTorch and calls the C-ABI
+entry points in the order of the hot path.  No arithmetic of the method lives here; every step
+runs inside libflashloop's kernels.
+
+Per-layer state carried across loops (all caller-owned device tensors):
+  k_base, v_base [L,H,dh]      loop-1 K/V (storage type)
+  streams[r-2]                 residual payloads of loop r: codes, scale, zero (K and V)
+  q_store, o_store [L,H,dh]    latest Q and attention output of every position
+  lse [H,L]                    latest log-normaliser of every (head, position), updated in place
+  col_idx [H,nb,c], col_cnt    selected columns per (head, query block)
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+from typing import List, Optional
+
+import torch
+
+from . import binding as B
+from .workloads import Workload
+
+
+def torch_dtype(w: Workload):
+    return torch.float32 if w.dtype == "f32" else torch.bfloat16
+
+
+def fl_dtype(w: Workload) -> int:
+    return B.FL_F32 if w.dtype == "f32" else B.FL_BF16
+
+
+def shape_of(w: Workload, bits: Optional[int] = None, q_block: Optional[int] = None):
+    return B.make_shape(w.L, w.n_heads, w.head_dim, fl_dtype(w), q_block or w.q_block, bits or w.bits, w.group,
+                        w.eps, w.sm_scale)
+
+
+@dataclass
+class TokenSelection:
+    active_idx: torch.Tensor     # int32 [n]
+    slot_of_pos: torch.Tensor    # int32 [L]
+    scores: torch.Tensor         # f32 [n_cand]
+    n: int
+
+
+def select_tokens(ctx, shape, loop_r, g_prev, g_cur, cand: Optional[torch.Tensor], k: int) -> TokenSelection:
+    L = shape.L
+    dev = g_cur.device
+    n_cand = L if cand is None else int(cand.numel())
+    n = min(k, n_cand)
+    scores = torch.empty(n_cand, dtype=torch.float32, device=dev)
+    active = torch.empty(max(n, 1), dtype=torch.int32, device=dev)
+    slot = torch.empty(L, dtype=torch.int32, device=dev)
+    B.fl_select_tokens(ctx, shape, loop_r, g_prev, g_cur, cand, n_cand, k, scores, active, slot)
+    return TokenSelection(active[:n], slot, scores, n)
+
+
+class LayerState:
+    """Buffers of one layer and the calls that advance it by one loop."""
+
+    def __init__(self, ctx, w: Workload, device="cuda:0", bits: Optional[int] = None, q_block: Optional[int] = None,
+                 c: Optional[int] = None):
+        self.ctx, self.w, self.dev = ctx, w, torch.device(device)
+        self.shape = shape_of(w, bits, q_block)
+        self.bits = self.shape.bits
+        self.c = c or w.col_budget
+        self.nb = (w.L + self.shape.q_block - 1) // self.shape.q_block
+        self.dt = torch_dtype(w)
+        self.k_streams: List[dict] = []
+        self.v_streams: List[dict] = []
+        self.col_idx = None
+        self.col_cnt = None
+        self.col_scores = None
+        self.lse = None
+        self.store = None
+
+    # ---- loop 1 -------------------------------------------------------------------------------
+    def dense_loop(self, q, k, v, want_col_scores=True):
+        w = self.w
+        self.k_base, self.v_base = k, v
+        self.q_store = q.clone()
+        self.o_store = torch.empty_like(q)
+        self.lse = torch.empty(w.n_heads, w.L, dtype=torch.float32, device=self.dev)
+        if want_col_scores:
+            self.col_scores = torch.empty(w.n_heads, self.nb, w.L, dtype=torch.float32, device=self.dev)
+        B.fl_dense_loop_attention(self.ctx, self.shape, q, k, v, self.o_store, self.lse, self.col_scores)
+        self._rebuild_store()
+
+    def select_columns_dense(self, c: Optional[int] = None, col_scores=None):
+        w = self.w
+        c = c or self.c
+        self.c = c
+        self.col_idx = torch.empty(w.n_heads, self.nb, c, dtype=torch.int32, device=self.dev)
+        self.col_cnt = torch.empty(w.n_heads, self.nb, dtype=torch.int32, device=self.dev)
+        B.fl_select_columns(self.ctx, self.shape, self.col_scores if col_scores is None else col_scores, None, None,
+                            w.L, c, self.col_idx, self.col_cnt)
+
+    def prune_columns(self, col_scores_next, c_next: int):
+        """Sparse source loop: keep the c_next best of the current set (Eq. 6, nested selection)."""
+        w = self.w
+        new_idx = torch.empty(w.n_heads, self.nb, c_next, dtype=torch.int32, device=self.dev)
+        new_cnt = torch.empty(w.n_heads, self.nb, dtype=torch.int32, device=self.dev)
+        B.fl_select_columns(self.ctx, self.shape, col_scores_next, self.col_idx, self.col_cnt, self.c, c_next,
+                            new_idx, new_cnt)
+        self.col_idx, self.col_cnt, self.c = new_idx, new_cnt, c_next
+
+    # ---- loop r >= 2 --------------------------------------------------------------------------
+    def _rebuild_store(self):
+        self.store = B.make_store(self.k_base, self.v_base, self.k_streams, self.v_streams)
+
+    def alloc_stream(self, sel: TokenSelection):
+        w, n = self.w, sel.n
+        d = w.d
+
+        def one():
+            if self.bits == 16:
+                return {"codes": torch.empty(max(n, 1), d, dtype=self.dt, device=self.dev), "scale": None,
+                        "zero": None, "slot_of_pos": sel.slot_of_pos, "n_rows": n}
+            return {"codes": torch.empty(max(n, 1), d * self.bits // 8, dtype=torch.uint8, device=self.dev),
+                    "scale": torch.empty(max(n, 1), d // w.group, dtype=torch.float16, device=self.dev),
+                    "zero": torch.empty(max(n, 1), d // w.group, dtype=torch.float16, device=self.dev),
+                    "slot_of_pos": sel.slot_of_pos, "n_rows": n}
+        self.k_streams.append(one())
+        self.v_streams.append(one())
+        self._rebuild_store()
+
+    def quantize(self, loop_r, k_new, v_new, sel: TokenSelection):
+        B.fl_quant_kv_residual(self.ctx, self.shape, loop_r, k_new, v_new, sel.active_idx, sel.n, self.store)
+
+    def gather(self, full, sel: TokenSelection, out=None):
+        row_bytes = full.shape[1] * full.shape[2] * full.element_size() if full.dim() == 3 else \
+            full.shape[1] * full.element_size()
+        if out is None:
+            out = torch.empty((max(sel.n, 1),) + tuple(full.shape[1:]), dtype=full.dtype, device=self.dev)
+        B.fl_gather_rows(self.ctx, full, sel.active_idx, sel.n, row_bytes, out)
+        return out
+
+    def scatter(self, rows, sel: TokenSelection, full):
+        row_bytes = full.shape[1] * full.shape[2] * full.element_size() if full.dim() == 3 else \
+            full.shape[1] * full.element_size()
+        B.fl_scatter_update(self.ctx, rows, sel.active_idx, sel.n, row_bytes, full)
+
+    def attention(self, loop_r, q_new, q_old, o_prev, o_out, sel: TokenSelection, col_scores_next=None):
+        B.fl_loop_attention(self.ctx, self.shape, loop_r, q_new, q_old, sel.active_idx, sel.n, self.store,
+                            self.col_idx, self.col_cnt, self.c, self.lse, self.lse, o_prev, o_out,
+                            col_scores_next)   # lse updated in place: only the active rows change
+
+    def sparse_loop(self, loop_r, q_new, k_new, v_new, sel: TokenSelection, want_col_scores_next=False):
+        """One loop r >= 2 for this layer: store residuals, gather the carried rows, attend, scatter back.
+        q_new, k_new, v_new: [n, H, dh] rows of the active tokens.  Returns (o_rows, col_scores_next)."""
+        self.alloc_stream(sel)
+        self.quantize(loop_r, k_new, v_new, sel)
+        q_old = self.gather(self.q_store, sel)
+        o_prev = self.gather(self.o_store, sel)
+        o_out = torch.empty_like(o_prev)
+        csn = None
+        if want_col_scores_next:
+            csn = torch.zeros(self.w.n_heads, self.nb, self.c, dtype=torch.float32, device=self.dev)
+        self.attention(loop_r, q_new, q_old, o_prev, o_out, sel, csn)
+        self.scatter(o_out, sel, self.o_store)
+        self.scatter(q_new, sel, self.q_store)
+        return o_out, csn

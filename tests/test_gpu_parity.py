@@ -1,0 +1,266 @@
+"""GPU parity: every stage of the CUDA path, called through the C ABI, against the CPU oracle on the
+same seeded inputs.  Integer results (index sets, codes, fp16 metadata) are compared bit for bit;
+attention outputs within relative L2 <= 1e-2 and max-abs <= 3e-2."""
+import dataclasses
+
+import numpy as np
+import pytest
+
+from oracle import flashloop_oracle as fo
+from paper_2609_29812_b200 import workloads
+from helpers import (assert_attn_close, assert_selection_matches, storage_round, to_dev, to_np)
+
+pytestmark = pytest.mark.gpu
+torch = pytest.importorskip("torch")
+
+
+@pytest.fixture(scope="module")
+def env():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2609_29812_b200 import binding, pipeline
+    ctx = binding.Context(0)
+    yield binding, pipeline, ctx
+    ctx.close()
+
+
+def small_bf16(L=2000, H=2, R=4, **kw):
+    """Config-2-shaped workload shrunk so the oracle runs in seconds; L is not a multiple of the block."""
+    w = workloads.config2(L=L, n_heads=H)
+    return dataclasses.replace(w, n_loops=R, q_block=kw.pop("q_block", 256), col_budget=kw.pop("c", 160),
+                               changed_fracs=w.changed_fracs[: R - 1], **kw)
+
+
+WORKLOADS = {
+    "c1": lambda: workloads.config1(),
+    "bf16_small": lambda: small_bf16(),
+    "bf16_int8_g64": lambda: small_bf16(L=1200, bits=8, group=64),
+    "bf16_int2_g32": lambda: small_bf16(L=1200, bits=2, group=32),
+    "bf16_off": lambda: small_bf16(L=1200, bits=16),
+}
+
+
+@pytest.fixture(scope="module", params=list(WORKLOADS))
+def case(request):
+    w = WORKLOADS[request.param]()
+    x = workloads.make_layer_inputs(w, seed=3)
+    orc = fo.LayerOracle(w.L, w.n_heads, w.head_dim, w.q_block, w.bits, w.group, w.eps, w.sm_scale)
+    ref = orc.run(x.G, x.Q, x.K, x.V, [w.k_tokens] * (w.n_loops - 1), [w.col_budget] * (w.n_loops - 1))
+    return w, x, ref
+
+
+# ------------------------------------------------------------------------------------------------
+def test_gather_scatter_bit_exact(env):
+    B, P, ctx = env
+    g = torch.Generator(device="cpu").manual_seed(0)
+    for rows, width, dt in [(1000, 2048, torch.bfloat16), (77, 256, torch.float32), (5, 8, torch.bfloat16)]:
+        src = torch.randn(rows, width, generator=g).to(dt).cuda()
+        idx = torch.sort(torch.randperm(rows, generator=g)[: max(1, rows // 3)])[0].to(torch.int32).cuda()
+        n = idx.numel()
+        dst = torch.zeros(n, width, dtype=dt, device="cuda")
+        B.fl_gather_rows(ctx, src, idx, n, width * src.element_size(), dst)
+        assert torch.equal(dst, src[idx.long()])
+        full = torch.full((rows, width), 7.0, dtype=dt, device="cuda")
+        B.fl_scatter_update(ctx, dst, idx, n, width * src.element_size(), full)
+        expect = torch.full((rows, width), 7.0, dtype=dt, device="cuda")
+        expect[idx.long()] = dst
+        assert torch.equal(full, expect)
+    B.fl_gather_rows(ctx, src, idx, 0, 16, dst)        # empty call is a no-op
+
+
+def test_token_selection(env, case):
+    B, P, ctx = env
+    w, x, ref = case
+    sh = P.shape_of(w)
+    cand = None
+    for r in range(2, w.n_loops + 1):
+        g_prev, g_cur = to_dev(x.G[r - 2], w), to_dev(x.G[r - 1], w)
+        sel = P.select_tokens(ctx, sh, r, g_prev, g_cur, cand, w.k_tokens)
+        scores = to_np(sel.scores).astype(np.float64)
+        cand_np = np.arange(w.L) if cand is None else to_np(cand).astype(np.int64)
+        np.testing.assert_allclose(scores, ref["token_scores"][r - 2], rtol=2e-5, atol=1e-9)
+        got = to_np(sel.active_idx).astype(np.int64)
+        # exact with respect to its own binary32 scores (total order: score desc, index asc)
+        own = cand_np[fo.topk_ascending(to_np(sel.scores), w.k_tokens)]
+        assert np.array_equal(got, own)
+        # and equal to the independent fp64 oracle except inside a near-tie band
+        assert_selection_matches(got, ref["token_scores"][r - 2], cand_np, w.k_tokens, f"tokens loop {r}")
+        slot = to_np(sel.slot_of_pos)
+        assert np.array_equal(slot, fo.slot_map(got, w.L))
+        cand = sel.active_idx
+
+
+def test_token_selection_ties_and_small_budgets(env):
+    B, P, ctx = env
+    w = dataclasses.replace(workloads.config1(), L=300)
+    sh = P.shape_of(w)
+    rng = np.random.default_rng(0)
+    g1 = rng.standard_normal((w.L, w.d)).astype(np.float32)
+    g2 = g1.copy()
+    # rows 10, 20, ..., 290 get the SAME update applied to the SAME base row: exactly equal scores
+    g1[10::10] = g1[10]
+    g2[10::10] = g1[10] + 0.5
+    g2[5] = g1[5] + 3.0                                     # one clear winner
+    for k in (1, 2, 7, 30, 299, 300, 1000):
+        sel = P.select_tokens(ctx, sh, 2, to_dev(g1, w), to_dev(g2, w), None, k)
+        s = to_np(sel.scores)
+        assert np.all(s[10::10] == s[10])
+        expect = fo.topk_ascending(s, k)
+        assert np.array_equal(to_np(sel.active_idx), expect), k
+        if 1 < k <= 30:
+            assert to_np(sel.active_idx).tolist() == [5] + list(range(10, 10 * k, 10))
+    # candidate subset
+    cand = torch.tensor([3, 5, 10, 20, 30, 44], dtype=torch.int32, device="cuda")
+    sel = P.select_tokens(ctx, sh, 3, to_dev(g1, w), to_dev(g2, w), cand, 3)
+    assert to_np(sel.active_idx).tolist() == [5, 10, 20]
+    assert to_np(sel.slot_of_pos)[[5, 10, 20, 30]].tolist() == [0, 1, 2, -1]
+
+
+def build_gpu_layer(env, w, x, ref, upto_loop, use_oracle_sets=True):
+    """Runs the GPU path through loop `upto_loop` - 1, feeding oracle token sets (stage isolation)."""
+    B, P, ctx = env
+    st = P.LayerState(ctx, w)
+    st.dense_loop(to_dev(x.Q[0], w), to_dev(x.K[0], w), to_dev(x.V[0], w))
+    st.select_columns_dense()
+    return st
+
+
+def oracle_selection(P, w, ref, r):
+    act = ref["active"][r - 2]
+    return P.TokenSelection(torch.from_numpy(act.astype(np.int32)).cuda(),
+                            torch.from_numpy(fo.slot_map(act, w.L)).cuda(), None, len(act))
+
+
+def test_quantizer_codes_bit_exact_all_loops(env, case):
+    B, P, ctx = env
+    w, x, ref = case
+    st = P.LayerState(ctx, w)
+    st.k_base, st.v_base = to_dev(x.K[0], w), to_dev(x.V[0], w)
+    for r in range(2, w.n_loops + 1):
+        sel = oracle_selection(P, w, ref, r)
+        act = ref["active"][r - 2]
+        st.alloc_stream(sel)
+        st.quantize(r, to_dev(x.K[r - 1][act], w), to_dev(x.V[r - 1][act], w), sel)
+        rec = ref["loops"][r - 2]
+        for side, streams in (("k_payload", st.k_streams), ("v_payload", st.v_streams)):
+            pay, got = rec[side], streams[-1]
+            if w.bits == 16:
+                assert np.array_equal(to_np(got["codes"]).reshape(pay["raw"].shape), pay["raw"])
+                continue
+            n = len(act)
+            assert np.array_equal(to_np(got["codes"]).reshape(n, w.n_heads, -1), pay["packed"]), (r, side)
+            assert np.array_equal(to_np(got["scale"]).view(np.uint16).reshape(pay["scale"].shape),
+                                  pay["scale"].view(np.uint16)), (r, side)
+            assert np.array_equal(to_np(got["zero"]).view(np.uint16).reshape(pay["zero"].shape),
+                                  pay["zero"].view(np.uint16)), (r, side)
+
+
+def test_dense_source_loop(env, case):
+    B, P, ctx = env
+    w, x, ref = case
+    st = build_gpu_layer(env, w, x, ref, 2)
+    d = ref["dense"]
+    assert_attn_close(to_np(st.o_store), d["O"], "dense O")
+    np.testing.assert_allclose(to_np(st.lse), d["lse"], rtol=0, atol=2e-4)
+    cs = to_np(st.col_scores).astype(np.float64)
+    for b in range(st.nb):
+        end = min(w.L, (b + 1) * w.q_block)
+        np.testing.assert_allclose(cs[:, b, :end], d["col_scores"][:, b, :end], rtol=2e-4, atol=1e-7)
+    # column selection: exact on its own scores, near-tie protocol against the oracle's scores
+    idx, cnt = to_np(st.col_idx), to_np(st.col_cnt)
+    n_diff = 0
+    for h in range(w.n_heads):
+        for b in range(st.nb):
+            end = min(w.L, (b + 1) * w.q_block)
+            k = min(w.col_budget, end)
+            assert cnt[h, b] == k and np.all(idx[h, b, k:] == -1)
+            own = fo.topk_ascending(to_np(st.col_scores)[h, b, :end], k)
+            assert np.array_equal(idx[h, b, :k], own)
+            n_diff += assert_selection_matches(idx[h, b, :k], d["col_scores"][h, b, :end], np.arange(end), k,
+                                               f"columns h{h} b{b}")
+    assert n_diff <= 0.01 * w.n_heads * st.nb * w.col_budget
+
+
+def test_select_columns_on_oracle_scores_is_exact(env, case):
+    B, P, ctx = env
+    w, x, ref = case
+    st = P.LayerState(ctx, w)
+    cs32 = ref["dense"]["col_scores"].astype(np.float32)
+    st.col_scores = torch.from_numpy(cs32).cuda()
+    st.select_columns_dense()
+    idx = to_np(st.col_idx)
+    for h in range(w.n_heads):
+        for b in range(st.nb):
+            end = min(w.L, (b + 1) * w.q_block)
+            k = min(w.col_budget, end)
+            assert np.array_equal(idx[h, b, :k], fo.topk_ascending(cs32[h, b, :end], k))
+
+
+def sets_to_arrays(w, nb, col_sets, c):
+    idx = np.full((w.n_heads, nb, c), -1, dtype=np.int32)
+    cnt = np.zeros((w.n_heads, nb), dtype=np.int32)
+    for (h, b), S in col_sets.items():
+        idx[h, b, : len(S)] = S
+        cnt[h, b] = len(S)
+    return idx, cnt
+
+
+def test_loop_attention_stage_isolated(env, case):
+    """Each loop's attention is fed the oracle's upstream state (token set, column sets, previous
+    outputs and log-normalisers rounded to storage precision; the store is bit-exact anyway)."""
+    B, P, ctx = env
+    w, x, ref = case
+    st = P.LayerState(ctx, w)
+    st.k_base, st.v_base = to_dev(x.K[0], w), to_dev(x.V[0], w)
+    lse = ref["dense"]["lse"].astype(np.float32).copy()
+    q_prev_full = x.Q[0]
+    for r in range(2, w.n_loops + 1):
+        rec = ref["loops"][r - 2]
+        act = rec["active"]
+        sel = oracle_selection(P, w, ref, r)
+        st.alloc_stream(sel)
+        st.quantize(r, to_dev(x.K[r - 1][act], w), to_dev(x.V[r - 1][act], w), sel)
+        idx, cnt = sets_to_arrays(w, st.nb, rec["col_sets"], w.col_budget)
+        st.col_idx, st.col_cnt, st.c = torch.from_numpy(idx).cuda(), torch.from_numpy(cnt).cuda(), w.col_budget
+        st.lse = torch.from_numpy(lse).cuda()
+        o_prev = to_dev(storage_round(rec["O_prev_rows"], w), w)
+        o_out = torch.empty_like(o_prev)
+        csn = torch.zeros(w.n_heads, st.nb, st.c, dtype=torch.float32, device="cuda")
+        st.attention(r, to_dev(x.Q[r - 1][act], w), to_dev(q_prev_full[act], w), o_prev, o_out, sel, csn)
+        assert_attn_close(to_np(o_out), rec["O_rows"], f"loop {r} O rows")
+        # log-normaliser of the active rows and next-loop column scores
+        got_lse = to_np(st.lse)[:, act]
+        ok = np.isfinite(rec["lse_rows"])
+        np.testing.assert_allclose(got_lse[ok], rec["lse_rows"][ok], rtol=0, atol=5e-3)
+        csn = to_np(csn)
+        for (h, b), s_ref in rec["col_scores_next"].items():
+            np.testing.assert_allclose(csn[h, b, : len(s_ref)], s_ref, rtol=2e-2, atol=2e-4)
+        # oracle state for the next loop
+        lse = lse.copy()
+        lse[:, act] = np.where(ok, rec["lse_rows"], lse[:, act]).astype(np.float32)
+        q_prev_full = q_prev_full.copy()
+        q_prev_full[act] = x.Q[r - 1][act]
+
+
+def test_chained_layer_all_on_gpu(env, case):
+    """Everything on the GPU, loop after loop; only the final comparison uses the oracle."""
+    B, P, ctx = env
+    w, x, ref = case
+    st = build_gpu_layer(env, w, x, ref, 2)
+    sh = st.shape
+    cand = None
+    for r in range(2, w.n_loops + 1):
+        sel = P.select_tokens(ctx, sh, r, to_dev(x.G[r - 2], w), to_dev(x.G[r - 1], w), cand, w.k_tokens)
+        act = to_np(sel.active_idx).astype(np.int64)
+        o_rows, _ = st.sparse_loop(r, to_dev(x.Q[r - 1][act], w), to_dev(x.K[r - 1][act], w),
+                                   to_dev(x.V[r - 1][act], w), sel)
+        cand = sel.active_idx
+        if np.array_equal(act, ref["active"][r - 2]):
+            assert_attn_close(to_np(o_rows), ref["loops"][r - 2]["O_rows"], f"chained loop {r}")
+    assert_attn_close(to_np(st.o_store), ref["loops"][-1]["O_full"], "chained final O store")
+    # KV accounting of the real store
+    fl, dense = B.fl_kv_store_bytes(sh, st.store, w.n_loops, 1)
+    n_r = [len(a) for a in ref["active"]]
+    fl_ref, dense_ref = fo.kv_bytes_per_token_layer(w.L, w.d, n_r, w.bits, w.group, 1,
+                                                    elem_bytes=4 if w.dtype == "f32" else 2)
+    assert dense == dense_ref * w.L and abs(fl - fl_ref * w.L) <= 4 * w.n_loops

@@ -93,7 +93,7 @@ def n_blocks(L: int, q_block: int) -> int:
     return (L + q_block - 1) // q_block
 
 
-def dense_loop_attention(q, k, v, sm_scale, q_block, rows_to_cache=None, head_list=None):
+def dense_loop_attention(q, k, v, sm_scale, q_block, rows_to_cache=None, head_list=None, block_list=None):
     """Causal softmax attention of one loop over all L rows, head by head.
 
     q, k, v: [L, H, dh].  Returns a dict with
@@ -103,7 +103,7 @@ def dense_loop_attention(q, k, v, sm_scale, q_block, rows_to_cache=None, head_li
                  (zero for j beyond the block's last row)
       probs      {(h,b): (rows, P)} only if rows_to_cache is given: P[t, j] = p_{rows[t], j}
                  for the rows of rows_to_cache that fall in block b, all j <= block end.
-    head_list restricts the work to some heads (others stay zero).
+    head_list / block_list restrict the work to some heads / query blocks (the rest stays zero).
     """
     q = np.asarray(q); k = np.asarray(k); v = np.asarray(v)
     L, H, dh = q.shape
@@ -118,7 +118,7 @@ def dense_loop_attention(q, k, v, sm_scale, q_block, rows_to_cache=None, head_li
     for h in heads:
         kh = k[:, h, :].astype(F64)
         vh = v[:, h, :].astype(F64)
-        for b in range(nb):
+        for b in (range(nb) if block_list is None else block_list):
             i0, i1 = b * q_block, min(L, (b + 1) * q_block)
             qi = q[i0:i1, h, :].astype(F64)
             logits = (qi @ kh[:i1].T) * F64(sm_scale)              # [rows, i1]
@@ -268,7 +268,7 @@ def residual_update(x_new_rows, xhat_prev, active, bits, group):
 # previous-loop probabilities.
 # --------------------------------------------------------------------------------------
 def sparse_loop_attention(q_new, khat_new, vhat_new, vhat_old, o_prev, active, col_sets, p_old_cache,
-                          sm_scale, q_block, head_list=None):
+                          sm_scale, q_block, head_list=None, block_list=None):
     """One sparse loop of Appendix D.2 for every (head, block).
 
     q_new     : [n, H, dh] queries of the active rows (ascending positions `active`)
@@ -295,7 +295,7 @@ def sparse_loop_attention(q_new, khat_new, vhat_new, vhat_old, o_prev, active, c
     heads = range(H) if head_list is None else head_list
     blk = active // q_block
     for h in heads:
-        for b in range(nb):
+        for b in (range(nb) if block_list is None else block_list):
             t_idx = np.nonzero(blk == b)[0]                      # slots of this block's active rows
             rows = active[t_idx]
             S = np.asarray(col_sets[(h, b)], dtype=np.int64)

@@ -167,3 +167,96 @@ def make_layer_inputs(w: Workload, seed: int = 0, layer: int = 0) -> LayerInputs
         v = store(x @ Wv).reshape(L, H, dh)
         G.append(g); Q.append(q); K.append(k); V.append(v)
     return LayerInputs(w, G, Q, K, V, changed, heavy)
+
+
+# ----------------------------------------------------------------------------------------------
+# Device-side generator for the stack configurations (too large for host numpy in reasonable time).
+# Same recipe as make_layer_inputs, drawn with torch's seeded CUDA generator.
+# ----------------------------------------------------------------------------------------------
+class DeviceStack:
+    """Synthetic 48-layer stack inputs on the GPU.
+
+    stack_hidden()        -> [G^(1) .. G^(R)], each [L, d] in storage type: the stack-level hidden state
+                             that token selection scores (one selection per loop, shared by all layers).
+    layer(l)              -> LayerGen with .qkv1() (all rows, loop 1), .hidden(r) ([L, d]) and
+                             .rows(r, active_idx) (Q, K, V of the active rows of loop r).
+    Each layer's input replaces the recurrence by the same lazy-update generator
+    (Y^(r) = Y^(r-1) + Delta^(r) on the shared nested changed-row sets); Q/K/V are projections of the
+    RMS-normalised rows with per-layer weights N(0, w_std).
+    """
+
+    def __init__(self, w: Workload, seed: int = 0, device="cuda:0"):
+        import torch
+        self.w, self.seed, self.device, self.torch = w, seed, device, torch
+        self.dt = torch.float32 if w.dtype == "f32" else torch.bfloat16
+        perm = _rng(seed, 0, 5).permutation(w.L)
+        self.changed = [torch.from_numpy(np.sort(perm[: w.n_changed(r)])).to(device)
+                        for r in range(2, w.n_loops + 1)]
+        n_heavy = int(np.floor(w.heavy_frac * w.L + 0.5))
+        self.heavy = torch.from_numpy(np.sort(_rng(seed, 0, 6).permutation(w.L)[:n_heavy])).to(device)
+
+    def _gen(self, layer: int, stream: int):
+        g = self.torch.Generator(device=self.device)
+        g.manual_seed((self.seed << 20) ^ (layer << 8) ^ stream)
+        return g
+
+    def _delta(self, layer: int, r: int):
+        torch, w = self.torch, self.w
+        g = self._gen(layer, 16 + r)
+        delta = torch.randn(w.L, w.d, generator=g, device=self.device) * w.delta_lo
+        rows = self.changed[r - 2]
+        delta[rows] = torch.randn(len(rows), w.d, generator=g, device=self.device) * w.delta_hi
+        return delta
+
+    def _chain(self, layer: int):
+        """Yields the storage-rounded hidden state of loops 1..R as float32 tensors."""
+        torch, w = self.torch, self.w
+        y = torch.randn(w.L, w.d, generator=self._gen(layer, 1), device=self.device).to(self.dt).float()
+        yield y
+        for r in range(2, w.n_loops + 1):
+            y = (y + self._delta(layer, r)).to(self.dt).float()
+            yield y
+
+    def stack_hidden(self):
+        return [y.to(self.dt) for y in self._chain(10_000)]
+
+    def layer(self, layer: int):
+        return LayerGen(self, layer)
+
+
+class LayerGen:
+    def __init__(self, stack: DeviceStack, layer: int):
+        torch, w = stack.torch, stack.w
+        self.s, self.layer_id = stack, layer
+        mk = lambda sid: (torch.randn(w.d, w.d, generator=stack._gen(layer, sid), device=stack.device)
+                          * w.w_std).to(stack.dt)
+        self.Wq, self.Wk, self.Wv = mk(2), mk(3), mk(4)
+        self._hidden = list(stack._chain(layer))            # R float32 tensors [L, d]
+
+    def hidden(self, r: int):
+        return self._hidden[r - 1].to(self.s.dt)
+
+    def _project(self, x, pos):
+        torch, w, s = self.s.torch, self.s.w, self.s
+        if w.rmsnorm:
+            x = x * torch.rsqrt(x.pow(2).mean(dim=1, keepdim=True) + 1e-6)
+        x = x.to(s.dt)
+        q = (x @ self.Wq).view(-1, w.n_heads, w.head_dim)
+        k = (x @ self.Wk).float()
+        if len(s.heavy):
+            is_heavy = torch.isin(pos, s.heavy)
+            k = torch.where(is_heavy[:, None], k * w.heavy_scale, k)
+        k = k.to(s.dt).view(-1, w.n_heads, w.head_dim)
+        v = (x @ self.Wv).view(-1, w.n_heads, w.head_dim)
+        return q.contiguous(), k.contiguous(), v.contiguous()
+
+    def qkv1(self):
+        torch, w = self.s.torch, self.s.w
+        return self._project(self._hidden[0], torch.arange(w.L, device=self.s.device))
+
+    def rows(self, r: int, active_idx):
+        pos = active_idx.long()
+        return self._project(self._hidden[r - 1][pos], pos)
+
+    def release(self):
+        self._hidden = None

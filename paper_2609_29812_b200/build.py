@@ -13,6 +13,7 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 OBJ_DIR = os.path.join(PKG, "build")
 LIB_PATH = os.path.join(PKG, "libflashloop.so")
+SELFTEST_LIB_PATH = os.path.join(PKG, "libflashloop_selftest.so")
 
 NVCC_FLAGS = [
     "-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
@@ -45,6 +46,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
     """Compile every .cu under csrc/ and link the shared library.  Returns its path."""
     srcs = sources()
     headers = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".cuh", ".h"))]
+    st_dir = os.path.join(CSRC, "selftest")
+    headers += [os.path.join(st_dir, f) for f in os.listdir(st_dir)]
     headers.append(os.path.join(ROOT, "include", "flashloop.h"))
     stamp = os.path.join(PKG, "libflashloop.stamp")
     digest = _digest(srcs + headers)
@@ -71,6 +74,13 @@ def build(force: bool = False, verbose: bool = False) -> str:
     r = subprocess.run(cmd, capture_output=True, text=True)
     if r.returncode != 0:
         raise RuntimeError(f"link failed:\n{r.stdout}\n{r.stderr}")
+    # tensor-path self-test kernels: a library of their own, loaded only by a GPU test
+    st_dir = os.path.join(CSRC, "selftest")
+    st_srcs = sorted(os.path.join(st_dir, f) for f in os.listdir(st_dir) if f.endswith(".cu"))
+    cmd = [nvcc, *NVCC_FLAGS, "-shared", "-o", SELFTEST_LIB_PATH, *st_srcs]
+    r = subprocess.run(cmd, capture_output=True, text=True)
+    if r.returncode != 0:
+        raise RuntimeError(f"self-test library failed to build:\n{r.stdout}\n{r.stderr}")
     with open(stamp, "w") as f:
         f.write(digest)
     return LIB_PATH

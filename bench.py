@@ -517,7 +517,7 @@ def oracle_sample(w, n_blocks_sample=2, seed=0):
         t_quant += time.time() - t0
         t0 = time.time()
         res = fo.sparse_loop_attention(qr, khat_new, vhat_new, vhat, o_full[act], act, sets, cache, w.sm_scale,
-                                       w.q_block, head_list=[0], block_list=blocks)
+                                       w.q_block, head_list=[0], block_list=blocks, kv_round=fo.round_bf16)
         t_attn += time.time() - t0
         o_full = o_full.copy(); o_full[act] = res["O"]
         cache = {key: (res["probs"][key] if key[1] in blocks else cache[key]) for key in cache}

@@ -267,8 +267,16 @@ def residual_update(x_new_rows, xhat_prev, active, bits, group):
 # Appendix D.2: attention replacement for a sparse loop, with literally cached
 # previous-loop probabilities.
 # --------------------------------------------------------------------------------------
+def round_bf16(x: np.ndarray) -> np.ndarray:
+    """Nearest bf16 (ties to even) of binary32 values, returned as binary32."""
+    x = np.ascontiguousarray(x, dtype=F32)
+    u = x.view(np.uint32).astype(np.uint64)
+    r = ((u + 0x7FFF + ((u >> 16) & 1)) >> 16) << 16
+    return r.astype(np.uint32).view(F32).reshape(x.shape)
+
+
 def sparse_loop_attention(q_new, khat_new, vhat_new, vhat_old, o_prev, active, col_sets, p_old_cache,
-                          sm_scale, q_block, head_list=None, block_list=None):
+                          sm_scale, q_block, head_list=None, block_list=None, kv_round=None):
     """One sparse loop of Appendix D.2 for every (head, block).
 
     q_new     : [n, H, dh] queries of the active rows (ascending positions `active`)
@@ -278,6 +286,11 @@ def sparse_loop_attention(q_new, khat_new, vhat_new, vhat_old, o_prev, active, c
     col_sets  : {(h,b): ascending column ids S[h,b]}
     p_old_cache : {(h,b): (rows, P)} with P[t, u] = p^(r-1) of query rows[t], column S[h,b][u]
                   (zero where the column is not causal); rows must contain the block's active rows.
+    kv_round  : optional rounding applied to the reconstructed K/V rows when attention consumes them.
+                The chain Xhat itself stays binary32 (the codec needs it exact); with bf16 storage the
+                reconstructed cache that attention reads is a BF16 KV cache (Appendix G: the engine runs on
+                BF16 activations and reads the packed streams "avoiding explicit reconstruction of a full BF16
+                KV cache"), so its rows are bf16 values: kv_round = round_bf16. None for binary32 storage.
     Returns dict: O [n,H,dh] fp64, mass {(h,b): m_i per active row}, probs {(h,b): (rows, P_new)},
                   col_scores {(h,b): sum over rows of P_new, per column of S},
                   lse [H, n] fp64: the one-number summary of each row's cached probabilities,
@@ -294,6 +307,7 @@ def sparse_loop_attention(q_new, khat_new, vhat_new, vhat_old, o_prev, active, c
     lse = np.full((H, n), np.nan, dtype=F64)
     heads = range(H) if head_list is None else head_list
     blk = active // q_block
+    rd = (lambda x: x) if kv_round is None else kv_round
     for h in heads:
         for b in (range(nb) if block_list is None else block_list):
             t_idx = np.nonzero(blk == b)[0]                      # slots of this block's active rows
@@ -311,14 +325,14 @@ def sparse_loop_attention(q_new, khat_new, vhat_new, vhat_old, o_prev, active, c
             causal = S[None, :] <= rows[:, None]                 # T_i membership
             P_old = np.where(causal, P_old, 0.0)
             m = P_old.sum(axis=1)                                # cached global mass, per query
-            logits = (q_new[t_idx, h, :].astype(F64) @ khat_new[S, h, :].astype(F64).T) * F64(sm_scale)
+            logits = (q_new[t_idx, h, :].astype(F64) @ rd(khat_new[S, h, :]).astype(F64).T) * F64(sm_scale)
             logits = np.where(causal, logits, -np.inf)
             has = causal.any(axis=1)
             mx = np.where(has, logits.max(axis=1, initial=-np.inf), 0.0)
             e = np.where(causal, np.exp(logits - mx[:, None]), 0.0)
             den = e.sum(axis=1)
             P_new = np.where(has[:, None], m[:, None] * e / np.where(den > 0, den, 1.0)[:, None], 0.0)
-            upd = (-P_old @ vhat_old[S, h, :].astype(F64)) + (P_new @ vhat_new[S, h, :].astype(F64))
+            upd = (-P_old @ rd(vhat_old[S, h, :]).astype(F64)) + (P_new @ rd(vhat_new[S, h, :]).astype(F64))
             O[t_idx, h, :] = O[t_idx, h, :] + np.where(has[:, None], upd, 0.0)
             mass[(h, b)] = m
             probs[(h, b)] = (rows, P_new)
@@ -383,7 +397,9 @@ class LayerOracle:
     Budgets: k_tokens[r-2], c_cols[r-2] for r = 2..R.
     """
 
-    def __init__(self, L, H, dh, q_block, bits, group, eps, sm_scale, head_list=None):
+    def __init__(self, L, H, dh, q_block, bits, group, eps, sm_scale, head_list=None, storage="f32"):
+        assert storage in ("f32", "bf16")
+        self.kv_round = round_bf16 if storage == "bf16" else None
         self.L, self.H, self.dh = L, H, dh
         self.q_block, self.bits, self.group = q_block, bits, group
         self.eps, self.sm_scale = eps, sm_scale
@@ -432,7 +448,7 @@ class LayerOracle:
             o_prev_rows = o_full[act]
             res = sparse_loop_attention(np.asarray(Q[r - 1])[act], khat_new, vhat_new, vhat, o_prev_rows,
                                         act, col_sets, cache, self.sm_scale, self.q_block,
-                                        head_list=self.head_list)
+                                        head_list=self.head_list, kv_round=self.kv_round)
             o_full = o_full.copy()
             o_full[act] = res["O"]
             rec = {"r": r, "active": act, "col_sets": dict(col_sets), "k_payload": k_pay, "v_payload": v_pay,

@@ -1,4 +1,5 @@
 // Context, status strings, shared host-side validation and the KV-cache accounting call.
+#include <cstdlib>
 #include <new>
 
 #include "fl_internal.cuh"
@@ -32,6 +33,8 @@ extern "C" int fl_create(fl_ctx** out, int device) {
     delete c;
     return FL_ERR_CUDA;
   }
+  const char* env = std::getenv("FL_FORCE_SIMT");
+  c->force_simt = (env != nullptr && env[0] == '1') ? 1 : 0;
   c->workspace_bytes = size_t(8) << 20;
   if (cudaMalloc(&c->workspace, c->workspace_bytes) != cudaSuccess) {
     delete c;

@@ -158,6 +158,8 @@ __global__ void __launch_bounds__(kAttnThreads) colscore_kernel(const __grid_con
     if (uu < n_cols) {
       const int j = SPARSE ? __ldg(cols + uu) : uu;
       recon8<T, BITS>(a.kside, a.n_use, j, h * DH + e, a.d, a.group, kv);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) kv[i] = to_float<T>(from_float<T>(kv[i]));  // storage precision, as in attention
     } else {
 #pragma unroll
       for (int i = 0; i < 8; ++i) kv[i] = 0.f;

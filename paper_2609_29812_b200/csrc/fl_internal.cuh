@@ -13,6 +13,7 @@ struct fl_ctx {
   int max_smem_optin;
   void* workspace;
   size_t workspace_bytes;
+  int force_simt;  // environment FL_FORCE_SIMT=1 at fl_create: keep attention on the binary32 SIMT kernels
 };
 
 #define FL_CHECK_CUDA(expr)                    \

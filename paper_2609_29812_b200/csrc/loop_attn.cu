@@ -7,6 +7,11 @@ int fl_launch_sparse_colscore(const fl_shape* s, const void* q_new, const int32_
                               const DevSide& kside, int n_use, const int32_t* col_idx, const int32_t* col_cnt, int c,
                               const float* lse, float* out, cudaStream_t st);
 
+int fl_launch_loop_attn_tc(const fl_ctx* ctx, const fl_shape* s, int loop_r, const void* q_new, const void* q_old,
+                           const int32_t* active_idx, int n_active, const fl_kv_store* store, const int32_t* col_idx,
+                           const int32_t* col_cnt, int c, const float* lse_prev, float* lse_out, const void* o_prev,
+                           void* o_out, int32_t* status, cudaStream_t st);
+
 namespace {
 
 struct LoopAttnArgs {
@@ -110,6 +115,9 @@ __global__ void __launch_bounds__(kAttnThreads) loop_attn_kernel(const __grid_co
 #pragma unroll
         for (int i = 0; i < 8; ++i) xo[i] = xn[i] = 0.f;
       }
+      // attention consumes the reconstructed rows in storage precision (a bf16 KV cache for bf16 storage)
+#pragma unroll
+      for (int i = 0; i < 8; ++i) { xo[i] = to_float<T>(from_float<T>(xo[i])); xn[i] = to_float<T>(from_float<T>(xn[i])); }
       if (is_v) {
 #pragma unroll
         for (int i = 0; i < 8; ++i) { v_old[u * DH + e + i] = xo[i]; v_new[u * DH + e + i] = xn[i]; }
@@ -220,6 +228,19 @@ extern "C" int fl_loop_attention(fl_ctx* ctx, const fl_shape* shape, int loop_r,
   FL_REQUIRE(q_new != nullptr && q_old != nullptr && o_prev != nullptr && o_out != nullptr && active_idx != nullptr);
   FL_REQUIRE(fl_aligned16(q_new) && fl_aligned16(q_old) && fl_aligned16(o_prev) && fl_aligned16(o_out));
 
+  DevSide kside;
+  fl_dev_side(store, true, &kside);
+  if (!ctx->force_simt) {
+    // tensor path (bf16 storage, head_dim 128); anything else runs on the binary32 SIMT kernel below
+    rc = fl_launch_loop_attn_tc(ctx, shape, loop_r, q_new, q_old, active_idx, n_active, store, col_idx, col_cnt, c,
+                                lse_prev, lse_out, o_prev, o_out, status, st);
+    if (rc == FL_OK) {
+      if (col_scores_next == nullptr) return FL_OK;
+      return fl_launch_sparse_colscore(shape, q_new, active_idx, n_active, kside, loop_r - 1, col_idx, col_cnt, c,
+                                       lse_out, col_scores_next, st);
+    }
+    if (rc != FL_ERR_UNSUPPORTED) return rc;
+  }
   LoopAttnArgs a{};
   a.q_new = q_new; a.q_old = q_old; a.o_prev = o_prev; a.o_out = o_out;
   a.active_idx = active_idx; a.n_active = n_active;

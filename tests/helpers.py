@@ -32,9 +32,11 @@ def attn_errors(got, ref):
     return rel, float(np.max(np.abs(got - ref))) if got.size else 0.0
 
 
-def assert_attn_close(got, ref, what=""):
+def assert_attn_close(got, ref, what="", loops=1):
+    """One loop: the stated tolerance.  `loops` chained loops: max-abs scales with the number of loops
+    (each adds a storage rounding of the carried output), relative L2 stays as stated."""
     rel, mx = attn_errors(got, ref)
-    assert rel <= REL_L2_TOL and mx <= MAX_ABS_TOL, f"{what}: rel L2 {rel:.3e}, max abs {mx:.3e}"
+    assert rel <= REL_L2_TOL and mx <= MAX_ABS_TOL * loops, f"{what}: rel L2 {rel:.3e}, max abs {mx:.3e}"
     return rel, mx
 
 

@@ -44,7 +44,8 @@ WORKLOADS = {
 def case(request):
     w = WORKLOADS[request.param]()
     x = workloads.make_layer_inputs(w, seed=3)
-    orc = fo.LayerOracle(w.L, w.n_heads, w.head_dim, w.q_block, w.bits, w.group, w.eps, w.sm_scale)
+    orc = fo.LayerOracle(w.L, w.n_heads, w.head_dim, w.q_block, w.bits, w.group, w.eps, w.sm_scale,
+                         storage=w.dtype)
     ref = orc.run(x.G, x.Q, x.K, x.V, [w.k_tokens] * (w.n_loops - 1), [w.col_budget] * (w.n_loops - 1))
     return w, x, ref
 
@@ -255,12 +256,40 @@ def test_chained_layer_all_on_gpu(env, case):
         o_rows, _ = st.sparse_loop(r, to_dev(x.Q[r - 1][act], w), to_dev(x.K[r - 1][act], w),
                                    to_dev(x.V[r - 1][act], w), sel)
         cand = sel.active_idx
+        # The GPU carries O between loops in storage precision (the oracle carries fp64), so every chained
+        # loop adds one storage rounding of O on top of that loop's own attention error: the max-abs bound
+        # grows linearly with the number of chained loops; the relative L2 bound is kept as stated.
         if np.array_equal(act, ref["active"][r - 2]):
-            assert_attn_close(to_np(o_rows), ref["loops"][r - 2]["O_rows"], f"chained loop {r}")
-    assert_attn_close(to_np(st.o_store), ref["loops"][-1]["O_full"], "chained final O store")
+            assert_attn_close(to_np(o_rows), ref["loops"][r - 2]["O_rows"], f"chained loop {r}", loops=r - 1)
+    assert_attn_close(to_np(st.o_store), ref["loops"][-1]["O_full"], "chained final O store", loops=w.n_loops - 1)
     # KV accounting of the real store
     fl, dense = B.fl_kv_store_bytes(sh, st.store, w.n_loops, 1)
     n_r = [len(a) for a in ref["active"]]
     fl_ref, dense_ref = fo.kv_bytes_per_token_layer(w.L, w.d, n_r, w.bits, w.group, 1,
                                                     elem_bytes=4 if w.dtype == "f32" else 2)
     assert dense == dense_ref * w.L and abs(fl - fl_ref * w.L) <= 4 * w.n_loops
+
+
+def test_binary32_simt_attention_path_on_bf16_storage(env):
+    """The SIMT attention kernels also serve bf16 storage (forced here; normally the tensor path runs)."""
+    import os
+    B, P, _ = env
+    w = small_bf16(L=900, H=2, R=3)
+    x = workloads.make_layer_inputs(w, seed=4)
+    ref = fo.LayerOracle(w.L, w.n_heads, w.head_dim, w.q_block, w.bits, w.group, w.eps, w.sm_scale,
+                         storage=w.dtype).run(x.G, x.Q, x.K, x.V, [w.k_tokens] * 2, [w.col_budget] * 2)
+    os.environ["FL_FORCE_SIMT"] = "1"
+    try:
+        ctx = B.Context(0)
+    finally:
+        del os.environ["FL_FORCE_SIMT"]
+    st = P.LayerState(ctx, w)
+    st.dense_loop(to_dev(x.Q[0], w), to_dev(x.K[0], w), to_dev(x.V[0], w))
+    st.select_columns_dense()
+    for r in (2, 3):
+        sel = oracle_selection(P, w, ref, r)
+        act = ref["active"][r - 2]
+        o_rows, _ = st.sparse_loop(r, to_dev(x.Q[r - 1][act], w), to_dev(x.K[r - 1][act], w),
+                                   to_dev(x.V[r - 1][act], w), sel)
+    assert_attn_close(to_np(st.o_store), ref["loops"][-1]["O_full"], "SIMT path final O store", loops=2)
+    ctx.close()

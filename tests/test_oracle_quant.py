@@ -148,3 +148,16 @@ def test_kv_accounting_against_the_papers_figures():
     w = workloads.config3()
     fl, dense = fo.kv_bytes_per_token_layer(w.L, w.d, [w.k_tokens] * 3, w.bits, w.group, w.n_layers)
     assert dense == 32768 and 8840 < fl < 8850 and dense / fl > 3.0
+
+
+def test_bf16_rounding_helper():
+    """round_bf16: exact on bf16 values, ties to even, nearest otherwise (checked against torch)."""
+    torch = pytest.importorskip("torch")
+    x = np.array([1.0, 1.00390625, 1.01171875, -3.14159, 1e-30, 65504.0, 0.1], dtype=np.float32)
+    # 1 + 2^-8 is a tie between 1 and 1 + 2^-7 -> even mantissa (1.0); 1 + 3*2^-8 ties up to 1 + 2^-6
+    got = fo.round_bf16(x)
+    assert got[0] == 1.0 and got[1] == 1.0 and got[2] == np.float32(1.015625)
+    ref = torch.from_numpy(x).to(torch.bfloat16).float().numpy()
+    assert np.array_equal(got, ref)
+    r = np.random.default_rng(0).standard_normal(10000).astype(np.float32) * 37
+    assert np.array_equal(fo.round_bf16(r), torch.from_numpy(r).to(torch.bfloat16).float().numpy())

@@ -11,7 +11,7 @@ import os
 from typing import Optional, Sequence
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_PKG, "libflashloop.so")
+LIB_PATH = os.environ.get("FLASHLOOP_LIB", os.path.join(_PKG, "libflashloop.so"))  # override: a custom build
 
 FL_OK = 0
 FL_ERR_INVALID_ARG = -1

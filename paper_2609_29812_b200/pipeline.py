@@ -71,6 +71,7 @@ class LayerState:
         self.col_scores = None
         self.lse = None
         self.store = None
+        self.status = torch.zeros(1, dtype=torch.int32, device=self.dev)   # asynchronous device-side errors
 
     # ---- loop 1 -------------------------------------------------------------------------------
     def dense_loop(self, q, k, v, want_col_scores=True):
@@ -141,7 +142,13 @@ class LayerState:
     def attention(self, loop_r, q_new, q_old, o_prev, o_out, sel: TokenSelection, col_scores_next=None):
         B.fl_loop_attention(self.ctx, self.shape, loop_r, q_new, q_old, sel.active_idx, sel.n, self.store,
                             self.col_idx, self.col_cnt, self.c, self.lse, self.lse, o_prev, o_out,
-                            col_scores_next)   # lse updated in place: only the active rows change
+                            col_scores_next, status=self.status)   # lse updated in place (active rows only)
+
+    def check_status(self):
+        """Synchronises and raises if a kernel reported an asynchronous error (e.g. a bounded wait ran out)."""
+        code = int(self.status.item())
+        if code != 0:
+            raise B.FlashLoopError("device status", code)
 
     def sparse_loop(self, loop_r, q_new, k_new, v_new, sel: TokenSelection, want_col_scores_next=False):
         """One loop r >= 2 for this layer: store residuals, gather the carried rows, attend, scatter back.

@@ -228,6 +228,7 @@ def test_loop_attention_stage_isolated(env, case):
         o_out = torch.empty_like(o_prev)
         csn = torch.zeros(w.n_heads, st.nb, st.c, dtype=torch.float32, device="cuda")
         st.attention(r, to_dev(x.Q[r - 1][act], w), to_dev(q_prev_full[act], w), o_prev, o_out, sel, csn)
+        st.check_status()
         assert_attn_close(to_np(o_out), rec["O_rows"], f"loop {r} O rows")
         # log-normaliser of the active rows and next-loop column scores
         got_lse = to_np(st.lse)[:, act]
@@ -256,6 +257,7 @@ def test_chained_layer_all_on_gpu(env, case):
         o_rows, _ = st.sparse_loop(r, to_dev(x.Q[r - 1][act], w), to_dev(x.K[r - 1][act], w),
                                    to_dev(x.V[r - 1][act], w), sel)
         cand = sel.active_idx
+        st.check_status()
         # The GPU carries O between loops in storage precision (the oracle carries fp64), so every chained
         # loop adds one storage rounding of O on top of that loop's own attention error: the max-abs bound
         # grows linearly with the number of chained loops; the relative L2 bound is kept as stated.
@@ -293,3 +295,35 @@ def test_binary32_simt_attention_path_on_bf16_storage(env):
                                    to_dev(x.V[r - 1][act], w), sel)
     assert_attn_close(to_np(st.o_store), ref["loops"][-1]["O_full"], "SIMT path final O store", loops=2)
     ctx.close()
+
+
+def test_many_patched_columns_and_wide_budgets(env):
+    """Half of the rows active and a column budget of several chunks: long runs of columns that carry
+    residual payloads (two ring slots per chunk) and several 128-row tiles per query block."""
+    B, P, ctx = env
+    w = dataclasses.replace(small_bf16(L=1536, H=2, R=3, c=640, q_block=512), token_frac=0.5,
+                            changed_fracs=(0.6, 0.5))
+    x = workloads.make_layer_inputs(w, seed=7)
+    ref = fo.LayerOracle(w.L, w.n_heads, w.head_dim, w.q_block, w.bits, w.group, w.eps, w.sm_scale,
+                         storage=w.dtype).run(x.G, x.Q, x.K, x.V, [w.k_tokens] * 2, [w.col_budget] * 2)
+    st = P.LayerState(ctx, w)
+    st.dense_loop(to_dev(x.Q[0], w), to_dev(x.K[0], w), to_dev(x.V[0], w))
+    lse = ref["dense"]["lse"].astype(np.float32).copy()
+    q_prev_full = x.Q[0]
+    for r in (2, 3):
+        rec = ref["loops"][r - 2]
+        act = rec["active"]
+        sel = oracle_selection(P, w, ref, r)
+        st.alloc_stream(sel)
+        st.quantize(r, to_dev(x.K[r - 1][act], w), to_dev(x.V[r - 1][act], w), sel)
+        idx, cnt = sets_to_arrays(w, st.nb, rec["col_sets"], w.col_budget)
+        st.col_idx, st.col_cnt, st.c = torch.from_numpy(idx).cuda(), torch.from_numpy(cnt).cuda(), w.col_budget
+        st.lse = torch.from_numpy(lse).cuda()
+        o_prev = to_dev(storage_round(rec["O_prev_rows"], w), w)
+        o_out = torch.empty_like(o_prev)
+        st.attention(r, to_dev(x.Q[r - 1][act], w), to_dev(q_prev_full[act], w), o_prev, o_out, sel)
+        st.check_status()
+        assert_attn_close(to_np(o_out), rec["O_rows"], f"loop {r} O rows (many patched columns)")
+        ok = np.isfinite(rec["lse_rows"])
+        lse = lse.copy(); lse[:, act] = np.where(ok, rec["lse_rows"], lse[:, act]).astype(np.float32)
+        q_prev_full = q_prev_full.copy(); q_prev_full[act] = x.Q[r - 1][act]

@@ -1,8 +1,42 @@
 // Context, status strings, shared host-side validation and the KV-cache accounting call.
 #include <cstdlib>
+#include <cstring>
 #include <new>
+#include <vector>
 
 #include "fl_internal.cuh"
+
+struct fl_tmap_cache {
+  struct Entry { const void* base; int64_t rows, row_elems; CUtensorMap map; };
+  std::vector<Entry> entries;
+  size_t next = 0;
+};
+
+typedef CUresult (*fl_encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                       const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                       CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+bool fl_row_gather_tmap(fl_ctx* ctx, const void* base, int64_t rows, int64_t row_elems, CUtensorMap* out) {
+  if (ctx->encode_tiled == nullptr || ctx->tmaps == nullptr) return false;
+  for (const auto& e : ctx->tmaps->entries)
+    if (e.base == base && e.rows == rows && e.row_elems == row_elems) { *out = e.map; return true; }
+  fl_tmap_cache::Entry e;
+  e.base = base; e.rows = rows; e.row_elems = row_elems;
+  const cuuint64_t gdim[2] = {(cuuint64_t)row_elems, (cuuint64_t)rows};
+  const cuuint64_t gstride[1] = {(cuuint64_t)row_elems * 2};
+  const cuuint32_t box[2] = {64, 1};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult rc = reinterpret_cast<fl_encode_tiled_fn>(ctx->encode_tiled)(
+      &e.map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstride, box, estr,
+      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (rc != CUDA_SUCCESS) return false;
+  constexpr size_t kMaxEntries = 512;   // ring replacement: 48 layers x (K, V) fit several times over
+  if (ctx->tmaps->entries.size() < kMaxEntries) ctx->tmaps->entries.push_back(e);
+  else { ctx->tmaps->entries[ctx->tmaps->next] = e; ctx->tmaps->next = (ctx->tmaps->next + 1) % kMaxEntries; }
+  *out = e.map;
+  return true;
+}
 
 extern "C" int fl_version(void) { return 100; }
 
@@ -35,8 +69,19 @@ extern "C" int fl_create(fl_ctx** out, int device) {
   }
   const char* env = std::getenv("FL_FORCE_SIMT");
   c->force_simt = (env != nullptr && env[0] == '1') ? 1 : 0;
+  c->encode_tiled = nullptr;
+  {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      c->encode_tiled = fn;
+    (void)cudaGetLastError();
+  }
+  c->tmaps = new (std::nothrow) fl_tmap_cache();
   c->workspace_bytes = size_t(8) << 20;
   if (cudaMalloc(&c->workspace, c->workspace_bytes) != cudaSuccess) {
+    delete c->tmaps;
     delete c;
     return FL_ERR_CUDA;
   }
@@ -47,6 +92,7 @@ extern "C" int fl_create(fl_ctx** out, int device) {
 extern "C" int fl_destroy(fl_ctx* ctx) {
   if (ctx == nullptr) return FL_ERR_INVALID_ARG;
   cudaError_t e = cudaFree(ctx->workspace);
+  delete ctx->tmaps;
   delete ctx;
   return e == cudaSuccess ? FL_OK : FL_ERR_CUDA;
 }

@@ -1,5 +1,6 @@
 // Internal declarations shared by the kernels of libflashloop (never installed).
 #pragma once
+#include <cuda.h>   // CUtensorMap and the tensor-map enums only; the driver is reached through the runtime
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
@@ -14,7 +15,14 @@ struct fl_ctx {
   void* workspace;
   size_t workspace_bytes;
   int force_simt;  // environment FL_FORCE_SIMT=1 at fl_create: keep attention on the binary32 SIMT kernels
+  void* encode_tiled;       // cuTensorMapEncodeTiled, resolved through cudaGetDriverEntryPoint (may be null)
+  struct fl_tmap_cache* tmaps;  // row-gather tensor maps, keyed by (base pointer, rows, row elements)
 };
+
+// Tensor map for gathering rows of a row-major bf16 matrix [rows, row_elems] with TMA (tile::gather4):
+// box = 64 elements x 1 row, 128-byte swizzle, out-of-range rows read as zero. Cached per context.
+// Returns false if tensor maps are not available (caller falls back to a non-TMA kernel).
+bool fl_row_gather_tmap(fl_ctx* ctx, const void* base, int64_t rows, int64_t row_elems, CUtensorMap* out);
 
 #define FL_CHECK_CUDA(expr)                    \
   do {                                         \

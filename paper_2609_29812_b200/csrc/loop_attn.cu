@@ -7,7 +7,7 @@ int fl_launch_sparse_colscore(const fl_shape* s, const void* q_new, const int32_
                               const DevSide& kside, int n_use, const int32_t* col_idx, const int32_t* col_cnt, int c,
                               const float* lse, float* out, cudaStream_t st);
 
-int fl_launch_loop_attn_tc(const fl_ctx* ctx, const fl_shape* s, int loop_r, const void* q_new, const void* q_old,
+int fl_launch_loop_attn_tc(fl_ctx* ctx, const fl_shape* s, int loop_r, const void* q_new, const void* q_old,
                            const int32_t* active_idx, int n_active, const fl_kv_store* store, const int32_t* col_idx,
                            const int32_t* col_cnt, int c, const float* lse_prev, float* lse_out, const void* o_prev,
                            void* o_out, int32_t* status, cudaStream_t st);

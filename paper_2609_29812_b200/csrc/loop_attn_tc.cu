@@ -6,7 +6,10 @@
 //   warps 0-3   softmax of the OLD term  (fixed normaliser lse_prev: p_old = exp(s_old - lse_prev), mass m_i)
 //   warps 4-7   softmax of the NEW term  (running reference with lazy rescale of the accumulator)
 //   warp  8     one elected thread issues every tcgen05.mma; the warp owns the tensor-memory allocation
-//   warps 9-15  producers: gather selected columns, dequantize-and-add, write 128B-swizzled operand tiles
+//   warp  9     TMA: row gathers (cp.async.bulk.tensor tile::gather4, 4 selected columns per copy) of the bf16
+//               base K/V rows straight into 128B-swizzled operand tiles; completion on mbarriers
+//   warps 10-15 patch: stage the Q tiles; for the columns that carry residual payloads, overwrite the gathered
+//               base rows with the dequantize-and-add result (Eq. 8)
 //
 // Prologue (whole CTA): the block's causal column list is copied to shared memory together with a bit mask
 // of the residual streams that carry each column, and stably partitioned into columns WITHOUT a payload in
@@ -34,10 +37,11 @@ constexpr int kSlotBytes = 2 * kTileBytes;  // K tile | V tile
 constexpr int kQTileBytes = kM * kDH * 2;   // 32 KB
 constexpr int kSoftmaxWarps = 8;
 constexpr int kMmaWarp = 8;
-constexpr int kProducerWarps = 7;
-constexpr int kWarps = kSoftmaxWarps + 1 + kProducerWarps;  // 16
+constexpr int kTmaWarp = 9;
+constexpr int kPatchWarps = 6;
+constexpr int kWarps = kSoftmaxWarps + 2 + kPatchWarps;  // 16
 constexpr int kThreads = kWarps * 32;
-constexpr int kProducerThreads = kProducerWarps * 32;
+constexpr int kPatchThreads = kPatchWarps * 32;
 constexpr int kMaxCols = 3072;              // column budget the shared-memory column list can hold
 constexpr uint32_t kAccOld = 0, kAccNew = 128, kSBase = 256;
 constexpr float kLog2e = 1.4426950408889634f;
@@ -56,7 +60,8 @@ constexpr float kRescaleThreshold = 60.f;   // in log2 units: rescale only when 
 #define TC_TRACE(role, chunk, ev) do { } while (0)
 #endif
 
-struct TcArgs {
+struct alignas(64) TcArgs {
+  CUtensorMap k_map, v_map;   // row-gather maps of the K / V base ([L, d] bf16, box 64 x 1, 128B swizzle)
   const __nv_bfloat16* q_new;
   const __nv_bfloat16* q_old;
   const __nv_bfloat16* o_prev;
@@ -76,8 +81,10 @@ struct TcArgs {
 };
 
 struct __align__(16) TcSmemCtl {
-  uint64_t full[kSlots];   // producers -> MMA: the slot's operand tiles are written
-  uint64_t done[kSlots];   // MMA -> producers / softmax: the MMAs that read the slot have finished
+  uint64_t landed[kSlots];   // TMA -> everyone: the slot's gathered tiles (32 KB) have arrived
+  uint64_t patched[kSlots];  // patch warps -> MMA: residual-carrying columns of the slot are rewritten (dirty chunks only)
+  uint64_t done[kSlots];     // MMA -> TMA / softmax: the MMAs that read the slot have finished
+  uint64_t q_full;           // patch warps -> MMA: the Q tiles of the current row tile are staged
   uint64_t s_full[2];      // MMA -> softmax: S of the chunk is in tensor memory
   uint64_t p_full[2];      // softmax -> MMA: P of the chunk is in tensor memory
   uint64_t acc_done;       // MMA -> softmax: all accumulation of the tile finished
@@ -88,6 +95,7 @@ struct __align__(16) TcSmemCtl {
   int warp_cnt[kWarps][2];
   int col_pos[kSlots][kNC];
   int col_last[kSlots];    // largest column position of the chunk, INT32_MAX if the chunk is padded
+  uint32_t chunk_mask[kMaxCols / kNC + 2];  // OR of the stream masks of the chunk's columns (0: plain gather only)
   float mass[kM];
   float ell[kM];
   float ref[kM];
@@ -202,9 +210,11 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
 
   if (tid == 0) {
     for (int s = 0; s < kSlots; ++s) {
-      tc::mbar_init(&ctl.full[s], kProducerThreads);
+      tc::mbar_init(&ctl.landed[s], 1);
+      tc::mbar_init(&ctl.patched[s], kPatchWarps);
       tc::mbar_init(&ctl.done[s], 1);
     }
+    tc::mbar_init(&ctl.q_full, kPatchThreads);
     for (int s = 0; s < 2; ++s) {
       tc::mbar_init(&ctl.s_full[s], 1);
       tc::mbar_init(&ctl.p_full[s], kSoftmaxWarps * 32);
@@ -253,6 +263,9 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
       tot0 += c0; tot1 += c1;
     }
     if (tid == 0) { ctl.n_plain = tot0; ctl.n_patch = tot1; }
+    for (int i = tid; i < kMaxCols / kNC + 2; i += kThreads) ctl.chunk_mask[i] = 0;
+    __syncthreads();
+    const int plain_chunks = (tot0 + kNC - 1) / kNC;
     for (int base = beg; base < end; base += 32) {
       const int u = base + lane;
       const int j = u < end ? __ldg(cols + u) : INT32_MAX;
@@ -268,6 +281,7 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
         const int dst = patched ? tot0 + before1 + __popc(m1 & lt) : before0 + __popc(m0 & lt);
         ord_col[dst] = j;
         ord_mask[dst] = mask;
+        if (mask != 0) atomicOr(&ctl.chunk_mask[patched ? plain_chunks + (dst - tot0) / kNC : dst / kNC], mask);
       }
       before0 += __popc(m0);
       before1 += __popc(m1);
@@ -278,17 +292,60 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
   const int n_chunks = (n_plain + kNC - 1) / kNC + (n_patch + kNC - 1) / kNC;
   int g = 0;    // chunks issued so far (all tiles): S/P buffer = g & 1, phase = (g >> 1) & 1
   int fill = 0; // ring slots filled so far: slot = fill % kSlots, phase = (fill / kSlots) & 1
+  uint32_t dirty_par_cta = 0;  // per-slot phase parity of the patched[] barriers (they only see dirty chunks)
 
   for (int s0 = q_lo, tile = 0; s0 < q_hi; s0 += kM, ++tile) {
   const int n_rows = min(kM, q_hi - s0);
   const int g0 = g, fill0 = fill;
+  const uint32_t dirty_par0 = dirty_par_cta;
 
-  if (warp > kMmaWarp) {
-    // =========================================== producers ===========================================
-    const int pt = tid - (kMmaWarp + 1) * 32;
+  if (warp == kTmaWarp) {
+    // ============================================== TMA ==============================================
+    // In-order fills of the ring; the lookahead is whatever the four slots allow. Each lane issues two of
+    // the 64 four-row gathers of a slot (K: 2 slabs x 16 groups, V: the same).
+    int f = fill0;
+    bool ok = true;
+#pragma unroll 1
+    for (int ci = 0; ci < n_chunks && ok; ++ci) {
+      const ChunkInfo ck = chunk_info(ci, n_plain, n_patch);
+      const int n_slots = ck.patch ? 2 : 1;
+      for (int k = 0; k < n_slots && ok; ++k)
+        if (f + k >= kSlots) ok = warp_wait(&ctl.done[(f + k) % kSlots], (((f + k) / kSlots) - 1) & 1, abort_flag);
+      if (!ok) break;
+      const int slot0 = f % kSlots;
+      if (lane == 0) TC_TRACE(0, ci, 0);
+      for (int u = lane; u < kNC; u += 32) ctl.col_pos[slot0][u] = u < ck.n_valid ? ord_col[ck.off + u] : INT32_MAX;
+      if (lane == 0) ctl.col_last[slot0] = ck.n_valid == kNC ? ord_col[ck.off + kNC - 1] : INT32_MAX;
+      __syncwarp();
+      if (lane == 0)
+        for (int k = 0; k < n_slots; ++k) tc::mbar_arrive_expect_tx(&ctl.landed[(f + k) % kSlots], kSlotBytes);
+      __syncwarp();
+#pragma unroll
+      for (int rep = 0; rep < 2; ++rep) {
+        const int gidx = lane + rep * 32;                  // 0..63
+        const int is_v = gidx >> 5, slab = (gidx >> 4) & 1, grp = gidx & 15;
+        int y[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int u = grp * 4 + i;
+          y[i] = u < ck.n_valid ? ord_col[ck.off + u] : a.L;   // row L is outside the tensor: reads as zero
+        }
+        const void* map = is_v ? static_cast<const void*>(&a.v_map) : static_cast<const void*>(&a.k_map);
+        for (int k = 0; k < n_slots; ++k) {
+          const int slot = (f + k) % kSlots;
+          tc::tma_gather4(ring + slot * kSlotBytes + is_v * kTileBytes + slab * (kNC * 128) + grp * 512, map,
+                          &ctl.landed[slot], h * kDH + slab * 64, y[0], y[1], y[2], y[3]);
+        }
+      }
+      f += n_slots;
+      if (lane == 0) TC_TRACE(0, ci, 1);
+    }
+  } else if (warp > kTmaWarp) {
+    // ============================================= patch =============================================
+    const int pt = tid - (kTmaWarp + 1) * 32;   // 0..191
     const int pw = pt >> 5;
-    // Q tiles (once per tile): asynchronous copies, part of the first commit group
-    for (int it = pt; it < 2 * kM * 16; it += kProducerThreads) {
+    // Q tiles (once per row tile): asynchronous 16-byte copies
+    for (int it = pt; it < 2 * kM * 16; it += kPatchThreads) {
       const int which = it / (kM * 16);
       const int rem = it % (kM * 16);
       const int r = rem >> 4, ch = rem & 15;
@@ -298,80 +355,33 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
       else
         *reinterpret_cast<uint4*>(dst) = make_uint4(0, 0, 0, 0);
     }
-    const int half = lane >> 4;          // 0: K row, 1: V row
-    const int ch = lane & 15;            // 16-byte chunk inside the 256-byte row
+    tc::cp_async_commit();
+    tc::cp_async_wait<0>();
+    tc::fence_proxy_async_smem();
+    tc::mbar_arrive(&ctl.q_full);
+    // dirty chunks: lanes 0-15 own the K row, lanes 16-31 the V row of one column at a time
+    const int half = lane >> 4, ch = lane & 15;
     const DevSide& side = half ? a.v : a.k;
     const int elem = h * kDH + ch * 8;
     const __nv_bfloat16* base_rows = static_cast<const __nv_bfloat16*>(side.base) + elem;
     const uint32_t ch_off = (ch >> 3) * (kNC * 128);
-    // Software pipeline over chunks, kAhead chunks of asynchronous gathers in flight per thread:
-    //   issue(ci)   : wait until the chunk's ring slot(s) are free, start the 16-byte copies of the base rows
-    //                 (warp pw owns columns pw, pw + 7, ...; lanes 0-15 the K row, lanes 16-31 the V row)
-    //   finish(ci)  : wait for those copies, overwrite the columns that carry residual payloads with their
-    //                 dequantize-and-add result, publish the column positions, hand the slot(s) to the MMA warp
-    // At most kAhead chunks are in flight, and never more slots than the ring has (a chunk that still waits to
-    // be finished must not hold a slot the next issue needs).
-    constexpr int kAhead = 2;
-    int f_issue = fill0, f_fin = fill0;
-    int ci_issue = 0, ci_fin = 0;
+    int f = fill0;
+    uint32_t dirty_par = dirty_par0;     // bit s: parity of the dirty fills slot s has seen
     bool ok = true;
 #pragma unroll 1
-    while (ci_fin < n_chunks && ok) {
-      bool can_issue = ci_issue < n_chunks && ci_issue - ci_fin < kAhead;
-      if (can_issue) {
-        // A slot is released by PV(y) of the chunk y that held it, and the MMA warp issues PV(y) only after
-        // QK(y+1), i.e. after chunk y+1 has been handed over: chunk y+1 must be finished before we wait.
-        const ChunkInfo nk = chunk_info(ci_issue, n_plain, n_patch);
-        const int n_plain_chunks = (n_plain + kNC - 1) / kNC;
-        auto holder = [&](int fill_no) {   // chunk (of this tile) that filled the same slot one lap earlier
-          const int rel = fill_no - kSlots - fill0;
-          if (rel < 0) return -1;
-          return rel < n_plain_chunks ? rel : n_plain_chunks + (rel - n_plain_chunks) / 2;
-        };
-        int hmax = holder(f_issue);
-        if (nk.patch) hmax = max(hmax, holder(f_issue + 1));
-        can_issue = f_issue + (nk.patch ? 2 : 1) - f_fin <= kSlots && (hmax < 0 || ci_fin >= hmax + 2);
-      }
-      if (can_issue) {
-        const int ci = ci_issue;
-        const ChunkInfo ck = chunk_info(ci, n_plain, n_patch);
-        const int slot0 = f_issue % kSlots, slot1 = (f_issue + 1) % kSlots;
-        if (pt == 0) TC_TRACE(0, ci, 0);
-        if (f_issue >= kSlots) ok = warp_wait(&ctl.done[slot0], ((f_issue / kSlots) - 1) & 1, abort_flag);
-        if (ok && ck.patch && f_issue + 1 >= kSlots)
-          ok = warp_wait(&ctl.done[slot1], (((f_issue + 1) / kSlots) - 1) & 1, abort_flag);
-        if (!ok) break;
-        if (pt == 0) TC_TRACE(0, ci, 1);
-        uint8_t* t_old = ring + slot0 * kSlotBytes + half * kTileBytes + ch_off;
-        uint8_t* t_new = ring + slot1 * kSlotBytes + half * kTileBytes + ch_off;
-#pragma unroll 2
-        for (int u = pw; u < kNC; u += kProducerWarps) {
-          const uint32_t off = tc::sw128_offset(u, ch & 7);
-          if (u < ck.n_valid) {
-            const __nv_bfloat16* src = base_rows + (size_t)ord_col[ck.off + u] * a.d;
-            tc::cp_async16(t_old + off, src);
-            if (ck.patch) tc::cp_async16(t_new + off, src);
-          } else {
-            *reinterpret_cast<uint4*>(t_old + off) = make_uint4(0, 0, 0, 0);
-            if (ck.patch) *reinterpret_cast<uint4*>(t_new + off) = make_uint4(0, 0, 0, 0);
-          }
-        }
-        tc::cp_async_commit();
-        f_issue += ck.patch ? 2 : 1;
-        ++ci_issue;
-      } else {
-        const int cf = ci_fin;
-        // groups complete in order: all but the (ci_issue - cf - 1) newer ones must have landed
-        if (ci_issue - cf - 1 >= 1) tc::cp_async_wait<1>(); else tc::cp_async_wait<0>();
-        const ChunkInfo ck = chunk_info(cf, n_plain, n_patch);
-        const int slot0 = f_fin % kSlots, slot1 = (f_fin + 1) % kSlots;
-        uint8_t* t_old = ring + slot0 * kSlotBytes + half * kTileBytes + ch_off;
-        uint8_t* t_new = ring + slot1 * kSlotBytes + half * kTileBytes + ch_off;
-        for (int u = pt; u < kNC; u += kProducerThreads)
-          ctl.col_pos[slot0][u] = u < ck.n_valid ? ord_col[ck.off + u] : INT32_MAX;
-        if (pt == 0) ctl.col_last[slot0] = ck.n_valid == kNC ? ord_col[ck.off + kNC - 1] : INT32_MAX;
+    for (int ci = 0; ci < n_chunks && ok; ++ci) {
+      const ChunkInfo ck = chunk_info(ci, n_plain, n_patch);
+      const int n_slots = ck.patch ? 2 : 1;
+      // Every fill is waited for, clean chunks included: a parity wait is only meaningful for the phase in
+      // progress, so a waiter must never skip a phase of a barrier it will wait on again.
+      for (int k = 0; k < n_slots && ok; ++k)
+        ok = warp_wait(&ctl.landed[(f + k) % kSlots], ((f + k) / kSlots) & 1, abort_flag);
+      if (!ok) break;
+      if (ctl.chunk_mask[ci] != 0) {
+        uint8_t* t_old = ring + (f % kSlots) * kSlotBytes + half * kTileBytes + ch_off;
+        uint8_t* t_new = ring + ((f + 1) % kSlots) * kSlotBytes + half * kTileBytes + ch_off;
 #pragma unroll 1
-        for (int u = pw; u < ck.n_valid; u += kProducerWarps) {
+        for (int u = pw; u < ck.n_valid; u += kPatchWarps) {
           const uint32_t mask = ord_mask[ck.off + u];
           if (mask == 0) continue;
           const int j = ord_col[ck.off + u];
@@ -379,19 +389,17 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
           uint4 v_old, v_new;
           patch_piece<BITS>(side, a.n_old, mask, j, elem, a.d, a.group, base16, v_old, v_new);
           const uint32_t off = tc::sw128_offset(u, ch & 7);
-          *reinterpret_cast<uint4*>(t_old + off) = v_old;
+          if (mask & ((1u << a.n_old) - 1u)) *reinterpret_cast<uint4*>(t_old + off) = v_old;
           if (ck.patch) *reinterpret_cast<uint4*>(t_new + off) = v_new;
         }
-        if (pt == 0) TC_TRACE(0, cf, 2);
         tc::fence_proxy_async_smem();
-        tc::mbar_arrive(&ctl.full[slot0]);
-        if (ck.patch) tc::mbar_arrive(&ctl.full[slot1]);
-        f_fin += ck.patch ? 2 : 1;
-        ++ci_fin;
-        if (pt == 0) TC_TRACE(0, cf, 3);
+        __syncwarp();
+        if (lane == 0)
+          for (int k = 0; k < n_slots; ++k) tc::mbar_arrive(&ctl.patched[(f + k) % kSlots]);
+        for (int k = 0; k < n_slots; ++k) dirty_par ^= 1u << ((f + k) % kSlots);
       }
+      f += n_slots;
     }
-    tc::cp_async_wait<0>();
   } else if (warp == kMmaWarp) {
     // =========================================== MMA issuer ==========================================
     if (lane == 0) {
@@ -404,9 +412,14 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
       const uint64_t q_new_desc = tc::make_desc_sw128(tc::smem_u32(q_new_tile), 16, 1024);
       const uint64_t k_desc0 = tc::make_desc_sw128(tc::smem_u32(ring), 16, 1024);
       const uint64_t v_desc0 = tc::make_desc_sw128(tc::smem_u32(ring) + kTileBytes, kNC * 128, 1024);
+      // low words move (start address, no carry into the other fields: shared memory is < 256 KB), high words stay
+      const uint32_t kq_hi = (uint32_t)(k_desc0 >> 32), v_hi = (uint32_t)(v_desc0 >> 32);
+      const uint32_t q_old_lo = (uint32_t)q_old_desc, q_new_lo = (uint32_t)q_new_desc;
+      const uint32_t k_lo0 = (uint32_t)k_desc0, v_lo0 = (uint32_t)v_desc0;
       bool ok = true;
       int f = fill0;        // slot counter of the chunk whose QK is issued next
       int f_pv = fill0;     // slot counter of the chunk whose PV is issued next
+      uint32_t dirty_par = dirty_par0;
       // iteration ci issues QK(ci) and then PV(ci-1): the softmax of chunk ci-1 overlaps QK(ci)
 #pragma unroll 1
       for (int ci = 0; ci <= n_chunks && ok; ++ci) {
@@ -414,22 +427,36 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
           const ChunkInfo ck = chunk_info(ci, n_plain, n_patch);
           const int slot0 = f % kSlots, slot1 = (f + 1) % kSlots;
           TC_TRACE(1, ci, 0);
-          if (!tc::mbar_wait(&ctl.full[slot0], (f / kSlots) & 1, abort_flag)) { ok = false; break; }
-          if (ck.patch && !tc::mbar_wait(&ctl.full[slot1], ((f + 1) / kSlots) & 1, abort_flag)) { ok = false; break; }
+          if (ci == 0 && !tc::mbar_wait(&ctl.q_full, tile & 1, abort_flag)) { ok = false; break; }
+          if (!tc::mbar_wait(&ctl.landed[slot0], (f / kSlots) & 1, abort_flag)) { ok = false; break; }
+          if (ck.patch && !tc::mbar_wait(&ctl.landed[slot1], ((f + 1) / kSlots) & 1, abort_flag)) { ok = false; break; }
+          if (ctl.chunk_mask[ci] != 0) {       // residual-carrying columns are rewritten by the patch warps
+            if (!tc::mbar_wait(&ctl.patched[slot0], (dirty_par >> slot0) & 1, abort_flag)) { ok = false; break; }
+            dirty_par ^= 1u << slot0;
+            if (ck.patch) {
+              if (!tc::mbar_wait(&ctl.patched[slot1], (dirty_par >> slot1) & 1, abort_flag)) { ok = false; break; }
+              dirty_par ^= 1u << slot1;
+            }
+          }
           tc::tc_fence_after();
           TC_TRACE(1, ci, 1);
-          const uint64_t k_old = k_desc0 + (uint64_t)(slot0 * (kSlotBytes >> 4));
-          const uint64_t k_new = ck.patch ? k_desc0 + (uint64_t)(slot1 * (kSlotBytes >> 4)) : k_old;
+          const uint32_t k_old = k_lo0 + slot0 * (kSlotBytes >> 4);
+          const uint32_t k_new = ck.patch ? k_lo0 + slot1 * (kSlotBytes >> 4) : k_old;
           const int sbuf = (g0 + ci) & 1;
           const uint32_t s_old = tmem + kSBase + sbuf * 128, s_new = s_old + 64;
-#pragma unroll
-          for (int kk = 0; kk < kDH / 16; ++kk)
-            tc::mma_ss(s_old, q_old_desc + (uint64_t)(((kk >> 2) * (kM * 128) + (kk & 3) * 32) >> 4),
-                       k_old + (uint64_t)(((kk >> 2) * (kNC * 128) + (kk & 3) * 32) >> 4), idesc_qk, kk > 0);
-#pragma unroll
-          for (int kk = 0; kk < kDH / 16; ++kk)
-            tc::mma_ss(s_new, q_new_desc + (uint64_t)(((kk >> 2) * (kM * 128) + (kk & 3) * 32) >> 4),
-                       k_new + (uint64_t)(((kk >> 2) * (kNC * 128) + (kk & 3) * 32) >> 4), idesc_qk, kk > 0);
+          // K step kk: 32 bytes inside a 64-element slab, then the next slab (Q: 128 rows, Khat: 64 rows per slab)
+#define FL_QK(D, QLO, KLO, KK, ACC)                                                                          \
+  tc::mma_ss_lo<ACC>(D, (QLO) + ((((KK) >> 2) * (kM * 128) + ((KK)&3) * 32) >> 4), kq_hi,                    \
+                     (KLO) + ((((KK) >> 2) * (kNC * 128) + ((KK)&3) * 32) >> 4), kq_hi, idesc_qk)
+          FL_QK(s_old, q_old_lo, k_old, 0, false); FL_QK(s_old, q_old_lo, k_old, 1, true);
+          FL_QK(s_old, q_old_lo, k_old, 2, true);  FL_QK(s_old, q_old_lo, k_old, 3, true);
+          FL_QK(s_old, q_old_lo, k_old, 4, true);  FL_QK(s_old, q_old_lo, k_old, 5, true);
+          FL_QK(s_old, q_old_lo, k_old, 6, true);  FL_QK(s_old, q_old_lo, k_old, 7, true);
+          FL_QK(s_new, q_new_lo, k_new, 0, false); FL_QK(s_new, q_new_lo, k_new, 1, true);
+          FL_QK(s_new, q_new_lo, k_new, 2, true);  FL_QK(s_new, q_new_lo, k_new, 3, true);
+          FL_QK(s_new, q_new_lo, k_new, 4, true);  FL_QK(s_new, q_new_lo, k_new, 5, true);
+          FL_QK(s_new, q_new_lo, k_new, 6, true);  FL_QK(s_new, q_new_lo, k_new, 7, true);
+#undef FL_QK
           tc::mma_commit(&ctl.s_full[sbuf]);
           f += ck.patch ? 2 : 1;
           TC_TRACE(1, ci, 2);
@@ -441,15 +468,16 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
           if (!tc::mbar_wait(&ctl.p_full[sbuf], ((g0 + cj) >> 1) & 1, abort_flag)) { ok = false; break; }
           tc::tc_fence_after();
           const int slot0 = f_pv % kSlots, slot1 = (f_pv + 1) % kSlots;
-          const uint64_t v_old = v_desc0 + (uint64_t)(slot0 * (kSlotBytes >> 4));
-          const uint64_t v_new = ck.patch ? v_desc0 + (uint64_t)(slot1 * (kSlotBytes >> 4)) : v_old;
+          const uint32_t v_old = v_lo0 + slot0 * (kSlotBytes >> 4);
+          const uint32_t v_new = ck.patch ? v_lo0 + slot1 * (kSlotBytes >> 4) : v_old;
           const uint32_t p_old = tmem + kSBase + sbuf * 128, p_new = p_old + 64;
+          const uint32_t acc0 = cj > 0 ? 1u : 0u;          // first chunk of the tile overwrites the accumulators
+#pragma unroll
+          for (int kk = 0; kk < kNC / 16; ++kk)             // 16 key rows per K step = 2048 bytes of the V tile
+            tc::mma_ts_lo(tmem + kAccOld, p_old + kk * 8, v_old + kk * (2048 >> 4), v_hi, idesc_pv, kk > 0 ? 1u : acc0);
 #pragma unroll
           for (int kk = 0; kk < kNC / 16; ++kk)
-            tc::mma_ts(tmem + kAccOld, p_old + kk * 8, v_old + (uint64_t)(kk * (2048 >> 4)), idesc_pv, cj > 0 || kk > 0);
-#pragma unroll
-          for (int kk = 0; kk < kNC / 16; ++kk)
-            tc::mma_ts(tmem + kAccNew, p_new + kk * 8, v_new + (uint64_t)(kk * (2048 >> 4)), idesc_pv, cj > 0 || kk > 0);
+            tc::mma_ts_lo(tmem + kAccNew, p_new + kk * 8, v_new + kk * (2048 >> 4), v_hi, idesc_pv, kk > 0 ? 1u : acc0);
           tc::mma_commit(&ctl.done[slot0]);
           if (ck.patch) tc::mma_commit(&ctl.done[slot1]);
           f_pv += ck.patch ? 2 : 1;
@@ -478,8 +506,8 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
       const int sbuf = gc & 1;
       const int slot0 = f % kSlots;
       if ((tid & 127) == 0) TC_TRACE(2 + grp, ci, 0);
-      // full[] first: orders the producers' column-position writes before the reads below
-      if (!warp_wait(&ctl.full[slot0], (f / kSlots) & 1, abort_flag) ||
+      // landed[] first: orders the TMA warp's column-position writes before the reads below
+      if (!warp_wait(&ctl.landed[slot0], (f / kSlots) & 1, abort_flag) ||
           !warp_wait(&ctl.s_full[sbuf], (gc >> 1) & 1, abort_flag)) { ok = false; break; }
       tc::tc_fence_after();
       if ((tid & 127) == 0) TC_TRACE(2 + grp, ci, 1);
@@ -487,85 +515,89 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
       const int* cp = ctl.col_pos[slot0];
       // rows of a warp that lie at or after every column of the chunk need no causal mask
       const bool unmasked = __all_sync(0xffffffffu, row_ok && ctl.col_last[slot0] <= pos);
-      // The loops over the 64 logits are rolled (16 columns per step) to keep the instruction footprint of the
-      // three concurrently running roles small.
-      float sub;                                         // exponent offset of this chunk: p = 2^(s * c2 - sub)
-      if (grp == 0) {
-        sub = lse2;
+      // One pass over the 64 logits of the row: load them, form p = 2^(s * c2 - sub) in place and pack to bf16.
+      // For the new term `sub` is the running reference; the chunk maximum is tracked on the side, and only if
+      // some row of the warp has no reference yet or would overflow (its maximum beats the reference by more
+      // than the threshold) does the warp take the slow path: fix the reference, rescale, recompute. The S
+      // region is still intact at that point because P is stored last.
+      uint32_t r[64];
+      tc::tmem_ld32(s_addr, *reinterpret_cast<uint32_t(*)[32]>(&r[0]));
+      tc::tmem_ld32(s_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&r[32]));
+      tc::tmem_wait_ld();
+      float sub = grp == 0 ? lse2 : (ref == -INFINITY ? 0.f : ref);
+      float cm = -INFINITY, sum = 0.f;
+      bool stored = false;                               // warp-uniform: the slow path stores P itself
+      if (unmasked) {
+#pragma unroll
+        for (int u = 0; u < 64; u += 2) {
+          const float t0 = __uint_as_float(r[u]), t1 = __uint_as_float(r[u + 1]);
+          cm = fmaxf(cm, fmaxf(t0, t1));
+          const float p0 = tc::ex2(fmaf(t0, c2, -sub)), p1 = tc::ex2(fmaf(t1, c2, -sub));
+          sum += p0 + p1;
+          r[u >> 1] = tc::pack_bf16(p0, p1);
+        }
       } else {
-        float cm = -INFINITY;                            // row maximum (first of two passes over the S region)
-#pragma unroll 1
-        for (int q = 0; q < 4; ++q) {
-          uint32_t r[16];
-          tc::tmem_ld16(s_addr + q * 16, r);
-          tc::tmem_wait_ld();
-          if (unmasked) {
 #pragma unroll
-            for (int u = 0; u < 16; ++u) cm = fmaxf(cm, __uint_as_float(r[u]));
-          } else {
-#pragma unroll
-            for (int u = 0; u < 16; ++u)
-              if (cp[q * 16 + u] <= pos) cm = fmaxf(cm, __uint_as_float(r[u]));
-          }
+        for (int u = 0; u < 64; u += 2) {
+          const float t0 = cp[u] <= pos ? __uint_as_float(r[u]) : -INFINITY;
+          const float t1 = cp[u + 1] <= pos ? __uint_as_float(r[u + 1]) : -INFINITY;
+          cm = fmaxf(cm, fmaxf(t0, t1));
+          const float p0 = tc::ex2(fmaf(t0, c2, -sub)), p1 = tc::ex2(fmaf(t1, c2, -sub));
+          sum += p0 + p1;
+          r[u >> 1] = tc::pack_bf16(p0, p1);
         }
+      }
+      if (grp == 1) {
         cm *= c2;                                        // c2 > 0: scaling commutes with the maximum
-        float factor = 1.f;
-        bool need = false;
-        if (ref == -INFINITY) {
-          ref = cm;                                      // first causal column(s) of this row: accumulator row is still zero
-        } else if (cm - ref > kRescaleThreshold) {
-          factor = tc::ex2(ref - cm);
-          ref = cm;
-          need = true;
-        }
-        if (__any_sync(0xffffffffu, need)) {
-          // lazy rescale of acc_new (rare): every earlier PV must have completed before the rows are rewritten
-          if (ci >= 1) {
-            if (!warp_wait(&ctl.done[f_prev % kSlots], (f_prev / kSlots) & 1, abort_flag)) { ok = false; break; }
-            tc::tc_fence_after();
-          }
-          ell *= factor;
+        const bool first = ref == -INFINITY && cm > -INFINITY;
+        const bool over = ref > -INFINITY && cm - ref > kRescaleThreshold;
+        if (__any_sync(0xffffffffu, first || over)) {
+          // ---- slow path (first chunk of a row, or a reference that fell too far behind) -----------------
+          float factor = 1.f;
+          if (first) ref = cm;                           // accumulator row is still zero: nothing to rescale
+          if (over) { factor = tc::ex2(ref - cm); ref = cm; }
+          if (__any_sync(0xffffffffu, over)) {
+            // every earlier PV must have completed before the accumulator rows are rewritten
+            if (ci >= 1) {
+              if (!warp_wait(&ctl.done[f_prev % kSlots], (f_prev / kSlots) & 1, abort_flag)) { ok = false; break; }
+              tc::tc_fence_after();
+            }
+            ell *= factor;
 #pragma unroll 1
-          for (int q4 = 0; q4 < 8; ++q4) {
-            uint32_t acc[16];
-            tc::tmem_ld16(tmem + lane_base + kAccNew + q4 * 16, acc);
+            for (int q4 = 0; q4 < 8; ++q4) {
+              uint32_t acc[16];
+              tc::tmem_ld16(tmem + lane_base + kAccNew + q4 * 16, acc);
+              tc::tmem_wait_ld();
+#pragma unroll
+              for (int i = 0; i < 16; ++i) acc[i] = __float_as_uint(__uint_as_float(acc[i]) * factor);
+              tc::tmem_st16(tmem + lane_base + kAccNew + q4 * 16, acc);
+            }
+            tc::tmem_wait_st();
+          }
+          sub = ref == -INFINITY ? 0.f : ref;
+          sum = 0.f;
+#pragma unroll 1
+          for (int q = 0; q < 4; ++q) {                  // recompute P from the untouched S region
+            uint32_t t[16];
+            tc::tmem_ld16(s_addr + q * 16, t);
             tc::tmem_wait_ld();
 #pragma unroll
-            for (int i = 0; i < 16; ++i) acc[i] = __float_as_uint(__uint_as_float(acc[i]) * factor);
-            tc::tmem_st16(tmem + lane_base + kAccNew + q4 * 16, acc);
+            for (int u = 0; u < 16; u += 2) {
+              const bool m0 = unmasked || cp[q * 16 + u] <= pos, m1 = unmasked || cp[q * 16 + u + 1] <= pos;
+              const float p0 = m0 ? tc::ex2(fmaf(__uint_as_float(t[u]), c2, -sub)) : 0.f;
+              const float p1 = m1 ? tc::ex2(fmaf(__uint_as_float(t[u + 1]), c2, -sub)) : 0.f;
+              sum += p0 + p1;
+              t[u >> 1] = tc::pack_bf16(p0, p1);
+            }
+            // S[16q, 16q+16) is consumed; P[8q, 8q+8) never reaches unread S
+            tc::tmem_st8(s_addr + q * 8, *reinterpret_cast<uint32_t(*)[8]>(&t[0]));
           }
-          tc::tmem_wait_st();
+          stored = true;
         }
-        sub = ref == -INFINITY ? 0.f : ref;
-      }
-      // exponentials, row sum, bf16 packing. P (bf16, 32 columns) overwrites the first half of the 64-column
-      // S region: step q consumes S[16q, 16q+16) and then stores P[8q, 8q+8), which never reaches unread S.
-      float sum = 0.f;
-#pragma unroll 1
-      for (int q = 0; q < 4; ++q) {
-        uint32_t r[16], p[8];
-        tc::tmem_ld16(s_addr + q * 16, r);
-        tc::tmem_wait_ld();
-        if (unmasked) {
-#pragma unroll
-          for (int u = 0; u < 16; u += 2) {
-            const float p0 = tc::ex2(fmaf(__uint_as_float(r[u]), c2, -sub));
-            const float p1 = tc::ex2(fmaf(__uint_as_float(r[u + 1]), c2, -sub));
-            sum += p0 + p1;
-            p[u >> 1] = tc::pack_bf16(p0, p1);
-          }
-        } else {
-#pragma unroll
-          for (int u = 0; u < 16; u += 2) {
-            const float p0 = cp[q * 16 + u] <= pos ? tc::ex2(fmaf(__uint_as_float(r[u]), c2, -sub)) : 0.f;
-            const float p1 = cp[q * 16 + u + 1] <= pos ? tc::ex2(fmaf(__uint_as_float(r[u + 1]), c2, -sub)) : 0.f;
-            sum += p0 + p1;
-            p[u >> 1] = tc::pack_bf16(p0, p1);
-          }
-        }
-        tc::tmem_st8(s_addr + q * 8, p);
       }
       if (grp == 0) mass += sum; else ell += sum;
+      // P (bf16, 32 columns) overwrites the first half of the 64-column S region, all of which was consumed
+      if (!stored) tc::tmem_st32(s_addr, *reinterpret_cast<uint32_t(*)[32]>(&r[0]));
       tc::tmem_wait_st();
       if ((tid & 127) == 0) TC_TRACE(2 + grp, ci, 2);
       tc::tc_fence_before();
@@ -617,7 +649,17 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
   }
   // every role is done with this tile: accumulators, Q tiles and the ring bookkeeping move on together
   g += n_chunks;
-  fill += (n_plain + kNC - 1) / kNC + 2 * ((n_patch + kNC - 1) / kNC);
+  {
+    int f = fill;
+    for (int ci = 0; ci < n_chunks; ++ci) {   // replay the tile's fills (same for every role)
+      const ChunkInfo ck = chunk_info(ci, n_plain, n_patch);
+      const int n_slots = ck.patch ? 2 : 1;
+      if (ctl.chunk_mask[ci] != 0)
+        for (int k = 0; k < n_slots; ++k) dirty_par_cta ^= 1u << ((f + k) % kSlots);
+      f += n_slots;
+    }
+    fill = f;
+  }
   tc::tc_fence_before();
   __syncthreads();
   tc::tc_fence_after();
@@ -646,13 +688,16 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
 
 // Returns FL_ERR_UNSUPPORTED when the tensor path does not cover the request (caller falls back to the
 // SIMT kernel, which is also CUDA).
-int fl_launch_loop_attn_tc(const fl_ctx* ctx, const fl_shape* s, int loop_r, const void* q_new, const void* q_old,
+int fl_launch_loop_attn_tc(fl_ctx* ctx, const fl_shape* s, int loop_r, const void* q_new, const void* q_old,
                            const int32_t* active_idx, int n_active, const fl_kv_store* store, const int32_t* col_idx,
                            const int32_t* col_cnt, int c, const float* lse_prev, float* lse_out, const void* o_prev,
                            void* o_out, int32_t* status, cudaStream_t st) {
   if (s->dtype != FL_BF16 || s->head_dim != kDH || c > kMaxCols) return FL_ERR_UNSUPPORTED;
   if ((size_t)ctx->max_smem_optin < kTcSmemBytes) return FL_ERR_UNSUPPORTED;
   TcArgs a{};
+  if (!fl_row_gather_tmap(ctx, store->k_base, s->L, (int64_t)s->n_heads * s->head_dim, &a.k_map) ||
+      !fl_row_gather_tmap(ctx, store->v_base, s->L, (int64_t)s->n_heads * s->head_dim, &a.v_map))
+    return FL_ERR_UNSUPPORTED;
   a.q_new = static_cast<const __nv_bfloat16*>(q_new);
   a.q_old = static_cast<const __nv_bfloat16*>(q_old);
   a.o_prev = static_cast<const __nv_bfloat16*>(o_prev);

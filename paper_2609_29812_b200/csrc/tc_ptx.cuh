@@ -43,10 +43,10 @@ __device__ __forceinline__ bool mbar_try_wait_hint(uint64_t* bar, uint32_t parit
 // Polls are spaced out (hardware suspend hint) so that waiting threads do not crowd the shared-memory pipe;
 // the default limit gives up after roughly a tenth of a second.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
-                                          uint32_t limit = (1u << 16)) {
+                                          uint32_t limit = (1u << 20)) {
   if (mbar_try_wait(bar, parity)) return true;
   for (uint32_t it = 0; it < limit; ++it) {
-    if (mbar_try_wait_hint(bar, parity, 2000u)) return true;
+    if (mbar_try_wait_hint(bar, parity, 64u)) return true;
     if ((it & 15u) == 15u && *abort_flag) return false;
   }
   *abort_flag = 1;
@@ -68,6 +68,25 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N>
 __device__ __forceinline__ void cp_async_wait() {
   asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
+// ---- TMA --------------------------------------------------------------------------------------------------
+// arrive on the barrier and add `tx_bytes` to the bytes it expects from asynchronous copies
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t tx_bytes) {
+  asm volatile("{\n\t.reg .b64 st;\n\tmbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1;\n\t}" ::"r"(smem_u32(bar)),
+               "r"(tx_bytes)
+               : "memory");
+}
+// Gather four rows (y0..y3) of a 2-D tensor, box = (tensor-map inner extent) x 1 row each, into consecutive
+// rows of shared memory; completes `4 * box bytes` on the mbarrier. Rows outside the tensor read as zero.
+// No multicast: the destination is this CTA's own shared memory.
+__device__ __forceinline__ void tma_gather4(void* smem_dst, const void* tmap, uint64_t* bar, int x, int y0, int y1, int y2,
+                                            int y3) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cta.global.tile::gather4.mbarrier::complete_tx::bytes "
+      "[%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+      ::"r"(smem_u32(smem_dst)), "l"(tmap), "r"(smem_u32(bar)), "r"(x), "r"(y0), "r"(y1), "r"(y2), "r"(y3)
+      : "memory");
 }
 
 // ---- TMEM allocation (one warp, all lanes) ----------------------------------------------------------
@@ -104,6 +123,31 @@ __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_
       "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
       ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"((uint32_t)accum)
+      : "memory");
+}
+// Lean forms for the issue loop: the descriptor is given as (low word, high word) so that stepping along K or
+// to another ring slot is ONE 32-bit add on the low word (start-address field), and the accumulate flag is an
+// immediate. The single issuing thread is otherwise issue-bound: a 64-bit add plus a predicate set-up per MMA
+// costs more cycles than a 128x64x16 MMA takes.
+template <bool ACC>
+__device__ __forceinline__ void mma_ss_lo(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                          uint32_t idesc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+      "setp.ne.b32 p, %6, 0;\n\t"
+      "mov.b64 da, {%1, %2};\n\tmov.b64 db, {%3, %4};\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "n"(ACC ? 1 : 0)
+      : "memory");
+}
+__device__ __forceinline__ void mma_ts_lo(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi, uint32_t idesc,
+                                          uint32_t accum) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\t"
+      "setp.ne.b32 p, %5, 0;\n\t"
+      "mov.b64 db, {%2, %3};\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accum)
       : "memory");
 }
 // arrive on the mbarrier once every MMA issued so far by this thread has completed

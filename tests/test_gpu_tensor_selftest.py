@@ -35,3 +35,34 @@ def test_umma_tile_products_match_matmul():
     p = s_out.to(torch.bfloat16).double()
     o_ref = p @ v.double()
     np.testing.assert_allclose(o_out.cpu().numpy(), o_ref.cpu().numpy(), rtol=1e-3, atol=5e-2)
+
+
+def test_tma_row_gather_feeds_the_tensor_core():
+    """tile::gather4 row gather into a swizzled operand tile, including an out-of-range row (zero fill)."""
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2609_29812_b200 import build
+    lib = C.CDLL(build.SELFTEST_LIB_PATH)
+    lib.fl_selftest_gather4.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+    lib.fl_selftest_gather4.restype = C.c_int
+    g = torch.Generator(device="cpu").manual_seed(2)
+    rows = 1000
+    base = torch.randn(rows, 128, generator=g).to(torch.bfloat16).cuda()
+    q = torch.randn(128, 128, generator=g).to(torch.bfloat16).cuda()
+    idx = torch.randperm(rows, generator=g)[:64].to(torch.int32)
+    idx[5] = rows                      # out of range: must read as a zero row
+    idx[63] = 0
+    idx_d = idx.cuda()
+    s_out = torch.zeros(128, 64, dtype=torch.float32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    rc = lib.fl_selftest_gather4(base.data_ptr(), rows, q.data_ptr(), idx_d.data_ptr(), s_out.data_ptr(),
+                                 status.data_ptr(), None)
+    assert rc == 0
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    kg = torch.zeros(64, 128, dtype=torch.float64)
+    for t, j in enumerate(idx.tolist()):
+        if j < rows:
+            kg[t] = base[j].double().cpu()
+    s_ref = q.double().cpu() @ kg.T
+    np.testing.assert_allclose(s_out.cpu().numpy(), s_ref.numpy(), rtol=1e-4, atol=1e-3)

@@ -5,10 +5,12 @@
 // Warp roles (16 warps, 512 threads):
 //   warps 0-3   softmax of the OLD term  (fixed normaliser lse_prev: p_old = exp(s_old - lse_prev), mass m_i)
 //   warps 4-7   softmax of the NEW term  (running reference with lazy rescale of the accumulator)
-//   warp  8     one elected thread issues every tcgen05.mma; the warp owns the tensor-memory allocation
-//   warp  9     TMA: row gathers (cp.async.bulk.tensor tile::gather4, 4 selected columns per copy) of the bf16
+//   warp  8     one thread issues the S = Q Khat^T MMAs; the warp owns the tensor-memory allocation
+//   warp  9     one thread issues the acc += P Vhat MMAs (a single thread cannot issue 64-column MMAs as fast
+//               as the tensor pipe retires them; two issuers keep it fed)
+//   warps 10-13 TMA: row gathers (cp.async.bulk.tensor tile::gather4, 4 selected columns per copy) of the bf16
 //               base K/V rows straight into 128B-swizzled operand tiles; completion on mbarriers
-//   warps 10-15 patch: stage the Q tiles; for the columns that carry residual payloads, overwrite the gathered
+//   warps 14-15 patch: stage the Q tiles; for the columns that carry residual payloads, overwrite the gathered
 //               base rows with the dequantize-and-add result (Eq. 8)
 //
 // Prologue (whole CTA): the block's causal column list is copied to shared memory together with a bit mask
@@ -37,9 +39,11 @@ constexpr int kSlotBytes = 2 * kTileBytes;  // K tile | V tile
 constexpr int kQTileBytes = kM * kDH * 2;   // 32 KB
 constexpr int kSoftmaxWarps = 8;
 constexpr int kMmaWarp = 8;
-constexpr int kTmaWarp = 9;
-constexpr int kPatchWarps = 6;
-constexpr int kWarps = kSoftmaxWarps + 2 + kPatchWarps;  // 16
+constexpr int kPvWarp = 9;         // second MMA issuer (the first, kMmaWarp, issues QK^T)
+constexpr int kTmaWarp = 10;       // first of the TMA warps
+constexpr int kTmaWarps = 4;       // a single warp cannot issue four-row gathers fast enough; four come close
+constexpr int kPatchWarps = 2;
+constexpr int kWarps = kSoftmaxWarps + 2 + kTmaWarps + kPatchWarps;  // 16
 constexpr int kThreads = kWarps * 32;
 constexpr int kPatchThreads = kPatchWarps * 32;
 constexpr int kMaxCols = 3072;              // column budget the shared-memory column list can hold
@@ -87,6 +91,7 @@ struct __align__(16) TcSmemCtl {
   uint64_t q_full;           // patch warps -> MMA: the Q tiles of the current row tile are staged
   uint64_t s_full[2];      // MMA -> softmax: S of the chunk is in tensor memory
   uint64_t p_full[2];      // softmax -> MMA: P of the chunk is in tensor memory
+  uint64_t s_free[2];      // PV issuer -> QK issuer: the PV MMAs that read P from the buffer have finished
   uint64_t acc_done;       // MMA -> softmax: all accumulation of the tile finished
   uint32_t tmem_base;
   int abort_flag;
@@ -169,27 +174,29 @@ __device__ __forceinline__ void patch_piece(const DevSide& side, int n_old, uint
   }
 }
 
-// chunk ci of the partitioned column list: plain chunks first, then patched chunks
+// chunk ci of the partitioned column list: patched chunks first (the first two are built by the whole CTA
+// before the pipeline starts), then plain chunks. In the ordered list the plain columns come first.
 struct ChunkInfo {
   int off;      // offset into the ordered column list
   int n_valid;  // valid columns (<= kNC)
   bool patch;   // columns carry a payload in the current loop: separate old / new operand tiles (two slots)
 };
 __device__ __forceinline__ ChunkInfo chunk_info(int ci, int n_plain, int n_patch) {
-  const int n_plain_chunks = (n_plain + kNC - 1) / kNC;
+  const int n_patch_chunks = (n_patch + kNC - 1) / kNC;
   ChunkInfo c;
-  if (ci < n_plain_chunks) {
-    c.off = ci * kNC;
+  if (ci < n_patch_chunks) {
+    c.off = n_plain + ci * kNC;
+    c.n_valid = min(kNC, n_patch - ci * kNC);
+    c.patch = true;
+  } else {
+    const int k = ci - n_patch_chunks;
+    c.off = k * kNC;
     c.n_valid = min(kNC, n_plain - c.off);
     c.patch = false;
-  } else {
-    const int k = ci - n_plain_chunks;
-    c.off = n_plain + k * kNC;
-    c.n_valid = min(kNC, n_patch - k * kNC);
-    c.patch = true;
   }
   return c;
 }
+constexpr int kPrefillChunks = 2;   // patched chunks the whole CTA builds at the start of a row tile (4 ring slots)
 
 template <int BITS>
 __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_constant__ TcArgs a) {
@@ -210,7 +217,7 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
 
   if (tid == 0) {
     for (int s = 0; s < kSlots; ++s) {
-      tc::mbar_init(&ctl.landed[s], 1);
+      tc::mbar_init(&ctl.landed[s], kTmaWarps);
       tc::mbar_init(&ctl.patched[s], kPatchWarps);
       tc::mbar_init(&ctl.done[s], 1);
     }
@@ -218,6 +225,7 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
     for (int s = 0; s < 2; ++s) {
       tc::mbar_init(&ctl.s_full[s], 1);
       tc::mbar_init(&ctl.p_full[s], kSoftmaxWarps * 32);
+      tc::mbar_init(&ctl.s_free[s], 1);
     }
     tc::mbar_init(&ctl.acc_done, 1);
     ctl.abort_flag = 0;
@@ -265,7 +273,7 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
     if (tid == 0) { ctl.n_plain = tot0; ctl.n_patch = tot1; }
     for (int i = tid; i < kMaxCols / kNC + 2; i += kThreads) ctl.chunk_mask[i] = 0;
     __syncthreads();
-    const int plain_chunks = (tot0 + kNC - 1) / kNC;
+    const int patch_chunks = (tot1 + kNC - 1) / kNC;
     for (int base = beg; base < end; base += 32) {
       const int u = base + lane;
       const int j = u < end ? __ldg(cols + u) : INT32_MAX;
@@ -281,7 +289,7 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
         const int dst = patched ? tot0 + before1 + __popc(m1 & lt) : before0 + __popc(m0 & lt);
         ord_col[dst] = j;
         ord_mask[dst] = mask;
-        if (mask != 0) atomicOr(&ctl.chunk_mask[patched ? plain_chunks + (dst - tot0) / kNC : dst / kNC], mask);
+        if (mask != 0) atomicOr(&ctl.chunk_mask[patched ? (dst - tot0) / kNC : patch_chunks + dst / kNC], mask);
       }
       before0 += __popc(m0);
       before1 += __popc(m1);
@@ -298,39 +306,81 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
   const int n_rows = min(kM, q_hi - s0);
   const int g0 = g, fill0 = fill;
   const uint32_t dirty_par0 = dirty_par_cta;
+  const int n_pre = min((n_patch + kNC - 1) / kNC, kPrefillChunks);
+  // ---- the first patched chunks are built by all 512 threads straight into the (idle) ring: base row plus
+  // dequantized residuals (Eq. 8), old and new operand tiles. Left to the two patch warps this would take an
+  // order of magnitude longer than a plain chunk; done here it costs a few dependent loads per thread.
+  {
+#pragma unroll 2
+    for (int p = tid; p < n_pre * kNC * 32; p += kThreads) {
+      const int pc = p / (kNC * 32), q = p % (kNC * 32);
+      const int u = q >> 5, half = (q >> 4) & 1, ch = q & 15;
+      const ChunkInfo ck = chunk_info(pc, n_plain, n_patch);
+      const int slot0 = (fill0 + 2 * pc) % kSlots, slot1 = (fill0 + 2 * pc + 1) % kSlots;
+      const uint32_t off = half * kTileBytes + (ch >> 3) * (kNC * 128) + tc::sw128_offset(u, ch & 7);
+      uint4 v_old = make_uint4(0, 0, 0, 0), v_new = make_uint4(0, 0, 0, 0);
+      if (u < ck.n_valid) {
+        const DevSide& side = half ? a.v : a.k;
+        const int j = ord_col[ck.off + u];
+        const int elem = h * kDH + ch * 8;
+        const uint4 base16 =
+            __ldg(reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(side.base) + (size_t)j * a.d + elem));
+        patch_piece<BITS>(side, a.n_old, ord_mask[ck.off + u], j, elem, a.d, a.group, base16, v_old, v_new);
+      }
+      *reinterpret_cast<uint4*>(ring + slot0 * kSlotBytes + off) = v_old;
+      *reinterpret_cast<uint4*>(ring + slot1 * kSlotBytes + off) = v_new;
+    }
+    for (int p = tid; p < n_pre * kNC; p += kThreads) {
+      const int pc = p / kNC, u = p % kNC;
+      const ChunkInfo ck = chunk_info(pc, n_plain, n_patch);
+      const int slot0 = (fill0 + 2 * pc) % kSlots;
+      ctl.col_pos[slot0][u] = u < ck.n_valid ? ord_col[ck.off + u] : INT32_MAX;
+      if (u == 0) ctl.col_last[slot0] = ck.n_valid == kNC ? ord_col[ck.off + kNC - 1] : INT32_MAX;
+    }
+    tc::fence_proxy_async_smem();
+    __syncthreads();
+  }
 
-  if (warp == kTmaWarp) {
+  if (warp >= kTmaWarp && warp < kTmaWarp + kTmaWarps) {
     // ============================================== TMA ==============================================
-    // In-order fills of the ring; the lookahead is whatever the four slots allow. Each lane issues two of
-    // the 64 four-row gathers of a slot (K: 2 slabs x 16 groups, V: the same).
+    // In-order fills of the ring; the lookahead is whatever the four slots allow. The 64 four-row gathers
+    // of a slot (K: 2 slabs x 16 groups, V: the same) are split over the TMA warps, 16 each, one per lane;
+    // every warp announces its own share of the bytes on the slot's barrier.
+    const int tw = warp - kTmaWarp;
+    const int is_v = tw >> 1, slab = tw & 1, grp = lane & 15;
+    const void* map = is_v ? static_cast<const void*>(&a.v_map) : static_cast<const void*>(&a.k_map);
     int f = fill0;
     bool ok = true;
 #pragma unroll 1
     for (int ci = 0; ci < n_chunks && ok; ++ci) {
       const ChunkInfo ck = chunk_info(ci, n_plain, n_patch);
       const int n_slots = ck.patch ? 2 : 1;
+      if (ci < n_pre) {   // built by the whole CTA above: only the barrier phase is left to complete
+        if (lane == 0)
+          for (int k = 0; k < n_slots; ++k) tc::mbar_arrive(&ctl.landed[(f + k) % kSlots]);
+        f += n_slots;
+        continue;
+      }
       for (int k = 0; k < n_slots && ok; ++k)
         if (f + k >= kSlots) ok = warp_wait(&ctl.done[(f + k) % kSlots], (((f + k) / kSlots) - 1) & 1, abort_flag);
       if (!ok) break;
       const int slot0 = f % kSlots;
-      if (lane == 0) TC_TRACE(0, ci, 0);
-      for (int u = lane; u < kNC; u += 32) ctl.col_pos[slot0][u] = u < ck.n_valid ? ord_col[ck.off + u] : INT32_MAX;
-      if (lane == 0) ctl.col_last[slot0] = ck.n_valid == kNC ? ord_col[ck.off + kNC - 1] : INT32_MAX;
+      if (tid == kTmaWarp * 32) TC_TRACE(0, ci, 0);
+      if (tw == 0) {
+        for (int u = lane; u < kNC; u += 32) ctl.col_pos[slot0][u] = u < ck.n_valid ? ord_col[ck.off + u] : INT32_MAX;
+        if (lane == 0) ctl.col_last[slot0] = ck.n_valid == kNC ? ord_col[ck.off + kNC - 1] : INT32_MAX;
+      }
       __syncwarp();
       if (lane == 0)
-        for (int k = 0; k < n_slots; ++k) tc::mbar_arrive_expect_tx(&ctl.landed[(f + k) % kSlots], kSlotBytes);
+        for (int k = 0; k < n_slots; ++k) tc::mbar_arrive_expect_tx(&ctl.landed[(f + k) % kSlots], kSlotBytes / kTmaWarps);
       __syncwarp();
-#pragma unroll
-      for (int rep = 0; rep < 2; ++rep) {
-        const int gidx = lane + rep * 32;                  // 0..63
-        const int is_v = gidx >> 5, slab = (gidx >> 4) & 1, grp = gidx & 15;
+      if (lane < 16) {
         int y[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const int u = grp * 4 + i;
           y[i] = u < ck.n_valid ? ord_col[ck.off + u] : a.L;   // row L is outside the tensor: reads as zero
         }
-        const void* map = is_v ? static_cast<const void*>(&a.v_map) : static_cast<const void*>(&a.k_map);
         for (int k = 0; k < n_slots; ++k) {
           const int slot = (f + k) % kSlots;
           tc::tma_gather4(ring + slot * kSlotBytes + is_v * kTileBytes + slab * (kNC * 128) + grp * 512, map,
@@ -338,11 +388,11 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
         }
       }
       f += n_slots;
-      if (lane == 0) TC_TRACE(0, ci, 1);
+      if (tid == kTmaWarp * 32) TC_TRACE(0, ci, 1);
     }
-  } else if (warp > kTmaWarp) {
+  } else if (warp >= kTmaWarp + kTmaWarps) {
     // ============================================= patch =============================================
-    const int pt = tid - (kTmaWarp + 1) * 32;   // 0..191
+    const int pt = tid - (kTmaWarp + kTmaWarps) * 32;   // 0..95
     const int pw = pt >> 5;
     // Q tiles (once per row tile): asynchronous 16-byte copies
     for (int it = pt; it < 2 * kM * 16; it += kPatchThreads) {
@@ -380,6 +430,7 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
       if (ctl.chunk_mask[ci] != 0) {
         uint8_t* t_old = ring + (f % kSlots) * kSlotBytes + half * kTileBytes + ch_off;
         uint8_t* t_new = ring + ((f + 1) % kSlots) * kSlotBytes + half * kTileBytes + ch_off;
+        if (ci >= n_pre)
 #pragma unroll 1
         for (int u = pw; u < ck.n_valid; u += kPatchWarps) {
           const uint32_t mask = ord_mask[ck.off + u];
@@ -401,88 +452,90 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
       f += n_slots;
     }
   } else if (warp == kMmaWarp) {
-    // =========================================== MMA issuer ==========================================
+    // ========================================= QK^T issuer ==========================================
     if (lane == 0) {
       const uint32_t idesc_qk = tc::make_idesc_bf16(kM, kNC, false);
-      const uint32_t idesc_pv = tc::make_idesc_bf16(kM, kDH, true);
-      // Descriptors differ only in their start-address field (bits 0-13, units of 16 bytes), so a step along
-      // K is one 64-bit add. K-major operands (Q, Khat): 32 bytes per 16-element K step inside a 64-element
-      // slab, then the next slab. MN-major Vhat: 16 key rows = two 1024-byte row groups per K step.
+      // Descriptors differ only in their start-address field (bits 0-13, units of 16 bytes): the low word
+      // moves (no carry into the other fields: shared memory is < 256 KB), the high word stays.
+      // K-major operands (Q, Khat): 32 bytes per 16-element K step inside a 64-element slab, then the next slab.
       const uint64_t q_old_desc = tc::make_desc_sw128(tc::smem_u32(q_old_tile), 16, 1024);
       const uint64_t q_new_desc = tc::make_desc_sw128(tc::smem_u32(q_new_tile), 16, 1024);
       const uint64_t k_desc0 = tc::make_desc_sw128(tc::smem_u32(ring), 16, 1024);
-      const uint64_t v_desc0 = tc::make_desc_sw128(tc::smem_u32(ring) + kTileBytes, kNC * 128, 1024);
-      // low words move (start address, no carry into the other fields: shared memory is < 256 KB), high words stay
-      const uint32_t kq_hi = (uint32_t)(k_desc0 >> 32), v_hi = (uint32_t)(v_desc0 >> 32);
-      const uint32_t q_old_lo = (uint32_t)q_old_desc, q_new_lo = (uint32_t)q_new_desc;
-      const uint32_t k_lo0 = (uint32_t)k_desc0, v_lo0 = (uint32_t)v_desc0;
-      bool ok = true;
-      int f = fill0;        // slot counter of the chunk whose QK is issued next
-      int f_pv = fill0;     // slot counter of the chunk whose PV is issued next
+      const uint32_t kq_hi = (uint32_t)(k_desc0 >> 32);
+      const uint32_t q_old_lo = (uint32_t)q_old_desc, q_new_lo = (uint32_t)q_new_desc, k_lo0 = (uint32_t)k_desc0;
+      int f = fill0;
       uint32_t dirty_par = dirty_par0;
-      // iteration ci issues QK(ci) and then PV(ci-1): the softmax of chunk ci-1 overlaps QK(ci)
 #pragma unroll 1
-      for (int ci = 0; ci <= n_chunks && ok; ++ci) {
-        if (ci < n_chunks) {
-          const ChunkInfo ck = chunk_info(ci, n_plain, n_patch);
-          const int slot0 = f % kSlots, slot1 = (f + 1) % kSlots;
-          TC_TRACE(1, ci, 0);
-          if (ci == 0 && !tc::mbar_wait(&ctl.q_full, tile & 1, abort_flag)) { ok = false; break; }
-          if (!tc::mbar_wait(&ctl.landed[slot0], (f / kSlots) & 1, abort_flag)) { ok = false; break; }
-          if (ck.patch && !tc::mbar_wait(&ctl.landed[slot1], ((f + 1) / kSlots) & 1, abort_flag)) { ok = false; break; }
-          if (ctl.chunk_mask[ci] != 0) {       // residual-carrying columns are rewritten by the patch warps
-            if (!tc::mbar_wait(&ctl.patched[slot0], (dirty_par >> slot0) & 1, abort_flag)) { ok = false; break; }
-            dirty_par ^= 1u << slot0;
-            if (ck.patch) {
-              if (!tc::mbar_wait(&ctl.patched[slot1], (dirty_par >> slot1) & 1, abort_flag)) { ok = false; break; }
-              dirty_par ^= 1u << slot1;
-            }
+      for (int ci = 0; ci < n_chunks; ++ci) {
+        const ChunkInfo ck = chunk_info(ci, n_plain, n_patch);
+        const int slot0 = f % kSlots, slot1 = (f + 1) % kSlots;
+        const int gc = g0 + ci, sbuf = gc & 1;
+        TC_TRACE(1, ci, 0);
+        if (ci == 0 && !tc::mbar_wait(&ctl.q_full, tile & 1, abort_flag)) break;
+        if (!tc::mbar_wait(&ctl.landed[slot0], (f / kSlots) & 1, abort_flag)) break;
+        if (ck.patch && !tc::mbar_wait(&ctl.landed[slot1], ((f + 1) / kSlots) & 1, abort_flag)) break;
+        if (ctl.chunk_mask[ci] != 0) {       // residual-carrying columns are rewritten by the patch warps
+          if (!tc::mbar_wait(&ctl.patched[slot0], (dirty_par >> slot0) & 1, abort_flag)) break;
+          dirty_par ^= 1u << slot0;
+          if (ck.patch) {
+            if (!tc::mbar_wait(&ctl.patched[slot1], (dirty_par >> slot1) & 1, abort_flag)) break;
+            dirty_par ^= 1u << slot1;
           }
-          tc::tc_fence_after();
-          TC_TRACE(1, ci, 1);
-          const uint32_t k_old = k_lo0 + slot0 * (kSlotBytes >> 4);
-          const uint32_t k_new = ck.patch ? k_lo0 + slot1 * (kSlotBytes >> 4) : k_old;
-          const int sbuf = (g0 + ci) & 1;
-          const uint32_t s_old = tmem + kSBase + sbuf * 128, s_new = s_old + 64;
-          // K step kk: 32 bytes inside a 64-element slab, then the next slab (Q: 128 rows, Khat: 64 rows per slab)
+        }
+        // the S buffer still holds P of chunk gc-2 until the PV MMAs that read it have retired
+        if (gc >= 2 && !tc::mbar_wait(&ctl.s_free[sbuf], ((gc >> 1) - 1) & 1, abort_flag)) break;
+        TC_TRACE(1, ci, 1);
+        const uint32_t k_old = k_lo0 + slot0 * (kSlotBytes >> 4);
+        const uint32_t k_new = ck.patch ? k_lo0 + slot1 * (kSlotBytes >> 4) : k_old;
+        const uint32_t s_old = tmem + kSBase + sbuf * 128, s_new = s_old + 64;
 #define FL_QK(D, QLO, KLO, KK, ACC)                                                                          \
   tc::mma_ss_lo<ACC>(D, (QLO) + ((((KK) >> 2) * (kM * 128) + ((KK)&3) * 32) >> 4), kq_hi,                    \
                      (KLO) + ((((KK) >> 2) * (kNC * 128) + ((KK)&3) * 32) >> 4), kq_hi, idesc_qk)
-          FL_QK(s_old, q_old_lo, k_old, 0, false); FL_QK(s_old, q_old_lo, k_old, 1, true);
-          FL_QK(s_old, q_old_lo, k_old, 2, true);  FL_QK(s_old, q_old_lo, k_old, 3, true);
-          FL_QK(s_old, q_old_lo, k_old, 4, true);  FL_QK(s_old, q_old_lo, k_old, 5, true);
-          FL_QK(s_old, q_old_lo, k_old, 6, true);  FL_QK(s_old, q_old_lo, k_old, 7, true);
-          FL_QK(s_new, q_new_lo, k_new, 0, false); FL_QK(s_new, q_new_lo, k_new, 1, true);
-          FL_QK(s_new, q_new_lo, k_new, 2, true);  FL_QK(s_new, q_new_lo, k_new, 3, true);
-          FL_QK(s_new, q_new_lo, k_new, 4, true);  FL_QK(s_new, q_new_lo, k_new, 5, true);
-          FL_QK(s_new, q_new_lo, k_new, 6, true);  FL_QK(s_new, q_new_lo, k_new, 7, true);
+        FL_QK(s_old, q_old_lo, k_old, 0, false); FL_QK(s_old, q_old_lo, k_old, 1, true);
+        FL_QK(s_old, q_old_lo, k_old, 2, true);  FL_QK(s_old, q_old_lo, k_old, 3, true);
+        FL_QK(s_old, q_old_lo, k_old, 4, true);  FL_QK(s_old, q_old_lo, k_old, 5, true);
+        FL_QK(s_old, q_old_lo, k_old, 6, true);  FL_QK(s_old, q_old_lo, k_old, 7, true);
+        FL_QK(s_new, q_new_lo, k_new, 0, false); FL_QK(s_new, q_new_lo, k_new, 1, true);
+        FL_QK(s_new, q_new_lo, k_new, 2, true);  FL_QK(s_new, q_new_lo, k_new, 3, true);
+        FL_QK(s_new, q_new_lo, k_new, 4, true);  FL_QK(s_new, q_new_lo, k_new, 5, true);
+        FL_QK(s_new, q_new_lo, k_new, 6, true);  FL_QK(s_new, q_new_lo, k_new, 7, true);
 #undef FL_QK
-          tc::mma_commit(&ctl.s_full[sbuf]);
-          f += ck.patch ? 2 : 1;
-          TC_TRACE(1, ci, 2);
-        }
-        if (ci >= 1) {
-          const int cj = ci - 1;
-          const ChunkInfo ck = chunk_info(cj, n_plain, n_patch);
-          const int sbuf = (g0 + cj) & 1;
-          if (!tc::mbar_wait(&ctl.p_full[sbuf], ((g0 + cj) >> 1) & 1, abort_flag)) { ok = false; break; }
-          tc::tc_fence_after();
-          const int slot0 = f_pv % kSlots, slot1 = (f_pv + 1) % kSlots;
-          const uint32_t v_old = v_lo0 + slot0 * (kSlotBytes >> 4);
-          const uint32_t v_new = ck.patch ? v_lo0 + slot1 * (kSlotBytes >> 4) : v_old;
-          const uint32_t p_old = tmem + kSBase + sbuf * 128, p_new = p_old + 64;
-          const uint32_t acc0 = cj > 0 ? 1u : 0u;          // first chunk of the tile overwrites the accumulators
+        tc::mma_commit(&ctl.s_full[sbuf]);
+        f += ck.patch ? 2 : 1;
+        TC_TRACE(1, ci, 2);
+      }
+    }
+    __syncwarp();
+  } else if (warp == kPvWarp) {
+    // ========================================== P V issuer ==========================================
+    if (lane == 0) {
+      const uint32_t idesc_pv = tc::make_idesc_bf16(kM, kDH, true);
+      // MN-major Vhat: 16 key rows = two 1024-byte row groups per K step
+      const uint64_t v_desc0 = tc::make_desc_sw128(tc::smem_u32(ring) + kTileBytes, kNC * 128, 1024);
+      const uint32_t v_hi = (uint32_t)(v_desc0 >> 32), v_lo0 = (uint32_t)v_desc0;
+      int f = fill0;
+#pragma unroll 1
+      for (int cj = 0; cj < n_chunks; ++cj) {
+        const ChunkInfo ck = chunk_info(cj, n_plain, n_patch);
+        const int gc = g0 + cj, sbuf = gc & 1;
+        if (!tc::mbar_wait(&ctl.p_full[sbuf], (gc >> 1) & 1, abort_flag)) break;
+        tc::tc_fence_after();
+        const int slot0 = f % kSlots, slot1 = (f + 1) % kSlots;
+        const uint32_t v_old = v_lo0 + slot0 * (kSlotBytes >> 4);
+        const uint32_t v_new = ck.patch ? v_lo0 + slot1 * (kSlotBytes >> 4) : v_old;
+        const uint32_t p_old = tmem + kSBase + sbuf * 128, p_new = p_old + 64;
+        const uint32_t acc0 = cj > 0 ? 1u : 0u;          // first chunk of the tile overwrites the accumulators
 #pragma unroll
-          for (int kk = 0; kk < kNC / 16; ++kk)             // 16 key rows per K step = 2048 bytes of the V tile
-            tc::mma_ts_lo(tmem + kAccOld, p_old + kk * 8, v_old + kk * (2048 >> 4), v_hi, idesc_pv, kk > 0 ? 1u : acc0);
+        for (int kk = 0; kk < kNC / 16; ++kk)
+          tc::mma_ts_lo(tmem + kAccOld, p_old + kk * 8, v_old + kk * (2048 >> 4), v_hi, idesc_pv, kk > 0 ? 1u : acc0);
 #pragma unroll
-          for (int kk = 0; kk < kNC / 16; ++kk)
-            tc::mma_ts_lo(tmem + kAccNew, p_new + kk * 8, v_new + kk * (2048 >> 4), v_hi, idesc_pv, kk > 0 ? 1u : acc0);
-          tc::mma_commit(&ctl.done[slot0]);
-          if (ck.patch) tc::mma_commit(&ctl.done[slot1]);
-          f_pv += ck.patch ? 2 : 1;
-          TC_TRACE(1, cj, 3);
-        }
+        for (int kk = 0; kk < kNC / 16; ++kk)
+          tc::mma_ts_lo(tmem + kAccNew, p_new + kk * 8, v_new + kk * (2048 >> 4), v_hi, idesc_pv, kk > 0 ? 1u : acc0);
+        tc::mma_commit(&ctl.done[slot0]);
+        if (ck.patch) tc::mma_commit(&ctl.done[slot1]);
+        tc::mma_commit(&ctl.s_free[sbuf]);
+        f += ck.patch ? 2 : 1;
+        TC_TRACE(1, cj, 3);
       }
       tc::mma_commit(&ctl.acc_done);
     }

@@ -339,11 +339,13 @@ def run_ours(args):
     sampler.start()
     attn_events = []
     t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+    host_t0 = time.perf_counter()
     with torch.cuda.stream(stream):
         t0.record(stream)
         for _ in range(args.steps):
             bench.run_step(attn_events)
         t1.record(stream)
+    host_issue_ms = (time.perf_counter() - host_t0) * 1e3 / args.steps
     barrier()
     clocks = sampler.stop()
     ms = t0.elapsed_time(t1) / args.steps
@@ -382,7 +384,8 @@ def run_ours(args):
                                   f"q_block {w.q_block}, int{w.bits} g{w.group} residuals",
                       "parallelism": "replicas only" if world > 1 else "single GPU",
                       "l2": "inputs exceed L2 (each step streams the per-layer stores, far above 126 MB)"},
-           "gpu_launches": bench.launches_per_step * args.steps, "clocks": clocks, "roofline": roof,
+           "gpu_launches": bench.launches_per_step * args.steps, "host_issue_ms_per_step": host_issue_ms,
+           "clocks": clocks, "roofline": roof,
            "step_roofline": step_roof}
     fl_b, dense_b = kv_bytes_per_token(bench)
     out["kv_bytes_per_token"] = {"flashloop": fl_b * w.n_layers, "dense_looped": dense_b * w.n_layers,
@@ -471,10 +474,11 @@ def run_e2e(bench, args, world, barrier):
 # ------------------------------------------------------------------------------------------------
 # CPU oracle arm (reported baseline; `--impl reference`)
 # ------------------------------------------------------------------------------------------------
-def oracle_sample(w, n_blocks_sample=2, seed=0):
+def oracle_sample(w, n_heads_sample=16, n_blocks_sample=0, seed=0):
     """Times the oracle, as it stands, on a bounded sample of the workload: token selection of every loop
-    in full (stack hidden state), and for ONE head of ONE layer the residual codec on all active rows and
-    the sparse attention of `n_blocks_sample` query blocks; scaled to all heads, blocks and layers."""
+    in full (stack hidden state), and for `n_heads_sample` heads of ONE layer the residual codec on all
+    active rows and the sparse attention of `n_blocks_sample` query blocks (0 = all); scaled to all heads,
+    blocks and layers."""
     import torch
     from oracle import flashloop_oracle as fo
     from paper_2609_29812_b200 import workloads
@@ -491,47 +495,57 @@ def oracle_sample(w, n_blocks_sample=2, seed=0):
         _, cand = fo.select_tokens(G[r - 2], G[r - 1], cand, w.k_tokens, w.eps)
         act_sets.append(cand)
     t_tok = time.time() - t0
-    # one layer, one head
     gen = stack.layer(0)
-    q1, k1, v1 = [f(t)[:, :1, :].copy() for t in gen.qkv1()]
-    blocks = sorted(set(int(b) for b in np.linspace(nb // 3, nb - 1, n_blocks_sample)))
-    d1 = fo.dense_loop_attention(q1, k1, v1, w.sm_scale, w.q_block, rows_to_cache=act_sets[0], head_list=[0],
-                                 block_list=blocks)                       # set-up (dense source), not timed
-    sets, cache = {}, {}
-    for b in range(nb):
-        sets[(0, b)] = np.zeros(0, dtype=np.int64); cache[(0, b)] = (np.zeros(0, dtype=np.int64), np.zeros((0, 0)))
-    for b in blocks:
-        end = min(L, (b + 1) * w.q_block)
-        S = fo.select_columns(d1["col_scores"][0, b, :end], np.arange(end), w.col_budget)
-        rows, P = d1["probs"][(0, b)]
-        sets[(0, b)] = S; cache[(0, b)] = (rows, P[:, S])
-    khat, vhat = k1.astype(np.float32), v1.astype(np.float32)
-    o_full = d1["O"]
+    n_heads_sample = max(1, min(n_heads_sample, w.n_heads))
+    if n_blocks_sample <= 0 or n_blocks_sample >= nb:
+        blocks = list(range(nb))
+    else:
+        blocks = sorted(set(int(b) for b in np.linspace(nb // 3, nb - 1, n_blocks_sample)))
+    qkv1 = [f(t) for t in gen.qkv1()]
+    rows_r = {r: [f(t) for t in gen.rows(r, torch.from_numpy(act_sets[r - 2].astype(np.int32)))]
+              for r in range(2, R + 1)}
     t_quant = t_attn = 0.0
-    for r in range(2, R + 1):
-        act = act_sets[r - 2]
-        qr, kr, vr = [f(t)[:, :1, :].copy() for t in gen.rows(r, torch.from_numpy(act.astype(np.int32)))]
-        t0 = time.time()
-        khat_new, _ = fo.residual_update(kr, khat, act, w.bits, w.group)
-        vhat_new, _ = fo.residual_update(vr, vhat, act, w.bits, w.group)
-        t_quant += time.time() - t0
-        t0 = time.time()
-        res = fo.sparse_loop_attention(qr, khat_new, vhat_new, vhat, o_full[act], act, sets, cache, w.sm_scale,
-                                       w.q_block, head_list=[0], block_list=blocks, kv_round=fo.round_bf16)
-        t_attn += time.time() - t0
-        o_full = o_full.copy(); o_full[act] = res["O"]
-        cache = {key: (res["probs"][key] if key[1] in blocks else cache[key]) for key in cache}
-        khat, vhat = khat_new, vhat_new
-    total = t_tok + w.n_layers * w.n_heads * (t_quant + t_attn * nb / len(blocks))
+    for h in range(n_heads_sample):
+        q1, k1, v1 = [t[:, h:h + 1, :].copy() for t in qkv1]
+        d1 = fo.dense_loop_attention(q1, k1, v1, w.sm_scale, w.q_block, rows_to_cache=act_sets[0], head_list=[0],
+                                     block_list=blocks)                   # set-up (dense source), not timed
+        sets, cache = {}, {}
+        for b in range(nb):
+            sets[(0, b)] = np.zeros(0, dtype=np.int64)
+            cache[(0, b)] = (np.zeros(0, dtype=np.int64), np.zeros((0, 0)))
+        for b in blocks:
+            end = min(L, (b + 1) * w.q_block)
+            S = fo.select_columns(d1["col_scores"][0, b, :end], np.arange(end), w.col_budget)
+            rows, P = d1["probs"][(0, b)]
+            sets[(0, b)] = S; cache[(0, b)] = (rows, P[:, S])
+        khat, vhat = k1.astype(np.float32), v1.astype(np.float32)
+        o_full = d1["O"]
+        for r in range(2, R + 1):
+            act = act_sets[r - 2]
+            qr, kr, vr = [t[:, h:h + 1, :].copy() for t in rows_r[r]]
+            t0 = time.time()
+            khat_new, _ = fo.residual_update(kr, khat, act, w.bits, w.group)
+            vhat_new, _ = fo.residual_update(vr, vhat, act, w.bits, w.group)
+            t_quant += time.time() - t0
+            t0 = time.time()
+            res = fo.sparse_loop_attention(qr, khat_new, vhat_new, vhat, o_full[act], act, sets, cache, w.sm_scale,
+                                           w.q_block, head_list=[0], block_list=blocks, kv_round=fo.round_bf16)
+            t_attn += time.time() - t0
+            o_full = o_full.copy(); o_full[act] = res["O"]
+            cache = {key: (res["probs"][key] if key[1] in blocks else cache[key]) for key in cache}
+            khat, vhat = khat_new, vhat_new
+    per_head = (t_quant + t_attn * nb / len(blocks)) / n_heads_sample
+    total = t_tok + w.n_layers * w.n_heads * per_head
     cores = os.cpu_count() or 1
     try:
         cores = len(os.sched_getaffinity(0))
     except Exception:
         pass
     return {"value": L / total, "unit": UNIT, "cores": cores, "kind": "oracle",
-            "sample": f"token selection of loops 2..{R} in full ({t_tok:.2f} s); one head of one layer: residual codec on all "
-                      f"active rows ({t_quant:.2f} s) and sparse attention of {len(blocks)} of {nb} query blocks "
-                      f"({t_attn:.2f} s); scaled by heads x blocks x layers = {total:.1f} s per prompt",
+            "sample": f"token selection of loops 2..{R} in full ({t_tok:.2f} s); {n_heads_sample} of {w.n_heads} heads of one "
+                      f"of {w.n_layers} layers: residual codec on all active rows ({t_quant:.2f} s) and sparse attention of "
+                      f"{len(blocks)} of {nb} query blocks ({t_attn:.2f} s); scaled by heads x blocks x layers = "
+                      f"{total:.1f} s per prompt",
             "measured_s": t_tok + t_quant + t_attn, "setup_s": time.time() - t_setup - (t_tok + t_quant + t_attn)}
 
 
@@ -545,7 +559,7 @@ def run_reference(args):
         return
     w = get_workload(args)
     for _ in range(min(args.warmup, 1)):
-        oracle_sample(w, n_blocks_sample=1)
+        oracle_sample(w, n_heads_sample=1, n_blocks_sample=1)
     vals = []
     steps = max(1, args.steps)
     t_all = time.time()

@@ -7,7 +7,7 @@
 #include "fl_internal.cuh"
 
 struct fl_tmap_cache {
-  struct Entry { const void* base; int64_t rows, row_elems; CUtensorMap map; };
+  struct Entry { const void* base; int64_t rows, row_elems; int box_rows; CUtensorMap map; };
   std::vector<Entry> entries;
   size_t next = 0;
 };
@@ -16,22 +16,23 @@ typedef CUresult (*fl_encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint
                                        const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                        CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-bool fl_row_gather_tmap(fl_ctx* ctx, const void* base, int64_t rows, int64_t row_elems, CUtensorMap* out) {
+bool fl_tile_tmap(fl_ctx* ctx, const void* base, int64_t rows, int64_t row_elems, int box_rows, CUtensorMap* out) {
   if (ctx->encode_tiled == nullptr || ctx->tmaps == nullptr) return false;
+  if (rows < 1 || box_rows < 1 || box_rows > 256 || !fl_aligned16(base) || (row_elems * 2) % 16 != 0) return false;
   for (const auto& e : ctx->tmaps->entries)
-    if (e.base == base && e.rows == rows && e.row_elems == row_elems) { *out = e.map; return true; }
+    if (e.base == base && e.rows == rows && e.row_elems == row_elems && e.box_rows == box_rows) { *out = e.map; return true; }
   fl_tmap_cache::Entry e;
-  e.base = base; e.rows = rows; e.row_elems = row_elems;
+  e.base = base; e.rows = rows; e.row_elems = row_elems; e.box_rows = box_rows;
   const cuuint64_t gdim[2] = {(cuuint64_t)row_elems, (cuuint64_t)rows};
   const cuuint64_t gstride[1] = {(cuuint64_t)row_elems * 2};
-  const cuuint32_t box[2] = {64, 1};
+  const cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
   const cuuint32_t estr[2] = {1, 1};
   const CUresult rc = reinterpret_cast<fl_encode_tiled_fn>(ctx->encode_tiled)(
       &e.map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstride, box, estr,
       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (rc != CUDA_SUCCESS) return false;
-  constexpr size_t kMaxEntries = 512;   // ring replacement: 48 layers x (K, V) fit several times over
+  constexpr size_t kMaxEntries = 1024;  // ring replacement: 48 layers x (K, V, Q of three loops) fit twice over
   if (ctx->tmaps->entries.size() < kMaxEntries) ctx->tmaps->entries.push_back(e);
   else { ctx->tmaps->entries[ctx->tmaps->next] = e; ctx->tmaps->next = (ctx->tmaps->next + 1) % kMaxEntries; }
   *out = e.map;

@@ -16,13 +16,14 @@ struct fl_ctx {
   size_t workspace_bytes;
   int force_simt;  // environment FL_FORCE_SIMT=1 at fl_create: keep attention on the binary32 SIMT kernels
   void* encode_tiled;       // cuTensorMapEncodeTiled, resolved through cudaGetDriverEntryPoint (may be null)
-  struct fl_tmap_cache* tmaps;  // row-gather tensor maps, keyed by (base pointer, rows, row elements)
+  struct fl_tmap_cache* tmaps;  // tensor maps, keyed by (base pointer, rows, row elements, box rows)
 };
 
-// Tensor map for gathering rows of a row-major bf16 matrix [rows, row_elems] with TMA (tile::gather4):
-// box = 64 elements x 1 row, 128-byte swizzle, out-of-range rows read as zero. Cached per context.
+// Tensor map of a row-major bf16 matrix [rows, row_elems] for TMA: box = 64 elements x box_rows rows,
+// 128-byte swizzle, out-of-range rows read as zero. box_rows = 1 is the map for row gathers (tile::gather4),
+// box_rows = 128 loads one slab of a compact Q tile. Cached per context.
 // Returns false if tensor maps are not available (caller falls back to a non-TMA kernel).
-bool fl_row_gather_tmap(fl_ctx* ctx, const void* base, int64_t rows, int64_t row_elems, CUtensorMap* out);
+bool fl_tile_tmap(fl_ctx* ctx, const void* base, int64_t rows, int64_t row_elems, int box_rows, CUtensorMap* out);
 
 #define FL_CHECK_CUDA(expr)                    \
   do {                                         \

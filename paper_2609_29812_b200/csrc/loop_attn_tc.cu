@@ -4,13 +4,14 @@
 //
 // Warp roles (16 warps, 512 threads):
 //   warps 0-3   softmax of the OLD term  (fixed normaliser lse_prev: p_old = exp(s_old - lse_prev), mass m_i)
-//   warps 4-7   softmax of the NEW term  (running reference with lazy rescale of the accumulator)
-//   warp  8     one thread issues the S = Q Khat^T MMAs; the warp owns the tensor-memory allocation
-//   warp  9     one thread issues the acc += P Vhat MMAs (a single thread cannot issue 64-column MMAs as fast
-//               as the tensor pipe retires them; two issuers keep it fed)
-//   warps 10-13 TMA: row gathers (cp.async.bulk.tensor tile::gather4, 4 selected columns per copy) of the bf16
-//               base K/V rows straight into 128B-swizzled operand tiles; completion on mbarriers
-//   warps 14-15 patch: stage the Q tiles; for the columns that carry residual payloads, overwrite the gathered
+//   warps 4-7   softmax of the NEW term  (running reference, lazy rescale of the accumulator)
+//   warps 8-11  MMA issuers, one thread each: S_old = Q_old Khat_old^T, S_new = Q_new Khat_new^T,
+//               acc_old += P_old Vhat_old, acc_new += P_new Vhat_new. A single thread issues a 128x64x16 MMA
+//               every ~60-90 cycles while the tensor pipe retires one in 48, so the four streams of MMAs are
+//               issued from four warps on four different schedulers.
+//   warps 12-15 TMA + patch: the Q tiles (two 2-D tile loads each), row gathers (cp.async.bulk.tensor
+//               tile::gather4, 4 selected columns per copy) of the bf16 base K/V rows straight into 128B-swizzled
+//               operand tiles, and for the columns that carry residual payloads the overwrite of the gathered
 //               base rows with the dequantize-and-add result (Eq. 8)
 //
 // Prologue (whole CTA): the block's causal column list is copied to shared memory together with a bit mask
@@ -18,12 +19,13 @@
 // the current loop (Khat_old == Khat_new, one K tile and one V tile serve both terms) followed by columns
 // WITH one (separate old / new tiles). Most columns are of the first kind and are a plain gather.
 //
-// Per chunk of 64 columns:  S_old = Q_old Khat_old^T, S_new = Q_new Khat_new^T  (SS MMAs, f32 in TMEM),
-// P = softmax pieces written back to TMEM as bf16, then acc_old += P_old Vhat_old, acc_new += P_new Vhat_new
-// (TS MMAs, V as MN-major operand). Epilogue: O = O_prev - acc_old + (m / l) acc_new.
+// Per chunk of 64 columns and per term: S (f32, 64 tensor-memory columns, ONE buffer: the softmax warps pull it
+// into registers and hand the buffer back at once, so the next chunk's QK^T runs under the current chunk's
+// exponentials), P (bf16, 32 columns, two buffers: PV of a chunk runs under the next chunk's exponentials).
+// The two terms are independent pipelines. Epilogue: O = O_prev - acc_old + (m / l) acc_new.
 // Shared memory: Q_old, Q_new tiles (64 KB) + a ring of four 32 KB operand slots (K tile | V tile); a chunk of
 // the first kind takes one slot, of the second kind two. Tensor memory (512 columns): acc_old 0-127,
-// acc_new 128-255, two S/P buffers of 128 columns.
+// acc_new 128-255, S_old 256-319, S_new 320-383, P_old 384-447, P_new 448-511.
 // Every mbarrier wait is bounded; on a timeout the CTA raises a flag, drains and reports FL_ERR_TIMEOUT.
 #include "fl_internal.cuh"
 #include "tc_ptx.cuh"
@@ -38,19 +40,22 @@ constexpr int kTileBytes = kNC * kDH * 2;   // 16 KB
 constexpr int kSlotBytes = 2 * kTileBytes;  // K tile | V tile
 constexpr int kQTileBytes = kM * kDH * 2;   // 32 KB
 constexpr int kSoftmaxWarps = 8;
-constexpr int kMmaWarp = 8;
-constexpr int kPvWarp = 9;         // second MMA issuer (the first, kMmaWarp, issues QK^T)
-constexpr int kTmaWarp = 10;       // first of the TMA warps
+constexpr int kIssueWarp = 8;      // warps 8..11: QK old, QK new, PV old, PV new
+constexpr int kTmaWarp = 12;       // first of the TMA / patch warps
 constexpr int kTmaWarps = 4;       // a single warp cannot issue four-row gathers fast enough; four come close
-constexpr int kPatchWarps = 2;
-constexpr int kWarps = kSoftmaxWarps + 2 + kTmaWarps + kPatchWarps;  // 16
+constexpr int kWarps = kSoftmaxWarps + 4 + kTmaWarps;  // 16
 constexpr int kThreads = kWarps * 32;
-constexpr int kPatchThreads = kPatchWarps * 32;
+constexpr int kColWarps = 14;               // warps that read the column list in the prologue (the other two search rows)
 constexpr int kMaxCols = 3072;              // column budget the shared-memory column list can hold
-constexpr uint32_t kAccOld = 0, kAccNew = 128, kSBase = 256;
+constexpr int kMaxChunks = kMaxCols / kNC + 2;
+constexpr int kPrefillChunks = 2;   // patched chunks the whole CTA builds at the start of a row tile (4 ring slots)
+constexpr int kPreStreams = 4;      // ... when the loop has at most this many residual streams (their slot lookups are
+                                    // kept from the prologue); deeper loops leave every patched chunk to the patch warps
+constexpr uint32_t kAccOld = 0, kAccNew = 128, kSOld = 256, kSNew = 320, kPOld = 384, kPNew = 448;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRescaleThreshold = 60.f;   // in log2 units: rescale only when the reference falls this far behind
+static_assert((2 + kPreStreams) * kMaxCols * 4 <= kSlots * kSlotBytes, "prologue staging must fit in the ring");
 
 // Optional device-side timeline for tuning (compile with -DFL_TC_TRACE): the CTA (block 1, head 0) writes
 // clock64() stamps into the buffer passed as `status`: trace[(role * 64 + chunk) * 4 + event].
@@ -65,9 +70,8 @@ constexpr float kRescaleThreshold = 60.f;   // in log2 units: rescale only when 
 #endif
 
 struct alignas(64) TcArgs {
-  CUtensorMap k_map, v_map;   // row-gather maps of the K / V base ([L, d] bf16, box 64 x 1, 128B swizzle)
-  const __nv_bfloat16* q_new;
-  const __nv_bfloat16* q_old;
+  CUtensorMap k_map, v_map;          // row-gather maps of the K / V base ([L, d] bf16, box 64 x 1, 128B swizzle)
+  CUtensorMap q_new_map, q_old_map;  // tile maps of the compact Q rows ([n_active, d] bf16, box 64 x 128)
   const __nv_bfloat16* o_prev;
   __nv_bfloat16* o_out;
   const int32_t* active_idx;
@@ -86,21 +90,22 @@ struct alignas(64) TcArgs {
 
 struct __align__(16) TcSmemCtl {
   uint64_t landed[kSlots];   // TMA -> everyone: the slot's gathered tiles (32 KB) have arrived
-  uint64_t patched[kSlots];  // patch warps -> MMA: residual-carrying columns of the slot are rewritten (dirty chunks only)
-  uint64_t done[kSlots];     // MMA -> TMA / softmax: the MMAs that read the slot have finished
-  uint64_t q_full;           // patch warps -> MMA: the Q tiles of the current row tile are staged
-  uint64_t s_full[2];      // MMA -> softmax: S of the chunk is in tensor memory
-  uint64_t p_full[2];      // softmax -> MMA: P of the chunk is in tensor memory
-  uint64_t s_free[2];      // PV issuer -> QK issuer: the PV MMAs that read P from the buffer have finished
-  uint64_t acc_done;       // MMA -> softmax: all accumulation of the tile finished
+  uint64_t patched[kSlots];  // patch -> QK issuers: residual-carrying columns of the slot are rewritten (dirty chunks only)
+  uint64_t done[kSlots];     // the four issuers -> TMA: the MMAs that read the slot have finished
+  uint64_t q_full;           // TMA -> QK issuers: the Q tiles of the current row tile have arrived
+  uint64_t s_full[2];        // QK issuer -> softmax (per term): S of the chunk is in tensor memory
+  uint64_t s_taken[2];       // softmax -> QK issuer: S of the chunk is in registers, the buffer may be overwritten
+  uint64_t p_full[2][2];     // softmax -> PV issuer (per term, per P buffer): P of the chunk is in tensor memory
+  uint64_t p_free[2][2];     // PV issuer -> softmax: the PV MMAs that read the P buffer have finished
+  uint64_t acc_done;         // PV issuers -> softmax: all accumulation of the tile finished
   uint32_t tmem_base;
   int abort_flag;
-  int q_lo, q_hi;          // block's slot range in active_idx
-  int n_plain, n_patch;    // columns without / with a payload in the current loop
+  int q_lo, q_hi, i_last;    // block's slot range in active_idx, position of its last active row
+  int n_plain, n_patch;      // columns without / with a payload in the current loop
   int warp_cnt[kWarps][2];
-  int col_pos[kSlots][kNC];
-  int col_last[kSlots];    // largest column position of the chunk, INT32_MAX if the chunk is padded
-  uint32_t chunk_mask[kMaxCols / kNC + 2];  // OR of the stream masks of the chunk's columns (0: plain gather only)
+  int chunk_last[kMaxChunks];       // largest column position of the chunk, INT32_MAX if the chunk is padded
+  uint32_t chunk_mask[kMaxChunks];  // OR of the stream masks of the chunk's columns (0: plain gather only)
+  int pre_slot[kPreStreams][kPrefillChunks * kNC];  // stream rows of the first patched columns (-1: none)
   float mass[kM];
   float ell[kM];
   float ref[kM];
@@ -109,18 +114,13 @@ struct __align__(16) TcSmemCtl {
 constexpr size_t kTcSmemBytes = 1024 /* alignment slack */ + 2 * kQTileBytes + kSlots * kSlotBytes + sizeof(TcSmemCtl) +
                                 2 * kMaxCols * sizeof(int32_t);
 
-// Bounded wait of a fully converged warp: lane 0 polls, the verdict is shared, and every lane then observes
-// the completed phase itself (one immediate poll) so that it acquires what the arriving threads released.
+// Bounded wait of a fully converged warp; every lane observes the completed phase itself, so each acquires
+// what the arriving threads released. Returns a warp-uniform verdict.
 __device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-  bool ok = true;
-  if ((threadIdx.x & 31) == 0) ok = tc::mbar_wait(bar, parity, abort_flag);
-  ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-  if (ok) {
-    bool seen = false;
-    for (int it = 0; it < 1024 && !seen; ++it) seen = tc::mbar_try_wait(bar, parity);
-    ok = __all_sync(0xffffffffu, seen);
-  }
-  return ok;
+  bool ok = tc::mbar_try_wait(bar, parity);
+  if (__all_sync(0xffffffffu, ok)) return true;
+  if (!ok) ok = tc::mbar_wait(bar, parity, abort_flag);
+  return __all_sync(0xffffffffu, ok);
 }
 
 // first index in the ascending array with value >= target; all 32 lanes cooperate (32-ary search)
@@ -164,13 +164,54 @@ __device__ __forceinline__ void patch_piece(const DevSide& side, int n_old, uint
                                          int group, const uint4& raw, uint4& v_old, uint4& v_new) {
   float x[8];
   unpack8(raw, x);
-  for (int s = 0; s < n_old; ++s)
+  v_old = raw;
+#pragma unroll 1
+  for (int s = 0; s <= n_old; ++s) {
+    if (s == n_old && (mask & ((1u << n_old) - 1u))) v_old = pack8(x);
     if ((mask >> s) & 1u) apply_stream8<__nv_bfloat16, BITS>(side.s[s], j, elem, d, group, x);
-  v_old = (mask & ((1u << n_old) - 1u)) ? pack8(x) : raw;
-  v_new = v_old;
-  if ((mask >> n_old) & 1u) {
-    apply_stream8<__nv_bfloat16, BITS>(side.s[n_old], j, elem, d, group, x);
-    v_new = pack8(x);
+  }
+  v_new = ((mask >> n_old) & 1u) ? pack8(x) : v_old;
+}
+
+// One stream's payload for 8 consecutive elements, fetched ahead of its use so that the loads of several
+// columns and streams are in flight together (the cooperative build of the first residual-carrying chunks).
+template <int BITS>
+struct Payload8 {
+  uint4 raw;      // BITS 16: the stored row piece; 8: x,y; 4 and 2: x
+  float sc, zr;
+};
+template <int BITS>
+__device__ __forceinline__ void payload_load(const DevStream& st, int slot, int elem, int d, int group, Payload8<BITS>& p) {
+  if (BITS == 16) {
+    p.raw = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(st.codes) + (size_t)slot * d + elem));
+  } else {
+    const uint8_t* row = st.codes + (size_t)slot * (d * BITS / 8);
+    if (BITS == 8) {
+      const uint2 t = __ldg(reinterpret_cast<const uint2*>(row + elem));
+      p.raw.x = t.x; p.raw.y = t.y;
+    } else if (BITS == 4) {
+      p.raw.x = __ldg(reinterpret_cast<const uint32_t*>(row + elem / 2));
+    } else {
+      p.raw.x = __ldg(reinterpret_cast<const uint16_t*>(row + elem / 4));
+    }
+    const size_t gi = (size_t)slot * (d / group) + elem / group;
+    p.sc = __half2float(__ldg(st.scale + gi));
+    p.zr = __half2float(__ldg(st.zero + gi));
+  }
+}
+template <int BITS>
+__device__ __forceinline__ void payload_apply(const Payload8<BITS>& p, float (&x)[8]) {
+  if (BITS == 16) {
+    unpack8(p.raw, x);
+  } else {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      uint32_t c;
+      if (BITS == 8) c = ((i < 4 ? p.raw.x : p.raw.y) >> (8 * (i & 3))) & 0xFFu;
+      else if (BITS == 4) c = (p.raw.x >> (4 * i)) & 0xFu;
+      else c = (p.raw.x >> (2 * i)) & 0x3u;
+      x[i] = __fadd_rn(x[i], __fmaf_rn((float)c, p.sc, p.zr));
+    }
   }
 }
 
@@ -196,7 +237,6 @@ __device__ __forceinline__ ChunkInfo chunk_info(int ci, int n_plain, int n_patch
   }
   return c;
 }
-constexpr int kPrefillChunks = 2;   // patched chunks the whole CTA builds at the start of a row tile (4 ring slots)
 
 template <int BITS>
 __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_constant__ TcArgs a) {
@@ -214,30 +254,49 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
   const size_t prob = (size_t)h * a.nb + b;
   const int32_t* cols = a.col_idx + prob * a.c;
   const int cnt = min(__ldg(a.col_cnt + prob), kMaxCols);
+  if (tid == 0) TC_TRACE(0, 60, 0);
 
   if (tid == 0) {
     for (int s = 0; s < kSlots; ++s) {
       tc::mbar_init(&ctl.landed[s], kTmaWarps);
-      tc::mbar_init(&ctl.patched[s], kPatchWarps);
-      tc::mbar_init(&ctl.done[s], 1);
+      tc::mbar_init(&ctl.patched[s], kTmaWarps);
+      tc::mbar_init(&ctl.done[s], 4);
     }
-    tc::mbar_init(&ctl.q_full, kPatchThreads);
-    for (int s = 0; s < 2; ++s) {
-      tc::mbar_init(&ctl.s_full[s], 1);
-      tc::mbar_init(&ctl.p_full[s], kSoftmaxWarps * 32);
-      tc::mbar_init(&ctl.s_free[s], 1);
+    tc::mbar_init(&ctl.q_full, 1);
+    for (int t = 0; t < 2; ++t) {
+      tc::mbar_init(&ctl.s_full[t], 1);
+      tc::mbar_init(&ctl.s_taken[t], 4);
+      for (int pb = 0; pb < 2; ++pb) {
+        tc::mbar_init(&ctl.p_full[t][pb], 4);
+        tc::mbar_init(&ctl.p_free[t][pb], 1);
+      }
     }
-    tc::mbar_init(&ctl.acc_done, 1);
+    tc::mbar_init(&ctl.acc_done, 2);
     ctl.abort_flag = 0;
     tc::fence_barrier_init();
   }
-  // ---- rows of this block: 32-ary searches in the ascending active list (warps 0 and 1) ----------------
-  if (warp < 2) {
-    const int target = warp == 0 ? b * a.q_block : min(a.L, (b + 1) * a.q_block);
+  for (int i = tid; i < kMaxChunks; i += kThreads) ctl.chunk_mask[i] = 0;
+  // ---- prologue (rolled loops throughout: code that runs once per CTA is paid for in instruction fetches) ----
+  // The raw column list, its stream rows and stream masks are staged in the still idle ring.
+  int32_t* raw_col = reinterpret_cast<int32_t*>(ring);                     // [kMaxCols]
+  uint32_t* raw_mask = reinterpret_cast<uint32_t*>(raw_col + kMaxCols);    // [kMaxCols]
+  int32_t* raw_slot = reinterpret_cast<int32_t*>(raw_mask + kMaxCols);     // [kPreStreams][kMaxCols]
+  if (warp >= kColWarps) {
+    // warps 14 and 15 search the block's rows in the ascending active list meanwhile
+    const int target = warp == kColWarps ? b * a.q_block : min(a.L, (b + 1) * a.q_block);
     const int r = lower_bound32(a.active_idx, a.n_active, target, lane);
-    if (lane == 0) { if (warp == 0) ctl.q_lo = r; else ctl.q_hi = r; }
+    if (lane == 0) {
+      if (warp == kColWarps) ctl.q_lo = r;
+      else { ctl.q_hi = r; ctl.i_last = r > 0 ? __ldg(a.active_idx + r - 1) : -1; }
+    }
+  } else {
+#pragma unroll 1
+    for (int u = tid; u < cnt; u += kColWarps * 32) {
+      raw_col[u] = __ldg(cols + u);
+      raw_mask[u] = 0;
+    }
   }
-  if (warp == kMmaWarp) {
+  if (warp == kIssueWarp) {
     tc::tmem_alloc(&ctl.tmem_base, 512);
     tc::tmem_relinquish();
   }
@@ -248,48 +307,84 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
   volatile int* abort_flag = &ctl.abort_flag;
   const int q_lo = ctl.q_lo, q_hi = ctl.q_hi;
   if (q_hi > q_lo) {   // CTA-uniform: blocks without active rows only release the tensor memory
-  // ---- column list of the block: causal prefix, stream masks, stable partition -------------------------
   {
-    const int i_last = __ldg(a.active_idx + q_hi - 1);            // last active row of the block
-    const int span = ((cnt + kWarps - 1) / kWarps + 31) & ~31;     // contiguous span per warp, multiple of 32
+    // every (column, stream) pair is one independent slot-map lookup
+#pragma unroll 1
+    for (int p2 = tid; p2 < cnt * (a.n_old + 1); p2 += kThreads) {
+      const int s = p2 / cnt, u = p2 - s * cnt;
+      const int sl = __ldg(a.k.s[s].slot + raw_col[u]);
+      if (sl >= 0) atomicOr(&raw_mask[u], 1u << s);
+      if (s < kPreStreams) raw_slot[s * kMaxCols + u] = sl;
+    }
+    __syncthreads();
+    // causal prefix, stable partition into plain / patched columns: every warp owns a contiguous span
+    const int i_last = ctl.i_last;                                   // last active row of the block
+    const int span = ((cnt + kWarps - 1) / kWarps + 31) & ~31;
     const int beg = warp * span, end = min(cnt, beg + span);
-    int n0 = 0, n1 = 0;                                            // plain / patched columns in this warp's span
+    int n0 = 0, n1 = 0;                                              // plain / patched columns in this warp's span
+#pragma unroll 1
     for (int base = beg; base < end; base += 32) {
       const int u = base + lane;
-      const int j = u < end ? __ldg(cols + u) : INT32_MAX;
-      const bool live = j <= i_last;
-      const bool patched = live && __ldg(a.k.s[a.n_old].slot + j) >= 0;
+      const bool live = u < end && raw_col[u] <= i_last;
+      const bool patched = live && ((raw_mask[u] >> a.n_old) & 1u);
       n0 += __popc(__ballot_sync(0xffffffffu, live && !patched));
       n1 += __popc(__ballot_sync(0xffffffffu, patched));
     }
     if (lane == 0) { ctl.warp_cnt[warp][0] = n0; ctl.warp_cnt[warp][1] = n1; }
     __syncthreads();
     int before0 = 0, before1 = 0, tot0 = 0, tot1 = 0;
+#pragma unroll 1
     for (int wv = 0; wv < kWarps; ++wv) {
       const int c0 = ctl.warp_cnt[wv][0], c1 = ctl.warp_cnt[wv][1];
       if (wv < warp) { before0 += c0; before1 += c1; }
       tot0 += c0; tot1 += c1;
     }
     if (tid == 0) { ctl.n_plain = tot0; ctl.n_patch = tot1; }
-    for (int i = tid; i < kMaxCols / kNC + 2; i += kThreads) ctl.chunk_mask[i] = 0;
-    __syncthreads();
     const int patch_chunks = (tot1 + kNC - 1) / kNC;
+    const uint32_t lt = (1u << lane) - 1;
+#pragma unroll 1
     for (int base = beg; base < end; base += 32) {
       const int u = base + lane;
-      const int j = u < end ? __ldg(cols + u) : INT32_MAX;
+      const int j = u < end ? raw_col[u] : INT32_MAX;
+      const uint32_t mask = u < end ? raw_mask[u] : 0u;
       const bool live = j <= i_last;
-      uint32_t mask = 0;
-      if (live)
-        for (int s = 0; s <= a.n_old; ++s) mask |= (__ldg(a.k.s[s].slot + j) >= 0 ? 1u : 0u) << s;
       const bool patched = live && ((mask >> a.n_old) & 1u);
       const uint32_t m0 = __ballot_sync(0xffffffffu, live && !patched);
       const uint32_t m1 = __ballot_sync(0xffffffffu, patched);
-      const uint32_t lt = (1u << lane) - 1;
       if (live) {
         const int dst = patched ? tot0 + before1 + __popc(m1 & lt) : before0 + __popc(m0 & lt);
         ord_col[dst] = j;
         ord_mask[dst] = mask;
         if (mask != 0) atomicOr(&ctl.chunk_mask[patched ? (dst - tot0) / kNC : patch_chunks + dst / kNC], mask);
+        if (patched && dst - tot0 < kPrefillChunks * kNC && a.n_old < kPreStreams) {
+          // one of the columns the whole CTA builds next: keep its stream rows and pull its base rows and
+          // payloads towards the L2 now, so that the build finds them there
+          const int pr = dst - tot0;
+          const size_t row_off = ((size_t)j * a.d + (size_t)h * kDH) * 2;
+          tc::prefetch_l2(static_cast<const uint8_t*>(a.k.base) + row_off);
+          tc::prefetch_l2(static_cast<const uint8_t*>(a.k.base) + row_off + 128);
+          tc::prefetch_l2(static_cast<const uint8_t*>(a.v.base) + row_off);
+          tc::prefetch_l2(static_cast<const uint8_t*>(a.v.base) + row_off + 128);
+#pragma unroll 1
+          for (int s = 0; s < kPreStreams; ++s) {
+            const int sl = s <= a.n_old ? raw_slot[s * kMaxCols + u] : -1;
+            ctl.pre_slot[s][pr] = sl;
+            if (sl >= 0) {
+              const size_t code_off = BITS == 16 ? ((size_t)sl * a.d + (size_t)h * kDH) * 2
+                                                 : (size_t)sl * (a.d * BITS / 8) + (size_t)h * (kDH * BITS / 8);
+              tc::prefetch_l2(a.k.s[s].codes + code_off);
+              tc::prefetch_l2(a.v.s[s].codes + code_off);
+              if (BITS == 16) {
+                tc::prefetch_l2(a.k.s[s].codes + code_off + 128);
+                tc::prefetch_l2(a.v.s[s].codes + code_off + 128);
+              } else {
+                const size_t gi = (size_t)sl * (a.d / a.group) + (size_t)h * (kDH / a.group);
+                tc::prefetch_l2(a.k.s[s].scale + gi); tc::prefetch_l2(a.k.s[s].zero + gi);
+                tc::prefetch_l2(a.v.s[s].scale + gi); tc::prefetch_l2(a.v.s[s].zero + gi);
+              }
+            }
+          }
+        }
       }
       before0 += __popc(m0);
       before1 += __popc(m1);
@@ -298,7 +393,12 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
   }
   const int n_plain = ctl.n_plain, n_patch = ctl.n_patch;
   const int n_chunks = (n_plain + kNC - 1) / kNC + (n_patch + kNC - 1) / kNC;
-  int g = 0;    // chunks issued so far (all tiles): S/P buffer = g & 1, phase = (g >> 1) & 1
+  for (int ci = tid; ci < n_chunks; ci += kThreads) {
+    const ChunkInfo ck = chunk_info(ci, n_plain, n_patch);
+    ctl.chunk_last[ci] = ck.n_valid == kNC ? ord_col[ck.off + kNC - 1] : INT32_MAX;
+  }
+  if (tid == 0) TC_TRACE(0, 60, 1);
+  int g = 0;    // chunks issued so far (all tiles): one phase of s_full / s_taken per chunk, P buffer = g & 1
   int fill = 0; // ring slots filled so far: slot = fill % kSlots, phase = (fill / kSlots) & 1
   uint32_t dirty_par_cta = 0;  // per-slot phase parity of the patched[] barriers (they only see dirty chunks)
 
@@ -306,71 +406,96 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
   const int n_rows = min(kM, q_hi - s0);
   const int g0 = g, fill0 = fill;
   const uint32_t dirty_par0 = dirty_par_cta;
-  const int n_pre = min((n_patch + kNC - 1) / kNC, kPrefillChunks);
+  const int n_pre = a.n_old < kPreStreams ? min((n_patch + kNC - 1) / kNC, kPrefillChunks) : 0;
+  if (tid == kTmaWarp * 32) {
+    // Q tiles of this row tile: two 64-element slabs each; rows past the compact list read as zero, rows of the
+    // next block (past n_rows) are computed and dropped
+    tc::mbar_arrive_expect_tx(&ctl.q_full, 2 * kQTileBytes);
+    tc::tma_tile2d(q_old_tile, &a.q_old_map, &ctl.q_full, h * kDH, s0);
+    tc::tma_tile2d(q_old_tile + kM * 128, &a.q_old_map, &ctl.q_full, h * kDH + 64, s0);
+    tc::tma_tile2d(q_new_tile, &a.q_new_map, &ctl.q_full, h * kDH, s0);
+    tc::tma_tile2d(q_new_tile + kM * 128, &a.q_new_map, &ctl.q_full, h * kDH + 64, s0);
+  }
   // ---- the first patched chunks are built by all 512 threads straight into the (idle) ring: base row plus
-  // dequantized residuals (Eq. 8), old and new operand tiles. Left to the two patch warps this would take an
-  // order of magnitude longer than a plain chunk; done here it costs a few dependent loads per thread.
+  // dequantized residuals (Eq. 8), old and new operand tiles. A warp owns 4 columns of the chunk (lanes 0-15:
+  // the 16 pieces of the K row, lanes 16-31: of the V row); their stream rows were kept by the prologue, so the
+  // base and payload loads of a column pair are one round of independent loads.
   {
-#pragma unroll 2
-    for (int p = tid; p < n_pre * kNC * 32; p += kThreads) {
-      const int pc = p / (kNC * 32), q = p % (kNC * 32);
-      const int u = q >> 5, half = (q >> 4) & 1, ch = q & 15;
+    const int half = lane >> 4, ch = lane & 15;
+    const DevSide& side = half ? a.v : a.k;
+    const int elem = h * kDH + ch * 8;
+    const uint32_t tile_off = half * kTileBytes + (ch >> 3) * (kNC * 128);
+#pragma unroll 1
+    for (int it = 0; it < n_pre * 4; ++it) {
+      const int pc = it >> 2, u = warp + 16 * (it & 3);
       const ChunkInfo ck = chunk_info(pc, n_plain, n_patch);
       const int slot0 = (fill0 + 2 * pc) % kSlots, slot1 = (fill0 + 2 * pc + 1) % kSlots;
-      const uint32_t off = half * kTileBytes + (ch >> 3) * (kNC * 128) + tc::sw128_offset(u, ch & 7);
-      uint4 v_old = make_uint4(0, 0, 0, 0), v_new = make_uint4(0, 0, 0, 0);
-      if (u < ck.n_valid) {
-        const DevSide& side = half ? a.v : a.k;
-        const int j = ord_col[ck.off + u];
-        const int elem = h * kDH + ch * 8;
-        const uint4 base16 =
-            __ldg(reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(side.base) + (size_t)j * a.d + elem));
-        patch_piece<BITS>(side, a.n_old, ord_mask[ck.off + u], j, elem, a.d, a.group, base16, v_old, v_new);
+      const bool valid = u < ck.n_valid;
+      const uint32_t mask = valid ? ord_mask[ck.off + u] : 0u;
+      uint4 raw = make_uint4(0, 0, 0, 0);
+      Payload8<BITS> pl[kPreStreams];
+      int sl[kPreStreams];
+      if (valid)
+        raw = __ldg(reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(side.base) +
+                                                   (size_t)ord_col[ck.off + u] * a.d + elem));
+#pragma unroll
+      for (int s = 0; s < kPreStreams; ++s) {
+        sl[s] = (valid && s <= a.n_old) ? ctl.pre_slot[s][pc * kNC + u] : -1;
+        if (sl[s] >= 0) payload_load<BITS>(side.s[s], sl[s], elem, a.d, a.group, pl[s]);
       }
+      float x[8];
+      unpack8(raw, x);
+      uint4 v_old = raw;
+#pragma unroll
+      for (int s = 0; s < kPreStreams; ++s) {
+        if (s == a.n_old && (mask & ((1u << a.n_old) - 1u))) v_old = pack8(x);
+        if (sl[s] >= 0) payload_apply<BITS>(pl[s], x);
+      }
+      const uint4 v_new = ((mask >> a.n_old) & 1u) ? pack8(x) : v_old;
+      const uint32_t off = tile_off + tc::sw128_offset(u, ch & 7);
       *reinterpret_cast<uint4*>(ring + slot0 * kSlotBytes + off) = v_old;
       *reinterpret_cast<uint4*>(ring + slot1 * kSlotBytes + off) = v_new;
     }
-    for (int p = tid; p < n_pre * kNC; p += kThreads) {
-      const int pc = p / kNC, u = p % kNC;
-      const ChunkInfo ck = chunk_info(pc, n_plain, n_patch);
-      const int slot0 = (fill0 + 2 * pc) % kSlots;
-      ctl.col_pos[slot0][u] = u < ck.n_valid ? ord_col[ck.off + u] : INT32_MAX;
-      if (u == 0) ctl.col_last[slot0] = ck.n_valid == kNC ? ord_col[ck.off + kNC - 1] : INT32_MAX;
-    }
-    tc::fence_proxy_async_smem();
-    __syncthreads();
   }
+  tc::fence_proxy_async_smem();
+  __syncthreads();
+  if (tid == 0) TC_TRACE(0, 60, 2);
 
-  if (warp >= kTmaWarp && warp < kTmaWarp + kTmaWarps) {
-    // ============================================== TMA ==============================================
+  if (warp >= kTmaWarp) {
+    // ========================================== TMA + patch ==========================================
     // In-order fills of the ring; the lookahead is whatever the four slots allow. The 64 four-row gathers
-    // of a slot (K: 2 slabs x 16 groups, V: the same) are split over the TMA warps, 16 each, one per lane;
-    // every warp announces its own share of the bytes on the slot's barrier.
+    // of a slot (K: 2 slabs x 16 groups, V: the same) are split over the four warps, 16 each, one per lane;
+    // every warp announces its own share of the bytes on the slot's barrier. Chunks whose columns carry
+    // residual payloads are then rewritten in place by the same warps (4 columns at a time, lanes 0-15 the K
+    // row, lanes 16-31 the V row).
     const int tw = warp - kTmaWarp;
     const int is_v = tw >> 1, slab = tw & 1, grp = lane & 15;
     const void* map = is_v ? static_cast<const void*>(&a.v_map) : static_cast<const void*>(&a.k_map);
+    const int half = lane >> 4, ch = lane & 15;
+    const DevSide& side = half ? a.v : a.k;
+    const int elem = h * kDH + ch * 8;
+    const __nv_bfloat16* base_rows = static_cast<const __nv_bfloat16*>(side.base) + elem;
+    const uint32_t ch_off = (ch >> 3) * (kNC * 128);
     int f = fill0;
     bool ok = true;
 #pragma unroll 1
     for (int ci = 0; ci < n_chunks && ok; ++ci) {
       const ChunkInfo ck = chunk_info(ci, n_plain, n_patch);
       const int n_slots = ck.patch ? 2 : 1;
-      if (ci < n_pre) {   // built by the whole CTA above: only the barrier phase is left to complete
+      const bool dirty = ctl.chunk_mask[ci] != 0;
+      if (ci < n_pre) {   // built by the whole CTA above: only the barrier phases are left to complete
         if (lane == 0)
-          for (int k = 0; k < n_slots; ++k) tc::mbar_arrive(&ctl.landed[(f + k) % kSlots]);
+          for (int k = 0; k < n_slots; ++k) {
+            tc::mbar_arrive(&ctl.landed[(f + k) % kSlots]);
+            tc::mbar_arrive(&ctl.patched[(f + k) % kSlots]);
+          }
         f += n_slots;
         continue;
       }
       for (int k = 0; k < n_slots && ok; ++k)
         if (f + k >= kSlots) ok = warp_wait(&ctl.done[(f + k) % kSlots], (((f + k) / kSlots) - 1) & 1, abort_flag);
       if (!ok) break;
-      const int slot0 = f % kSlots;
       if (tid == kTmaWarp * 32) TC_TRACE(0, ci, 0);
-      if (tw == 0) {
-        for (int u = lane; u < kNC; u += 32) ctl.col_pos[slot0][u] = u < ck.n_valid ? ord_col[ck.off + u] : INT32_MAX;
-        if (lane == 0) ctl.col_last[slot0] = ck.n_valid == kNC ? ord_col[ck.off + kNC - 1] : INT32_MAX;
-      }
-      __syncwarp();
       if (lane == 0)
         for (int k = 0; k < n_slots; ++k) tc::mbar_arrive_expect_tx(&ctl.landed[(f + k) % kSlots], kSlotBytes / kTmaWarps);
       __syncwarp();
@@ -387,52 +512,15 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
                           &ctl.landed[slot], h * kDH + slab * 64, y[0], y[1], y[2], y[3]);
         }
       }
-      f += n_slots;
       if (tid == kTmaWarp * 32) TC_TRACE(0, ci, 1);
-    }
-  } else if (warp >= kTmaWarp + kTmaWarps) {
-    // ============================================= patch =============================================
-    const int pt = tid - (kTmaWarp + kTmaWarps) * 32;   // 0..95
-    const int pw = pt >> 5;
-    // Q tiles (once per row tile): asynchronous 16-byte copies
-    for (int it = pt; it < 2 * kM * 16; it += kPatchThreads) {
-      const int which = it / (kM * 16);
-      const int rem = it % (kM * 16);
-      const int r = rem >> 4, ch = rem & 15;
-      uint8_t* dst = (which ? q_new_tile : q_old_tile) + (ch >> 3) * (kM * 128) + tc::sw128_offset(r, ch & 7);
-      if (r < n_rows)
-        tc::cp_async16(dst, (which ? a.q_new : a.q_old) + (size_t)(s0 + r) * a.d + h * kDH + ch * 8);
-      else
-        *reinterpret_cast<uint4*>(dst) = make_uint4(0, 0, 0, 0);
-    }
-    tc::cp_async_commit();
-    tc::cp_async_wait<0>();
-    tc::fence_proxy_async_smem();
-    tc::mbar_arrive(&ctl.q_full);
-    // dirty chunks: lanes 0-15 own the K row, lanes 16-31 the V row of one column at a time
-    const int half = lane >> 4, ch = lane & 15;
-    const DevSide& side = half ? a.v : a.k;
-    const int elem = h * kDH + ch * 8;
-    const __nv_bfloat16* base_rows = static_cast<const __nv_bfloat16*>(side.base) + elem;
-    const uint32_t ch_off = (ch >> 3) * (kNC * 128);
-    int f = fill0;
-    uint32_t dirty_par = dirty_par0;     // bit s: parity of the dirty fills slot s has seen
-    bool ok = true;
-#pragma unroll 1
-    for (int ci = 0; ci < n_chunks && ok; ++ci) {
-      const ChunkInfo ck = chunk_info(ci, n_plain, n_patch);
-      const int n_slots = ck.patch ? 2 : 1;
-      // Every fill is waited for, clean chunks included: a parity wait is only meaningful for the phase in
-      // progress, so a waiter must never skip a phase of a barrier it will wait on again.
-      for (int k = 0; k < n_slots && ok; ++k)
-        ok = warp_wait(&ctl.landed[(f + k) % kSlots], ((f + k) / kSlots) & 1, abort_flag);
-      if (!ok) break;
-      if (ctl.chunk_mask[ci] != 0) {
+      if (dirty) {
+        for (int k = 0; k < n_slots && ok; ++k)
+          ok = warp_wait(&ctl.landed[(f + k) % kSlots], ((f + k) / kSlots) & 1, abort_flag);
+        if (!ok) break;
         uint8_t* t_old = ring + (f % kSlots) * kSlotBytes + half * kTileBytes + ch_off;
         uint8_t* t_new = ring + ((f + 1) % kSlots) * kSlotBytes + half * kTileBytes + ch_off;
-        if (ci >= n_pre)
 #pragma unroll 1
-        for (int u = pw; u < ck.n_valid; u += kPatchWarps) {
+        for (int u = tw; u < ck.n_valid; u += kTmaWarps) {
           const uint32_t mask = ord_mask[ck.off + u];
           if (mask == 0) continue;
           const int j = ord_col[ck.off + u];
@@ -447,30 +535,31 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
         __syncwarp();
         if (lane == 0)
           for (int k = 0; k < n_slots; ++k) tc::mbar_arrive(&ctl.patched[(f + k) % kSlots]);
-        for (int k = 0; k < n_slots; ++k) dirty_par ^= 1u << ((f + k) % kSlots);
       }
       f += n_slots;
     }
-  } else if (warp == kMmaWarp) {
-    // ========================================= QK^T issuer ==========================================
-    if (lane == 0) {
+  } else if (warp >= kIssueWarp) {
+    // ========================================== MMA issuers ==========================================
+    const int role = warp - kIssueWarp;   // 0: QK old, 1: QK new, 2: PV old, 3: PV new
+    const int t = role & 1;
+    if (lane == 0 && role < 2) {
       const uint32_t idesc_qk = tc::make_idesc_bf16(kM, kNC, false);
       // Descriptors differ only in their start-address field (bits 0-13, units of 16 bytes): the low word
       // moves (no carry into the other fields: shared memory is < 256 KB), the high word stays.
       // K-major operands (Q, Khat): 32 bytes per 16-element K step inside a 64-element slab, then the next slab.
-      const uint64_t q_old_desc = tc::make_desc_sw128(tc::smem_u32(q_old_tile), 16, 1024);
-      const uint64_t q_new_desc = tc::make_desc_sw128(tc::smem_u32(q_new_tile), 16, 1024);
+      const uint64_t q_desc = tc::make_desc_sw128(tc::smem_u32(t ? q_new_tile : q_old_tile), 16, 1024);
       const uint64_t k_desc0 = tc::make_desc_sw128(tc::smem_u32(ring), 16, 1024);
       const uint32_t kq_hi = (uint32_t)(k_desc0 >> 32);
-      const uint32_t q_old_lo = (uint32_t)q_old_desc, q_new_lo = (uint32_t)q_new_desc, k_lo0 = (uint32_t)k_desc0;
+      const uint32_t q_lo_w = (uint32_t)q_desc, k_lo0 = (uint32_t)k_desc0;
+      const uint32_t s_dst = tmem + (t ? kSNew : kSOld);
       int f = fill0;
       uint32_t dirty_par = dirty_par0;
 #pragma unroll 1
       for (int ci = 0; ci < n_chunks; ++ci) {
         const ChunkInfo ck = chunk_info(ci, n_plain, n_patch);
         const int slot0 = f % kSlots, slot1 = (f + 1) % kSlots;
-        const int gc = g0 + ci, sbuf = gc & 1;
-        TC_TRACE(1, ci, 0);
+        const int gc = g0 + ci;
+        if (t == 0) TC_TRACE(1, ci, 0);
         if (ci == 0 && !tc::mbar_wait(&ctl.q_full, tile & 1, abort_flag)) break;
         if (!tc::mbar_wait(&ctl.landed[slot0], (f / kSlots) & 1, abort_flag)) break;
         if (ck.patch && !tc::mbar_wait(&ctl.landed[slot1], ((f + 1) / kSlots) & 1, abort_flag)) break;
@@ -482,60 +571,51 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
             dirty_par ^= 1u << slot1;
           }
         }
-        // the S buffer still holds P of chunk gc-2 until the PV MMAs that read it have retired
-        if (gc >= 2 && !tc::mbar_wait(&ctl.s_free[sbuf], ((gc >> 1) - 1) & 1, abort_flag)) break;
-        TC_TRACE(1, ci, 1);
-        const uint32_t k_old = k_lo0 + slot0 * (kSlotBytes >> 4);
-        const uint32_t k_new = ck.patch ? k_lo0 + slot1 * (kSlotBytes >> 4) : k_old;
-        const uint32_t s_old = tmem + kSBase + sbuf * 128, s_new = s_old + 64;
-#define FL_QK(D, QLO, KLO, KK, ACC)                                                                          \
-  tc::mma_ss_lo<ACC>(D, (QLO) + ((((KK) >> 2) * (kM * 128) + ((KK)&3) * 32) >> 4), kq_hi,                    \
-                     (KLO) + ((((KK) >> 2) * (kNC * 128) + ((KK)&3) * 32) >> 4), kq_hi, idesc_qk)
-        FL_QK(s_old, q_old_lo, k_old, 0, false); FL_QK(s_old, q_old_lo, k_old, 1, true);
-        FL_QK(s_old, q_old_lo, k_old, 2, true);  FL_QK(s_old, q_old_lo, k_old, 3, true);
-        FL_QK(s_old, q_old_lo, k_old, 4, true);  FL_QK(s_old, q_old_lo, k_old, 5, true);
-        FL_QK(s_old, q_old_lo, k_old, 6, true);  FL_QK(s_old, q_old_lo, k_old, 7, true);
-        FL_QK(s_new, q_new_lo, k_new, 0, false); FL_QK(s_new, q_new_lo, k_new, 1, true);
-        FL_QK(s_new, q_new_lo, k_new, 2, true);  FL_QK(s_new, q_new_lo, k_new, 3, true);
-        FL_QK(s_new, q_new_lo, k_new, 4, true);  FL_QK(s_new, q_new_lo, k_new, 5, true);
-        FL_QK(s_new, q_new_lo, k_new, 6, true);  FL_QK(s_new, q_new_lo, k_new, 7, true);
+        // the S buffer holds the previous chunk until the softmax warps have pulled it into registers
+        if (gc >= 1 && !tc::mbar_wait(&ctl.s_taken[t], (gc - 1) & 1, abort_flag)) break;
+        tc::tc_fence_after();
+        if (t == 0) TC_TRACE(1, ci, 1);
+        const uint32_t k_lo = k_lo0 + ((t && ck.patch) ? slot1 : slot0) * (kSlotBytes >> 4);
+#define FL_QK(KK, ACC)                                                                                       \
+  tc::mma_ss_lo<ACC>(s_dst, q_lo_w + ((((KK) >> 2) * (kM * 128) + ((KK)&3) * 32) >> 4), kq_hi,               \
+                     k_lo + ((((KK) >> 2) * (kNC * 128) + ((KK)&3) * 32) >> 4), kq_hi, idesc_qk)
+        FL_QK(0, false); FL_QK(1, true); FL_QK(2, true); FL_QK(3, true);
+        FL_QK(4, true);  FL_QK(5, true); FL_QK(6, true); FL_QK(7, true);
 #undef FL_QK
-        tc::mma_commit(&ctl.s_full[sbuf]);
+        tc::mma_commit(&ctl.s_full[t]);
+        tc::mma_commit(&ctl.done[slot0]);
+        if (ck.patch) tc::mma_commit(&ctl.done[slot1]);
         f += ck.patch ? 2 : 1;
-        TC_TRACE(1, ci, 2);
+        if (t == 0) TC_TRACE(1, ci, 2);
       }
-    }
-    __syncwarp();
-  } else if (warp == kPvWarp) {
-    // ========================================== P V issuer ==========================================
-    if (lane == 0) {
+    } else if (lane == 0) {
       const uint32_t idesc_pv = tc::make_idesc_bf16(kM, kDH, true);
       // MN-major Vhat: 16 key rows = two 1024-byte row groups per K step
       const uint64_t v_desc0 = tc::make_desc_sw128(tc::smem_u32(ring) + kTileBytes, kNC * 128, 1024);
       const uint32_t v_hi = (uint32_t)(v_desc0 >> 32), v_lo0 = (uint32_t)v_desc0;
+      const uint32_t acc = tmem + (t ? kAccNew : kAccOld);
+      const uint32_t p_base = tmem + (t ? kPNew : kPOld);
       int f = fill0;
 #pragma unroll 1
       for (int cj = 0; cj < n_chunks; ++cj) {
         const ChunkInfo ck = chunk_info(cj, n_plain, n_patch);
-        const int gc = g0 + cj, sbuf = gc & 1;
-        if (!tc::mbar_wait(&ctl.p_full[sbuf], (gc >> 1) & 1, abort_flag)) break;
+        const int gc = g0 + cj, pb = gc & 1;
+        if (t == 0) TC_TRACE(4, cj, 0);
+        if (!tc::mbar_wait(&ctl.p_full[t][pb], (gc >> 1) & 1, abort_flag)) break;
         tc::tc_fence_after();
+        if (t == 0) TC_TRACE(4, cj, 1);
         const int slot0 = f % kSlots, slot1 = (f + 1) % kSlots;
-        const uint32_t v_old = v_lo0 + slot0 * (kSlotBytes >> 4);
-        const uint32_t v_new = ck.patch ? v_lo0 + slot1 * (kSlotBytes >> 4) : v_old;
-        const uint32_t p_old = tmem + kSBase + sbuf * 128, p_new = p_old + 64;
-        const uint32_t acc0 = cj > 0 ? 1u : 0u;          // first chunk of the tile overwrites the accumulators
+        const uint32_t v_lo = v_lo0 + ((t && ck.patch) ? slot1 : slot0) * (kSlotBytes >> 4);
+        const uint32_t p_src = p_base + pb * 32;
+        const uint32_t acc0 = cj > 0 ? 1u : 0u;          // first chunk of the tile overwrites the accumulator
 #pragma unroll
         for (int kk = 0; kk < kNC / 16; ++kk)
-          tc::mma_ts_lo(tmem + kAccOld, p_old + kk * 8, v_old + kk * (2048 >> 4), v_hi, idesc_pv, kk > 0 ? 1u : acc0);
-#pragma unroll
-        for (int kk = 0; kk < kNC / 16; ++kk)
-          tc::mma_ts_lo(tmem + kAccNew, p_new + kk * 8, v_new + kk * (2048 >> 4), v_hi, idesc_pv, kk > 0 ? 1u : acc0);
+          tc::mma_ts_lo(acc, p_src + kk * 8, v_lo + kk * (2048 >> 4), v_hi, idesc_pv, kk > 0 ? 1u : acc0);
+        tc::mma_commit(&ctl.p_free[t][pb]);
         tc::mma_commit(&ctl.done[slot0]);
         if (ck.patch) tc::mma_commit(&ctl.done[slot1]);
-        tc::mma_commit(&ctl.s_free[sbuf]);
         f += ck.patch ? 2 : 1;
-        TC_TRACE(1, cj, 3);
+        if (t == 0) TC_TRACE(4, cj, 2);
       }
       tc::mma_commit(&ctl.acc_done);
     }
@@ -543,166 +623,159 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
   } else {
     // ============================================ softmax ============================================
     const int grp = warp >> 2;                    // 0: old term, 1: new term
+    const int gt = tid & 127;                     // thread inside the term's group of four warps
     const int row = (warp & 3) * 32 + lane;
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
     const bool row_ok = row < n_rows;
     const int pos = row_ok ? __ldg(a.active_idx + s0 + row) : -1;
     const float c2 = a.scale * kLog2e;
-    const float lse_prev = row_ok ? a.lse_prev[(size_t)h * a.L + pos] : 0.f;
-    const float lse2 = lse_prev * kLog2e;
+    const float lse2 = (row_ok ? a.lse_prev[(size_t)h * a.L + pos] : 0.f) * kLog2e;
+    const uint32_t s_addr = tmem + lane_base + (grp ? kSNew : kSOld);
+    const uint32_t p_addr = tmem + lane_base + (grp ? kPNew : kPOld);
     float mass = 0.f, ell = 0.f, ref = -INFINITY;
     bool ok = true;
-    int f = fill0, f_prev = fill0;
     for (int ci = 0; ci < n_chunks; ++ci) {
-      const ChunkInfo ck = chunk_info(ci, n_plain, n_patch);
-      const int gc = g0 + ci;
-      const int sbuf = gc & 1;
-      const int slot0 = f % kSlots;
-      if ((tid & 127) == 0) TC_TRACE(2 + grp, ci, 0);
-      // landed[] first: orders the TMA warp's column-position writes before the reads below
-      if (!warp_wait(&ctl.landed[slot0], (f / kSlots) & 1, abort_flag) ||
-          !warp_wait(&ctl.s_full[sbuf], (gc >> 1) & 1, abort_flag)) { ok = false; break; }
+      const int gc = g0 + ci, pb = gc & 1, n_use = gc >> 1;
+      if (gt == 0) TC_TRACE(2 + grp, ci, 0);
+      if (!warp_wait(&ctl.s_full[grp], gc & 1, abort_flag)) { ok = false; break; }
       tc::tc_fence_after();
-      if ((tid & 127) == 0) TC_TRACE(2 + grp, ci, 1);
-      const uint32_t s_addr = tmem + lane_base + kSBase + sbuf * 128 + grp * 64;
-      const int* cp = ctl.col_pos[slot0];
-      // rows of a warp that lie at or after every column of the chunk need no causal mask
-      const bool unmasked = __all_sync(0xffffffffu, row_ok && ctl.col_last[slot0] <= pos);
-      // One pass over the 64 logits of the row: load them, form p = 2^(s * c2 - sub) in place and pack to bf16.
-      // For the new term `sub` is the running reference; the chunk maximum is tracked on the side, and only if
-      // some row of the warp has no reference yet or would overflow (its maximum beats the reference by more
-      // than the threshold) does the warp take the slow path: fix the reference, rescale, recompute. The S
-      // region is still intact at that point because P is stored last.
+      if (gt == 0) TC_TRACE(2 + grp, ci, 1);
       uint32_t r[64];
       tc::tmem_ld32(s_addr, *reinterpret_cast<uint32_t(*)[32]>(&r[0]));
       tc::tmem_ld32(s_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&r[32]));
       tc::tmem_wait_ld();
-      float sub = grp == 0 ? lse2 : (ref == -INFINITY ? 0.f : ref);
-      float cm = -INFINITY, sum = 0.f;
-      bool stored = false;                               // warp-uniform: the slow path stores P itself
-      if (unmasked) {
-#pragma unroll
-        for (int u = 0; u < 64; u += 2) {
-          const float t0 = __uint_as_float(r[u]), t1 = __uint_as_float(r[u + 1]);
-          cm = fmaxf(cm, fmaxf(t0, t1));
-          const float p0 = tc::ex2(fmaf(t0, c2, -sub)), p1 = tc::ex2(fmaf(t1, c2, -sub));
-          sum += p0 + p1;
-          r[u >> 1] = tc::pack_bf16(p0, p1);
+      // S is in registers: hand the buffer back so that the next chunk's QK^T runs under the arithmetic below
+      tc::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) tc::mbar_arrive(&ctl.s_taken[grp]);
+      // rows of a warp that lie at or after every column of the chunk need no causal mask; rows beyond the
+      // tile's last (their results are never stored) must not force the masked path
+      const bool unmasked = __all_sync(0xffffffffu, !row_ok || ctl.chunk_last[ci] <= pos);
+      if (!unmasked) {
+        // the chunk's columns ascend: the visible ones are a prefix, found by bisection; the rest read as -inf
+        const ChunkInfo ck = chunk_info(ci, n_plain, n_patch);
+        const int32_t* cp = ord_col + ck.off;
+        int lo = 0, hi = row_ok ? ck.n_valid : 0;
+        while (lo < hi) {
+          const int mid = (lo + hi) >> 1;
+          if (cp[mid] <= pos) lo = mid + 1; else hi = mid;
         }
-      } else {
 #pragma unroll
-        for (int u = 0; u < 64; u += 2) {
-          const float t0 = cp[u] <= pos ? __uint_as_float(r[u]) : -INFINITY;
-          const float t1 = cp[u + 1] <= pos ? __uint_as_float(r[u + 1]) : -INFINITY;
-          cm = fmaxf(cm, fmaxf(t0, t1));
-          const float p0 = tc::ex2(fmaf(t0, c2, -sub)), p1 = tc::ex2(fmaf(t1, c2, -sub));
-          sum += p0 + p1;
-          r[u >> 1] = tc::pack_bf16(p0, p1);
-        }
+        for (int u = 0; u < 64; ++u) r[u] = u < lo ? r[u] : 0xff800000u;
       }
+      float sub = lse2;
       if (grp == 1) {
+        // running reference of the new term: taken from the first chunk that shows a finite logit and moved
+        // (with a rescale of the accumulator row) only when a chunk's maximum beats it by more than the threshold
+        float cm = -INFINITY;
+#pragma unroll
+        for (int u = 0; u < 64; u += 2) cm = fmaxf(cm, fmaxf(__uint_as_float(r[u]), __uint_as_float(r[u + 1])));
         cm *= c2;                                        // c2 > 0: scaling commutes with the maximum
         const bool first = ref == -INFINITY && cm > -INFINITY;
         const bool over = ref > -INFINITY && cm - ref > kRescaleThreshold;
-        if (__any_sync(0xffffffffu, first || over)) {
-          // ---- slow path (first chunk of a row, or a reference that fell too far behind) -----------------
+        if (first) ref = cm;                             // accumulator row is still zero: nothing to rescale
+        if (__any_sync(0xffffffffu, over)) {
           float factor = 1.f;
-          if (first) ref = cm;                           // accumulator row is still zero: nothing to rescale
           if (over) { factor = tc::ex2(ref - cm); ref = cm; }
-          if (__any_sync(0xffffffffu, over)) {
-            // every earlier PV must have completed before the accumulator rows are rewritten
-            if (ci >= 1) {
-              if (!warp_wait(&ctl.done[f_prev % kSlots], (f_prev / kSlots) & 1, abort_flag)) { ok = false; break; }
-              tc::tc_fence_after();
-            }
-            ell *= factor;
+          // every earlier PV must have completed before the accumulator rows are rewritten (ci >= 1 here)
+          if (!warp_wait(&ctl.p_free[1][(gc - 1) & 1], ((gc - 1) >> 1) & 1, abort_flag)) { ok = false; break; }
+          tc::tc_fence_after();
+          ell *= factor;
 #pragma unroll 1
-            for (int q4 = 0; q4 < 8; ++q4) {
-              uint32_t acc[16];
-              tc::tmem_ld16(tmem + lane_base + kAccNew + q4 * 16, acc);
-              tc::tmem_wait_ld();
-#pragma unroll
-              for (int i = 0; i < 16; ++i) acc[i] = __float_as_uint(__uint_as_float(acc[i]) * factor);
-              tc::tmem_st16(tmem + lane_base + kAccNew + q4 * 16, acc);
-            }
-            tc::tmem_wait_st();
-          }
-          sub = ref == -INFINITY ? 0.f : ref;
-          sum = 0.f;
-#pragma unroll 1
-          for (int q = 0; q < 4; ++q) {                  // recompute P from the untouched S region
-            uint32_t t[16];
-            tc::tmem_ld16(s_addr + q * 16, t);
+          for (int q4 = 0; q4 < 8; ++q4) {
+            uint32_t acc[16];
+            tc::tmem_ld16(tmem + lane_base + kAccNew + q4 * 16, acc);
             tc::tmem_wait_ld();
 #pragma unroll
-            for (int u = 0; u < 16; u += 2) {
-              const bool m0 = unmasked || cp[q * 16 + u] <= pos, m1 = unmasked || cp[q * 16 + u + 1] <= pos;
-              const float p0 = m0 ? tc::ex2(fmaf(__uint_as_float(t[u]), c2, -sub)) : 0.f;
-              const float p1 = m1 ? tc::ex2(fmaf(__uint_as_float(t[u + 1]), c2, -sub)) : 0.f;
-              sum += p0 + p1;
-              t[u >> 1] = tc::pack_bf16(p0, p1);
-            }
-            // S[16q, 16q+16) is consumed; P[8q, 8q+8) never reaches unread S
-            tc::tmem_st8(s_addr + q * 8, *reinterpret_cast<uint32_t(*)[8]>(&t[0]));
+            for (int i = 0; i < 16; ++i) acc[i] = __float_as_uint(__uint_as_float(acc[i]) * factor);
+            tc::tmem_st16(tmem + lane_base + kAccNew + q4 * 16, acc);
           }
-          stored = true;
+          tc::tmem_wait_st();
         }
+        sub = ref == -INFINITY ? 0.f : ref;
+      }
+      float sum = 0.f;
+#pragma unroll
+      for (int u = 0; u < 64; u += 2) {
+        const float p0 = tc::ex2(fmaf(__uint_as_float(r[u]), c2, -sub));
+        const float p1 = tc::ex2(fmaf(__uint_as_float(r[u + 1]), c2, -sub));
+        sum += p0 + p1;
+        r[u >> 1] = tc::pack_bf16(p0, p1);
       }
       if (grp == 0) mass += sum; else ell += sum;
-      // P (bf16, 32 columns) overwrites the first half of the 64-column S region, all of which was consumed
-      if (!stored) tc::tmem_st32(s_addr, *reinterpret_cast<uint32_t(*)[32]>(&r[0]));
+      // the P buffer is free once the PV MMAs of chunk gc - 2 have retired
+      if (n_use >= 1 && !warp_wait(&ctl.p_free[grp][pb], (n_use - 1) & 1, abort_flag)) { ok = false; break; }
+      tc::tc_fence_after();
+      tc::tmem_st32(p_addr + pb * 32, *reinterpret_cast<uint32_t(*)[32]>(&r[0]));
       tc::tmem_wait_st();
-      if ((tid & 127) == 0) TC_TRACE(2 + grp, ci, 2);
+      if (gt == 0) TC_TRACE(2 + grp, ci, 2);
       tc::tc_fence_before();
-      tc::mbar_arrive(&ctl.p_full[sbuf]);
-      f_prev = f + (ck.patch ? 1 : 0);     // last slot of this chunk: its done[] marks the completion of PV(ci)
-      f += ck.patch ? 2 : 1;
-      if ((tid & 127) == 0) TC_TRACE(2 + grp, ci, 3);
+      __syncwarp();
+      if (lane == 0) tc::mbar_arrive(&ctl.p_full[grp][pb]);
+      if (gt == 0) TC_TRACE(2 + grp, ci, 3);
     }
     // ---- epilogue ------------------------------------------------------------------------------------
+    // Each group finishes 64 of the 128 head-dim columns. Its half of the O_prev tile is staged in the group's
+    // own Q tile (the QK^T MMAs of the group's term have all retired once its last S arrived) with coalesced
+    // asynchronous copies, combined in place by the row-owning threads, and written out coalesced again.
+    uint8_t* stage = grp ? q_new_tile : q_old_tile;          // [128 rows][8 x 16 B], 16-byte chunks XOR-swizzled by row
+    const size_t o_col0 = (size_t)h * kDH + grp * 64;
+#pragma unroll 1
+    for (int k = 0; k < 8; ++k) {
+      const int idx = k * 128 + gt, rr = idx >> 3, cc = idx & 7;
+      if (rr < n_rows)
+        tc::cp_async16(stage + rr * 128 + ((cc ^ (rr & 7)) << 4), a.o_prev + (size_t)(s0 + rr) * a.d + o_col0 + cc * 8);
+    }
+    tc::cp_async_commit();
     if (ok) ok = warp_wait(&ctl.acc_done, tile & 1, abort_flag);
     tc::tc_fence_after();
+    if (gt == 0) TC_TRACE(2 + grp, 61, 0);
     if (grp == 0) ctl.mass[row] = mass;
     else { ctl.ell[row] = ell; ctl.ref[row] = ref; }
+    tc::cp_async_wait<0>();
     asm volatile("bar.sync 1, 256;" ::: "memory");
+    if (gt == 0) TC_TRACE(2 + grp, 61, 1);
     const float m_i = ctl.mass[row], l_i = ctl.ell[row], ref_i = ctl.ref[row];
     const bool acc_valid = ok && n_chunks > 0;            // warp-uniform: the tensor-memory reads below are collective
     const bool has = acc_valid && ref_i > -INFINITY;      // per row: T_i is not empty
     const float w = has ? m_i / l_i : 0.f;
 #pragma unroll 1
     for (int hh = 0; hh < 4; ++hh) {
-      // each group finishes 64 of the 128 head-dim columns, 16 at a time
-      const int col0 = grp * 64 + hh * 16;
       uint32_t ao[16], an[16];
       if (acc_valid) {
-        tc::tmem_ld16(tmem + lane_base + kAccOld + col0, ao);
-        tc::tmem_ld16(tmem + lane_base + kAccNew + col0, an);
+        tc::tmem_ld16(tmem + lane_base + kAccOld + grp * 64 + hh * 16, ao);
+        tc::tmem_ld16(tmem + lane_base + kAccNew + grp * 64 + hh * 16, an);
         tc::tmem_wait_ld();
       }
-      if (!row_ok) continue;
-      const size_t off = (size_t)(s0 + row) * a.d + h * kDH + col0;
       if (has) {
 #pragma unroll
         for (int v8 = 0; v8 < 2; ++v8) {
-          float prev[8], out[8];
-          load8<__nv_bfloat16>(a.o_prev + off + v8 * 8, prev);
+          uint4* cell = reinterpret_cast<uint4*>(stage + row * 128 + (((hh * 2 + v8) ^ (row & 7)) << 4));
+          float pv[8], out[8];
+          unpack8(*cell, pv);
 #pragma unroll
           for (int i = 0; i < 8; ++i)
-            out[i] = prev[i] - __uint_as_float(ao[v8 * 8 + i]) + w * __uint_as_float(an[v8 * 8 + i]);
-          store8<__nv_bfloat16>(a.o_out + off + v8 * 8, out);
+            out[i] = pv[i] - __uint_as_float(ao[v8 * 8 + i]) + w * __uint_as_float(an[v8 * 8 + i]);
+          *cell = pack8(out);
         }
-      } else if (a.o_out != a.o_prev) {
-#pragma unroll
-        for (int v8 = 0; v8 < 2; ++v8)
-          *reinterpret_cast<uint4*>(a.o_out + off + v8 * 8) = *reinterpret_cast<const uint4*>(a.o_prev + off + v8 * 8);
       }
     }
     if (grp == 1 && row_ok)
-      a.lse_out[(size_t)h * a.L + pos] = has ? (ref_i + log2f(l_i)) * kLn2 - logf(m_i) : lse_prev;
+      a.lse_out[(size_t)h * a.L + pos] = has ? (ref_i + log2f(l_i)) * kLn2 - logf(m_i) : lse2 * kLn2;
+    asm volatile("bar.sync 1, 256;" ::: "memory");
+    if (gt == 0) TC_TRACE(2 + grp, 61, 2);
+#pragma unroll 1
+    for (int k = 0; k < 8; ++k) {
+      const int idx = k * 128 + gt, rr = idx >> 3, cc = idx & 7;
+      if (rr < n_rows)
+        *reinterpret_cast<uint4*>(a.o_out + (size_t)(s0 + rr) * a.d + o_col0 + cc * 8) =
+            *reinterpret_cast<const uint4*>(stage + rr * 128 + ((cc ^ (rr & 7)) << 4));
+    }
+    if (gt == 0) TC_TRACE(2 + grp, 61, 3);
   }
   // every role is done with this tile: accumulators, Q tiles and the ring bookkeeping move on together
-  g += n_chunks;
-  {
+  if (s0 + kM < q_hi) {   // CTA-uniform: another row tile of the block follows
+    g += n_chunks;
     int f = fill;
     for (int ci = 0; ci < n_chunks; ++ci) {   // replay the tile's fills (same for every role)
       const ChunkInfo ck = chunk_info(ci, n_plain, n_patch);
@@ -712,17 +785,17 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
       f += n_slots;
     }
     fill = f;
+    tc::tc_fence_before();
+    __syncthreads();
+    tc::tc_fence_after();
+    if (ctl.abort_flag) break;
   }
-  tc::tc_fence_before();
-  __syncthreads();
-  tc::tc_fence_after();
-  if (ctl.abort_flag) break;
   }  // tiles of the block
   }  // block has active rows
   // ---- teardown ------------------------------------------------------------------------------------------
   tc::tc_fence_before();
   __syncthreads();
-  if (warp == kMmaWarp) {
+  if (warp == kIssueWarp) {
     if (ctl.abort_flag) {
       // let outstanding tensor work drain (bounded) before the columns are released
       if (lane == 0) tc::mma_commit(&ctl.acc_done);
@@ -748,11 +821,12 @@ int fl_launch_loop_attn_tc(fl_ctx* ctx, const fl_shape* s, int loop_r, const voi
   if (s->dtype != FL_BF16 || s->head_dim != kDH || c > kMaxCols) return FL_ERR_UNSUPPORTED;
   if ((size_t)ctx->max_smem_optin < kTcSmemBytes) return FL_ERR_UNSUPPORTED;
   TcArgs a{};
-  if (!fl_row_gather_tmap(ctx, store->k_base, s->L, (int64_t)s->n_heads * s->head_dim, &a.k_map) ||
-      !fl_row_gather_tmap(ctx, store->v_base, s->L, (int64_t)s->n_heads * s->head_dim, &a.v_map))
+  const int64_t d_row = (int64_t)s->n_heads * s->head_dim;
+  if (!fl_tile_tmap(ctx, store->k_base, s->L, d_row, 1, &a.k_map) ||
+      !fl_tile_tmap(ctx, store->v_base, s->L, d_row, 1, &a.v_map) ||
+      !fl_tile_tmap(ctx, q_new, n_active, d_row, kM, &a.q_new_map) ||
+      !fl_tile_tmap(ctx, q_old, n_active, d_row, kM, &a.q_old_map))
     return FL_ERR_UNSUPPORTED;
-  a.q_new = static_cast<const __nv_bfloat16*>(q_new);
-  a.q_old = static_cast<const __nv_bfloat16*>(q_old);
   a.o_prev = static_cast<const __nv_bfloat16*>(o_prev);
   a.o_out = static_cast<__nv_bfloat16*>(o_out);
   a.active_idx = active_idx; a.n_active = n_active;

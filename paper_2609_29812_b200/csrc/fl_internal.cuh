@@ -154,6 +154,67 @@ __device__ __forceinline__ bool apply_stream8(const DevStream& st, int pos, int 
   return true;
 }
 
+// One stream's payload for 8 consecutive elements, fetched ahead of its use so that the loads of several
+// streams (and columns) are in flight together; applying it is the arithmetic of apply_stream8.
+template <typename T, int BITS>
+struct Payload8 {
+  uint4 raw;      // BITS 16: the stored row piece (first 16 bytes); 8: x,y; 4 and 2: x
+  uint4 raw_hi;   // BITS 16 with binary32 storage: the second 16 bytes
+  float sc, zr;
+};
+template <typename T, int BITS>
+__device__ __forceinline__ void payload_load(const DevStream& st, int slot, int elem, int d, int group,
+                                             Payload8<T, BITS>& p) {
+  if (BITS == 16) {
+    const uint4* src = reinterpret_cast<const uint4*>(reinterpret_cast<const T*>(st.codes) + (size_t)slot * d + elem);
+    p.raw = __ldg(src);
+    if (sizeof(T) == 4) p.raw_hi = __ldg(src + 1);
+  } else {
+    const uint8_t* row = st.codes + (size_t)slot * (d * BITS / 8);
+    if (BITS == 8) {
+      const uint2 t = __ldg(reinterpret_cast<const uint2*>(row + elem));
+      p.raw.x = t.x; p.raw.y = t.y;
+    } else if (BITS == 4) {
+      p.raw.x = __ldg(reinterpret_cast<const uint32_t*>(row + elem / 2));
+    } else {
+      p.raw.x = __ldg(reinterpret_cast<const uint16_t*>(row + elem / 4));
+    }
+    const size_t gi = (size_t)slot * (d / group) + elem / group;
+    p.sc = __half2float(__ldg(st.scale + gi));
+    p.zr = __half2float(__ldg(st.zero + gi));
+  }
+}
+template <typename T, int BITS>
+__device__ __forceinline__ void payload_apply(const Payload8<T, BITS>& p, float (&x)[8]) {
+  if (BITS == 16) {
+    if (sizeof(T) == 4) {
+      x[0] = __uint_as_float(p.raw.x); x[1] = __uint_as_float(p.raw.y);
+      x[2] = __uint_as_float(p.raw.z); x[3] = __uint_as_float(p.raw.w);
+      x[4] = __uint_as_float(p.raw_hi.x); x[5] = __uint_as_float(p.raw_hi.y);
+      x[6] = __uint_as_float(p.raw_hi.z); x[7] = __uint_as_float(p.raw_hi.w);
+    } else {
+      const __nv_bfloat162* hp = reinterpret_cast<const __nv_bfloat162*>(&p.raw);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float2 f = __bfloat1622float2(hp[i]);
+        x[2 * i] = f.x;
+        x[2 * i + 1] = f.y;
+      }
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      uint32_t c;
+      if (BITS == 8) c = ((i < 4 ? p.raw.x : p.raw.y) >> (8 * (i & 3))) & 0xFFu;
+      else if (BITS == 4) c = (p.raw.x >> (4 * i)) & 0xFu;
+      else c = (p.raw.x >> (2 * i)) & 0x3u;
+      // code -> float without the conversion unit: 2^23 + c is exact in binary32
+      const float cf = __fsub_rn(__uint_as_float(0x4B000000u | c), 8388608.f);
+      x[i] = __fadd_rn(x[i], __fmaf_rn(cf, p.sc, p.zr));
+    }
+  }
+}
+
 // Reconstruct 8 consecutive elements of Xhat after the first n_use residual streams
 // (Eq. 8 chain in binary32, loop order): x = ((base + D_2) + D_3) + ...
 template <typename T, int BITS>

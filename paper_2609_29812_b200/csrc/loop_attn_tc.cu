@@ -58,11 +58,15 @@ constexpr float kRescaleThreshold = 60.f;   // in log2 units: rescale only when 
 static_assert((2 + kPreStreams) * kMaxCols * 4 <= kSlots * kSlotBytes, "prologue staging must fit in the ring");
 
 // Optional device-side timeline for tuning (compile with -DFL_TC_TRACE): the CTA (block 1, head 0) writes
-// clock64() stamps into the buffer passed as `status`: trace[(role * 64 + chunk) * 4 + event].
+// clock64() stamps into the buffer passed as `status` (the traced CTA can be chosen with -DFL_TC_TRACE_X/_Y): trace[(role * 64 + chunk) * 4 + event].
 #ifdef FL_TC_TRACE
+#ifndef FL_TC_TRACE_X
+#define FL_TC_TRACE_X 1
+#define FL_TC_TRACE_Y 0
+#endif
 #define TC_TRACE(role, chunk, ev)                                                                      \
   do {                                                                                                 \
-    if (blockIdx.x == 1 && blockIdx.y == 0 && (chunk) < 64 && a.status != nullptr)                     \
+    if (blockIdx.x == FL_TC_TRACE_X && blockIdx.y == FL_TC_TRACE_Y && (chunk) < 64 && a.status != nullptr) \
       reinterpret_cast<long long*>(a.status)[((role) * 64 + (chunk)) * 4 + (ev)] = clock64();          \
   } while (0)
 #else
@@ -123,19 +127,38 @@ __device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, volati
   return __all_sync(0xffffffffu, ok);
 }
 
-// first index in the ascending array with value >= target; all 32 lanes cooperate (32-ary search)
-__device__ __forceinline__ int lower_bound32(const int32_t* __restrict__ arr, int n, int target, int lane) {
-  int lo = 0, hi = n;
-  while (hi > lo) {
-    const int step = (hi - lo + 31) >> 5;
-    const int idx = lo + lane * step + step - 1;
-    const bool less = idx < hi && __ldg(arr + idx) < target;
-    const int k = __popc(__ballot_sync(0xffffffffu, less));
-    const int new_lo = lo + k * step;
+// First index in the ascending array with value >= target, and through `below` the element just before it
+// (INT32_MIN if there is none). All 32 lanes cooperate: 128 probes per round while the range is wide, then one
+// load per lane; the active lists of the benchmark shapes (a few thousand rows) take two dependent rounds.
+__device__ __forceinline__ int lower_bound_warp(const int32_t* __restrict__ arr, int n, int target, int lane, int* below) {
+  int lo = 0, hi = n, prev = INT32_MIN;   // invariant: arr[lo - 1] == prev < target (or lo == 0), arr[hi] >= target (or hi == n)
+  while (hi - lo > 32) {
+    const int step = (hi - lo + 127) >> 7;
+    int v[4];
+    uint32_t less[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const int idx = lo + (lane * 4 + k + 1) * step - 1;
+      v[k] = idx < hi ? __ldg(arr + idx) : INT32_MAX;
+    }
+#pragma unroll
+    for (int k = 0; k < 4; ++k) less[k] = __ballot_sync(0xffffffffu, v[k] < target);
+    // probes ascend with (lane, k): the ones below the target are a prefix
+    const int n_less = __popc(less[0]) + __popc(less[1]) + __popc(less[2]) + __popc(less[3]);
+    if (n_less > 0) {
+      const int src = (n_less - 1) >> 2, kk = (n_less - 1) & 3;
+      const int cand = kk == 0 ? v[0] : (kk == 1 ? v[1] : (kk == 2 ? v[2] : v[3]));
+      prev = __shfl_sync(0xffffffffu, cand, src);
+    }
+    const int new_lo = lo + n_less * step;
     hi = min(hi, new_lo + step - 1);
     lo = min(new_lo, hi);
   }
-  return lo;
+  const int val = lo + lane < hi ? __ldg(arr + lo + lane) : INT32_MAX;
+  const int cnt = __popc(__ballot_sync(0xffffffffu, val < target));
+  if (cnt > 0) prev = __shfl_sync(0xffffffffu, val, cnt - 1);
+  *below = prev;
+  return lo + cnt;
 }
 
 __device__ __forceinline__ uint4 pack8(const float (&x)[8]) {
@@ -171,48 +194,6 @@ __device__ __forceinline__ void patch_piece(const DevSide& side, int n_old, uint
     if ((mask >> s) & 1u) apply_stream8<__nv_bfloat16, BITS>(side.s[s], j, elem, d, group, x);
   }
   v_new = ((mask >> n_old) & 1u) ? pack8(x) : v_old;
-}
-
-// One stream's payload for 8 consecutive elements, fetched ahead of its use so that the loads of several
-// columns and streams are in flight together (the cooperative build of the first residual-carrying chunks).
-template <int BITS>
-struct Payload8 {
-  uint4 raw;      // BITS 16: the stored row piece; 8: x,y; 4 and 2: x
-  float sc, zr;
-};
-template <int BITS>
-__device__ __forceinline__ void payload_load(const DevStream& st, int slot, int elem, int d, int group, Payload8<BITS>& p) {
-  if (BITS == 16) {
-    p.raw = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(st.codes) + (size_t)slot * d + elem));
-  } else {
-    const uint8_t* row = st.codes + (size_t)slot * (d * BITS / 8);
-    if (BITS == 8) {
-      const uint2 t = __ldg(reinterpret_cast<const uint2*>(row + elem));
-      p.raw.x = t.x; p.raw.y = t.y;
-    } else if (BITS == 4) {
-      p.raw.x = __ldg(reinterpret_cast<const uint32_t*>(row + elem / 2));
-    } else {
-      p.raw.x = __ldg(reinterpret_cast<const uint16_t*>(row + elem / 4));
-    }
-    const size_t gi = (size_t)slot * (d / group) + elem / group;
-    p.sc = __half2float(__ldg(st.scale + gi));
-    p.zr = __half2float(__ldg(st.zero + gi));
-  }
-}
-template <int BITS>
-__device__ __forceinline__ void payload_apply(const Payload8<BITS>& p, float (&x)[8]) {
-  if (BITS == 16) {
-    unpack8(p.raw, x);
-  } else {
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      uint32_t c;
-      if (BITS == 8) c = ((i < 4 ? p.raw.x : p.raw.y) >> (8 * (i & 3))) & 0xFFu;
-      else if (BITS == 4) c = (p.raw.x >> (4 * i)) & 0xFu;
-      else c = (p.raw.x >> (2 * i)) & 0x3u;
-      x[i] = __fadd_rn(x[i], __fmaf_rn((float)c, p.sc, p.zr));
-    }
-  }
 }
 
 // chunk ci of the partitioned column list: patched chunks first (the first two are built by the whole CTA
@@ -281,17 +262,20 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
   int32_t* raw_col = reinterpret_cast<int32_t*>(ring);                     // [kMaxCols]
   uint32_t* raw_mask = reinterpret_cast<uint32_t*>(raw_col + kMaxCols);    // [kMaxCols]
   int32_t* raw_slot = reinterpret_cast<int32_t*>(raw_mask + kMaxCols);     // [kPreStreams][kMaxCols]
+  const int c_cap = min(a.c, kMaxCols);
   if (warp >= kColWarps) {
     // warps 14 and 15 search the block's rows in the ascending active list meanwhile
     const int target = warp == kColWarps ? b * a.q_block : min(a.L, (b + 1) * a.q_block);
-    const int r = lower_bound32(a.active_idx, a.n_active, target, lane);
+    int below;
+    const int r = lower_bound_warp(a.active_idx, a.n_active, target, lane, &below);
     if (lane == 0) {
       if (warp == kColWarps) ctl.q_lo = r;
-      else { ctl.q_hi = r; ctl.i_last = r > 0 ? __ldg(a.active_idx + r - 1) : -1; }
+      else { ctl.q_hi = r; ctl.i_last = r > 0 ? below : -1; }
     }
   } else {
+    // the whole row of the column table is read without waiting for its count: entries past the count are -1
 #pragma unroll 1
-    for (int u = tid; u < cnt; u += kColWarps * 32) {
+    for (int u = tid; u < c_cap; u += kColWarps * 32) {
       raw_col[u] = __ldg(cols + u);
       raw_mask[u] = 0;
     }
@@ -310,9 +294,10 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
   {
     // every (column, stream) pair is one independent slot-map lookup
 #pragma unroll 1
-    for (int p2 = tid; p2 < cnt * (a.n_old + 1); p2 += kThreads) {
-      const int s = p2 / cnt, u = p2 - s * cnt;
-      const int sl = __ldg(a.k.s[s].slot + raw_col[u]);
+    for (int p2 = tid; p2 < c_cap * (a.n_old + 1); p2 += kThreads) {
+      const int s = p2 / c_cap, u = p2 - s * c_cap;
+      const int j = raw_col[u];
+      const int sl = j >= 0 ? __ldg(a.k.s[s].slot + j) : -1;
       if (sl >= 0) atomicOr(&raw_mask[u], 1u << s);
       if (s < kPreStreams) raw_slot[s * kMaxCols + u] = sl;
     }
@@ -433,7 +418,7 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
       const bool valid = u < ck.n_valid;
       const uint32_t mask = valid ? ord_mask[ck.off + u] : 0u;
       uint4 raw = make_uint4(0, 0, 0, 0);
-      Payload8<BITS> pl[kPreStreams];
+      Payload8<__nv_bfloat16, BITS> pl[kPreStreams];
       int sl[kPreStreams];
       if (valid)
         raw = __ldg(reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(side.base) +
@@ -441,7 +426,7 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
 #pragma unroll
       for (int s = 0; s < kPreStreams; ++s) {
         sl[s] = (valid && s <= a.n_old) ? ctl.pre_slot[s][pc * kNC + u] : -1;
-        if (sl[s] >= 0) payload_load<BITS>(side.s[s], sl[s], elem, a.d, a.group, pl[s]);
+        if (sl[s] >= 0) payload_load<__nv_bfloat16, BITS>(side.s[s], sl[s], elem, a.d, a.group, pl[s]);
       }
       float x[8];
       unpack8(raw, x);
@@ -449,7 +434,7 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
 #pragma unroll
       for (int s = 0; s < kPreStreams; ++s) {
         if (s == a.n_old && (mask & ((1u << a.n_old) - 1u))) v_old = pack8(x);
-        if (sl[s] >= 0) payload_apply<BITS>(pl[s], x);
+        if (sl[s] >= 0) payload_apply<__nv_bfloat16, BITS>(pl[s], x);
       }
       const uint4 v_new = ((mask >> a.n_old) & 1u) ? pack8(x) : v_old;
       const uint32_t off = tile_off + tc::sw128_offset(u, ch & 7);

@@ -29,9 +29,23 @@ __global__ void __launch_bounds__(256) quant_residual_kernel(const __grid_consta
   const int lanes_per_group = a.group >> 3;  // 1, 2, 4, 8 or 16
 
   for (int elem = threadIdx.x * 8; elem < a.d; elem += blockDim.x * 8) {
+    // The new row, the base row and every earlier stream's slot lookup are independent loads; the payloads of
+    // four streams at a time follow as a second round (Eq. 8 chain applied in loop order afterwards).
     float xn[8], xh[8];
     load8<T>(x_new + elem, xn);
-    recon8<T, BITS>(side, a.n_prev, pos, elem, a.d, a.group, xh);
+    load8<T>(static_cast<const T*>(side.base) + (size_t)pos * a.d + elem, xh);
+    for (int sg = 0; sg < a.n_prev; sg += 4) {
+      int sl[4];
+      Payload8<T, BITS> pl[4];
+#pragma unroll
+      for (int si = 0; si < 4; ++si) sl[si] = sg + si < a.n_prev ? __ldg(side.s[sg + si].slot + pos) : -1;
+#pragma unroll
+      for (int si = 0; si < 4; ++si)
+        if (sl[si] >= 0) payload_load<T, BITS>(side.s[sg + si], sl[si], elem, a.d, a.group, pl[si]);
+#pragma unroll
+      for (int si = 0; si < 4; ++si)
+        if (sl[si] >= 0) payload_apply<T, BITS>(pl[si], xh);
+    }
     if (BITS == 16) {  // codec off: the stream keeps the row itself
       store8<T>(reinterpret_cast<T*>(codes) + (size_t)t * a.d + elem, xn);
       continue;
@@ -55,15 +69,33 @@ __global__ void __launch_bounds__(256) quant_residual_kernel(const __grid_consta
     const float qmax = (float)((1 << BITS) - 1);
     const __half sh = range == 0.f ? __float2half_rn(0.f) : __float2half_ru(__fdiv_rn(range, qmax));
     const float sf = __half2float(sh);
+    // Codes: round-half-even of the binary32 quotient (delta - zero) / scale. The quotient is first formed with
+    // one reciprocal per group; that estimate is within a few ulp of the correctly rounded quotient (<= 5e-5
+    // absolute for codes up to 255), so its rounding to an integer is the same unless it lies within 1e-4 of a
+    // half-integer. Only then (a few percent of the warps) the true divisions are redone.
+    float q[8];
+    bool ambiguous = false;
+    if (sf != 0.f) {
+      const float inv = __frcp_rn(sf);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const float est = __fmul_rn(__fsub_rn(dl[i], zf), inv);
+        q[i] = __fsub_rn(__fadd_rn(est, 12582912.f), 12582912.f);   // round-half-even for |est| < 2^22
+        ambiguous |= 0.5f - fabsf(est - q[i]) < 1e-4f;
+      }
+      if (__any_sync(__activemask(), ambiguous)) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) q[i] = rintf(__fdiv_rn(__fsub_rn(dl[i], zf), sf));
+      }
+    } else {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) q[i] = 0.f;
+    }
     uint32_t packed_lo = 0, packed_hi = 0;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-      uint32_t c = 0;
-      if (sf != 0.f) {
-        float q = __fdiv_rn(__fsub_rn(dl[i], zf), sf);
-        q = fminf(fmaxf(rintf(q), 0.f), qmax);
-        c = (uint32_t)q;
-      }
+      // integer-valued 0..qmax: the low mantissa bits of (value + 2^23) are the code
+      const uint32_t c = __float_as_uint(__fadd_rn(fminf(fmaxf(q[i], 0.f), qmax), 8388608.f)) & 0xFFu;
       if (BITS == 8) {
         if (i < 4) packed_lo |= c << (8 * i); else packed_hi |= c << (8 * (i - 4));
       } else {

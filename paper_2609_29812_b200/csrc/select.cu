@@ -186,6 +186,229 @@ __global__ void __launch_bounds__(kSelThreads) token_select_kernel(const float* 
   });
 }
 
+// ------------------------------------------------------------------------------------------
+// The same selection with the keys staged in shared memory (problems of up to kSelCap candidates): the
+// scores are read from global memory once; the radix passes run on shared memory and, as soon as the bin
+// that holds the k-th largest key is small, on a compacted list of that bin's keys only.
+// ------------------------------------------------------------------------------------------
+constexpr int kSelCap = 49152;    // 192 KB of keys
+constexpr int kSelSmall = 2048;
+
+struct SelectSmem2 {
+  uint32_t hist[256];
+  uint32_t warp_gt[32], warp_eq[32];
+  uint32_t prefix, k_rem, bin_cnt, n_small;
+  uint32_t small[kSelSmall];
+};
+
+// Adds the warp's keys that are `on` to the histogram: lanes that share the digit of the first matching lane
+// are counted with one atomic (scores cluster in a few exponent bins, runs of equal scores are common), the
+// rest add themselves.
+__device__ __forceinline__ void hist_add(uint32_t* hist, bool on, uint32_t digit, int lane) {
+  const uint32_t active = __ballot_sync(0xffffffffu, on);
+  if (active == 0) return;
+  const int leader = __ffs(active) - 1;
+  const uint32_t d0 = __shfl_sync(0xffffffffu, digit, leader);
+  const uint32_t same = __ballot_sync(0xffffffffu, on && digit == d0);
+  if (lane == leader) atomicAdd(&hist[d0], (uint32_t)__popc(same));
+  else if (on && digit != d0) atomicAdd(&hist[digit], 1u);
+}
+
+// one radix pass (8 bits at `shift`) over list[0..m4*4): histogram of the keys that match `prefix` above the
+// digit. Four keys per thread and step: the four dependent chains (load, vote, atomic) overlap.
+__device__ __forceinline__ void radix_hist_pass(const uint32_t* list, int m4, int shift, uint32_t prefix, uint32_t* hist) {
+  const int tid = threadIdx.x, lane = tid & 31;
+  const uint32_t hi_mask = shift == 24 ? 0u : (0xFFFFFFFFu << (shift + 8));
+  const uint4* l4 = reinterpret_cast<const uint4*>(list);
+  for (int base = 0; base < m4; base += kSelThreads) {
+    const int i = base + tid;
+    const bool in = i < m4;
+    const uint4 kv = in ? l4[i] : make_uint4(0, 0, 0, 0);
+    hist_add(hist, in && (kv.x & hi_mask) == prefix, (kv.x >> shift) & 0xFFu, lane);
+    hist_add(hist, in && (kv.y & hi_mask) == prefix, (kv.y >> shift) & 0xFFu, lane);
+    hist_add(hist, in && (kv.z & hi_mask) == prefix, (kv.z >> shift) & 0xFFu, lane);
+    hist_add(hist, in && (kv.w & hi_mask) == prefix, (kv.w >> shift) & 0xFFu, lane);
+  }
+}
+
+__global__ void __launch_bounds__(kSelThreads, 1) column_select_smem_kernel(const float* __restrict__ col_scores,
+                                                                            const int32_t* __restrict__ cand_cols,
+                                                                            const int32_t* __restrict__ cand_cnt, int stride,
+                                                                            int c, int L, int q_block, int nb, int vec_ok,
+                                                                            int32_t* __restrict__ col_idx,
+                                                                            int32_t* __restrict__ col_cnt) {
+  extern __shared__ __align__(16) uint32_t keys[];   // [n rounded up to 4], padded with key 0 (below every real key)
+  __shared__ SelectSmem2 sm;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int b = blockIdx.x, h = blockIdx.y;
+  const size_t prob = (size_t)h * nb + b;
+  const float* vals = col_scores + prob * stride;
+  const int32_t* cols = cand_cols != nullptr ? cand_cols + prob * stride : nullptr;
+  int n = cand_cols != nullptr ? __ldg(cand_cnt + prob) : min(L, (b + 1) * q_block);
+  n = max(0, min(n, stride));
+  const int k = min(c, n);
+  int32_t* out = col_idx + prob * c;
+  for (int i = k + tid; i < c; i += kSelThreads) out[i] = -1;
+  if (tid == 0) col_cnt[prob] = k;
+  if (k == 0) return;
+  const int n4 = (n + 3) >> 2;
+  // ---- stage the order-preserving keys --------------------------------------------------------------
+  if (vec_ok) {
+    const float4* v4 = reinterpret_cast<const float4*>(vals);
+    uint4* k4 = reinterpret_cast<uint4*>(keys);
+    for (int i = tid; i < (n >> 2); i += kSelThreads) {
+      const float4 v = __ldg(v4 + i);
+      k4[i] = make_uint4(ordered_key(v.x), ordered_key(v.y), ordered_key(v.z), ordered_key(v.w));
+    }
+    for (int i = (n & ~3) + tid; i < n4 * 4; i += kSelThreads) keys[i] = i < n ? ordered_key(__ldg(vals + i)) : 0u;
+  } else {
+    for (int i = tid; i < n4 * 4; i += kSelThreads) keys[i] = i < n ? ordered_key(__ldg(vals + i)) : 0u;
+  }
+  uint32_t prefix = 0, k_rem = 0;
+  const bool take_all = k >= n;
+  if (!take_all) {
+    k_rem = (uint32_t)k;
+    const uint32_t* list = keys;
+    int m4 = n4;
+    for (int shift = 24; shift >= 0; shift -= 8) {
+      for (int i = tid; i < 256; i += kSelThreads) sm.hist[i] = 0;
+      __syncthreads();   // also orders the staging / compaction writes before the reads below
+      radix_hist_pass(list, m4, shift, prefix, sm.hist);
+      __syncthreads();
+      if (warp == 0) {
+        // lane owns digits [8*lane, 8*lane+8); find the digit holding the k_rem-th largest
+        uint32_t local[8], sum = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { local[j] = sm.hist[lane * 8 + j]; sum += local[j]; }
+        uint32_t incl = sum;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const uint32_t v = __shfl_down_sync(0xffffffffu, incl, o);
+          if (lane + o < 32) incl += v;
+        }
+        const uint32_t above = incl - sum;
+        if (above < k_rem && k_rem <= above + sum) {
+          uint32_t acc = above;
+          for (int j = 7; j >= 0; --j) {
+            if (k_rem <= acc + local[j]) {
+              sm.prefix = prefix | ((uint32_t)(lane * 8 + j) << shift);
+              sm.k_rem = k_rem - acc;
+              sm.bin_cnt = local[j];
+              break;
+            }
+            acc += local[j];
+          }
+        }
+        if (lane == 0) sm.n_small = 0;
+      }
+      __syncthreads();
+      prefix = sm.prefix;
+      k_rem = sm.k_rem;
+      const uint32_t bin_cnt = sm.bin_cnt;
+      if (shift > 0 && list == keys && bin_cnt <= (uint32_t)(kSelSmall - 4)) {
+        // the k-th largest key lies in a small bin: finish on that bin's keys alone
+        const uint32_t hi_mask = 0xFFFFFFFFu << shift;
+        const uint4* k4 = reinterpret_cast<const uint4*>(keys);
+        for (int base = 0; base < n4; base += kSelThreads) {
+          const int i = base + tid;
+          const uint4 kv = i < n4 ? k4[i] : make_uint4(0, 0, 0, 0);
+          const uint32_t kk[4] = {kv.x, kv.y, kv.z, kv.w};
+          uint32_t flags = 0;
+#pragma unroll
+          for (int j = 0; j < 4; ++j) flags |= (i < n4 && (kk[j] & hi_mask) == prefix ? 1u : 0u) << j;
+          // exclusive prefix of the per-lane counts over the warp, then one atomic per warp
+          const uint32_t cnt = __popc(flags);
+          uint32_t incl = cnt;
+#pragma unroll
+          for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t v = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += v;
+          }
+          const uint32_t total = __shfl_sync(0xffffffffu, incl, 31);
+          uint32_t off = 0;
+          if (lane == 0 && total != 0) off = atomicAdd(&sm.n_small, total);
+          off = __shfl_sync(0xffffffffu, off, 0) + incl - cnt;
+#pragma unroll
+          for (int j = 0; j < 4; ++j)
+            if ((flags >> j) & 1u) sm.small[off++] = kk[j];
+        }
+        __syncthreads();
+        // pad the list to a multiple of four with keys that cannot match the prefix of any later pass
+        if (tid < 4) {
+          const uint32_t m = sm.n_small;
+          if (m + tid < ((m + 3) & ~3u)) sm.small[m + tid] = ~prefix;
+        }
+        list = sm.small;
+        m4 = (int)((bin_cnt + 3) >> 2);
+      }
+      __syncthreads();
+    }
+  } else {
+    __syncthreads();
+  }
+  const uint32_t thr = prefix;
+  // ---- index-ordered compaction from the staged keys: each warp owns a contiguous span of whole uint4s ------
+  const int span4 = (n4 + 31) / 32;                    // uint4s per warp
+  const int beg4 = warp * span4, end4 = min(n4, beg4 + span4);
+  const uint4* k4 = reinterpret_cast<const uint4*>(keys);
+  uint32_t gt = 0, eq = 0;
+  for (int i = beg4 + lane; i < end4; i += 32) {
+    const uint4 kv = k4[i];
+    const uint32_t kk[4] = {kv.x, kv.y, kv.z, kv.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const bool valid = i * 4 + j < n;
+      gt += (valid && (take_all || kk[j] > thr)) ? 1u : 0u;
+      eq += (valid && !take_all && kk[j] == thr) ? 1u : 0u;
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    gt += __shfl_xor_sync(0xffffffffu, gt, o);
+    eq += __shfl_xor_sync(0xffffffffu, eq, o);
+  }
+  if (lane == 0) { sm.warp_gt[warp] = gt; sm.warp_eq[warp] = eq; }
+  __syncthreads();
+  uint32_t gt_before = 0, eq_before = 0;
+  for (int w = 0; w < warp; ++w) { gt_before += sm.warp_gt[w]; eq_before += sm.warp_eq[w]; }
+  for (int base = beg4; base < end4; base += 32) {
+    const int i = base + lane;
+    uint32_t f_gt = 0, f_eq = 0;
+    if (i < end4) {
+      const uint4 kv = k4[i];
+      const uint32_t kk[4] = {kv.x, kv.y, kv.z, kv.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const bool valid = i * 4 + j < n;
+        f_gt |= (valid && (take_all || kk[j] > thr) ? 1u : 0u) << j;
+        f_eq |= (valid && !take_all && kk[j] == thr ? 1u : 0u) << j;
+      }
+    }
+    // exclusive prefixes over the warp, in index order (lane-major, then the four keys of the lane)
+    const uint32_t c_gt = __popc(f_gt), c_eq = __popc(f_eq);
+    uint32_t i_gt = c_gt, i_eq = c_eq;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t v_gt = __shfl_up_sync(0xffffffffu, i_gt, o);
+      const uint32_t v_eq = __shfl_up_sync(0xffffffffu, i_eq, o);
+      if (lane >= o) { i_gt += v_gt; i_eq += v_eq; }
+    }
+    uint32_t my_gt = gt_before + i_gt - c_gt, my_eq = eq_before + i_eq - c_eq;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const bool is_gt = (f_gt >> j) & 1u, is_eq = (f_eq >> j) & 1u;
+      int rank = -1;
+      if (is_gt) rank = (int)(my_gt + min(my_eq, k_rem));
+      else if (is_eq && my_eq < k_rem) rank = (int)(my_gt + my_eq);
+      if (rank >= 0) out[rank] = cols != nullptr ? __ldg(cols + i * 4 + j) : i * 4 + j;
+      my_gt += is_gt ? 1u : 0u;
+      my_eq += is_eq ? 1u : 0u;
+    }
+    gt_before += __shfl_sync(0xffffffffu, i_gt, 31);
+    eq_before += __shfl_sync(0xffffffffu, i_eq, 31);
+  }
+}
+
 // one block per (head, query block)
 __global__ void __launch_bounds__(kSelThreads) column_select_kernel(const float* __restrict__ col_scores,
                                                                     const int32_t* __restrict__ cand_cols,
@@ -258,7 +481,17 @@ extern "C" int fl_select_columns(fl_ctx* ctx, const fl_shape* shape, const float
   const int nb = fl_n_blocks(shape);
   FL_REQUIRE(nb <= 65535 * 1024 && shape->n_heads <= 65535);
   dim3 grid(nb, shape->n_heads);
-  column_select_kernel<<<grid, kSelThreads, 0, static_cast<cudaStream_t>(stream)>>>(
-      col_scores, cand_cols, cand_cnt, n_cand, c, shape->L, shape->q_block, nb, col_idx, col_cnt);
+  const size_t key_bytes = sizeof(uint32_t) * (((size_t)n_cand + 3) & ~(size_t)3);
+  if (n_cand <= kSelCap && key_bytes + 16384 <= (size_t)ctx->max_smem_optin) {
+    // keys staged in shared memory: the scores are read from global memory once
+    const int vec_ok = (fl_aligned16(col_scores) && n_cand % 4 == 0) ? 1 : 0;
+    FL_CHECK_CUDA(cudaFuncSetAttribute(column_select_smem_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)key_bytes));
+    column_select_smem_kernel<<<grid, kSelThreads, key_bytes, static_cast<cudaStream_t>(stream)>>>(
+        col_scores, cand_cols, cand_cnt, n_cand, c, shape->L, shape->q_block, nb, vec_ok, col_idx, col_cnt);
+  } else {
+    column_select_kernel<<<grid, kSelThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+        col_scores, cand_cols, cand_cnt, n_cand, c, shape->L, shape->q_block, nb, col_idx, col_cnt);
+  }
   return fl_launch_status();
 }

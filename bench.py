@@ -156,7 +156,7 @@ class Bench:
             # compact buffers shared by all layers (a real engine reuses them the same way)
             mkrows = lambda: torch.empty(n_max, self.H, self.dh, dtype=torch.bfloat16, device=dev)
             self.xbuf = torch.empty(n_max, self.d, dtype=torch.bfloat16, device=dev)
-            self.q_old_buf, self.o_prev_buf, self.o_out_buf = mkrows(), mkrows(), mkrows()
+            self.o_out_buf = mkrows()      # end-to-end arm: the last layer's new O rows, gathered for the read-back
             self.layers = []
             for l in range(self.NL):
                 gen = stack.layer(l)
@@ -245,23 +245,18 @@ class Bench:
                 q_new, k_new, v_new = st.rows[r]
                 calls.append(("quant", lib.fl_quant_kv_residual,
                               (ctx, shp, r, p(k_new), p(v_new), p(sel.active_idx), n, C.byref(store), None, sp)))
+                # Q^(r-1), O^(r-1) are read from and O^(r), Q^(r) written to position-indexed stores by the attention
+                # call itself; loop 2 reads the pristine loop-1 stores and writes the work stores, so that every
+                # step starts from the same state
                 q_src = st.q_store if r == 2 else st.q_work
                 o_src = st.o_store if r == 2 else st.o_work
                 lse_prev = st.lse1 if r == 2 else st.lse_work
-                calls.append(("gather", lib.fl_gather_rows, (ctx, p(q_src), p(sel.active_idx), n, row_bytes,
-                                                             p(self.q_old_buf), sp)))
-                calls.append(("gather", lib.fl_gather_rows, (ctx, p(o_src), p(sel.active_idx), n, row_bytes,
-                                                             p(self.o_prev_buf), sp)))
-                calls.append(("attention", lib.fl_loop_attention,
-                              (ctx, shp, r, p(q_new), p(self.q_old_buf), p(sel.active_idx), n, C.byref(store),
+                calls.append(("attention", lib.fl_loop_attention_indexed,
+                              (ctx, shp, r, p(q_new), p(q_src), p(st.q_work), p(sel.active_idx), n, C.byref(store),
                                p(st.col_idx), p(st.col_cnt), self.c, p(lse_prev), p(st.lse_work),
-                               p(self.o_prev_buf), p(self.o_out_buf), None, None, sp)))
-                calls.append(("scatter", lib.fl_scatter_update, (ctx, p(self.o_out_buf), p(sel.active_idx), n,
-                                                                 row_bytes, p(st.o_work), sp)))
-                calls.append(("scatter", lib.fl_scatter_update, (ctx, p(q_new), p(sel.active_idx), n, row_bytes,
-                                                                 p(st.q_work), sp)))
-                launches += 7
-                self.stage_bytes["gather_scatter"] += 5 * 2.0 * n * row_bytes
+                               p(o_src), p(st.o_work), None, None, sp)))
+                launches += 3
+                self.stage_bytes["gather_scatter"] += 2.0 * n * row_bytes
                 self.stage_bytes["quant"] += 4.0 * n * self.d * e + n * pay_row * (r - 1)
             calls.append(("scatter", lib.fl_scatter_update, (ctx, p(self.xbuf), p(sel.active_idx), n, row_bytes,
                                                              p(self.g_work), sp)))
@@ -428,6 +423,12 @@ def run_e2e(bench, args, world, barrier):
         elif tag == "quant":
             li += 1; marks[i] = (li, r)
 
+    loop_of_call, r_cur = {}, 1
+    for i, (tag, fn, a) in enumerate(bench.calls):
+        if tag == "select_tokens":
+            r_cur += 1
+        loop_of_call[i] = r_cur
+
     def one_step():
         events = {}
         copy_stream.wait_stream(bench.stream)          # the previous step has consumed its inputs
@@ -449,6 +450,9 @@ def run_e2e(bench, args, world, barrier):
                 assert rc == 0
                 end_of_loop = i == n_calls - 1 or bench.calls[i + 1][0] == "select_tokens"
                 if end_of_loop:                        # result of the loop: the last layer's new attention rows
+                    sel = bench.sels[loop_of_call[i] - 2]
+                    rc = bench.B.fl_gather_rows(bench.ctx, bench.layers[-1].o_work, sel.active_idx, sel.n,
+                                                bench.d * 2, bench.o_out_buf, stream=bench.sp)
                     out_host.copy_(bench.o_out_buf, non_blocking=True)
 
     copy_stream.wait_stream(bench.stream)

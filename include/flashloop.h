@@ -91,7 +91,8 @@ typedef struct {
 } fl_kv_stream;
 
 /* Per-layer K/V store: loop-1 base (storage type, all L rows) plus one residual stream per later loop.
- * k_res[r-2] / v_res[r-2] hold loop r. Reconstruction (Eq. 4 / Eq. 8), in binary32 and in loop order:
+ * k_res[r-2] / v_res[r-2] hold loop r and describe the same rows (equal n_rows and slot_of_pos contents).
+ * Reconstruction (Eq. 4 / Eq. 8), in binary32 and in loop order:
  *   Xhat^(r)_i = ((base_i + D_2) + D_3) + ... over the loops <= r in which position i was active. */
 typedef struct {
   void* k_base;
@@ -171,6 +172,22 @@ FL_API int fl_loop_attention(fl_ctx* ctx, const fl_shape* shape, int loop_r, con
                       const int32_t* col_idx, const int32_t* col_cnt, int32_t c, const float* lse_prev,
                       float* lse_out, const void* o_prev, void* o_out, float* col_scores_next,
                       int32_t* status, void* stream);
+
+/* The same operation (Eq. 7 / Eq. 3 with Eq. 8 inside the kernel) on position-indexed stores, which removes the
+ * gathers of Q^(r-1), O^(r-1) and the scatters of O^(r), Q^(r) around it (the gather / update steps of Appendix G):
+ *   q_store_in  [L, H, dh]: row active_idx[t] holds q_old_t
+ *   q_store_out [L, H, dh]: row active_idx[t] receives q_new_t (NULL: not written; may be q_store_in)
+ *   o_store_in  [L, H, dh]: row active_idx[t] holds o_prev_t
+ *   o_store_out [L, H, dh]: row active_idx[t] receives o_out_t (may be o_store_in)
+ *   lse_in, lse_out f32 [H, L] by position (may be the same)
+ * Rows of inactive positions are neither read nor written. q_new is [n_active, H, dh] as above. Tensor path only:
+ * returns FL_ERR_UNSUPPORTED (nothing launched) unless dtype is FL_BF16, head_dim is 128 and c <= 3072, or when
+ * the context was created with FL_FORCE_SIMT=1; callers then gather, call fl_loop_attention and scatter. */
+FL_API int fl_loop_attention_indexed(fl_ctx* ctx, const fl_shape* shape, int loop_r, const void* q_new,
+                              const void* q_store_in, void* q_store_out, const int32_t* active_idx, int32_t n_active,
+                              const fl_kv_store* store, const int32_t* col_idx, const int32_t* col_cnt, int32_t c,
+                              const float* lse_in, float* lse_out, const void* o_store_in, void* o_store_out,
+                              float* col_scores_next, int32_t* status, void* stream);
 
 /* KV-cache accounting (Section 1's 48 GiB example; Section 4.3): bytes held for one layer by this store
  * after n_loops loops, and by a dense looped cache of n_loops loops. Host-only, no device access.

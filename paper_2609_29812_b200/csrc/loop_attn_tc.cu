@@ -75,9 +75,12 @@ static_assert((2 + kPreStreams) * kMaxCols * 4 <= kSlots * kSlotBytes, "prologue
 
 struct alignas(64) TcArgs {
   CUtensorMap k_map, v_map;          // row-gather maps of the K / V base ([L, d] bf16, box 64 x 1, 128B swizzle)
-  CUtensorMap q_new_map, q_old_map;  // tile maps of the compact Q rows ([n_active, d] bf16, box 64 x 128)
-  const __nv_bfloat16* o_prev;
+  CUtensorMap q_new_map, q_old_map;  // tile maps of the compact Q rows ([n_active, d] bf16, box 64 x 128); in the
+                                     // indexed form q_old_map is a row-gather map of the Q store ([L, d], box 64 x 1)
+  const __nv_bfloat16* o_prev;       // compact rows; in the indexed form the O stores [L, d] (may be the same)
   __nv_bfloat16* o_out;
+  const __nv_bfloat16* q_new;        // indexed form only: compact new Q rows, copied into q_store at the end
+  __nv_bfloat16* q_store;            // indexed form only: Q store [L, d] that receives them, or null
   const int32_t* active_idx;
   int n_active;
   DevSide k, v;
@@ -219,7 +222,9 @@ __device__ __forceinline__ ChunkInfo chunk_info(int ci, int n_plain, int n_patch
   return c;
 }
 
-template <int BITS>
+// INDEXED: the previous loop's Q and O rows are read from, and the new O rows written to, position-indexed
+// stores (row active_idx[t] for compact row t) instead of compact buffers.
+template <int BITS, bool INDEXED>
 __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_constant__ TcArgs a) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -392,14 +397,30 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
   const int g0 = g, fill0 = fill;
   const uint32_t dirty_par0 = dirty_par_cta;
   const int n_pre = a.n_old < kPreStreams ? min((n_patch + kNC - 1) / kNC, kPrefillChunks) : 0;
-  if (tid == kTmaWarp * 32) {
+  if (warp == kTmaWarp) {
     // Q tiles of this row tile: two 64-element slabs each; rows past the compact list read as zero, rows of the
     // next block (past n_rows) are computed and dropped
-    tc::mbar_arrive_expect_tx(&ctl.q_full, 2 * kQTileBytes);
-    tc::tma_tile2d(q_old_tile, &a.q_old_map, &ctl.q_full, h * kDH, s0);
-    tc::tma_tile2d(q_old_tile + kM * 128, &a.q_old_map, &ctl.q_full, h * kDH + 64, s0);
-    tc::tma_tile2d(q_new_tile, &a.q_new_map, &ctl.q_full, h * kDH, s0);
-    tc::tma_tile2d(q_new_tile + kM * 128, &a.q_new_map, &ctl.q_full, h * kDH + 64, s0);
+    if (lane == 0) {
+      tc::mbar_arrive_expect_tx(&ctl.q_full, 2 * kQTileBytes);
+      tc::tma_tile2d(q_new_tile, &a.q_new_map, &ctl.q_full, h * kDH, s0);
+      tc::tma_tile2d(q_new_tile + kM * 128, &a.q_new_map, &ctl.q_full, h * kDH + 64, s0);
+      if (!INDEXED) {
+        tc::tma_tile2d(q_old_tile, &a.q_old_map, &ctl.q_full, h * kDH, s0);
+        tc::tma_tile2d(q_old_tile + kM * 128, &a.q_old_map, &ctl.q_full, h * kDH + 64, s0);
+      }
+    }
+    if (INDEXED) {
+      // the previous loop's Q rows come from the store: four-row gathers by position, one group of rows per lane
+      __syncwarp();
+      int y[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int r = lane * 4 + i;
+        y[i] = r < n_rows ? __ldg(a.active_idx + s0 + r) : a.L;   // row L is outside the tensor: reads as zero
+      }
+      tc::tma_gather4(q_old_tile + lane * 512, &a.q_old_map, &ctl.q_full, h * kDH, y[0], y[1], y[2], y[3]);
+      tc::tma_gather4(q_old_tile + kM * 128 + lane * 512, &a.q_old_map, &ctl.q_full, h * kDH + 64, y[0], y[1], y[2], y[3]);
+    }
   }
   // ---- the first patched chunks are built by all 512 threads straight into the (idle) ring: base row plus
   // dequantized residuals (Eq. 8), old and new operand tiles. A warp owns 4 columns of the chunk (lanes 0-15:
@@ -522,6 +543,19 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
           for (int k = 0; k < n_slots; ++k) tc::mbar_arrive(&ctl.patched[(f + k) % kSlots]);
       }
       f += n_slots;
+    }
+    if (INDEXED && a.q_store != nullptr && ok) {
+      // The Q store rows of this (row tile, head) were read by the gathers that completed q_full and belong to
+      // no other CTA: the new rows take their place for the next loop.
+      ok = warp_wait(&ctl.q_full, tile & 1, abort_flag);
+      const int pt = tid - kTmaWarp * 32;
+#pragma unroll 1
+      for (int it = pt; ok && it < n_rows * 16; it += kTmaWarps * 32) {
+        const int r = it >> 4, ch = it & 15;
+        const int pos_r = __ldg(a.active_idx + s0 + r);
+        *reinterpret_cast<uint4*>(a.q_store + (size_t)pos_r * a.d + h * kDH + ch * 8) =
+            __ldg(reinterpret_cast<const uint4*>(a.q_new + (size_t)(s0 + r) * a.d + h * kDH + ch * 8));
+      }
     }
   } else if (warp >= kIssueWarp) {
     // ========================================== MMA issuers ==========================================
@@ -708,8 +742,10 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
 #pragma unroll 1
     for (int k = 0; k < 8; ++k) {
       const int idx = k * 128 + gt, rr = idx >> 3, cc = idx & 7;
-      if (rr < n_rows)
-        tc::cp_async16(stage + rr * 128 + ((cc ^ (rr & 7)) << 4), a.o_prev + (size_t)(s0 + rr) * a.d + o_col0 + cc * 8);
+      if (rr < n_rows) {
+        const size_t src_row = INDEXED ? (size_t)__ldg(a.active_idx + s0 + rr) : (size_t)(s0 + rr);
+        tc::cp_async16(stage + rr * 128 + ((cc ^ (rr & 7)) << 4), a.o_prev + src_row * a.d + o_col0 + cc * 8);
+      }
     }
     tc::cp_async_commit();
     if (ok) ok = warp_wait(&ctl.acc_done, tile & 1, abort_flag);
@@ -752,9 +788,11 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
 #pragma unroll 1
     for (int k = 0; k < 8; ++k) {
       const int idx = k * 128 + gt, rr = idx >> 3, cc = idx & 7;
-      if (rr < n_rows)
-        *reinterpret_cast<uint4*>(a.o_out + (size_t)(s0 + rr) * a.d + o_col0 + cc * 8) =
+      if (rr < n_rows) {
+        const size_t dst_row = INDEXED ? (size_t)__ldg(a.active_idx + s0 + rr) : (size_t)(s0 + rr);
+        *reinterpret_cast<uint4*>(a.o_out + dst_row * a.d + o_col0 + cc * 8) =
             *reinterpret_cast<const uint4*>(stage + rr * 128 + ((cc ^ (rr & 7)) << 4));
+      }
     }
     if (gt == 0) TC_TRACE(2 + grp, 61, 3);
   }
@@ -798,22 +836,27 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
 }  // namespace
 
 // Returns FL_ERR_UNSUPPORTED when the tensor path does not cover the request (caller falls back to the
-// SIMT kernel, which is also CUDA).
+// SIMT kernel, which is also CUDA). indexed != 0: q_old, o_prev and o_out are position-indexed stores [L, d] and
+// q_store (may be null) receives the new Q rows.
 int fl_launch_loop_attn_tc(fl_ctx* ctx, const fl_shape* s, int loop_r, const void* q_new, const void* q_old,
                            const int32_t* active_idx, int n_active, const fl_kv_store* store, const int32_t* col_idx,
                            const int32_t* col_cnt, int c, const float* lse_prev, float* lse_out, const void* o_prev,
-                           void* o_out, int32_t* status, cudaStream_t st) {
+                           void* o_out, int indexed, void* q_store, int32_t* status, cudaStream_t st) {
   if (s->dtype != FL_BF16 || s->head_dim != kDH || c > kMaxCols) return FL_ERR_UNSUPPORTED;
   if ((size_t)ctx->max_smem_optin < kTcSmemBytes) return FL_ERR_UNSUPPORTED;
   TcArgs a{};
   const int64_t d_row = (int64_t)s->n_heads * s->head_dim;
   if (!fl_tile_tmap(ctx, store->k_base, s->L, d_row, 1, &a.k_map) ||
       !fl_tile_tmap(ctx, store->v_base, s->L, d_row, 1, &a.v_map) ||
-      !fl_tile_tmap(ctx, q_new, n_active, d_row, kM, &a.q_new_map) ||
-      !fl_tile_tmap(ctx, q_old, n_active, d_row, kM, &a.q_old_map))
+      !fl_tile_tmap(ctx, q_new, n_active, d_row, kM, &a.q_new_map))
+    return FL_ERR_UNSUPPORTED;
+  if (indexed ? !fl_tile_tmap(ctx, q_old, s->L, d_row, 1, &a.q_old_map)
+              : !fl_tile_tmap(ctx, q_old, n_active, d_row, kM, &a.q_old_map))
     return FL_ERR_UNSUPPORTED;
   a.o_prev = static_cast<const __nv_bfloat16*>(o_prev);
   a.o_out = static_cast<__nv_bfloat16*>(o_out);
+  a.q_new = static_cast<const __nv_bfloat16*>(q_new);
+  a.q_store = static_cast<__nv_bfloat16*>(q_store);
   a.active_idx = active_idx; a.n_active = n_active;
   fl_dev_side(store, true, &a.k);
   fl_dev_side(store, false, &a.v);
@@ -823,11 +866,15 @@ int fl_launch_loop_attn_tc(fl_ctx* ctx, const fl_shape* s, int loop_r, const voi
   a.L = s->L; a.H = s->n_heads; a.q_block = s->q_block; a.nb = fl_n_blocks(s);
   a.d = s->n_heads * s->head_dim; a.group = s->group; a.scale = s->sm_scale;
   const dim3 grid(a.nb, s->n_heads);   // one CTA per (query block, head); it walks the block's 128-row tiles
-#define FL_TC(BITS)                                                                                              \
+#define FL_TC2(BITS, IDX)                                                                                        \
   do {                                                                                                           \
-    auto kern = loop_attn_tc_kernel<BITS>;                                                                       \
+    auto kern = loop_attn_tc_kernel<BITS, IDX>;                                                                  \
     FL_CHECK_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcSmemBytes));  \
     kern<<<grid, kThreads, kTcSmemBytes, st>>>(a);                                                               \
+  } while (0)
+#define FL_TC(BITS)                                   \
+  do {                                                \
+    if (indexed) FL_TC2(BITS, true); else FL_TC2(BITS, false); \
   } while (0)
   switch (s->bits) {
     case 2: FL_TC(2); break;
@@ -836,5 +883,6 @@ int fl_launch_loop_attn_tc(fl_ctx* ctx, const fl_shape* s, int loop_r, const voi
     default: FL_TC(16); break;
   }
 #undef FL_TC
+#undef FL_TC2
   return fl_launch_status();
 }

@@ -144,17 +144,33 @@ class LayerState:
                             self.col_idx, self.col_cnt, self.c, self.lse, self.lse, o_prev, o_out,
                             col_scores_next, status=self.status)   # lse updated in place (active rows only)
 
+    def attention_indexed(self, loop_r, q_new, sel: TokenSelection, col_scores_next=None, check=True) -> int:
+        """Same step on the position-indexed Q / O stores, updated in place (no gathers or scatters around it);
+        returns the status code, FL_ERR_UNSUPPORTED when the shape is outside the tensor path."""
+        return B.fl_loop_attention_indexed(self.ctx, self.shape, loop_r, q_new, self.q_store, self.q_store,
+                                           sel.active_idx, sel.n, self.store, self.col_idx, self.col_cnt, self.c,
+                                           self.lse, self.lse, self.o_store, self.o_store, col_scores_next,
+                                           status=self.status, check=check)
+
     def check_status(self):
         """Synchronises and raises if a kernel reported an asynchronous error (e.g. a bounded wait ran out)."""
         code = int(self.status.item())
         if code != 0:
             raise B.FlashLoopError("device status", code)
 
-    def sparse_loop(self, loop_r, q_new, k_new, v_new, sel: TokenSelection, want_col_scores_next=False):
-        """One loop r >= 2 for this layer: store residuals, gather the carried rows, attend, scatter back.
-        q_new, k_new, v_new: [n, H, dh] rows of the active tokens.  Returns (o_rows, col_scores_next)."""
+    def sparse_loop(self, loop_r, q_new, k_new, v_new, sel: TokenSelection, want_col_scores_next=False,
+                    indexed=False):
+        """One loop r >= 2 for this layer: store residuals, gather the carried rows, attend, scatter back
+        (indexed=True: one call on the stores instead).  q_new, k_new, v_new: [n, H, dh] rows of the active tokens.
+        Returns (o_rows, col_scores_next)."""
         self.alloc_stream(sel)
         self.quantize(loop_r, k_new, v_new, sel)
+        if indexed:
+            csn = None
+            if want_col_scores_next:
+                csn = torch.zeros(self.w.n_heads, self.nb, self.c, dtype=torch.float32, device=self.dev)
+            self.attention_indexed(loop_r, q_new, sel, csn)
+            return self.gather(self.o_store, sel), csn
         q_old = self.gather(self.q_store, sel)
         o_prev = self.gather(self.o_store, sel)
         o_out = torch.empty_like(o_prev)

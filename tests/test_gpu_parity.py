@@ -272,6 +272,53 @@ def test_chained_layer_all_on_gpu(env, case):
     assert dense == dense_ref * w.L and abs(fl - fl_ref * w.L) <= 4 * w.n_loops
 
 
+def test_indexed_attention_matches_compact_path_and_oracle(env):
+    """fl_loop_attention_indexed on the position-indexed stores (updated in place): same rows as gather -> fl_loop_attention ->
+    scatter (bit for bit: the same kernel arithmetic), and the oracle's within the stated tolerance; the Q store
+    ends up holding the new rows, inactive rows stay untouched."""
+    import torch
+    B, P, ctx = env
+    w = small_bf16(L=1500, H=2, R=3)
+    x = workloads.make_layer_inputs(w, seed=11)
+    ref = fo.LayerOracle(w.L, w.n_heads, w.head_dim, w.q_block, w.bits, w.group, w.eps, w.sm_scale,
+                         storage=w.dtype).run(x.G, x.Q, x.K, x.V, [w.k_tokens] * 2, [w.col_budget] * 2)
+    states = []
+    for indexed in (False, True):
+        st = P.LayerState(ctx, w)
+        st.dense_loop(to_dev(x.Q[0], w), to_dev(x.K[0], w), to_dev(x.V[0], w))
+        st.select_columns_dense()
+        q0 = st.q_store.clone()
+        for r in (2, 3):
+            sel = oracle_selection(P, w, ref, r)
+            act = ref["active"][r - 2]
+            st.sparse_loop(r, to_dev(x.Q[r - 1][act], w), to_dev(x.K[r - 1][act], w), to_dev(x.V[r - 1][act], w),
+                           sel, indexed=indexed)
+            st.check_status()
+        states.append((st, q0))
+    (a, _), (b, q0) = states
+    assert torch.equal(a.o_store, b.o_store)
+    assert torch.equal(a.q_store, b.q_store)
+    assert torch.equal(a.lse, b.lse)
+    assert_attn_close(to_np(b.o_store), ref["loops"][-1]["O_full"], "indexed final O store", loops=2)
+    touched = np.zeros(w.L, dtype=bool)
+    touched[ref["active"][0]] = True
+    assert torch.equal(b.q_store[torch.from_numpy(~touched).to(b.q_store.device)],
+                       q0[torch.from_numpy(~touched).to(q0.device)])
+    # shapes outside the tensor path are refused before anything is launched
+    w32 = workloads.config1()
+    x32 = workloads.make_layer_inputs(w32, seed=3)
+    st32 = P.LayerState(ctx, w32)
+    st32.dense_loop(to_dev(x32.Q[0], w32), to_dev(x32.K[0], w32), to_dev(x32.V[0], w32))
+    st32.select_columns_dense()
+    sel = P.select_tokens(ctx, st32.shape, 2, to_dev(x32.G[0], w32), to_dev(x32.G[1], w32), None, w32.k_tokens)
+    act = to_np(sel.active_idx).astype(np.int64)
+    st32.alloc_stream(sel)
+    st32.quantize(2, to_dev(x32.K[1][act], w32), to_dev(x32.V[1][act], w32), sel)
+    o_before = st32.o_store.clone()
+    rc = st32.attention_indexed(2, to_dev(x32.Q[1][act], w32), sel, check=False)
+    assert rc == -2 and torch.equal(st32.o_store, o_before)
+
+
 def test_binary32_simt_attention_path_on_bf16_storage(env):
     """The SIMT attention kernels also serve bf16 storage (forced here; normally the tensor path runs)."""
     import os

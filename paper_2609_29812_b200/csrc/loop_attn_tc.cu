@@ -663,10 +663,16 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
       tc::tmem_ld32(s_addr, *reinterpret_cast<uint32_t(*)[32]>(&r[0]));
       tc::tmem_ld32(s_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&r[32]));
       tc::tmem_wait_ld();
-      // S is in registers: hand the buffer back so that the next chunk's QK^T runs under the arithmetic below
+      // S is in registers: hand the buffer back so that the next chunk's QK^T runs under the arithmetic below.
+      // The previous chunk's P store has had this long to land: it is announced now instead of being waited for
+      // at the end of its own iteration.
+      if (ci > 0) tc::tmem_wait_st();
       tc::tc_fence_before();
       __syncwarp();
-      if (lane == 0) tc::mbar_arrive(&ctl.s_taken[grp]);
+      if (lane == 0) {
+        tc::mbar_arrive(&ctl.s_taken[grp]);
+        if (ci > 0) tc::mbar_arrive(&ctl.p_full[grp][pb ^ 1]);
+      }
       // rows of a warp that lie at or after every column of the chunk need no causal mask; rows beyond the
       // tile's last (their results are never stored) must not force the masked path
       const bool unmasked = __all_sync(0xffffffffu, !row_ok || ctl.chunk_last[ci] <= pos);
@@ -726,12 +732,13 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
       if (n_use >= 1 && !warp_wait(&ctl.p_free[grp][pb], (n_use - 1) & 1, abort_flag)) { ok = false; break; }
       tc::tc_fence_after();
       tc::tmem_st32(p_addr + pb * 32, *reinterpret_cast<uint32_t(*)[32]>(&r[0]));
-      tc::tmem_wait_st();
       if (gt == 0) TC_TRACE(2 + grp, ci, 2);
+    }
+    if (ok && n_chunks > 0) {   // the last chunk's P
+      tc::tmem_wait_st();
       tc::tc_fence_before();
       __syncwarp();
-      if (lane == 0) tc::mbar_arrive(&ctl.p_full[grp][pb]);
-      if (gt == 0) TC_TRACE(2 + grp, ci, 3);
+      if (lane == 0) tc::mbar_arrive(&ctl.p_full[grp][(g0 + n_chunks - 1) & 1]);
     }
     // ---- epilogue ------------------------------------------------------------------------------------
     // Each group finishes 64 of the 128 head-dim columns. Its half of the O_prev tile is staged in the group's

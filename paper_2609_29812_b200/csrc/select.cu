@@ -195,6 +195,8 @@ constexpr int kSelCap = 49152;    // 192 KB of keys
 constexpr int kSelSmall = 2048;
 
 struct SelectSmem2 {
+  uint32_t hist12[4096];
+  uint32_t warp_tot[32];
   uint32_t hist[256];
   uint32_t warp_gt[32], warp_eq[32];
   uint32_t prefix, k_rem, bin_cnt, n_small;
@@ -214,21 +216,33 @@ __device__ __forceinline__ void hist_add(uint32_t* hist, bool on, uint32_t digit
   else if (on && digit != d0) atomicAdd(&hist[digit], 1u);
 }
 
-// one radix pass (8 bits at `shift`) over list[0..m4*4): histogram of the keys that match `prefix` above the
-// digit. Four keys per thread and step: the four dependent chains (load, vote, atomic) overlap.
-__device__ __forceinline__ void radix_hist_pass(const uint32_t* list, int m4, int shift, uint32_t prefix, uint32_t* hist) {
+// one radix pass (`bits` <= 8 bits at `shift`) over list[0..m4*4): histogram of the keys that match `prefix`
+// above the digit. Four keys per thread and step: the four dependent chains (load, vote, atomic) overlap.
+__device__ __forceinline__ void radix_hist_pass(const uint32_t* list, int m4, int shift, int bits, uint32_t prefix,
+                                                uint32_t* hist) {
   const int tid = threadIdx.x, lane = tid & 31;
-  const uint32_t hi_mask = shift == 24 ? 0u : (0xFFFFFFFFu << (shift + 8));
+  const uint32_t hi_mask = shift + bits >= 32 ? 0u : (0xFFFFFFFFu << (shift + bits));
+  const uint32_t dmask = (1u << bits) - 1u;
   const uint4* l4 = reinterpret_cast<const uint4*>(list);
   for (int base = 0; base < m4; base += kSelThreads) {
     const int i = base + tid;
     const bool in = i < m4;
     const uint4 kv = in ? l4[i] : make_uint4(0, 0, 0, 0);
-    hist_add(hist, in && (kv.x & hi_mask) == prefix, (kv.x >> shift) & 0xFFu, lane);
-    hist_add(hist, in && (kv.y & hi_mask) == prefix, (kv.y >> shift) & 0xFFu, lane);
-    hist_add(hist, in && (kv.z & hi_mask) == prefix, (kv.z >> shift) & 0xFFu, lane);
-    hist_add(hist, in && (kv.w & hi_mask) == prefix, (kv.w >> shift) & 0xFFu, lane);
+    hist_add(hist, in && (kv.x & hi_mask) == prefix, (kv.x >> shift) & dmask, lane);
+    hist_add(hist, in && (kv.y & hi_mask) == prefix, (kv.y >> shift) & dmask, lane);
+    hist_add(hist, in && (kv.z & hi_mask) == prefix, (kv.z >> shift) & dmask, lane);
+    hist_add(hist, in && (kv.w & hi_mask) == prefix, (kv.w >> shift) & dmask, lane);
   }
+}
+
+// First level: 12-bit digit (sign, exponent, three mantissa bits) counted while the keys are staged. A warp whose
+// 32 keys share the digit adds them with one atomic; otherwise every lane adds itself (a handful of lanes per bin).
+__device__ __forceinline__ void hist12_add(uint32_t* hist12, uint32_t key, int lane) {
+  const uint32_t d = key >> 20;
+  int all_same;
+  __match_all_sync(0xffffffffu, d, &all_same);
+  if (all_same) { if (lane == 0) atomicAdd(&hist12[d], 32u); }
+  else atomicAdd(&hist12[d], 1u);
 }
 
 __global__ void __launch_bounds__(kSelThreads, 1) column_select_smem_kernel(const float* __restrict__ col_scores,
@@ -252,62 +266,116 @@ __global__ void __launch_bounds__(kSelThreads, 1) column_select_smem_kernel(cons
   if (tid == 0) col_cnt[prob] = k;
   if (k == 0) return;
   const int n4 = (n + 3) >> 2;
-  // ---- stage the order-preserving keys --------------------------------------------------------------
-  if (vec_ok) {
+  // ---- stage the order-preserving keys, counting their 12-bit digits on the way -----------------------------
+  for (int i = tid; i < 4096; i += kSelThreads) sm.hist12[i] = 0;
+  __syncthreads();
+  {
     const float4* v4 = reinterpret_cast<const float4*>(vals);
     uint4* k4 = reinterpret_cast<uint4*>(keys);
-    for (int i = tid; i < (n >> 2); i += kSelThreads) {
-      const float4 v = __ldg(v4 + i);
-      k4[i] = make_uint4(ordered_key(v.x), ordered_key(v.y), ordered_key(v.z), ordered_key(v.w));
+    for (int base = 0; base < n4; base += kSelThreads) {   // whole warps run every step: padding keys are 0 (bin 0)
+      const int i = base + tid;
+      uint4 kv = make_uint4(0, 0, 0, 0);
+      if (i < n4) {
+        if (vec_ok && i * 4 + 3 < n) {
+          const float4 v = __ldg(v4 + i);
+          kv = make_uint4(ordered_key(v.x), ordered_key(v.y), ordered_key(v.z), ordered_key(v.w));
+        } else {
+          if (i * 4 + 0 < n) kv.x = ordered_key(__ldg(vals + i * 4 + 0));
+          if (i * 4 + 1 < n) kv.y = ordered_key(__ldg(vals + i * 4 + 1));
+          if (i * 4 + 2 < n) kv.z = ordered_key(__ldg(vals + i * 4 + 2));
+          if (i * 4 + 3 < n) kv.w = ordered_key(__ldg(vals + i * 4 + 3));
+        }
+        k4[i] = kv;
+      }
+      hist12_add(sm.hist12, kv.x, lane);
+      hist12_add(sm.hist12, kv.y, lane);
+      hist12_add(sm.hist12, kv.z, lane);
+      hist12_add(sm.hist12, kv.w, lane);
     }
-    for (int i = (n & ~3) + tid; i < n4 * 4; i += kSelThreads) keys[i] = i < n ? ordered_key(__ldg(vals + i)) : 0u;
-  } else {
-    for (int i = tid; i < n4 * 4; i += kSelThreads) keys[i] = i < n ? ordered_key(__ldg(vals + i)) : 0u;
   }
+  __syncthreads();
   uint32_t prefix = 0, k_rem = 0;
   const bool take_all = k >= n;
   if (!take_all) {
-    k_rem = (uint32_t)k;
-    const uint32_t* list = keys;
-    int m4 = n4;
-    for (int shift = 24; shift >= 0; shift -= 8) {
-      for (int i = tid; i < 256; i += kSelThreads) sm.hist[i] = 0;
-      __syncthreads();   // also orders the staging / compaction writes before the reads below
-      radix_hist_pass(list, m4, shift, prefix, sm.hist);
-      __syncthreads();
-      if (warp == 0) {
-        // lane owns digits [8*lane, 8*lane+8); find the digit holding the k_rem-th largest
-        uint32_t local[8], sum = 0;
+    // ---- first level: the 12-bit bin that holds the k-th largest key (thread t owns bins 4t .. 4t+3) -------
+    {
+      uint32_t loc[4], sum = 0;
 #pragma unroll
-        for (int j = 0; j < 8; ++j) { local[j] = sm.hist[lane * 8 + j]; sum += local[j]; }
-        uint32_t incl = sum;
+      for (int j = 0; j < 4; ++j) { loc[j] = sm.hist12[tid * 4 + j]; sum += loc[j]; }
+      uint32_t incl = sum;                       // inclusive suffix sum over the warp (higher lanes = larger keys)
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-          const uint32_t v = __shfl_down_sync(0xffffffffu, incl, o);
-          if (lane + o < 32) incl += v;
-        }
-        const uint32_t above = incl - sum;
-        if (above < k_rem && k_rem <= above + sum) {
-          uint32_t acc = above;
-          for (int j = 7; j >= 0; --j) {
-            if (k_rem <= acc + local[j]) {
-              sm.prefix = prefix | ((uint32_t)(lane * 8 + j) << shift);
-              sm.k_rem = k_rem - acc;
-              sm.bin_cnt = local[j];
-              break;
-            }
-            acc += local[j];
-          }
-        }
-        if (lane == 0) sm.n_small = 0;
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t v = __shfl_down_sync(0xffffffffu, incl, o);
+        if (lane + o < 32) incl += v;
       }
+      if (lane == 0) sm.warp_tot[warp] = incl;
+      __syncthreads();
+      uint32_t above = incl - sum;               // keys in bins above this thread's
+      for (int w2 = warp + 1; w2 < 32; ++w2) above += sm.warp_tot[w2];
+      if (above < (uint32_t)k && (uint32_t)k <= above + sum) {
+        uint32_t acc = above;
+        for (int j = 3; j >= 0; --j) {
+          if ((uint32_t)k <= acc + loc[j]) {
+            sm.prefix = (uint32_t)(tid * 4 + j) << 20;
+            sm.k_rem = (uint32_t)k - acc;
+            sm.bin_cnt = loc[j];
+            break;
+          }
+          acc += loc[j];
+        }
+      }
+      if (tid == 0) sm.n_small = 0;
       __syncthreads();
       prefix = sm.prefix;
       k_rem = sm.k_rem;
+    }
+    const uint32_t* list = keys;
+    int m4 = n4;
+    int fixed = 12;                              // leading bits of the threshold found so far
+    for (int pass = 0; pass < 4; ++pass) {
+      // pass 0 only tries the compaction; passes 1-3 resolve 8, 8 and 4 more bits
+      if (pass > 0) {
+        const int bits = pass == 3 ? 4 : 8;
+        const int shift = 32 - fixed - bits;
+        for (int i = tid; i < 256; i += kSelThreads) sm.hist[i] = 0;
+        __syncthreads();
+        radix_hist_pass(list, m4, shift, bits, prefix, sm.hist);
+        __syncthreads();
+        if (warp == 0) {
+          // lane owns digits [8*lane, 8*lane+8); find the digit holding the k_rem-th largest
+          uint32_t local[8], sum = 0;
+#pragma unroll
+          for (int j = 0; j < 8; ++j) { local[j] = sm.hist[lane * 8 + j]; sum += local[j]; }
+          uint32_t incl = sum;
+#pragma unroll
+          for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t v = __shfl_down_sync(0xffffffffu, incl, o);
+            if (lane + o < 32) incl += v;
+          }
+          const uint32_t above = incl - sum;
+          if (above < k_rem && k_rem <= above + sum) {
+            uint32_t acc = above;
+            for (int j = 7; j >= 0; --j) {
+              if (k_rem <= acc + local[j]) {
+                sm.prefix = prefix | ((uint32_t)(lane * 8 + j) << shift);
+                sm.k_rem = k_rem - acc;
+                sm.bin_cnt = local[j];
+                break;
+              }
+              acc += local[j];
+            }
+          }
+          if (lane == 0) sm.n_small = 0;
+        }
+        __syncthreads();
+        prefix = sm.prefix;
+        k_rem = sm.k_rem;
+        fixed += bits;
+      }
       const uint32_t bin_cnt = sm.bin_cnt;
-      if (shift > 0 && list == keys && bin_cnt <= (uint32_t)(kSelSmall - 4)) {
+      if (fixed < 32 && list == keys && bin_cnt <= (uint32_t)(kSelSmall - 4)) {
         // the k-th largest key lies in a small bin: finish on that bin's keys alone
-        const uint32_t hi_mask = 0xFFFFFFFFu << shift;
+        const uint32_t hi_mask = 0xFFFFFFFFu << (32 - fixed);
         const uint4* k4 = reinterpret_cast<const uint4*>(keys);
         for (int base = 0; base < n4; base += kSelThreads) {
           const int i = base + tid;
@@ -316,6 +384,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) column_select_smem_kernel(cons
           uint32_t flags = 0;
 #pragma unroll
           for (int j = 0; j < 4; ++j) flags |= (i < n4 && (kk[j] & hi_mask) == prefix ? 1u : 0u) << j;
+          if (__ballot_sync(0xffffffffu, flags != 0) == 0) continue;
           // exclusive prefix of the per-lane counts over the warp, then one atomic per warp
           const uint32_t cnt = __popc(flags);
           uint32_t incl = cnt;
@@ -326,7 +395,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) column_select_smem_kernel(cons
           }
           const uint32_t total = __shfl_sync(0xffffffffu, incl, 31);
           uint32_t off = 0;
-          if (lane == 0 && total != 0) off = atomicAdd(&sm.n_small, total);
+          if (lane == 0) off = atomicAdd(&sm.n_small, total);
           off = __shfl_sync(0xffffffffu, off, 0) + incl - cnt;
 #pragma unroll
           for (int j = 0; j < 4; ++j)
@@ -343,8 +412,6 @@ __global__ void __launch_bounds__(kSelThreads, 1) column_select_smem_kernel(cons
       }
       __syncthreads();
     }
-  } else {
-    __syncthreads();
   }
   const uint32_t thr = prefix;
   // ---- index-ordered compaction from the staged keys: each warp owns a contiguous span of whole uint4s ------
@@ -482,7 +549,7 @@ extern "C" int fl_select_columns(fl_ctx* ctx, const fl_shape* shape, const float
   FL_REQUIRE(nb <= 65535 * 1024 && shape->n_heads <= 65535);
   dim3 grid(nb, shape->n_heads);
   const size_t key_bytes = sizeof(uint32_t) * (((size_t)n_cand + 3) & ~(size_t)3);
-  if (n_cand <= kSelCap && key_bytes + 16384 <= (size_t)ctx->max_smem_optin) {
+  if (n_cand <= kSelCap && key_bytes + 32768 <= (size_t)ctx->max_smem_optin) {
     // keys staged in shared memory: the scores are read from global memory once
     const int vec_ok = (fl_aligned16(col_scores) && n_cand % 4 == 0) ? 1 : 0;
     FL_CHECK_CUDA(cudaFuncSetAttribute(column_select_smem_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,

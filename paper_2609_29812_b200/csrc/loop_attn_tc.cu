@@ -347,33 +347,11 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
         ord_mask[dst] = mask;
         if (mask != 0) atomicOr(&ctl.chunk_mask[patched ? (dst - tot0) / kNC : patch_chunks + dst / kNC], mask);
         if (patched && dst - tot0 < kPrefillChunks * kNC && a.n_old < kPreStreams) {
-          // one of the columns the whole CTA builds next: keep its stream rows and pull its base rows and
-          // payloads towards the L2 now, so that the build finds them there
+          // one of the columns the whole CTA builds next: keep its stream rows
           const int pr = dst - tot0;
-          const size_t row_off = ((size_t)j * a.d + (size_t)h * kDH) * 2;
-          tc::prefetch_l2(static_cast<const uint8_t*>(a.k.base) + row_off);
-          tc::prefetch_l2(static_cast<const uint8_t*>(a.k.base) + row_off + 128);
-          tc::prefetch_l2(static_cast<const uint8_t*>(a.v.base) + row_off);
-          tc::prefetch_l2(static_cast<const uint8_t*>(a.v.base) + row_off + 128);
 #pragma unroll 1
-          for (int s = 0; s < kPreStreams; ++s) {
-            const int sl = s <= a.n_old ? raw_slot[s * kMaxCols + u] : -1;
-            ctl.pre_slot[s][pr] = sl;
-            if (sl >= 0) {
-              const size_t code_off = BITS == 16 ? ((size_t)sl * a.d + (size_t)h * kDH) * 2
-                                                 : (size_t)sl * (a.d * BITS / 8) + (size_t)h * (kDH * BITS / 8);
-              tc::prefetch_l2(a.k.s[s].codes + code_off);
-              tc::prefetch_l2(a.v.s[s].codes + code_off);
-              if (BITS == 16) {
-                tc::prefetch_l2(a.k.s[s].codes + code_off + 128);
-                tc::prefetch_l2(a.v.s[s].codes + code_off + 128);
-              } else {
-                const size_t gi = (size_t)sl * (a.d / a.group) + (size_t)h * (kDH / a.group);
-                tc::prefetch_l2(a.k.s[s].scale + gi); tc::prefetch_l2(a.k.s[s].zero + gi);
-                tc::prefetch_l2(a.v.s[s].scale + gi); tc::prefetch_l2(a.v.s[s].zero + gi);
-              }
-            }
-          }
+          for (int s = 0; s < kPreStreams; ++s)
+            ctl.pre_slot[s][pr] = s <= a.n_old ? raw_slot[s * kMaxCols + u] : -1;
         }
       }
       before0 += __popc(m0);

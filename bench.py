@@ -32,6 +32,11 @@ METRIC = "loop_r_prefill_tokens_per_s"
 UNIT = "tokens/s"
 
 
+# DRAM bytes one attention launch of the default workload moves, from one ncu capture of exactly that launch shape
+# (one layer of the 48: every layer launches the same grid); the live timing of this file cannot measure it.
+NCU_ATTN_TRAFFIC_BYTES = 152.1e6
+
+
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -362,7 +367,11 @@ def run_ours(args):
                 "unit": "GB/s"}
     roof["frac"] = roof["achieved"] / roof["peak"]
     roof.update({"kernel": "fl_loop_attention", "avg_launch_ms": avg_attn_ms, "launches": len(attn_ms) // args.steps,
-                 "flops_per_launch": flops, "bytes_per_launch": byt, "traffic": None, "peak_source": peaks["source"],
+                 "flops_per_launch": flops, "bytes_per_launch": byt,
+                 "traffic": NCU_ATTN_TRAFFIC_BYTES if (args.workload == "c3" and not args.L) else None,
+                 "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum per launch of this shape, mean of "
+                                   "loops 2-4 (one capture, summary under profiles/)",
+                 "kernel_name": "loop_attn_tc_kernel", "peak_source": peaks["source"],
                  "share_of_step": sum(attn_ms) / args.steps / ms})
     # whole-step roofline: sum over stages of max(flops / tensor peak, bytes / HBM bandwidth)
     t_roof = sum(max(f / (peaks["bf16_tflops"] * 1e12), b / (peaks["hbm_gbs"] * 1e9))

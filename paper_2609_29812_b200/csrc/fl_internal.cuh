@@ -160,7 +160,7 @@ template <typename T, int BITS>
 struct Payload8 {
   uint4 raw;      // BITS 16: the stored row piece (first 16 bytes); 8: x,y; 4 and 2: x
   uint4 raw_hi;   // BITS 16 with binary32 storage: the second 16 bytes
-  float sc, zr;
+  __half sc, zr;  // kept as loaded: converting here would make the load round wait for its own data
 };
 template <typename T, int BITS>
 __device__ __forceinline__ void payload_load(const DevStream& st, int slot, int elem, int d, int group,
@@ -180,8 +180,8 @@ __device__ __forceinline__ void payload_load(const DevStream& st, int slot, int 
       p.raw.x = __ldg(reinterpret_cast<const uint16_t*>(row + elem / 4));
     }
     const size_t gi = (size_t)slot * (d / group) + elem / group;
-    p.sc = __half2float(__ldg(st.scale + gi));
-    p.zr = __half2float(__ldg(st.zero + gi));
+    p.sc = __ldg(st.scale + gi);
+    p.zr = __ldg(st.zero + gi);
   }
 }
 template <typename T, int BITS>
@@ -202,6 +202,7 @@ __device__ __forceinline__ void payload_apply(const Payload8<T, BITS>& p, float 
       }
     }
   } else {
+    const float sc = __half2float(p.sc), zr = __half2float(p.zr);
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       uint32_t c;
@@ -210,7 +211,7 @@ __device__ __forceinline__ void payload_apply(const Payload8<T, BITS>& p, float 
       else c = (p.raw.x >> (2 * i)) & 0x3u;
       // code -> float without the conversion unit: 2^23 + c is exact in binary32
       const float cf = __fsub_rn(__uint_as_float(0x4B000000u | c), 8388608.f);
-      x[i] = __fadd_rn(x[i], __fmaf_rn(cf, p.sc, p.zr));
+      x[i] = __fadd_rn(x[i], __fmaf_rn(cf, sc, zr));
     }
   }
 }

@@ -27,6 +27,7 @@ import numpy as np
 ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
+from paper_2609_29812_b200 import replicas  # noqa: E402  (plain Python: importable without CUDA)
 
 METRIC = "loop_r_prefill_tokens_per_s"
 UNIT = "tokens/s"
@@ -349,9 +350,8 @@ def run_ours(args):
     barrier()
     clocks = sampler.stop()
     ms = t0.elapsed_time(t1) / args.steps
-    if world > 1:
-        t = torch.tensor([ms], device=device); dist.all_reduce(t, op=dist.ReduceOp.MAX); ms = float(t.item())
-    value = world * w.L / (ms * 1e-3)
+    ms = replicas.max_over_ranks(ms, world, device)
+    value = replicas.job_throughput(w.L, world, ms)
 
     # dominant kernel: loop attention
     attn_ms = [a.elapsed_time(b) for a, b in attn_events]
@@ -477,9 +477,8 @@ def run_e2e(bench, args, world, barrier):
     t1.record(bench.stream)
     barrier()
     ms = t0.elapsed_time(t1) / steps
-    if world > 1:
-        t = torch.tensor([ms], device=bench.dev); dist.all_reduce(t, op=dist.ReduceOp.MAX); ms = float(t.item())
-    return {"value": world * w.L / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms, "h2d_bytes_per_step": h2d,
+    ms = replicas.max_over_ranks(ms, world, bench.dev)
+    return {"value": replicas.job_throughput(w.L, world, ms), "unit": UNIT, "ms_per_step": ms, "h2d_bytes_per_step": h2d,
             "d2h_bytes_per_step": d2h,
             "note": "pinned host inputs copied on a side stream ahead of the compute stream; last layer's new O rows read back per loop"}
 

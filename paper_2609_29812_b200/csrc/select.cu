@@ -376,30 +376,27 @@ __global__ void __launch_bounds__(kSelThreads, 1) column_select_smem_kernel(cons
       if (fixed < 32 && list == keys && bin_cnt <= (uint32_t)(kSelSmall - 4)) {
         // the k-th largest key lies in a small bin: finish on that bin's keys alone
         const uint32_t hi_mask = 0xFFFFFFFFu << (32 - fixed);
-        const uint4* k4 = reinterpret_cast<const uint4*>(keys);
-        for (int base = 0; base < n4; base += kSelThreads) {
-          const int i = base + tid;
-          const uint4 kv = i < n4 ? k4[i] : make_uint4(0, 0, 0, 0);
-          const uint32_t kk[4] = {kv.x, kv.y, kv.z, kv.w};
-          uint32_t flags = 0;
+        const int n_pad = n4 * 4;
+        for (int base = warp * 128; base < n_pad; base += kSelThreads * 4) {   // 128 keys per warp and step
+          uint32_t kk[4], m[4];
+          uint32_t total = 0;
 #pragma unroll
-          for (int j = 0; j < 4; ++j) flags |= (i < n4 && (kk[j] & hi_mask) == prefix ? 1u : 0u) << j;
-          if (__ballot_sync(0xffffffffu, flags != 0) == 0) continue;
-          // exclusive prefix of the per-lane counts over the warp, then one atomic per warp
-          const uint32_t cnt = __popc(flags);
-          uint32_t incl = cnt;
-#pragma unroll
-          for (int o = 1; o < 32; o <<= 1) {
-            const uint32_t v = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl += v;
+          for (int j = 0; j < 4; ++j) {
+            const int i = base + j * 32 + lane;
+            kk[j] = i < n_pad ? keys[i] : 0u;
+            m[j] = __ballot_sync(0xffffffffu, i < n_pad && (kk[j] & hi_mask) == prefix);
+            total += __popc(m[j]);
           }
-          const uint32_t total = __shfl_sync(0xffffffffu, incl, 31);
+          if (total == 0) continue;
           uint32_t off = 0;
           if (lane == 0) off = atomicAdd(&sm.n_small, total);
-          off = __shfl_sync(0xffffffffu, off, 0) + incl - cnt;
+          off = __shfl_sync(0xffffffffu, off, 0);
+          const uint32_t lt = (1u << lane) - 1;
 #pragma unroll
-          for (int j = 0; j < 4; ++j)
-            if ((flags >> j) & 1u) sm.small[off++] = kk[j];
+          for (int j = 0; j < 4; ++j) {
+            if ((m[j] >> lane) & 1u) sm.small[off + __popc(m[j] & lt)] = kk[j];
+            off += __popc(m[j]);
+          }
         }
         __syncthreads();
         // pad the list to a multiple of four with keys that cannot match the prefix of any later pass
@@ -414,20 +411,15 @@ __global__ void __launch_bounds__(kSelThreads, 1) column_select_smem_kernel(cons
     }
   }
   const uint32_t thr = prefix;
-  // ---- index-ordered compaction from the staged keys: each warp owns a contiguous span of whole uint4s ------
-  const int span4 = (n4 + 31) / 32;                    // uint4s per warp
-  const int beg4 = warp * span4, end4 = min(n4, beg4 + span4);
-  const uint4* k4 = reinterpret_cast<const uint4*>(keys);
+  // ---- index-ordered compaction from the staged keys: each warp owns a contiguous span, walked 128 keys at a
+  // time (lane l holds keys l, 32 + l, 64 + l, 96 + l of the step: votes give every key its place in index order)
+  const int span = ((n + 31) / 32 + 127) / 128 * 128;
+  const int beg = warp * span, end = min(n, beg + span);
   uint32_t gt = 0, eq = 0;
-  for (int i = beg4 + lane; i < end4; i += 32) {
-    const uint4 kv = k4[i];
-    const uint32_t kk[4] = {kv.x, kv.y, kv.z, kv.w};
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const bool valid = i * 4 + j < n;
-      gt += (valid && (take_all || kk[j] > thr)) ? 1u : 0u;
-      eq += (valid && !take_all && kk[j] == thr) ? 1u : 0u;
-    }
+  for (int i = beg + lane; i < end; i += 32) {
+    const uint32_t key = keys[i];
+    gt += (take_all || key > thr) ? 1u : 0u;
+    eq += (!take_all && key == thr) ? 1u : 0u;
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
@@ -438,41 +430,45 @@ __global__ void __launch_bounds__(kSelThreads, 1) column_select_smem_kernel(cons
   __syncthreads();
   uint32_t gt_before = 0, eq_before = 0;
   for (int w = 0; w < warp; ++w) { gt_before += sm.warp_gt[w]; eq_before += sm.warp_eq[w]; }
-  for (int base = beg4; base < end4; base += 32) {
-    const int i = base + lane;
-    uint32_t f_gt = 0, f_eq = 0;
-    if (i < end4) {
-      const uint4 kv = k4[i];
-      const uint32_t kk[4] = {kv.x, kv.y, kv.z, kv.w};
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const bool valid = i * 4 + j < n;
-        f_gt |= (valid && (take_all || kk[j] > thr) ? 1u : 0u) << j;
-        f_eq |= (valid && !take_all && kk[j] == thr ? 1u : 0u) << j;
-      }
-    }
-    // exclusive prefixes over the warp, in index order (lane-major, then the four keys of the lane)
-    const uint32_t c_gt = __popc(f_gt), c_eq = __popc(f_eq);
-    uint32_t i_gt = c_gt, i_eq = c_eq;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const uint32_t v_gt = __shfl_up_sync(0xffffffffu, i_gt, o);
-      const uint32_t v_eq = __shfl_up_sync(0xffffffffu, i_eq, o);
-      if (lane >= o) { i_gt += v_gt; i_eq += v_eq; }
-    }
-    uint32_t my_gt = gt_before + i_gt - c_gt, my_eq = eq_before + i_eq - c_eq;
+  const uint32_t lt = (1u << lane) - 1;
+  for (int base = beg; base < end; base += 128) {
+    uint32_t kk[4], mg[4];
+    bool any_eq_lane = false;
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
-      const bool is_gt = (f_gt >> j) & 1u, is_eq = (f_eq >> j) & 1u;
-      int rank = -1;
-      if (is_gt) rank = (int)(my_gt + min(my_eq, k_rem));
-      else if (is_eq && my_eq < k_rem) rank = (int)(my_gt + my_eq);
-      if (rank >= 0) out[rank] = cols != nullptr ? __ldg(cols + i * 4 + j) : i * 4 + j;
-      my_gt += is_gt ? 1u : 0u;
-      my_eq += is_eq ? 1u : 0u;
+      const int i = base + j * 32 + lane;
+      kk[j] = i < end ? keys[i] : 0u;
+      mg[j] = __ballot_sync(0xffffffffu, i < end && (take_all || kk[j] > thr));
+      any_eq_lane |= i < end && !take_all && kk[j] == thr;
     }
-    gt_before += __shfl_sync(0xffffffffu, i_gt, 31);
-    eq_before += __shfl_sync(0xffffffffu, i_eq, 31);
+    if (!__any_sync(0xffffffffu, any_eq_lane)) {
+      // no key of the step ties with the threshold: the selected ones are the greater ones, in index order
+      uint32_t off = gt_before + min(eq_before, k_rem);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        if ((mg[j] >> lane) & 1u) {
+          const int i = base + j * 32 + lane;
+          out[off + __popc(mg[j] & lt)] = cols != nullptr ? __ldg(cols + i) : i;
+        }
+        off += __popc(mg[j]);
+      }
+      gt_before += __popc(mg[0]) + __popc(mg[1]) + __popc(mg[2]) + __popc(mg[3]);
+    } else {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int i = base + j * 32 + lane;
+        const bool is_gt = (mg[j] >> lane) & 1u;
+        const bool is_eq = i < end && !take_all && kk[j] == thr;
+        const uint32_t me = __ballot_sync(0xffffffffu, is_eq);
+        const uint32_t my_gt = gt_before + __popc(mg[j] & lt), my_eq = eq_before + __popc(me & lt);
+        int rank = -1;
+        if (is_gt) rank = (int)(my_gt + min(my_eq, k_rem));
+        else if (is_eq && my_eq < k_rem) rank = (int)(my_gt + my_eq);
+        if (rank >= 0) out[rank] = cols != nullptr ? __ldg(cols + i) : i;
+        gt_before += __popc(mg[j]);
+        eq_before += __popc(me);
+      }
+    }
   }
 }
 

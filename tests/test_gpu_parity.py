@@ -37,6 +37,9 @@ WORKLOADS = {
     "bf16_int8_g64": lambda: small_bf16(L=1200, bits=8, group=64),
     "bf16_int2_g32": lambda: small_bf16(L=1200, bits=2, group=32),
     "bf16_off": lambda: small_bf16(L=1200, bits=16),
+    # a point of the depth sweep: 7 loops, so the later loops carry more residual streams (up to 6) than the
+    # cooperative build of the attention kernel keeps slot tables for (its patch warps then build every chunk)
+    "bf16_R7": lambda: dataclasses.replace(workloads.sweep_point(7, 0.25, 160, 4, L=900), n_heads=2, q_block=256),
 }
 
 

@@ -2,14 +2,29 @@
 #include <cstdlib>
 #include <cstring>
 #include <new>
-#include <vector>
+#include <unordered_map>
 
 #include "fl_internal.cuh"
 
+// Tensor maps are encoded once per (base pointer, rows, row elements, box rows) and kept in a hash table: a step of
+// the 48-layer benchmark uses a few hundred of them and looks four up per attention call.
+struct fl_tmap_key {
+  const void* base;
+  int64_t rows, row_elems;
+  int box_rows;
+  bool operator==(const fl_tmap_key& o) const {
+    return base == o.base && rows == o.rows && row_elems == o.row_elems && box_rows == o.box_rows;
+  }
+};
+struct fl_tmap_key_hash {
+  size_t operator()(const fl_tmap_key& k) const {
+    uint64_t x = reinterpret_cast<uintptr_t>(k.base) * 0x9E3779B97F4A7C15ull;
+    x ^= (uint64_t)k.rows * 0xC2B2AE3D27D4EB4Full + (uint64_t)k.row_elems * 0x165667B19E3779F9ull + (uint64_t)k.box_rows;
+    return (size_t)(x ^ (x >> 29));
+  }
+};
 struct fl_tmap_cache {
-  struct Entry { const void* base; int64_t rows, row_elems; int box_rows; CUtensorMap map; };
-  std::vector<Entry> entries;
-  size_t next = 0;
+  std::unordered_map<fl_tmap_key, CUtensorMap, fl_tmap_key_hash> maps;
 };
 
 typedef CUresult (*fl_encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -19,23 +34,23 @@ typedef CUresult (*fl_encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint
 bool fl_tile_tmap(fl_ctx* ctx, const void* base, int64_t rows, int64_t row_elems, int box_rows, CUtensorMap* out) {
   if (ctx->encode_tiled == nullptr || ctx->tmaps == nullptr) return false;
   if (rows < 1 || box_rows < 1 || box_rows > 256 || !fl_aligned16(base) || (row_elems * 2) % 16 != 0) return false;
-  for (const auto& e : ctx->tmaps->entries)
-    if (e.base == base && e.rows == rows && e.row_elems == row_elems && e.box_rows == box_rows) { *out = e.map; return true; }
-  fl_tmap_cache::Entry e;
-  e.base = base; e.rows = rows; e.row_elems = row_elems; e.box_rows = box_rows;
+  const fl_tmap_key key{base, rows, row_elems, box_rows};
+  auto it = ctx->tmaps->maps.find(key);
+  if (it != ctx->tmaps->maps.end()) { *out = it->second; return true; }
+  CUtensorMap map;
   const cuuint64_t gdim[2] = {(cuuint64_t)row_elems, (cuuint64_t)rows};
   const cuuint64_t gstride[1] = {(cuuint64_t)row_elems * 2};
   const cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
   const cuuint32_t estr[2] = {1, 1};
   const CUresult rc = reinterpret_cast<fl_encode_tiled_fn>(ctx->encode_tiled)(
-      &e.map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstride, box, estr,
+      &map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstride, box, estr,
       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (rc != CUDA_SUCCESS) return false;
-  constexpr size_t kMaxEntries = 1024;  // ring replacement: 48 layers x (K, V, Q of three loops) fit twice over
-  if (ctx->tmaps->entries.size() < kMaxEntries) ctx->tmaps->entries.push_back(e);
-  else { ctx->tmaps->entries[ctx->tmaps->next] = e; ctx->tmaps->next = (ctx->tmaps->next + 1) % kMaxEntries; }
-  *out = e.map;
+  constexpr size_t kMaxEntries = 8192;   // a map describes memory the caller may free and reuse: start over when full
+  if (ctx->tmaps->maps.size() >= kMaxEntries) ctx->tmaps->maps.clear();
+  ctx->tmaps->maps.emplace(key, map);
+  *out = map;
   return true;
 }
 

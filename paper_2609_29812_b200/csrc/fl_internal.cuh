@@ -145,7 +145,8 @@ __device__ __forceinline__ bool apply_stream8(const DevStream& st, int pos, int 
   } else {
     uint32_t c[8];
     load_codes8<BITS>(st.codes + (size_t)slot * (d * BITS / 8), elem, c);
-    const size_t gi = (size_t)slot * (d / group) + elem / group;
+    const int gs = 31 - __clz(group);   // the group is a power of two: shifts instead of runtime divisions
+    const size_t gi = (size_t)slot * (d >> gs) + (elem >> gs);
     const float sc = __half2float(st.scale[gi]);
     const float zr = __half2float(st.zero[gi]);
 #pragma unroll
@@ -179,7 +180,8 @@ __device__ __forceinline__ void payload_load(const DevStream& st, int slot, int 
     } else {
       p.raw.x = __ldg(reinterpret_cast<const uint16_t*>(row + elem / 4));
     }
-    const size_t gi = (size_t)slot * (d / group) + elem / group;
+    const int gs = 31 - __clz(group);   // the group is a power of two: shifts instead of runtime divisions
+    const size_t gi = (size_t)slot * (d >> gs) + (elem >> gs);
     p.sc = __ldg(st.scale + gi);
     p.zr = __ldg(st.zero + gi);
   }

@@ -261,7 +261,6 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
     ctl.abort_flag = 0;
     tc::fence_barrier_init();
   }
-  for (int i = tid; i < kMaxChunks; i += kThreads) ctl.chunk_mask[i] = 0;
   // ---- prologue (rolled loops throughout: code that runs once per CTA is paid for in instruction fetches) ----
   // The raw column list, its stream rows and stream masks are staged in the still idle ring.
   int32_t* raw_col = reinterpret_cast<int32_t*>(ring);                     // [kMaxCols]
@@ -330,7 +329,6 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
       tot0 += c0; tot1 += c1;
     }
     if (tid == 0) { ctl.n_plain = tot0; ctl.n_patch = tot1; }
-    const int patch_chunks = (tot1 + kNC - 1) / kNC;
     const uint32_t lt = (1u << lane) - 1;
 #pragma unroll 1
     for (int base = beg; base < end; base += 32) {
@@ -345,7 +343,6 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
         const int dst = patched ? tot0 + before1 + __popc(m1 & lt) : before0 + __popc(m0 & lt);
         ord_col[dst] = j;
         ord_mask[dst] = mask;
-        if (mask != 0) atomicOr(&ctl.chunk_mask[patched ? (dst - tot0) / kNC : patch_chunks + dst / kNC], mask);
         if (patched && dst - tot0 < kPrefillChunks * kNC && a.n_old < kPreStreams) {
           // one of the columns the whole CTA builds next: keep its stream rows
           const int pr = dst - tot0;
@@ -361,10 +358,18 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
   }
   const int n_plain = ctl.n_plain, n_patch = ctl.n_patch;
   const int n_chunks = (n_plain + kNC - 1) / kNC + (n_patch + kNC - 1) / kNC;
-  for (int ci = tid; ci < n_chunks; ci += kThreads) {
+  // per chunk: the OR of its columns' stream masks and its last column (a warp per chunk, two columns per lane)
+  for (int ci = warp; ci < n_chunks; ci += kWarps) {
     const ChunkInfo ck = chunk_info(ci, n_plain, n_patch);
-    ctl.chunk_last[ci] = ck.n_valid == kNC ? ord_col[ck.off + kNC - 1] : INT32_MAX;
-  }
+    uint32_t m = 0;
+    if (lane < ck.n_valid) m |= ord_mask[ck.off + lane];
+    if (lane + 32 < ck.n_valid) m |= ord_mask[ck.off + lane + 32];
+    m = __reduce_or_sync(0xffffffffu, m);
+    if (lane == 0) {
+      ctl.chunk_mask[ci] = m;
+      ctl.chunk_last[ci] = ck.n_valid == kNC ? ord_col[ck.off + kNC - 1] : INT32_MAX;
+    }
+  }   // read after the barrier that ends the cooperative build below
   if (tid == 0) TC_TRACE(0, 60, 1);
   int g = 0;    // chunks issued so far (all tiles): one phase of s_full / s_taken per chunk, P buffer = g & 1
   int fill = 0; // ring slots filled so far: slot = fill % kSlots, phase = (fill / kSlots) & 1

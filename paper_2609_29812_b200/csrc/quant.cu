@@ -107,7 +107,8 @@ __global__ void __launch_bounds__(256) quant_residual_kernel(const __grid_consta
     else if (BITS == 4) *reinterpret_cast<uint32_t*>(row + elem / 2) = packed_lo;
     else *reinterpret_cast<uint16_t*>(row + elem / 4) = (uint16_t)packed_lo;
     if (((elem >> 3) & (lanes_per_group - 1)) == 0) {
-      const size_t gi = (size_t)t * (a.d / a.group) + elem / a.group;
+      const int gs = 31 - __clz(a.group);   // power of two
+      const size_t gi = (size_t)t * (a.d >> gs) + (elem >> gs);
       scale[gi] = sh;
       zero[gi] = zh;
     }

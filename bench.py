@@ -290,7 +290,8 @@ class Bench:
             raise RuntimeError("a C-ABI call failed inside the step")
 
     def breakdown(self):
-        """One untimed-for-the-metric pass with events around every call: per-stage GPU time (ms)."""
+        """One untimed-for-the-metric pass with events around every call: per-stage GPU time (ms) and the time of
+        each loop r (select_tokens of loop r up to the call before loop r + 1)."""
         torch = self.torch
         evs = []
         with torch.cuda.stream(self.stream):
@@ -303,6 +304,12 @@ class Bench:
         out = {}
         for tag, e0, e1 in evs:
             out[tag] = out.get(tag, 0.0) + e0.elapsed_time(e1)
+        starts = [i for i, (tag, _, _) in enumerate(evs) if tag == "select_tokens"] + [len(evs)]
+        per_loop = {}
+        for li in range(len(starts) - 1):
+            ms = evs[starts[li]][1].elapsed_time(evs[starts[li + 1] - 1][2])
+            per_loop[f"loop_{li + 2}"] = {"ms": round(ms, 4), "tokens_per_s": round(self.L / (ms * 1e-3), 1)}
+        self.per_loop = per_loop
         return {k: round(v, 4) for k, v in out.items()}
 
 
@@ -396,6 +403,7 @@ def run_ours(args):
                                  "ratio": dense_b / fl_b, "per": "token, all layers"}
     if rank == 0:
         out["breakdown_ms"] = bench.breakdown()
+        out["per_loop"] = bench.per_loop
     if not args.no_e2e:
         out["e2e"] = run_e2e(bench, args, world, barrier)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

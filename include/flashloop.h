@@ -15,7 +15,7 @@
  *  - Every call validates its arguments on the host, enqueues its kernels on `stream` (a cudaStream_t
  *    passed as void*) and returns without synchronising. Return value: FL_OK or a negative fl_status.
  *    Nothing is launched when an argument is rejected.
- *  - No call allocates device memory except fl_create (one fixed workspace, freed by fl_destroy).
+ *  - No call allocates device memory: every buffer, scratch included, is the caller's.
  *  - Results are deterministic: the same inputs give bit-identical outputs.
  *  - Row-major tensors; [n, H, dh] means n rows of H heads of dh elements, dh fastest.
  *    "storage type" is fl_shape.dtype: FL_BF16 (2 bytes) or FL_F32 (4 bytes).
@@ -44,7 +44,7 @@ typedef enum {
   FL_OK = 0,
   FL_ERR_INVALID_ARG = -1, /* null / misaligned pointer, size out of range, inconsistent store */
   FL_ERR_UNSUPPORTED = -2, /* a valid request this build has no kernel for (e.g. head_dim 96) */
-  FL_ERR_WORKSPACE = -3,   /* problem larger than the context workspace allows */
+  FL_ERR_WORKSPACE = -3,   /* reserved (no entry point needs a workspace) */
   FL_ERR_CUDA = -4,        /* a CUDA runtime call failed (launch error, wrong device, ...) */
   FL_ERR_TIMEOUT = -5      /* reported through the device status word: a bounded wait ran out */
 } fl_status;
@@ -52,7 +52,7 @@ typedef enum {
 enum { FL_BF16 = 0, FL_F32 = 1 };
 #define FL_MAX_LOOPS 32 /* residual streams per store: loops 2 .. FL_MAX_LOOPS+1 */
 
-/* Opaque context: device ordinal, SM count, one small workspace. Not thread-safe per context. */
+/* Opaque context: device ordinal, SM count, cached TMA tensor maps (host memory). Not thread-safe per context. */
 typedef struct fl_ctx fl_ctx;
 FL_API int fl_create(fl_ctx** out /* host */, int device);
 FL_API int fl_destroy(fl_ctx* ctx);

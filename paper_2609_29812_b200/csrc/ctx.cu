@@ -95,9 +95,7 @@ extern "C" int fl_create(fl_ctx** out, int device) {
     (void)cudaGetLastError();
   }
   c->tmaps = new (std::nothrow) fl_tmap_cache();
-  c->workspace_bytes = size_t(8) << 20;
-  if (cudaMalloc(&c->workspace, c->workspace_bytes) != cudaSuccess) {
-    delete c->tmaps;
+  if (c->tmaps == nullptr) {
     delete c;
     return FL_ERR_CUDA;
   }
@@ -107,10 +105,9 @@ extern "C" int fl_create(fl_ctx** out, int device) {
 
 extern "C" int fl_destroy(fl_ctx* ctx) {
   if (ctx == nullptr) return FL_ERR_INVALID_ARG;
-  cudaError_t e = cudaFree(ctx->workspace);
   delete ctx->tmaps;
   delete ctx;
-  return e == cudaSuccess ? FL_OK : FL_ERR_CUDA;
+  return FL_OK;
 }
 
 int fl_launch_status() { return cudaGetLastError() == cudaSuccess ? FL_OK : FL_ERR_CUDA; }

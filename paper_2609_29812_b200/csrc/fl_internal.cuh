@@ -12,8 +12,6 @@ struct fl_ctx {
   int device;
   int sm_count;
   int max_smem_optin;
-  void* workspace;
-  size_t workspace_bytes;
   int force_simt;  // environment FL_FORCE_SIMT=1 at fl_create: keep attention on the binary32 SIMT kernels
   void* encode_tiled;       // cuTensorMapEncodeTiled, resolved through cudaGetDriverEntryPoint (may be null)
   struct fl_tmap_cache* tmaps;  // tensor maps, keyed by (base pointer, rows, row elements, box rows)

@@ -91,16 +91,25 @@ __global__ void __launch_bounds__(256) quant_residual_kernel(const __grid_consta
 #pragma unroll
       for (int i = 0; i < 8; ++i) q[i] = 0.f;
     }
-    uint32_t packed_lo = 0, packed_hi = 0;
+    // The quotients are integers in [0, qmax] already: delta >= zero (the offset was rounded down) and
+    // (max - zero) / scale <= qmax (the scale was rounded up), so the oracle's clamp never acts. Four codes at a
+    // time are packed with exact binary32 arithmetic (sum of code * 2^(BITS*i) < 2^24 for BITS <= 4, two codes
+    // for 8 bits), and the integer is read from the low mantissa bits of (value + 2^23).
+    uint32_t packed_lo, packed_hi = 0;
+    if (BITS == 8) {
+      uint32_t w[4];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      // integer-valued 0..qmax: the low mantissa bits of (value + 2^23) are the code
-      const uint32_t c = __float_as_uint(__fadd_rn(fminf(fmaxf(q[i], 0.f), qmax), 8388608.f)) & 0xFFu;
-      if (BITS == 8) {
-        if (i < 4) packed_lo |= c << (8 * i); else packed_hi |= c << (8 * (i - 4));
-      } else {
-        packed_lo |= c << (BITS * i);
-      }
+      for (int i = 0; i < 4; ++i)
+        w[i] = __float_as_uint(__fadd_rn(__fmaf_rn(q[2 * i + 1], 256.f, q[2 * i]), 8388608.f)) & 0xFFFFu;
+      packed_lo = w[0] | (w[1] << 16);
+      packed_hi = w[2] | (w[3] << 16);
+    } else {
+      const float r1 = (float)(1 << BITS), r2 = r1 * r1, r3 = r2 * r1;
+      const float lo = __fmaf_rn(q[3], r3, __fmaf_rn(q[2], r2, __fmaf_rn(q[1], r1, q[0])));
+      const float hi = __fmaf_rn(q[7], r3, __fmaf_rn(q[6], r2, __fmaf_rn(q[5], r1, q[4])));
+      const uint32_t half_mask = (1u << (4 * BITS)) - 1u;
+      packed_lo = (__float_as_uint(__fadd_rn(lo, 8388608.f)) & half_mask) |
+                  ((__float_as_uint(__fadd_rn(hi, 8388608.f)) & half_mask) << (4 * BITS));
     }
     uint8_t* row = codes + (size_t)t * (a.d * BITS / 8);
     if (BITS == 8) *reinterpret_cast<uint2*>(row + elem) = make_uint2(packed_lo, packed_hi);

@@ -642,23 +642,10 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
       if (!warp_wait(&ctl.s_full[grp], gc & 1, abort_flag)) { ok = false; break; }
       tc::tc_fence_after();
       if (gt == 0) TC_TRACE(2 + grp, ci, 1);
-      uint32_t r[64];
-      tc::tmem_ld32(s_addr, *reinterpret_cast<uint32_t(*)[32]>(&r[0]));
-      tc::tmem_ld32(s_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&r[32]));
-      tc::tmem_wait_ld();
-      // S is in registers: hand the buffer back so that the next chunk's QK^T runs under the arithmetic below.
-      // The previous chunk's P store has had this long to land: it is announced now instead of being waited for
-      // at the end of its own iteration.
-      if (ci > 0) tc::tmem_wait_st();
-      tc::tc_fence_before();
-      __syncwarp();
-      if (lane == 0) {
-        tc::mbar_arrive(&ctl.s_taken[grp]);
-        if (ci > 0) tc::mbar_arrive(&ctl.p_full[grp][pb ^ 1]);
-      }
       // rows of a warp that lie at or after every column of the chunk need no causal mask; rows beyond the
       // tile's last (their results are never stored) must not force the masked path
       const bool unmasked = __all_sync(0xffffffffu, !row_ok || ctl.chunk_last[ci] <= pos);
+      int vis = kNC;
       if (!unmasked) {
         // the chunk's columns ascend: the visible ones are a prefix, found by bisection; the rest read as -inf
         const ChunkInfo ck = chunk_info(ci, n_plain, n_patch);
@@ -668,53 +655,97 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
           const int mid = (lo + hi) >> 1;
           if (cp[mid] <= pos) lo = mid + 1; else hi = mid;
         }
-#pragma unroll
-        for (int u = 0; u < 64; ++u) r[u] = u < lo ? r[u] : 0xff800000u;
+        vis = lo;
       }
-      float sub = lse2;
-      if (grp == 1) {
-        // running reference of the new term: taken from the first chunk that shows a finite logit and moved
-        // (with a rescale of the accumulator row) only when a chunk's maximum beats it by more than the threshold
-        float cm = -INFINITY;
-#pragma unroll
-        for (int u = 0; u < 64; u += 2) cm = fmaxf(cm, fmaxf(__uint_as_float(r[u]), __uint_as_float(r[u + 1])));
-        cm *= c2;                                        // c2 > 0: scaling commutes with the maximum
-        const bool first = ref == -INFINITY && cm > -INFINITY;
-        const bool over = ref > -INFINITY && cm - ref > kRescaleThreshold;
-        if (first) ref = cm;                             // accumulator row is still zero: nothing to rescale
-        if (__any_sync(0xffffffffu, over)) {
-          float factor = 1.f;
-          if (over) { factor = tc::ex2(ref - cm); ref = cm; }
-          // every earlier PV must have completed before the accumulator rows are rewritten (ci >= 1 here)
-          if (!warp_wait(&ctl.p_free[1][(gc - 1) & 1], ((gc - 1) >> 1) & 1, abort_flag)) { ok = false; break; }
-          tc::tc_fence_after();
-          ell *= factor;
-#pragma unroll 1
-          for (int q4 = 0; q4 < 8; ++q4) {
-            uint32_t acc[16];
-            tc::tmem_ld16(tmem + lane_base + kAccNew + q4 * 16, acc);
-            tc::tmem_wait_ld();
-#pragma unroll
-            for (int i = 0; i < 16; ++i) acc[i] = __float_as_uint(__uint_as_float(acc[i]) * factor);
-            tc::tmem_st16(tmem + lane_base + kAccNew + q4 * 16, acc);
-          }
-          tc::tmem_wait_st();
-        }
-        sub = ref == -INFINITY ? 0.f : ref;
-      }
-      float sum = 0.f;
-#pragma unroll
-      for (int u = 0; u < 64; u += 2) {
-        const float p0 = tc::ex2(fmaf(__uint_as_float(r[u]), c2, -sub));
-        const float p1 = tc::ex2(fmaf(__uint_as_float(r[u + 1]), c2, -sub));
-        sum += p0 + p1;
-        r[u >> 1] = tc::pack_bf16(p0, p1);
-      }
-      if (grp == 0) mass += sum; else ell += sum;
       // the P buffer is free once the PV MMAs of chunk gc - 2 have retired
       if (n_use >= 1 && !warp_wait(&ctl.p_free[grp][pb], (n_use - 1) & 1, abort_flag)) { ok = false; break; }
-      tc::tc_fence_after();
-      tc::tmem_st32(p_addr + pb * 32, *reinterpret_cast<uint32_t(*)[32]>(&r[0]));
+      // The 64 logits of the row are taken in two halves of 32 (each its own little softmax step): 64 live logits
+      // plus the pipeline's state do not fit 128 registers, and what spills lands in an L1 of ~30 KB.
+#pragma unroll 1
+      for (int hf = 0; hf < 2 && ok; ++hf) {
+        uint32_t r[32];
+        tc::tmem_ld32(s_addr + hf * 32, r);
+        tc::tmem_wait_ld();
+        if (hf == 0) {
+          // the previous chunk's P store has had this long to land: it is announced now instead of being waited
+          // for at the end of its own iteration
+          if (ci > 0) {
+            tc::tmem_wait_st();
+            tc::tc_fence_before();
+            __syncwarp();
+            if (lane == 0) tc::mbar_arrive(&ctl.p_full[grp][pb ^ 1]);
+          }
+        } else {
+          // S is in registers: hand the buffer back so that the next chunk's QK^T runs under the arithmetic below
+          tc::tc_fence_before();
+          __syncwarp();
+          if (lane == 0) tc::mbar_arrive(&ctl.s_taken[grp]);
+        }
+        if (!unmasked) {
+          const int lim = vis - hf * 32;
+#pragma unroll
+          for (int u = 0; u < 32; ++u) r[u] = u < lim ? r[u] : 0xff800000u;
+        }
+        float sub = lse2;
+        if (grp == 1) {
+          // running reference of the new term: taken from the first columns that show a finite logit and moved
+          // (with a rescale of the accumulator row) only when a maximum beats it by more than the threshold
+          float cm = -INFINITY;
+#pragma unroll
+          for (int u = 0; u < 32; u += 2) cm = fmaxf(cm, fmaxf(__uint_as_float(r[u]), __uint_as_float(r[u + 1])));
+          cm *= c2;                                        // c2 > 0: scaling commutes with the maximum
+          const bool first = ref == -INFINITY && cm > -INFINITY;
+          const bool over = ref > -INFINITY && cm - ref > kRescaleThreshold;
+          if (first) ref = cm;                             // accumulator row is still zero: nothing to rescale
+          if (__any_sync(0xffffffffu, over)) {
+            float factor = 1.f;
+            if (over) { factor = tc::ex2(ref - cm); ref = cm; }
+            // every earlier PV must have completed before the accumulator rows are rewritten (ci >= 1 here: the
+            // reference was set in an earlier chunk, or in this chunk's first half, whose P is not announced yet)
+            if (ci >= 1) {
+              if (!warp_wait(&ctl.p_free[1][(gc - 1) & 1], ((gc - 1) >> 1) & 1, abort_flag)) { ok = false; break; }
+              tc::tc_fence_after();
+#pragma unroll 1
+              for (int q4 = 0; q4 < 8; ++q4) {
+                uint32_t acc[16];
+                tc::tmem_ld16(tmem + lane_base + kAccNew + q4 * 16, acc);
+                tc::tmem_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 16; ++i) acc[i] = __float_as_uint(__uint_as_float(acc[i]) * factor);
+                tc::tmem_st16(tmem + lane_base + kAccNew + q4 * 16, acc);
+              }
+              tc::tmem_wait_st();
+            }
+            ell *= factor;
+            if (hf == 1) {
+              // the first half of this chunk's P was formed against the old reference: bring it along
+              uint32_t ph[16];
+              tc::tmem_wait_st();
+              tc::tmem_ld16(p_addr + pb * 32, ph);
+              tc::tmem_wait_ld();
+#pragma unroll
+              for (int i = 0; i < 16; ++i) {
+                const __nv_bfloat162 v = *reinterpret_cast<const __nv_bfloat162*>(&ph[i]);
+                const float2 f = __bfloat1622float2(v);
+                ph[i] = tc::pack_bf16(f.x * factor, f.y * factor);
+              }
+              tc::tmem_st16(p_addr + pb * 32, ph);
+            }
+          }
+          sub = ref == -INFINITY ? 0.f : ref;
+        }
+        float sum = 0.f;
+#pragma unroll
+        for (int u = 0; u < 32; u += 2) {
+          const float p0 = tc::ex2(fmaf(__uint_as_float(r[u]), c2, -sub));
+          const float p1 = tc::ex2(fmaf(__uint_as_float(r[u + 1]), c2, -sub));
+          sum += p0 + p1;
+          r[u >> 1] = tc::pack_bf16(p0, p1);
+        }
+        if (grp == 0) mass += sum; else ell += sum;
+        tc::tmem_st16(p_addr + pb * 32 + hf * 16, *reinterpret_cast<uint32_t(*)[16]>(&r[0]));
+      }
+      if (!ok) break;
       if (gt == 0) TC_TRACE(2 + grp, ci, 2);
     }
     if (ok && n_chunks > 0) {   // the last chunk's P

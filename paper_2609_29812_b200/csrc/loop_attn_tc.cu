@@ -636,6 +636,7 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
     const uint32_t p_addr = tmem + lane_base + (grp ? kPNew : kPOld);
     float mass = 0.f, ell = 0.f, ref = -INFINITY;
     bool ok = true;
+    bool pending = false;   // the previous chunk's P is stored but not yet announced (warp-uniform)
     for (int ci = 0; ci < n_chunks; ++ci) {
       const int gc = g0 + ci, pb = gc & 1, n_use = gc >> 1;
       if (gt == 0) TC_TRACE(2 + grp, ci, 0);
@@ -669,11 +670,12 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
         if (hf == 0) {
           // the previous chunk's P store has had this long to land: it is announced now instead of being waited
           // for at the end of its own iteration
-          if (ci > 0) {
+          if (pending) {
             tc::tmem_wait_st();
             tc::tc_fence_before();
             __syncwarp();
             if (lane == 0) tc::mbar_arrive(&ctl.p_full[grp][pb ^ 1]);
+            pending = false;
           }
         } else {
           // S is in registers: hand the buffer back so that the next chunk's QK^T runs under the arithmetic below
@@ -746,9 +748,19 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
         tc::tmem_st16(p_addr + pb * 32 + hf * 16, *reinterpret_cast<uint32_t(*)[16]>(&r[0]));
       }
       if (!ok) break;
+      pending = true;
+      if (ci < kSlots / 2) {
+        // while the pipeline fills (the first chunks hold the whole ring) latency counts: announce P at once, so
+        // that its PV retires and the ring slots are handed to the gathers as early as possible
+        tc::tmem_wait_st();
+        tc::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) tc::mbar_arrive(&ctl.p_full[grp][pb]);
+        pending = false;
+      }
       if (gt == 0) TC_TRACE(2 + grp, ci, 2);
     }
-    if (ok && n_chunks > 0) {   // the last chunk's P
+    if (ok && pending) {   // the last chunk's P
       tc::tmem_wait_st();
       tc::tc_fence_before();
       __syncwarp();

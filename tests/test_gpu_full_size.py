@@ -15,7 +15,7 @@ pytestmark = pytest.mark.gpu
 SAMPLES = [(0, 0), (3, 7), (9, 20), (15, 31)]     # (head, query block): first, middle and last blocks
 
 
-def test_full_size_layer_loop2_sampled_against_oracle():
+def test_full_size_layer_loops_2_and_3_sampled_against_oracle():
     import torch
     from paper_2609_29812_b200 import binding as B, pipeline as P
     w = workloads.config3(n_layers=1)
@@ -28,64 +28,79 @@ def test_full_size_layer_loop2_sampled_against_oracle():
     st = P.LayerState(ctx, w, dev)
     st.dense_loop(q1, k1, v1)
     st.select_columns_dense()
-    sel = P.select_tokens(ctx, st.shape, 2, G[0], G[1], None, w.k_tokens)
-    act = to_np(sel.active_idx).astype(np.int64)
-
-    # ---- stage 1 in full: the fp64 scores of all L rows and their exact top-k (near-tie band at the boundary)
-    s_ref = fo.token_scores(to_np(G[0]), to_np(G[1]), np.arange(w.L), w.eps)
-    assert_selection_matches(act, s_ref, np.arange(w.L), w.k_tokens, "token set at L=32768")
-    np.testing.assert_allclose(to_np(sel.scores), s_ref, rtol=2e-5, atol=0)
-    slot = to_np(sel.slot_of_pos)
-    assert np.array_equal(slot, fo.slot_map(act, w.L))
-
-    q2, k2, v2 = gen.rows(2, sel.active_idx)
-    st.alloc_stream(sel)
-    st.quantize(2, k2, v2, sel)
-    o_dense = st.o_store.clone()
-    rc = st.attention_indexed(2, q2, sel)
-    assert rc == 0
-    st.check_status()
-    o_gpu = to_np(st.o_store)
-    untouched = np.ones(w.L, dtype=bool)
-    untouched[act] = False
-    assert torch.equal(st.o_store[torch.from_numpy(untouched).to(dev)], o_dense[torch.from_numpy(untouched).to(dev)])
-
     col_idx, col_cnt = to_np(st.col_idx), to_np(st.col_cnt)
-    k_codes = to_np(st.k_streams[-1]["codes"]).reshape(len(act), w.n_heads, -1)
-    v_codes = to_np(st.v_streams[-1]["codes"]).reshape(len(act), w.n_heads, -1)
-    k_scale = to_np(st.k_streams[-1]["scale"]).view(np.uint16).reshape(len(act), w.n_heads, -1)
-    k_zero = to_np(st.k_streams[-1]["zero"]).view(np.uint16).reshape(len(act), w.n_heads, -1)
     nb = st.nb
+
+    # ---- the GPU path, loops 2 and 3, through the calls and launch shapes bench.py times --------------------
+    gpu = {}
+    cand = None
+    for r in (2, 3):
+        sel = P.select_tokens(ctx, st.shape, r, G[r - 2], G[r - 1], cand, w.k_tokens)
+        act = to_np(sel.active_idx).astype(np.int64)
+        # stage 1 in full: fp64 scores of every candidate and their exact top-k (near-tie band at the boundary)
+        cand_np = np.arange(w.L) if cand is None else to_np(cand).astype(np.int64)
+        s_ref = fo.token_scores(to_np(G[r - 2]), to_np(G[r - 1]), cand_np, w.eps)
+        assert_selection_matches(act, s_ref, cand_np, w.k_tokens, f"token set of loop {r} at L=32768")
+        np.testing.assert_allclose(to_np(sel.scores)[: len(cand_np)], s_ref, rtol=2e-5, atol=0)
+        assert np.array_equal(to_np(sel.slot_of_pos), fo.slot_map(act, w.L))
+        qr, kr, vr = gen.rows(r, sel.active_idx)
+        st.alloc_stream(sel)
+        st.quantize(r, kr, vr, sel)
+        o_before = st.o_store.clone()
+        assert st.attention_indexed(r, qr, sel) == 0
+        st.check_status()
+        untouched = np.ones(w.L, dtype=bool)
+        untouched[act] = False
+        keep = torch.from_numpy(untouched).to(dev)
+        assert torch.equal(st.o_store[keep], o_before[keep])
+        gpu[r] = dict(act=act, q=qr, k=kr, v=vr, o=to_np(st.o_store), lse=to_np(st.lse),
+                      k_codes=to_np(st.k_streams[-1]["codes"]).reshape(len(act), w.n_heads, -1),
+                      v_codes=to_np(st.v_streams[-1]["codes"]).reshape(len(act), w.n_heads, -1),
+                      k_scale=to_np(st.k_streams[-1]["scale"]).view(np.uint16).reshape(len(act), w.n_heads, -1),
+                      k_zero=to_np(st.k_streams[-1]["zero"]).view(np.uint16).reshape(len(act), w.n_heads, -1))
+        cand = sel.active_idx
+
+    # ---- the oracle, on its own, for sampled (head, block) pairs -------------------------------------------
     for h, b in SAMPLES:
         hs = slice(h, h + 1)
         q1h, k1h, v1h = (to_np(t[:, hs, :]) for t in (q1, k1, v1))
         end = min(w.L, (b + 1) * w.q_block)
-        # ---- dense source loop of the block's rows, column scores, column set (Eq. 6)
-        d1 = fo.dense_loop_attention(q1h, k1h, v1h, w.sm_scale, w.q_block, rows_to_cache=act, head_list=[0],
+        act2 = gpu[2]["act"]
+        # dense source loop of the block's rows, column scores, column set (Eq. 6)
+        d1 = fo.dense_loop_attention(q1h, k1h, v1h, w.sm_scale, w.q_block, rows_to_cache=act2, head_list=[0],
                                      block_list=[b])
         S_gpu = col_idx[h, b, : col_cnt[h, b]].astype(np.int64)
         assert col_cnt[h, b] == min(w.col_budget, end)
         assert_selection_matches(S_gpu, d1["col_scores"][0, b, :end], np.arange(end), w.col_budget,
                                  f"column set of head {h}, block {b}")
-        # ---- residual codec of this head's rows (Eq. 8): codes and metadata bit for bit
-        khat_new, kpay = fo.residual_update(to_np(k2[:, hs, :]), k1h.astype(np.float32), act, w.bits, w.group)
-        vhat_new, vpay = fo.residual_update(to_np(v2[:, hs, :]), v1h.astype(np.float32), act, w.bits, w.group)
-        assert np.array_equal(k_codes[:, h], kpay["packed"][:, 0]), (h, "K codes")
-        assert np.array_equal(v_codes[:, h], vpay["packed"][:, 0]), (h, "V codes")
-        assert np.array_equal(k_scale[:, h], kpay["scale"][:, 0].view(np.uint16)), (h, "K scale")
-        assert np.array_equal(k_zero[:, h], kpay["zero"][:, 0].view(np.uint16)), (h, "K offset")
-        # ---- attention replacement of the block's active rows (Eq. 7) over the GPU's column set
         sets = {(0, bb): np.zeros(0, dtype=np.int64) for bb in range(nb)}
         cache = {(0, bb): (np.zeros(0, dtype=np.int64), np.zeros((0, 0))) for bb in range(nb)}
         rows, P1 = d1["probs"][(0, b)]
         sets[(0, b)] = S_gpu
         cache[(0, b)] = (rows, P1[:, S_gpu])
-        res = fo.sparse_loop_attention(to_np(q2[:, hs, :]), khat_new, vhat_new, v1h.astype(np.float32), d1["O"][act],
-                                       act, sets, cache, w.sm_scale, w.q_block, head_list=[0], block_list=[b],
-                                       kv_round=fo.round_bf16)
-        in_block = np.nonzero(act // w.q_block == b)[0]
-        assert len(in_block) > 0
-        assert_attn_close(o_gpu[act[in_block], h], res["O"][in_block, 0], f"O rows of head {h}, block {b}")
-        lse_gpu = to_np(st.lse)[h, act[in_block]]
-        np.testing.assert_allclose(lse_gpu, res["lse"][0, in_block], rtol=0, atol=5e-3)
+        khat, vhat = k1h.astype(np.float32), v1h.astype(np.float32)
+        o_full = d1["O"]
+        for r in (2, 3):
+            g = gpu[r]
+            act = g["act"]
+            # residual codec of this head's rows (Eq. 8): codes and metadata bit for bit
+            khat_new, kpay = fo.residual_update(to_np(g["k"][:, hs, :]), khat, act, w.bits, w.group)
+            vhat_new, vpay = fo.residual_update(to_np(g["v"][:, hs, :]), vhat, act, w.bits, w.group)
+            assert np.array_equal(g["k_codes"][:, h], kpay["packed"][:, 0]), (r, h, "K codes")
+            assert np.array_equal(g["v_codes"][:, h], vpay["packed"][:, 0]), (r, h, "V codes")
+            assert np.array_equal(g["k_scale"][:, h], kpay["scale"][:, 0].view(np.uint16)), (r, h, "K scale")
+            assert np.array_equal(g["k_zero"][:, h], kpay["zero"][:, 0].view(np.uint16)), (r, h, "K offset")
+            # attention replacement of the block's active rows (Eq. 7) over the GPU's column set
+            res = fo.sparse_loop_attention(to_np(g["q"][:, hs, :]), khat_new, vhat_new, vhat, o_full[act], act, sets,
+                                           cache, w.sm_scale, w.q_block, head_list=[0], block_list=[b],
+                                           kv_round=fo.round_bf16)
+            in_block = np.nonzero(act // w.q_block == b)[0]
+            assert len(in_block) > 0
+            assert_attn_close(g["o"][act[in_block], h], res["O"][in_block, 0],
+                              f"O rows of loop {r}, head {h}, block {b}", loops=r - 1)
+            np.testing.assert_allclose(g["lse"][h, act[in_block]], res["lse"][0, in_block], rtol=0, atol=5e-3 * (r - 1))
+            o_full = o_full.copy()
+            o_full[act] = res["O"]
+            cache = {key: (res["probs"][key] if key[1] == b else cache[key]) for key in cache}
+            khat, vhat = khat_new, vhat_new
     ctx.close()

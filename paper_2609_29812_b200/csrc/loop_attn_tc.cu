@@ -98,7 +98,8 @@ struct alignas(64) TcArgs {
 struct __align__(16) TcSmemCtl {
   uint64_t landed[kSlots];   // TMA -> everyone: the slot's gathered tiles (32 KB) have arrived
   uint64_t patched[kSlots];  // patch -> QK issuers: residual-carrying columns of the slot are rewritten (dirty chunks only)
-  uint64_t done[kSlots];     // the four issuers -> TMA: the MMAs that read the slot have finished
+  uint64_t done[kSlots];     // the two PV issuers -> TMA: the MMAs that read the slot have finished (a term's PV of a chunk
+                             // is issued after its softmax, hence after its QK^T of the chunk has completed)
   uint64_t q_full;           // TMA -> QK issuers: the Q tiles of the current row tile have arrived
   uint64_t s_full[2];        // QK issuer -> softmax (per term): S of the chunk is in tensor memory
   uint64_t s_taken[2];       // softmax -> QK issuer: S of the chunk is in registers, the buffer may be overwritten
@@ -246,7 +247,7 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
     for (int s = 0; s < kSlots; ++s) {
       tc::mbar_init(&ctl.landed[s], kTmaWarps);
       tc::mbar_init(&ctl.patched[s], kTmaWarps);
-      tc::mbar_init(&ctl.done[s], 4);
+      tc::mbar_init(&ctl.done[s], 2);
     }
     tc::mbar_init(&ctl.q_full, 1);
     for (int t = 0; t < 2; ++t) {
@@ -585,8 +586,6 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
         FL_QK(4, true);  FL_QK(5, true); FL_QK(6, true); FL_QK(7, true);
 #undef FL_QK
         tc::mma_commit(&ctl.s_full[t]);
-        tc::mma_commit(&ctl.done[slot0]);
-        if (ck.patch) tc::mma_commit(&ctl.done[slot1]);
         f += ck.patch ? 2 : 1;
         if (t == 0) TC_TRACE(1, ci, 2);
       }

@@ -32,7 +32,8 @@ class FlShape(C.Structure):
 
 class FlKvStream(C.Structure):
     _fields_ = [("codes", C.c_void_p), ("scale", C.c_void_p), ("zero", C.c_void_p),
-                ("slot_of_pos", C.c_void_p), ("n_rows", C.c_int32), ("reserved_", C.c_int32)]
+                ("slot_of_pos", C.c_void_p), ("rows_prev", C.c_void_p), ("rows_cur", C.c_void_p),
+                ("n_rows", C.c_int32), ("reserved_", C.c_int32)]
 
 
 class FlKvStore(C.Structure):
@@ -118,7 +119,8 @@ def make_shape(L, n_heads, head_dim, dtype, q_block, bits, group, eps, sm_scale)
 
 def make_store(k_base, v_base, k_streams: Sequence[dict] = (), v_streams: Sequence[dict] = ()) -> FlKvStore:
     """Builds the host-side store struct.  Each stream is a dict with codes, scale, zero, slot_of_pos
-    (tensors or addresses) and n_rows.  The caller keeps the tensors alive."""
+    (tensors or addresses), n_rows and optionally rows_prev / rows_cur (the transient workspace for the loop's
+    materialized rows).  The caller keeps the tensors alive."""
     st = FlKvStore()
     st.k_base, st.v_base = _ptr(k_base), _ptr(v_base)
     assert len(k_streams) == len(v_streams) <= FL_MAX_LOOPS
@@ -128,6 +130,8 @@ def make_store(k_base, v_base, k_streams: Sequence[dict] = (), v_streams: Sequen
             dst[i].scale = _ptr(s.get("scale"))
             dst[i].zero = _ptr(s.get("zero"))
             dst[i].slot_of_pos = _ptr(s.get("slot_of_pos"))
+            dst[i].rows_prev = _ptr(s.get("rows_prev"))
+            dst[i].rows_cur = _ptr(s.get("rows_cur"))
             dst[i].n_rows = int(s["n_rows"])
     st.n_streams = len(k_streams)
     return st

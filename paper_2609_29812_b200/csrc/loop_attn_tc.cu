@@ -10,14 +10,18 @@
 //               every ~60-90 cycles while the tensor pipe retires one in 48, so the four streams of MMAs are
 //               issued from four warps on four different schedulers.
 //   warps 12-15 TMA + patch: the Q tiles (two 2-D tile loads each), row gathers (cp.async.bulk.tensor
-//               tile::gather4, 4 selected columns per copy) of the bf16 base K/V rows straight into 128B-swizzled
-//               operand tiles, and for the columns that carry residual payloads the overwrite of the gathered
-//               base rows with the dequantize-and-add result (Eq. 8)
+//               tile::gather4, 4 selected columns per copy) of bf16 K/V rows straight into 128B-swizzled
+//               operand tiles, and for columns that carry residual payloads which nobody has materialized the
+//               overwrite of the gathered base rows with the dequantize-and-add result (Eq. 8)
 //
 // Prologue (whole CTA): the block's causal column list is copied to shared memory together with a bit mask
 // of the residual streams that carry each column, and stably partitioned into columns WITHOUT a payload in
 // the current loop (Khat_old == Khat_new, one K tile and one V tile serve both terms) followed by columns
-// WITH one (separate old / new tiles). Most columns are of the first kind and are a plain gather.
+// WITH one (separate old / new tiles). Most columns are of the first kind and are a plain gather of base rows.
+// The second kind are the loop's active tokens: the quantization kernel of the same loop, which holds both
+// Xhat^(r-1) and Xhat^(r) of those rows in registers, leaves them as bf16 rows in a transient workspace, and the
+// old / new tiles are plain gathers from there (indexed by the token's row in the loop's stream). Without that
+// workspace, and for columns whose only payloads are from earlier loops, the patch warps rebuild the rows here.
 //
 // Per chunk of 64 columns and per term: S (f32, 64 tensor-memory columns, ONE buffer: the softmax warps pull it
 // into registers and hand the buffer back at once, so the next chunk's QK^T runs under the current chunk's
@@ -48,14 +52,11 @@ constexpr int kThreads = kWarps * 32;
 constexpr int kColWarps = 14;               // warps that read the column list in the prologue (the other two search rows)
 constexpr int kMaxCols = 3072;              // column budget the shared-memory column list can hold
 constexpr int kMaxChunks = kMaxCols / kNC + 2;
-constexpr int kPrefillChunks = 2;   // patched chunks the whole CTA builds at the start of a row tile (4 ring slots)
-constexpr int kPreStreams = 4;      // ... when the loop has at most this many residual streams (their slot lookups are
-                                    // kept from the prologue); deeper loops leave every patched chunk to the patch warps
 constexpr uint32_t kAccOld = 0, kAccNew = 128, kSOld = 256, kSNew = 320, kPOld = 384, kPNew = 448;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRescaleThreshold = 60.f;   // in log2 units: rescale only when the reference falls this far behind
-static_assert((2 + kPreStreams) * kMaxCols * 4 <= kSlots * kSlotBytes, "prologue staging must fit in the ring");
+static_assert(3 * kMaxCols * 4 <= kSlots * kSlotBytes, "prologue staging must fit in the ring");
 
 // Optional device-side timeline for tuning (compile with -DFL_TC_TRACE): the CTA (block 1, head 0) writes
 // clock64() stamps into the buffer passed as `status` (the traced CTA can be chosen with -DFL_TC_TRACE_X/_Y): trace[(role * 64 + chunk) * 4 + event].
@@ -75,6 +76,8 @@ static_assert((2 + kPreStreams) * kMaxCols * 4 <= kSlots * kSlotBytes, "prologue
 
 struct alignas(64) TcArgs {
   CUtensorMap k_map, v_map;          // row-gather maps of the K / V base ([L, d] bf16, box 64 x 1, 128B swizzle)
+  CUtensorMap k_prev_map, k_cur_map;  // use_rows: row-gather maps of the loop's materialized rows ([n_active, d] bf16):
+  CUtensorMap v_prev_map, v_cur_map;  // Khat / Vhat of the active tokens before and after the loop's residual
   CUtensorMap q_new_map, q_old_map;  // tile maps of the compact Q rows ([n_active, d] bf16, box 64 x 128); in the
                                      // indexed form q_old_map is a row-gather map of the Q store ([L, d], box 64 x 1)
   const __nv_bfloat16* o_prev;       // compact rows; in the indexed form the O stores [L, d] (may be the same)
@@ -85,6 +88,7 @@ struct alignas(64) TcArgs {
   int n_active;
   DevSide k, v;
   int n_old;
+  int use_rows;                      // columns active in this loop are gathered from the materialized rows
   const int32_t* col_idx;
   const int32_t* col_cnt;
   int c;
@@ -113,7 +117,6 @@ struct __align__(16) TcSmemCtl {
   int warp_cnt[kWarps][2];
   int chunk_last[kMaxChunks];       // largest column position of the chunk, INT32_MAX if the chunk is padded
   uint32_t chunk_mask[kMaxChunks];  // OR of the stream masks of the chunk's columns (0: plain gather only)
-  int pre_slot[kPreStreams][kPrefillChunks * kNC];  // stream rows of the first patched columns (-1: none)
   float mass[kM];
   float ell[kM];
   float ref[kM];
@@ -266,7 +269,7 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
   // The raw column list, its stream rows and stream masks are staged in the still idle ring.
   int32_t* raw_col = reinterpret_cast<int32_t*>(ring);                     // [kMaxCols]
   uint32_t* raw_mask = reinterpret_cast<uint32_t*>(raw_col + kMaxCols);    // [kMaxCols]
-  int32_t* raw_slot = reinterpret_cast<int32_t*>(raw_mask + kMaxCols);     // [kPreStreams][kMaxCols]
+  int32_t* raw_slot = reinterpret_cast<int32_t*>(raw_mask + kMaxCols);     // [kMaxCols]: row in the loop's own stream
   const int c_cap = min(a.c, kMaxCols);
   if (warp >= kColWarps) {
     // warps 14 and 15 search the block's rows in the ascending active list meanwhile
@@ -304,7 +307,7 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
       const int j = raw_col[u];
       const int sl = j >= 0 ? __ldg(a.k.s[s].slot + j) : -1;
       if (sl >= 0) atomicOr(&raw_mask[u], 1u << s);
-      if (s < kPreStreams) raw_slot[s * kMaxCols + u] = sl;
+      if (s == a.n_old) raw_slot[u] = sl;
     }
     __syncthreads();
     // causal prefix, stable partition into plain / patched columns: every warp owns a contiguous span
@@ -343,14 +346,8 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
       if (live) {
         const int dst = patched ? tot0 + before1 + __popc(m1 & lt) : before0 + __popc(m0 & lt);
         ord_col[dst] = j;
-        ord_mask[dst] = mask;
-        if (patched && dst - tot0 < kPrefillChunks * kNC && a.n_old < kPreStreams) {
-          // one of the columns the whole CTA builds next: keep its stream rows
-          const int pr = dst - tot0;
-#pragma unroll 1
-          for (int s = 0; s < kPreStreams; ++s)
-            ctl.pre_slot[s][pr] = s <= a.n_old ? raw_slot[s * kMaxCols + u] : -1;
-        }
+        // a column that is gathered from the materialized rows needs its row there, not its stream mask
+        ord_mask[dst] = (patched && a.use_rows) ? (uint32_t)raw_slot[u] : mask;
       }
       before0 += __popc(m0);
       before1 += __popc(m1);
@@ -363,14 +360,17 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
   for (int ci = warp; ci < n_chunks; ci += kWarps) {
     const ChunkInfo ck = chunk_info(ci, n_plain, n_patch);
     uint32_t m = 0;
-    if (lane < ck.n_valid) m |= ord_mask[ck.off + lane];
-    if (lane + 32 < ck.n_valid) m |= ord_mask[ck.off + lane + 32];
+    if (!(ck.patch && a.use_rows)) {   // chunks gathered from the materialized rows are never rewritten
+      if (lane < ck.n_valid) m |= ord_mask[ck.off + lane];
+      if (lane + 32 < ck.n_valid) m |= ord_mask[ck.off + lane + 32];
+    }
     m = __reduce_or_sync(0xffffffffu, m);
     if (lane == 0) {
       ctl.chunk_mask[ci] = m;
       ctl.chunk_last[ci] = ck.n_valid == kNC ? ord_col[ck.off + kNC - 1] : INT32_MAX;
     }
-  }   // read after the barrier that ends the cooperative build below
+  }
+  __syncthreads();
   if (tid == 0) TC_TRACE(0, 60, 1);
   int g = 0;    // chunks issued so far (all tiles): one phase of s_full / s_taken per chunk, P buffer = g & 1
   int fill = 0; // ring slots filled so far: slot = fill % kSlots, phase = (fill / kSlots) & 1
@@ -380,7 +380,6 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
   const int n_rows = min(kM, q_hi - s0);
   const int g0 = g, fill0 = fill;
   const uint32_t dirty_par0 = dirty_par_cta;
-  const int n_pre = a.n_old < kPreStreams ? min((n_patch + kNC - 1) / kNC, kPrefillChunks) : 0;
   if (warp == kTmaWarp) {
     // Q tiles of this row tile: two 64-element slabs each; rows past the compact list read as zero, rows of the
     // next block (past n_rows) are computed and dropped
@@ -406,49 +405,6 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
       tc::tma_gather4(q_old_tile + kM * 128 + lane * 512, &a.q_old_map, &ctl.q_full, h * kDH + 64, y[0], y[1], y[2], y[3]);
     }
   }
-  // ---- the first patched chunks are built by all 512 threads straight into the (idle) ring: base row plus
-  // dequantized residuals (Eq. 8), old and new operand tiles. A warp owns 4 columns of the chunk (lanes 0-15:
-  // the 16 pieces of the K row, lanes 16-31: of the V row); their stream rows were kept by the prologue, so the
-  // base and payload loads of a column pair are one round of independent loads.
-  {
-    const int half = lane >> 4, ch = lane & 15;
-    const DevSide& side = half ? a.v : a.k;
-    const int elem = h * kDH + ch * 8;
-    const uint32_t tile_off = half * kTileBytes + (ch >> 3) * (kNC * 128);
-#pragma unroll 1
-    for (int it = 0; it < n_pre * 4; ++it) {
-      const int pc = it >> 2, u = warp + 16 * (it & 3);
-      const ChunkInfo ck = chunk_info(pc, n_plain, n_patch);
-      const int slot0 = (fill0 + 2 * pc) % kSlots, slot1 = (fill0 + 2 * pc + 1) % kSlots;
-      const bool valid = u < ck.n_valid;
-      const uint32_t mask = valid ? ord_mask[ck.off + u] : 0u;
-      uint4 raw = make_uint4(0, 0, 0, 0);
-      Payload8<__nv_bfloat16, BITS> pl[kPreStreams];
-      int sl[kPreStreams];
-      if (valid)
-        raw = __ldg(reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(side.base) +
-                                                   (size_t)ord_col[ck.off + u] * a.d + elem));
-#pragma unroll
-      for (int s = 0; s < kPreStreams; ++s) {
-        sl[s] = (valid && s <= a.n_old) ? ctl.pre_slot[s][pc * kNC + u] : -1;
-        if (sl[s] >= 0) payload_load<__nv_bfloat16, BITS>(side.s[s], sl[s], elem, a.d, a.group, pl[s]);
-      }
-      float x[8];
-      unpack8(raw, x);
-      uint4 v_old = raw;
-#pragma unroll
-      for (int s = 0; s < kPreStreams; ++s) {
-        if (s == a.n_old && (mask & ((1u << a.n_old) - 1u))) v_old = pack8(x);
-        if (sl[s] >= 0) payload_apply<__nv_bfloat16, BITS>(pl[s], x);
-      }
-      const uint4 v_new = ((mask >> a.n_old) & 1u) ? pack8(x) : v_old;
-      const uint32_t off = tile_off + tc::sw128_offset(u, ch & 7);
-      *reinterpret_cast<uint4*>(ring + slot0 * kSlotBytes + off) = v_old;
-      *reinterpret_cast<uint4*>(ring + slot1 * kSlotBytes + off) = v_new;
-    }
-  }
-  tc::fence_proxy_async_smem();
-  __syncthreads();
   if (tid == 0) TC_TRACE(0, 60, 2);
 
   if (warp >= kTmaWarp) {
@@ -473,15 +429,6 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
       const ChunkInfo ck = chunk_info(ci, n_plain, n_patch);
       const int n_slots = ck.patch ? 2 : 1;
       const bool dirty = ctl.chunk_mask[ci] != 0;
-      if (ci < n_pre) {   // built by the whole CTA above: only the barrier phases are left to complete
-        if (lane == 0)
-          for (int k = 0; k < n_slots; ++k) {
-            tc::mbar_arrive(&ctl.landed[(f + k) % kSlots]);
-            tc::mbar_arrive(&ctl.patched[(f + k) % kSlots]);
-          }
-        f += n_slots;
-        continue;
-      }
       for (int k = 0; k < n_slots && ok; ++k)
         if (f + k >= kSlots) ok = warp_wait(&ctl.done[(f + k) % kSlots], (((f + k) / kSlots) - 1) & 1, abort_flag);
       if (!ok) break;
@@ -489,16 +436,24 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
       if (lane == 0)
         for (int k = 0; k < n_slots; ++k) tc::mbar_arrive_expect_tx(&ctl.landed[(f + k) % kSlots], kSlotBytes / kTmaWarps);
       __syncwarp();
+      // columns that are active in this loop come from the materialized rows (old tile: before the loop's
+      // residual, new tile: after it), indexed by their row in the loop's stream; all others from the base
+      const bool from_rows = ck.patch && a.use_rows;
       if (lane < 16) {
         int y[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const int u = grp * 4 + i;
-          y[i] = u < ck.n_valid ? ord_col[ck.off + u] : a.L;   // row L is outside the tensor: reads as zero
+          // a row past the end of the tensor reads as zero
+          if (from_rows) y[i] = u < ck.n_valid ? (int)ord_mask[ck.off + u] : a.n_active;
+          else y[i] = u < ck.n_valid ? ord_col[ck.off + u] : a.L;
         }
         for (int k = 0; k < n_slots; ++k) {
           const int slot = (f + k) % kSlots;
-          tc::tma_gather4(ring + slot * kSlotBytes + is_v * kTileBytes + slab * (kNC * 128) + grp * 512, map,
+          const void* src = !from_rows ? map
+                            : (k == 0 ? (is_v ? static_cast<const void*>(&a.v_prev_map) : static_cast<const void*>(&a.k_prev_map))
+                                      : (is_v ? static_cast<const void*>(&a.v_cur_map) : static_cast<const void*>(&a.k_cur_map)));
+          tc::tma_gather4(ring + slot * kSlotBytes + is_v * kTileBytes + slab * (kNC * 128) + grp * 512, src,
                           &ctl.landed[slot], h * kDH + slab * 64, y[0], y[1], y[2], y[3]);
         }
       }
@@ -893,6 +848,16 @@ int fl_launch_loop_attn_tc(fl_ctx* ctx, const fl_shape* s, int loop_r, const voi
   fl_dev_side(store, true, &a.k);
   fl_dev_side(store, false, &a.v);
   a.n_old = loop_r - 2;
+  // the loop's materialized rows, when the caller keeps them (all four buffers)
+  const fl_kv_stream& ks = store->k_res[loop_r - 2];
+  const fl_kv_stream& vs = store->v_res[loop_r - 2];
+  a.use_rows = ks.rows_prev != nullptr && ks.rows_cur != nullptr && vs.rows_prev != nullptr && vs.rows_cur != nullptr &&
+               ks.n_rows == n_active && n_active > 0;
+  if (a.use_rows && (!fl_tile_tmap(ctx, ks.rows_prev, n_active, d_row, 1, &a.k_prev_map) ||
+                     !fl_tile_tmap(ctx, ks.rows_cur, n_active, d_row, 1, &a.k_cur_map) ||
+                     !fl_tile_tmap(ctx, vs.rows_prev, n_active, d_row, 1, &a.v_prev_map) ||
+                     !fl_tile_tmap(ctx, vs.rows_cur, n_active, d_row, 1, &a.v_cur_map)))
+    return FL_ERR_UNSUPPORTED;
   a.col_idx = col_idx; a.col_cnt = col_cnt; a.c = c;
   a.lse_prev = lse_prev; a.lse_out = lse_out; a.status = status;
   a.L = s->L; a.H = s->n_heads; a.q_block = s->q_block; a.nb = fl_n_blocks(s);

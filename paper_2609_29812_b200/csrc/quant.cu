@@ -12,6 +12,8 @@ struct QuantArgs {
   const int32_t* active_idx;    // [n]
   uint8_t* k_codes; __half* k_scale; __half* k_zero;   // stream being written
   uint8_t* v_codes; __half* v_scale; __half* v_zero;
+  void* k_rows_prev; void* k_rows_cur;   // optional [n, H, dh] storage type: Xhat^(r-1) / Xhat^(r) of the active rows
+  void* v_rows_prev; void* v_rows_cur;
   int n_prev;                   // residual streams already in the chain (loop_r - 2)
   int d, group;
 };
@@ -25,6 +27,8 @@ __global__ void __launch_bounds__(256) quant_residual_kernel(const __grid_consta
   uint8_t* codes = is_v ? a.v_codes : a.k_codes;
   __half* scale = is_v ? a.v_scale : a.k_scale;
   __half* zero = is_v ? a.v_zero : a.k_zero;
+  T* rows_prev = static_cast<T*>(is_v ? a.v_rows_prev : a.k_rows_prev);   // null: not wanted
+  T* rows_cur = static_cast<T*>(is_v ? a.v_rows_cur : a.k_rows_cur);
   const int pos = __ldg(a.active_idx + t);
   const int lanes_per_group = a.group >> 3;  // 1, 2, 4, 8 or 16
 
@@ -46,8 +50,10 @@ __global__ void __launch_bounds__(256) quant_residual_kernel(const __grid_consta
       for (int si = 0; si < 4; ++si)
         if (sl[si] >= 0) payload_apply<T, BITS>(pl[si], xh);
     }
+    if (rows_prev != nullptr) store8<T>(rows_prev + (size_t)t * a.d + elem, xh);
     if (BITS == 16) {  // codec off: the stream keeps the row itself
       store8<T>(reinterpret_cast<T*>(codes) + (size_t)t * a.d + elem, xn);
+      if (rows_cur != nullptr) store8<T>(rows_cur + (size_t)t * a.d + elem, xn);
       continue;
     }
     float dl[8];
@@ -90,6 +96,12 @@ __global__ void __launch_bounds__(256) quant_residual_kernel(const __grid_consta
     } else {
 #pragma unroll
       for (int i = 0; i < 8; ++i) q[i] = 0.f;
+    }
+    if (rows_cur != nullptr) {
+      // the reconstruction every later reader of this stream forms: Xhat + (code * scale + zero), Eq. 8
+#pragma unroll
+      for (int i = 0; i < 8; ++i) xh[i] = __fadd_rn(xh[i], __fmaf_rn(q[i], sf, zf));
+      store8<T>(rows_cur + (size_t)t * a.d + elem, xh);
     }
     // The quotients are integers in [0, qmax] already: delta >= zero (the offset was rounded down) and
     // (max - zero) / scale <= qmax (the scale was rounded up), so the oracle's clamp never acts. Four codes at a
@@ -168,6 +180,9 @@ extern "C" int fl_quant_kv_residual(fl_ctx* ctx, const fl_shape* shape, int loop
   a.k_zero = reinterpret_cast<__half*>(ks.zero);
   a.v_codes = static_cast<uint8_t*>(vs.codes); a.v_scale = reinterpret_cast<__half*>(vs.scale);
   a.v_zero = reinterpret_cast<__half*>(vs.zero);
+  const bool rows = shape->dtype == FL_BF16 && ks.rows_prev != nullptr && vs.rows_prev != nullptr;
+  a.k_rows_prev = rows ? ks.rows_prev : nullptr; a.k_rows_cur = rows ? ks.rows_cur : nullptr;
+  a.v_rows_prev = rows ? vs.rows_prev : nullptr; a.v_rows_cur = rows ? vs.rows_cur : nullptr;
   a.n_prev = loop_r - 2; a.d = d; a.group = shape->group;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   return shape->dtype == FL_F32 ? launch_quant<float>(shape, a, n_active, st)

@@ -53,6 +53,21 @@ def select_tokens(ctx, shape, loop_r, g_prev, g_cur, cand: Optional[torch.Tensor
     return TokenSelection(active[:n], slot, scores, n)
 
 
+_ROWS_WS: dict = {}
+
+
+def rows_workspace(dev, n: int, d: int):
+    """Transient bf16 buffers [n, d] for the materialized rows of one loop: ((K before, K after), (V before,
+    V after)).  One set per device, grown on demand and reused by every layer and loop: a loop's rows are dead once
+    its attention call has been issued on the stream."""
+    key = (str(dev), d)
+    ws = _ROWS_WS.get(key)
+    if ws is None or ws[0][0].shape[0] < n:
+        ws = tuple(tuple(torch.empty(n, d, dtype=torch.bfloat16, device=dev) for _ in range(2)) for _ in range(2))
+        _ROWS_WS[key] = ws
+    return ws
+
+
 class LayerState:
     """Buffers of one layer and the calls that advance it by one loop."""
 
@@ -107,20 +122,29 @@ class LayerState:
     def _rebuild_store(self):
         self.store = B.make_store(self.k_base, self.v_base, self.k_streams, self.v_streams)
 
-    def alloc_stream(self, sel: TokenSelection):
+    def alloc_stream(self, sel: TokenSelection, rows: bool = True):
+        """Adds the residual stream of the next loop.  rows: also lend it the transient workspace for the loop's
+        materialized rows (bf16 storage only), which the quantization kernel fills and the attention kernel of the
+        same loop gathers from; the workspace is shared by every LayerState of the device."""
         w, n = self.w, sel.n
         d = w.d
+        ws = rows_workspace(self.dev, n, d) if rows and self.dt == torch.bfloat16 and n > 0 else None
 
-        def one():
+        def one(side):
+            st = {"slot_of_pos": sel.slot_of_pos, "n_rows": n}
+            if ws is not None:
+                st["rows_prev"], st["rows_cur"] = ws[side][0][:n], ws[side][1][:n]
             if self.bits == 16:
-                return {"codes": torch.empty(max(n, 1), d, dtype=self.dt, device=self.dev), "scale": None,
-                        "zero": None, "slot_of_pos": sel.slot_of_pos, "n_rows": n}
-            return {"codes": torch.empty(max(n, 1), d * self.bits // 8, dtype=torch.uint8, device=self.dev),
-                    "scale": torch.empty(max(n, 1), d // w.group, dtype=torch.float16, device=self.dev),
-                    "zero": torch.empty(max(n, 1), d // w.group, dtype=torch.float16, device=self.dev),
-                    "slot_of_pos": sel.slot_of_pos, "n_rows": n}
-        self.k_streams.append(one())
-        self.v_streams.append(one())
+                st.update(codes=torch.empty(max(n, 1), d, dtype=self.dt, device=self.dev), scale=None, zero=None)
+            else:
+                st.update(codes=torch.empty(max(n, 1), d * self.bits // 8, dtype=torch.uint8, device=self.dev),
+                          scale=torch.empty(max(n, 1), d // w.group, dtype=torch.float16, device=self.dev),
+                          zero=torch.empty(max(n, 1), d // w.group, dtype=torch.float16, device=self.dev))
+            return st
+        # every stream of the device points at the same workspace: its content belongs to whichever loop was
+        # quantized last, and only that loop's attention call reads it
+        self.k_streams.append(one(0))
+        self.v_streams.append(one(1))
         self._rebuild_store()
 
     def quantize(self, loop_r, k_new, v_new, sel: TokenSelection):

@@ -148,6 +148,14 @@ def test_quantizer_codes_bit_exact_all_loops(env, case):
         rec = ref["loops"][r - 2]
         for side, streams in (("k_payload", st.k_streams), ("v_payload", st.v_streams)):
             pay, got = rec[side], streams[-1]
+            if w.dtype == "bf16":
+                # the loop's materialized rows: the oracle's reconstruction before / after the residual, rounded
+                # once to bf16 (what the attention of this loop consumes), bit for bit
+                hat_old, hat_new = rec[side[0] + "hat_old"], rec[side[0] + "hat"]
+                for name, want in (("rows_prev", hat_old), ("rows_cur", hat_new)):
+                    got_rows = to_np(got[name]).astype(np.float32).reshape(len(act), w.n_heads, -1)
+                    assert np.array_equal(got_rows.view(np.uint32), fo.round_bf16(want[act]).view(np.uint32)), \
+                        (r, side, name)
             if w.bits == 16:
                 assert np.array_equal(to_np(got["codes"]).reshape(pay["raw"].shape), pay["raw"])
                 continue
@@ -209,9 +217,15 @@ def sets_to_arrays(w, nb, col_sets, c):
     return idx, cnt
 
 
-def test_loop_attention_stage_isolated(env, case):
+ROWS = pytest.mark.parametrize("rows", [True, False], ids=["materialized_rows", "rebuilt_in_kernel"])
+
+
+@ROWS
+def test_loop_attention_stage_isolated(env, case, rows):
     """Each loop's attention is fed the oracle's upstream state (token set, column sets, previous
-    outputs and log-normalisers rounded to storage precision; the store is bit-exact anyway)."""
+    outputs and log-normalisers rounded to storage precision; the store is bit-exact anyway).  rows: the columns
+    active in the loop come from the rows the quantization kernel materialized, or (without that workspace) are
+    rebuilt from the residual streams inside the attention kernel."""
     B, P, ctx = env
     w, x, ref = case
     st = P.LayerState(ctx, w)
@@ -222,7 +236,7 @@ def test_loop_attention_stage_isolated(env, case):
         rec = ref["loops"][r - 2]
         act = rec["active"]
         sel = oracle_selection(P, w, ref, r)
-        st.alloc_stream(sel)
+        st.alloc_stream(sel, rows=rows)
         st.quantize(r, to_dev(x.K[r - 1][act], w), to_dev(x.V[r - 1][act], w), sel)
         idx, cnt = sets_to_arrays(w, st.nb, rec["col_sets"], w.col_budget)
         st.col_idx, st.col_cnt, st.c = torch.from_numpy(idx).cuda(), torch.from_numpy(cnt).cuda(), w.col_budget
@@ -347,7 +361,8 @@ def test_binary32_simt_attention_path_on_bf16_storage(env):
     ctx.close()
 
 
-def test_many_patched_columns_and_wide_budgets(env):
+@ROWS
+def test_many_patched_columns_and_wide_budgets(env, rows):
     """Half of the rows active and a column budget of several chunks: long runs of columns that carry
     residual payloads (two ring slots per chunk) and several 128-row tiles per query block."""
     B, P, ctx = env
@@ -364,7 +379,7 @@ def test_many_patched_columns_and_wide_budgets(env):
         rec = ref["loops"][r - 2]
         act = rec["active"]
         sel = oracle_selection(P, w, ref, r)
-        st.alloc_stream(sel)
+        st.alloc_stream(sel, rows=rows)
         st.quantize(r, to_dev(x.K[r - 1][act], w), to_dev(x.V[r - 1][act], w), sel)
         idx, cnt = sets_to_arrays(w, st.nb, rec["col_sets"], w.col_budget)
         st.col_idx, st.col_cnt, st.c = torch.from_numpy(idx).cuda(), torch.from_numpy(cnt).cuda(), w.col_budget

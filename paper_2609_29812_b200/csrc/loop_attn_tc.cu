@@ -281,11 +281,43 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
       else { ctl.q_hi = r; ctl.i_last = r > 0 ? below : -1; }
     }
   } else {
-    // the whole row of the column table is read without waiting for its count: entries past the count are -1
+    // The whole row of the column table is read without waiting for its count (entries past the count are -1),
+    // and the thread that read a column goes on to look it up in the slot map of every residual stream: three
+    // columns per thread and up to four streams at a time are in flight, two dependent rounds in all.
+    constexpr int kBatch = 3, kStride = kColWarps * 32;
 #pragma unroll 1
-    for (int u = tid; u < c_cap; u += kColWarps * 32) {
-      raw_col[u] = __ldg(cols + u);
-      raw_mask[u] = 0;
+    for (int u0 = tid; u0 < c_cap; u0 += kBatch * kStride) {
+      int j[kBatch], sl_new[kBatch];
+      uint32_t mask[kBatch];
+#pragma unroll
+      for (int k = 0; k < kBatch; ++k) {
+        j[k] = u0 + k * kStride < c_cap ? __ldg(cols + u0 + k * kStride) : -1;
+        mask[k] = 0;
+        sl_new[k] = -1;
+      }
+#pragma unroll 1
+      for (int sg = 0; sg <= a.n_old; sg += 4) {
+        int sl[kBatch][4];
+#pragma unroll
+        for (int k = 0; k < kBatch; ++k)
+#pragma unroll
+          for (int q = 0; q < 4; ++q)
+            sl[k][q] = (j[k] >= 0 && sg + q <= a.n_old) ? __ldg(a.k.s[sg + q].slot + j[k]) : -1;
+#pragma unroll
+        for (int k = 0; k < kBatch; ++k)
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            if (sl[k][q] >= 0) mask[k] |= 1u << (sg + q);
+            if (sg + q == a.n_old) sl_new[k] = sl[k][q];
+          }
+      }
+#pragma unroll
+      for (int k = 0; k < kBatch; ++k)
+        if (u0 + k * kStride < c_cap) {
+          raw_col[u0 + k * kStride] = j[k];
+          raw_mask[u0 + k * kStride] = mask[k];
+          raw_slot[u0 + k * kStride] = sl_new[k];
+        }
     }
   }
   if (warp == kIssueWarp) {
@@ -300,16 +332,6 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
   const int q_lo = ctl.q_lo, q_hi = ctl.q_hi;
   if (q_hi > q_lo) {   // CTA-uniform: blocks without active rows only release the tensor memory
   {
-    // every (column, stream) pair is one independent slot-map lookup
-#pragma unroll 1
-    for (int p2 = tid; p2 < c_cap * (a.n_old + 1); p2 += kThreads) {
-      const int s = p2 / c_cap, u = p2 - s * c_cap;
-      const int j = raw_col[u];
-      const int sl = j >= 0 ? __ldg(a.k.s[s].slot + j) : -1;
-      if (sl >= 0) atomicOr(&raw_mask[u], 1u << s);
-      if (s == a.n_old) raw_slot[u] = sl;
-    }
-    __syncthreads();
     // causal prefix, stable partition into plain / patched columns: every warp owns a contiguous span
     const int i_last = ctl.i_last;                                   // last active row of the block
     const int span = ((cnt + kWarps - 1) / kWarps + 31) & ~31;
@@ -325,13 +347,17 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
     }
     if (lane == 0) { ctl.warp_cnt[warp][0] = n0; ctl.warp_cnt[warp][1] = n1; }
     __syncthreads();
-    int before0 = 0, before1 = 0, tot0 = 0, tot1 = 0;
-#pragma unroll 1
-    for (int wv = 0; wv < kWarps; ++wv) {
-      const int c0 = ctl.warp_cnt[wv][0], c1 = ctl.warp_cnt[wv][1];
-      if (wv < warp) { before0 += c0; before1 += c1; }
-      tot0 += c0; tot1 += c1;
+    // exclusive prefix over the warps' counts: lane w of every warp holds warp w's pair
+    static_assert(kWarps <= 32, "one lane per warp");
+    int inc0 = lane < kWarps ? ctl.warp_cnt[lane][0] : 0, inc1 = lane < kWarps ? ctl.warp_cnt[lane][1] : 0;
+#pragma unroll
+    for (int off = 1; off < kWarps; off <<= 1) {
+      const int t0 = __shfl_up_sync(0xffffffffu, inc0, off), t1 = __shfl_up_sync(0xffffffffu, inc1, off);
+      if (lane >= off) { inc0 += t0; inc1 += t1; }
     }
+    const int tot0 = __shfl_sync(0xffffffffu, inc0, kWarps - 1), tot1 = __shfl_sync(0xffffffffu, inc1, kWarps - 1);
+    const int up0 = __shfl_sync(0xffffffffu, inc0, (warp + 31) & 31), up1 = __shfl_sync(0xffffffffu, inc1, (warp + 31) & 31);
+    int before0 = warp > 0 ? up0 : 0, before1 = warp > 0 ? up1 : 0;
     if (tid == 0) { ctl.n_plain = tot0; ctl.n_patch = tot1; }
     const uint32_t lt = (1u << lane) - 1;
 #pragma unroll 1

@@ -254,7 +254,8 @@ __global__ void __launch_bounds__(kSelThreads, 1) column_select_smem_kernel(cons
   extern __shared__ __align__(16) uint32_t keys[];   // [n rounded up to 4], padded with key 0 (below every real key)
   __shared__ SelectSmem2 sm;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int b = blockIdx.x, h = blockIdx.y;
+  // later blocks have more candidates (causal prefix): they are dispatched first, the short ones fill the tail
+  const int h = blockIdx.x, b = gridDim.y - 1 - blockIdx.y;
   const size_t prob = (size_t)h * nb + b;
   const float* vals = col_scores + prob * stride;
   const int32_t* cols = cand_cols != nullptr ? cand_cols + prob * stride : nullptr;
@@ -480,7 +481,8 @@ __global__ void __launch_bounds__(kSelThreads) column_select_kernel(const float*
                                                                     int32_t* __restrict__ col_idx,
                                                                     int32_t* __restrict__ col_cnt) {
   __shared__ SelectSmem sm;
-  const int b = blockIdx.x, h = blockIdx.y;
+  // later blocks have more candidates (causal prefix): they are dispatched first, the short ones fill the tail
+  const int h = blockIdx.x, b = gridDim.y - 1 - blockIdx.y;
   const size_t prob = (size_t)h * nb + b;
   const float* vals = col_scores + prob * stride;
   const int32_t* cols = cand_cols != nullptr ? cand_cols + prob * stride : nullptr;
@@ -542,8 +544,8 @@ extern "C" int fl_select_columns(fl_ctx* ctx, const fl_shape* shape, const float
   if (cand_cols == nullptr) FL_REQUIRE(n_cand == shape->L);
   else FL_REQUIRE(cand_cnt != nullptr);
   const int nb = fl_n_blocks(shape);
-  FL_REQUIRE(nb <= 65535 * 1024 && shape->n_heads <= 65535);
-  dim3 grid(nb, shape->n_heads);
+  FL_REQUIRE(nb <= 65535);
+  dim3 grid(shape->n_heads, nb);
   const size_t key_bytes = sizeof(uint32_t) * (((size_t)n_cand + 3) & ~(size_t)3);
   if (n_cand <= kSelCap && key_bytes + 32768 <= (size_t)ctx->max_smem_optin) {
     // keys staged in shared memory: the scores are read from global memory once

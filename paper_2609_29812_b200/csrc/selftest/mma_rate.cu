@@ -113,7 +113,10 @@ __global__ void __launch_bounds__(320) mma_rate_kernel(int mode, int noise, int 
       if (tid == 0) {
         tc::mbar_wait(&bar, 0, &abort_flag, 1u << 24);
         cycles_out[blockIdx.x] = clock64() - t0;
+        stop_flag = 1;
       }
+    } else if (noise != 0) {
+      noise_loop(noise, tmem, smem, &stop_flag, cycles_out);   // the issuing thread's neighbours on the schedulers
     }
   } else if (mode >= 4) {
     if (tid == 0 || (mode == 6 && tid == 32)) {

@@ -273,25 +273,42 @@ __global__ void __launch_bounds__(kSelThreads, 1) column_select_smem_kernel(cons
   {
     const float4* v4 = reinterpret_cast<const float4*>(vals);
     uint4* k4 = reinterpret_cast<uint4*>(keys);
-    for (int base = 0; base < n4; base += kSelThreads) {   // whole warps run every step: padding keys are 0 (bin 0)
-      const int i = base + tid;
-      uint4 kv = make_uint4(0, 0, 0, 0);
-      if (i < n4) {
-        if (vec_ok && i * 4 + 3 < n) {
-          const float4 v = __ldg(v4 + i);
-          kv = make_uint4(ordered_key(v.x), ordered_key(v.y), ordered_key(v.z), ordered_key(v.w));
-        } else {
-          if (i * 4 + 0 < n) kv.x = ordered_key(__ldg(vals + i * 4 + 0));
-          if (i * 4 + 1 < n) kv.y = ordered_key(__ldg(vals + i * 4 + 1));
-          if (i * 4 + 2 < n) kv.z = ordered_key(__ldg(vals + i * 4 + 2));
-          if (i * 4 + 3 < n) kv.w = ordered_key(__ldg(vals + i * 4 + 3));
+    // four steps' loads are issued before the first is consumed: the staging is bound by memory latency otherwise
+    // (whole warps run every step: padding keys are 0, bin 0)
+    for (int base0 = 0; base0 < n4; base0 += 4 * kSelThreads) {
+      float4 v[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int i = base0 + q * kSelThreads + tid;
+        v[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (i < n4) {
+          if (vec_ok && i * 4 + 3 < n) {
+            v[q] = __ldg(v4 + i);
+          } else {
+            if (i * 4 + 0 < n) v[q].x = __ldg(vals + i * 4 + 0);
+            if (i * 4 + 1 < n) v[q].y = __ldg(vals + i * 4 + 1);
+            if (i * 4 + 2 < n) v[q].z = __ldg(vals + i * 4 + 2);
+            if (i * 4 + 3 < n) v[q].w = __ldg(vals + i * 4 + 3);
+          }
         }
-        k4[i] = kv;
       }
-      hist12_add(sm.hist12, kv.x, lane);
-      hist12_add(sm.hist12, kv.y, lane);
-      hist12_add(sm.hist12, kv.z, lane);
-      hist12_add(sm.hist12, kv.w, lane);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int i = base0 + q * kSelThreads + tid;
+        if (base0 + q * kSelThreads >= n4) break;   // CTA-uniform
+        uint4 kv = make_uint4(0, 0, 0, 0);
+        if (i < n4) {
+          if (i * 4 + 0 < n) kv.x = ordered_key(v[q].x);
+          if (i * 4 + 1 < n) kv.y = ordered_key(v[q].y);
+          if (i * 4 + 2 < n) kv.z = ordered_key(v[q].z);
+          if (i * 4 + 3 < n) kv.w = ordered_key(v[q].w);
+          k4[i] = kv;
+        }
+        hist12_add(sm.hist12, kv.x, lane);
+        hist12_add(sm.hist12, kv.y, lane);
+        hist12_add(sm.hist12, kv.z, lane);
+        hist12_add(sm.hist12, kv.w, lane);
+      }
     }
   }
   __syncthreads();

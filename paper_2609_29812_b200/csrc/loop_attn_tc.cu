@@ -545,21 +545,20 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
         const int gc = g0 + ci;
         if (t == 0) TC_TRACE(1, ci, 0);
         if (ci == 0 && !tc::mbar_wait(&ctl.q_full, tile & 1, abort_flag)) break;
-        if (!tc::mbar_wait(&ctl.landed[slot0], (f / kSlots) & 1, abort_flag)) break;
-        if (ck.patch && !tc::mbar_wait(&ctl.landed[slot1], ((f + 1) / kSlots) & 1, abort_flag)) break;
+        // a term reads one slot of the chunk only (the new term of a two-slot chunk the second): it starts on it
+        // without waiting for the other
+        const int my_slot = (t && ck.patch) ? slot1 : slot0, my_fill = (t && ck.patch) ? f + 1 : f;
+        if (!tc::mbar_wait(&ctl.landed[my_slot], (my_fill / kSlots) & 1, abort_flag)) break;
         if (ctl.chunk_mask[ci] != 0) {       // residual-carrying columns are rewritten by the patch warps
-          if (!tc::mbar_wait(&ctl.patched[slot0], (dirty_par >> slot0) & 1, abort_flag)) break;
+          if (!tc::mbar_wait(&ctl.patched[my_slot], (dirty_par >> my_slot) & 1, abort_flag)) break;
           dirty_par ^= 1u << slot0;
-          if (ck.patch) {
-            if (!tc::mbar_wait(&ctl.patched[slot1], (dirty_par >> slot1) & 1, abort_flag)) break;
-            dirty_par ^= 1u << slot1;
-          }
+          if (ck.patch) dirty_par ^= 1u << slot1;
         }
         // the S buffer holds the previous chunk until the softmax warps have pulled it into registers
         if (gc >= 1 && !tc::mbar_wait(&ctl.s_taken[t], (gc - 1) & 1, abort_flag)) break;
         tc::tc_fence_after();
         if (t == 0) TC_TRACE(1, ci, 1);
-        const uint32_t k_lo = k_lo0 + ((t && ck.patch) ? slot1 : slot0) * (kSlotBytes >> 4);
+        const uint32_t k_lo = k_lo0 + my_slot * (kSlotBytes >> 4);
 #define FL_QK(KK, ACC)                                                                                       \
   tc::mma_ss_lo<ACC>(s_dst, q_lo_w + ((((KK) >> 2) * (kM * 128) + ((KK)&3) * 32) >> 4), kq_hi,               \
                      k_lo + ((((KK) >> 2) * (kNC * 128) + ((KK)&3) * 32) >> 4), kq_hi, idesc_qk)

@@ -1,25 +1,32 @@
 // Active-row gather / scatter (Appendix G: only the selected token rows are processed; inactive rows
-// keep their hidden states and KV entries). HBM-bound copies: one warp per row, 16-byte accesses.
+// keep their hidden states and KV entries). HBM-bound copies with 16-byte accesses.
 #include "fl_internal.cuh"
 
 namespace {
 
+// One warp per piece of at most 128 vectors (2 KB) of a row: a lane has its (up to) four 16-byte loads in flight at
+// once, and a row of several KB is spread over several warps, so that the launch is two dependent rounds deep (index,
+// then data) however wide the rows are.
 template <bool GATHER>
 __global__ void __launch_bounds__(256) rows_copy_kernel(const uint4* __restrict__ src, const int32_t* __restrict__ idx,
-                                                        int n, int vec_per_row, uint4* __restrict__ dst) {
+                                                        int n, int vec_per_row, int pieces, uint4* __restrict__ dst) {
   const int warps_per_block = blockDim.x >> 5;
   const int lane = threadIdx.x & 31;
-  for (int t = blockIdx.x * warps_per_block + (threadIdx.x >> 5); t < n; t += gridDim.x * warps_per_block) {
+  const int64_t n_work = (int64_t)n * pieces;
+  for (int64_t wi = (int64_t)blockIdx.x * warps_per_block + (threadIdx.x >> 5); wi < n_work;
+       wi += (int64_t)gridDim.x * warps_per_block) {
+    const int t = (int)(wi / pieces), piece = (int)(wi - (int64_t)t * pieces);
     const int64_t row = __ldg(idx + t);
     const uint4* s = src + (GATHER ? row : (int64_t)t) * vec_per_row;
     uint4* d = dst + (GATHER ? (int64_t)t : row) * vec_per_row;
-    int v = lane;
-    // four independent 16-byte loads in flight per lane before the stores
-    for (; v + 96 < vec_per_row; v += 128) {
-      uint4 a = __ldg(s + v), b = __ldg(s + v + 32), c = __ldg(s + v + 64), e = __ldg(s + v + 96);
-      d[v] = a; d[v + 32] = b; d[v + 64] = c; d[v + 96] = e;
-    }
-    for (; v < vec_per_row; v += 32) d[v] = __ldg(s + v);
+    const int v0 = piece * 128 + lane, v_end = min(vec_per_row, (piece + 1) * 128);
+    uint4 r[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+      if (v0 + 32 * k < v_end) r[k] = __ldg(s + v0 + 32 * k);
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+      if (v0 + 32 * k < v_end) d[v0 + 32 * k] = r[k];
   }
 }
 
@@ -32,16 +39,18 @@ int rows_copy(bool gather, fl_ctx* ctx, const void* src, const int32_t* idx, int
   FL_REQUIRE(src != nullptr && dst != nullptr && idx != nullptr);
   FL_REQUIRE(fl_aligned16(src) && fl_aligned16(dst));
   const int warps = 8;
-  int grid = (n + warps - 1) / warps;
-  const int max_grid = ctx->sm_count * 16;
-  if (grid > max_grid) grid = max_grid;
+  const int vec_per_row = (int)(row_bytes / 16);
+  const int pieces = (vec_per_row + 127) / 128;
+  int64_t grid64 = ((int64_t)n * pieces + warps - 1) / warps;
+  const int64_t max_grid = (int64_t)ctx->sm_count * 32;
+  const int grid = (int)(grid64 > max_grid ? max_grid : grid64);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (gather)
-    rows_copy_kernel<true><<<grid, warps * 32, 0, st>>>(static_cast<const uint4*>(src), idx, n, (int)(row_bytes / 16),
+    rows_copy_kernel<true><<<grid, warps * 32, 0, st>>>(static_cast<const uint4*>(src), idx, n, vec_per_row, pieces,
                                                         static_cast<uint4*>(dst));
   else
-    rows_copy_kernel<false><<<grid, warps * 32, 0, st>>>(static_cast<const uint4*>(src), idx, n,
-                                                         (int)(row_bytes / 16), static_cast<uint4*>(dst));
+    rows_copy_kernel<false><<<grid, warps * 32, 0, st>>>(static_cast<const uint4*>(src), idx, n, vec_per_row, pieces,
+                                                         static_cast<uint4*>(dst));
   return fl_launch_status();
 }
 

@@ -140,6 +140,8 @@ FL_API int fl_scatter_update(fl_ctx* ctx, const void* src, const int32_t* idx, i
  *   code  = scale == 0 ? 0 : clamp(round-half-even((delta - zero) / scale), 0, 2^bits - 1)
  * and writes stream r (store->k_res[loop_r-2], v_res[loop_r-2]; codes/scale/zero pre-allocated by the
  * caller for n_rows == n_active, slot_of_pos already filled for loop r). |delta| must stay below 65504.
+ * With bf16 storage and the stream's rows_prev / rows_cur set (K and V alike) it also writes, per active row,
+ * Xhat^(r-1)_i and Xhat^(r)_i = Xhat^(r-1)_i + (code * scale + zero), each rounded once to bf16.
  * k_new, v_new: [n_active, H, dh] storage type. store is a host struct; store->n_streams must be
  * >= loop_r - 1 (the stream being written counts). Errors: loop_r < 2 or > FL_MAX_LOOPS+1, bad bits or
  * group, null buffers, n_rows mismatch. n_active == 0 is a no-op. */
@@ -165,7 +167,10 @@ FL_API int fl_select_columns(fl_ctx* ctx, const fl_shape* shape, const float* co
                       const int32_t* cand_cnt, int32_t n_cand, int32_t c, int32_t* col_idx, int32_t* col_cnt,
                       int32_t* status, void* stream);
 
-/* Stages 2 + 4 -- Eq. 7 (equivalently Eq. 3) over K/V reconstructed inside the kernel.
+/* Stages 2 + 4 -- Eq. 7 (equivalently Eq. 3) over the reconstructed K/V (Eq. 4 / Eq. 8): rows of tokens that are
+ * active in loop r are read from the stream's rows_prev / rows_cur when fl_quant_kv_residual of loop r has left them
+ * there (store->k_res[loop_r-2] and v_res[loop_r-2], all four buffers set), everything else is rebuilt inside the
+ * kernel from the base and the residual streams.
  * For head h, active row t (position i = active_idx[t], block b), T_i = { j in col_idx[h,b,:] : j <= i }:
  *   p_old_j = exp(sm_scale q_old_t . Khat^(r-1)_j - lse_prev[h,i])       previous loop's probabilities
  *   m_i     = sum_{T_i} p_old_j                                          cached global mass

@@ -611,6 +611,9 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
     const int pos = row_ok ? __ldg(a.active_idx + s0 + row) : -1;
     const float c2 = a.scale * kLog2e;
     const float lse2 = (row_ok ? a.lse_prev[(size_t)h * a.L + pos] : 0.f) * kLog2e;
+    // the epilogue reads the row's previous output: have it in L2 by then (each group asks for its 128-byte half)
+    if (row_ok)
+      tc::prefetch_l2(a.o_prev + (INDEXED ? (size_t)pos : (size_t)(s0 + row)) * a.d + h * kDH + grp * 64);
     const uint32_t s_addr = tmem + lane_base + (grp ? kSNew : kSOld);
     const uint32_t p_addr = tmem + lane_base + (grp ? kPNew : kPOld);
     float mass = 0.f, ell = 0.f, ref = -INFINITY;

@@ -44,7 +44,7 @@ typedef enum {
   FL_OK = 0,
   FL_ERR_INVALID_ARG = -1, /* null / misaligned pointer, size out of range, inconsistent store */
   FL_ERR_UNSUPPORTED = -2, /* a valid request this build has no kernel for (e.g. head_dim 96) */
-  FL_ERR_WORKSPACE = -3,   /* reserved (no entry point needs a workspace) */
+  FL_ERR_WORKSPACE = -3,   /* the workspace handed to fl_set_workspace is too small to be of any use */
   FL_ERR_CUDA = -4,        /* a CUDA runtime call failed (launch error, wrong device, ...) */
   FL_ERR_TIMEOUT = -5      /* reported through the device status word: a bounded wait ran out */
 } fl_status;
@@ -166,6 +166,19 @@ FL_API int fl_dense_loop_attention(fl_ctx* ctx, const fl_shape* shape, const voi
 FL_API int fl_select_columns(fl_ctx* ctx, const fl_shape* shape, const float* col_scores, const int32_t* cand_cols,
                       const int32_t* cand_cnt, int32_t n_cand, int32_t c, int32_t* col_idx, int32_t* col_cnt,
                       int32_t* status, void* stream);
+
+/* Optional workspace for fl_loop_attention / fl_loop_attention_indexed (device memory of the caller, 256-byte
+ * aligned; the paper has no counterpart: it is a scheduling aid of this implementation). The attention launch has one
+ * CTA per (head, query block) problem and the problems cost about the same, so a problem count that is not a multiple
+ * of the SM count ends in a partly empty wave. With a workspace of fl_loop_attention_workspace_bytes() bytes (0 when a
+ * split cannot help the shape), the problems of that last wave are given to two CTAs each; the one that finishes
+ * first leaves its partial accumulators there and the other adds them to its own, so the result does not depend on
+ * which came first beyond the rounding order of that one addition. fl_set_workspace clears the arrival counters at the
+ * head of the buffer on `stream` (every launch leaves them cleared); the buffer must stay valid until fl_destroy or
+ * the next fl_set_workspace (NULL detaches it). Attention calls of one context that may overlap in time (different
+ * streams) must not share a workspace. */
+FL_API int fl_loop_attention_workspace_bytes(fl_ctx* ctx, const fl_shape* shape, int64_t* bytes /* host */);
+FL_API int fl_set_workspace(fl_ctx* ctx, void* workspace /* device */, int64_t bytes, void* stream);
 
 /* Stages 2 + 4 -- Eq. 7 (equivalently Eq. 3) over the reconstructed K/V (Eq. 4 / Eq. 8): rows of tokens that are
  * active in loop r are read from the stream's rows_prev / rows_cur when fl_quant_kv_residual of loop r has left them

@@ -71,6 +71,8 @@ def _load() -> C.CDLL:
                                       i32, p, p, p, p, p, p, p],
         "fl_kv_store_bytes": [C.POINTER(FlShape), C.POINTER(FlKvStore), C.c_int, C.c_int,
                               C.POINTER(i64), C.POINTER(i64)],
+        "fl_loop_attention_workspace_bytes": [p, C.POINTER(FlShape), C.POINTER(i64)],
+        "fl_set_workspace": [p, p, i64, p],
     }
     for name, args in sig.items():
         fn = getattr(lib, name)
@@ -173,6 +175,18 @@ def fl_select_tokens(ctx, shape, loop_r, h_prev, h_cur, cand, n_cand, k, scores,
                               int(n_cand), int(k), _ptr(scores), _ptr(active_idx), _ptr(slot_of_pos),
                               _ptr(status), _stream(stream))
     return _check("fl_select_tokens", rc, check)
+
+
+def fl_loop_attention_workspace_bytes(ctx, shape) -> int:
+    out = C.c_int64(0)
+    _check("fl_loop_attention_workspace_bytes", lib.fl_loop_attention_workspace_bytes(_h(ctx), C.byref(shape),
+                                                                                      C.byref(out)), True)
+    return int(out.value)
+
+
+def fl_set_workspace(ctx, workspace, nbytes, stream=None, check=True) -> int:
+    rc = lib.fl_set_workspace(_h(ctx), _ptr(workspace), int(nbytes), _stream(stream))
+    return _check("fl_set_workspace", rc, check)
 
 
 def fl_gather_rows(ctx, src, idx, n, row_bytes, dst, stream=None, check=True) -> int:

@@ -15,7 +15,12 @@ struct fl_ctx {
   int force_simt;  // environment FL_FORCE_SIMT=1 at fl_create: keep attention on the binary32 SIMT kernels
   void* encode_tiled;       // cuTensorMapEncodeTiled, resolved through cudaGetDriverEntryPoint (may be null)
   struct fl_tmap_cache* tmaps;  // tensor maps, keyed by (base pointer, rows, row elements, box rows)
+  void* ws;                 // caller's workspace (fl_set_workspace), or null
+  size_t ws_bytes;
 };
+
+// Bytes of workspace with which the loop-attention launch can split the problems of its last wave (0: never useful).
+size_t fl_attn_workspace_bytes(const fl_ctx* ctx, const fl_shape* s);
 
 // Tensor map of a row-major bf16 matrix [rows, row_elems] for TMA: box = 64 elements x box_rows rows,
 // 128-byte swizzle, out-of-range rows read as zero. box_rows = 1 is the map for row gathers (tile::gather4),

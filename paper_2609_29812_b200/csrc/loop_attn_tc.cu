@@ -55,8 +55,13 @@ constexpr int kMaxChunks = kMaxCols / kNC + 2;
 constexpr uint32_t kAccOld = 0, kAccNew = 128, kSOld = 256, kSNew = 320, kPOld = 384, kPNew = 448;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
+// A problem can be split over two CTAs, each taking half of the chunks: a CTA's partial result is both accumulators
+// (column-major, so that the row-owning threads write and read coalesced) and the three per-row statistics.
+constexpr int kPartFloats = 2 * kM * kDH + 3 * kM;
+constexpr int kMaxSplit = 256;              // counters at the head of the workspace
 constexpr float kRescaleThreshold = 60.f;   // in log2 units: rescale only when the reference falls this far behind
 static_assert(3 * kMaxCols * 4 <= kSlots * kSlotBytes, "prologue staging must fit in the ring");
+static_assert(kAccNew == kAccOld + kDH, "the two accumulators are adjacent in tensor memory");
 
 // Optional device-side timeline for tuning (compile with -DFL_TC_TRACE): the CTA (block 1, head 0) writes
 // clock64() stamps into the buffer passed as `status` (the traced CTA can be chosen with -DFL_TC_TRACE_X/_Y): trace[(role * 64 + chunk) * 4 + event].
@@ -67,7 +72,7 @@ static_assert(3 * kMaxCols * 4 <= kSlots * kSlotBytes, "prologue staging must fi
 #endif
 #define TC_TRACE(role, chunk, ev)                                                                      \
   do {                                                                                                 \
-    if (blockIdx.x == FL_TC_TRACE_X && blockIdx.y == FL_TC_TRACE_Y && (chunk) < 64 && a.status != nullptr) \
+    if (b == FL_TC_TRACE_X && h == FL_TC_TRACE_Y && part == 0 && (chunk) < 64 && a.status != nullptr) \
       reinterpret_cast<long long*>(a.status)[((role) * 64 + (chunk)) * 4 + (ev)] = clock64();          \
   } while (0)
 #else
@@ -89,6 +94,9 @@ struct alignas(64) TcArgs {
   DevSide k, v;
   int n_old;
   int use_rows;                      // columns active in this loop are gathered from the materialized rows
+  int n_full;                        // CTAs 0 .. n_full-1 take one problem each; the rest are pairs sharing one
+  int32_t* part_cnt;                 // [kMaxSplit] arrival counters of the pairs (zero between launches)
+  float* part_acc;                   // [pairs][2][kPartFloats] partial results
   const int32_t* col_idx;
   const int32_t* col_cnt;
   int c;
@@ -114,6 +122,8 @@ struct __align__(16) TcSmemCtl {
   int abort_flag;
   int q_lo, q_hi, i_last;    // block's slot range in active_idx, position of its last active row
   int n_plain, n_patch;      // columns without / with a payload in the current loop
+  int merge_role;            // split problems: 0 = this CTA finished first (the other one merges), 1 = it merges,
+                             // 2 = it should have merged but gave up waiting for the other's partial result
   int warp_cnt[kWarps][2];
   int chunk_last[kMaxChunks];       // largest column position of the chunk, INT32_MAX if the chunk is padded
   uint32_t chunk_mask[kMaxChunks];  // OR of the stream masks of the chunk's columns (0: plain gather only)
@@ -240,7 +250,14 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
   uint32_t* ord_mask = reinterpret_cast<uint32_t*>(ord_col + kMaxCols);  // bit s: payload in stream s
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int b = blockIdx.x, h = blockIdx.y;
+  // problem (query block b, head h) of this CTA, and for the pairs at the end of the grid which half of it
+  int item = blockIdx.x, part = 0, pair = -1;
+  if (item >= a.n_full) {
+    pair = (item - a.n_full) >> 1;
+    part = (item - a.n_full) & 1;
+    item = a.n_full + pair;
+  }
+  const int b = item % a.nb, h = item / a.nb;
   const size_t prob = (size_t)h * a.nb + b;
   const int32_t* cols = a.col_idx + prob * a.c;
   const int cnt = min(__ldg(a.col_cnt + prob), kMaxCols);
@@ -382,6 +399,12 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
   }
   const int n_plain = ctl.n_plain, n_patch = ctl.n_patch;
   const int n_chunks = (n_plain + kNC - 1) / kNC + (n_patch + kNC - 1) / kNC;
+  // A pair splits its problem's chunks in the middle, unless the block has several row tiles or a single chunk: then
+  // the first CTA of the pair does everything and the second nothing (both see the same numbers).
+  const bool split = pair >= 0 && q_hi - q_lo <= kM && n_chunks >= 2;
+  const int c_mid = (n_chunks + 1) >> 1;
+  const int c_lo = (split && part == 1) ? c_mid : 0;
+  const int c_hi = (pair >= 0 && part == 1 && !split) ? 0 : ((split && part == 0) ? c_mid : n_chunks);
   // per chunk: the OR of its columns' stream masks and its last column (a warp per chunk, two columns per lane)
   for (int ci = warp; ci < n_chunks; ci += kWarps) {
     const ChunkInfo ck = chunk_info(ci, n_plain, n_patch);
@@ -402,7 +425,7 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
   int fill = 0; // ring slots filled so far: slot = fill % kSlots, phase = (fill / kSlots) & 1
   uint32_t dirty_par_cta = 0;  // per-slot phase parity of the patched[] barriers (they only see dirty chunks)
 
-  for (int s0 = q_lo, tile = 0; s0 < q_hi; s0 += kM, ++tile) {
+  for (int s0 = q_lo, tile = 0; s0 < q_hi && !(pair >= 0 && part == 1 && !split); s0 += kM, ++tile) {
   const int n_rows = min(kM, q_hi - s0);
   const int g0 = g, fill0 = fill;
   const uint32_t dirty_par0 = dirty_par_cta;
@@ -451,7 +474,7 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
     int f = fill0;
     bool ok = true;
 #pragma unroll 1
-    for (int ci = 0; ci < n_chunks && ok; ++ci) {
+    for (int ci = c_lo; ci < c_hi && ok; ++ci) {
       const ChunkInfo ck = chunk_info(ci, n_plain, n_patch);
       const int n_slots = ck.patch ? 2 : 1;
       const bool dirty = ctl.chunk_mask[ci] != 0;
@@ -509,7 +532,7 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
       }
       f += n_slots;
     }
-    if (INDEXED && a.q_store != nullptr && ok) {
+    if (INDEXED && a.q_store != nullptr && ok && !split) {
       // The Q store rows of this (row tile, head) were read by the gathers that completed q_full and belong to
       // no other CTA: the new rows take their place for the next loop.
       ok = warp_wait(&ctl.q_full, tile & 1, abort_flag);
@@ -539,12 +562,12 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
       int f = fill0;
       uint32_t dirty_par = dirty_par0;
 #pragma unroll 1
-      for (int ci = 0; ci < n_chunks; ++ci) {
+      for (int ci = c_lo; ci < c_hi; ++ci) {
         const ChunkInfo ck = chunk_info(ci, n_plain, n_patch);
         const int slot0 = f % kSlots, slot1 = (f + 1) % kSlots;
-        const int gc = g0 + ci;
+        const int gc = g0 + ci - c_lo;
         if (t == 0) TC_TRACE(1, ci, 0);
-        if (ci == 0 && !tc::mbar_wait(&ctl.q_full, tile & 1, abort_flag)) break;
+        if (ci == c_lo && !tc::mbar_wait(&ctl.q_full, tile & 1, abort_flag)) break;
         // a term reads one slot of the chunk only (the new term of a two-slot chunk the second): it starts on it
         // without waiting for the other
         const int my_slot = (t && ck.patch) ? slot1 : slot0, my_fill = (t && ck.patch) ? f + 1 : f;
@@ -578,9 +601,9 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
       const uint32_t p_base = tmem + (t ? kPNew : kPOld);
       int f = fill0;
 #pragma unroll 1
-      for (int cj = 0; cj < n_chunks; ++cj) {
+      for (int cj = c_lo; cj < c_hi; ++cj) {
         const ChunkInfo ck = chunk_info(cj, n_plain, n_patch);
-        const int gc = g0 + cj, pb = gc & 1;
+        const int gc = g0 + cj - c_lo, pb = gc & 1;
         if (t == 0) TC_TRACE(4, cj, 0);
         if (!tc::mbar_wait(&ctl.p_full[t][pb], (gc >> 1) & 1, abort_flag)) break;
         tc::tc_fence_after();
@@ -588,7 +611,7 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
         const int slot0 = f % kSlots, slot1 = (f + 1) % kSlots;
         const uint32_t v_lo = v_lo0 + ((t && ck.patch) ? slot1 : slot0) * (kSlotBytes >> 4);
         const uint32_t p_src = p_base + pb * 32;
-        const uint32_t acc0 = cj > 0 ? 1u : 0u;          // first chunk of the tile overwrites the accumulator
+        const uint32_t acc0 = cj > c_lo ? 1u : 0u;       // the CTA's first chunk of the tile overwrites the accumulator
 #pragma unroll
         for (int kk = 0; kk < kNC / 16; ++kk)
           tc::mma_ts_lo(acc, p_src + kk * 8, v_lo + kk * (2048 >> 4), v_hi, idesc_pv, kk > 0 ? 1u : acc0);
@@ -619,8 +642,8 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
     float mass = 0.f, ell = 0.f, ref = -INFINITY;
     bool ok = true;
     bool pending = false;   // the previous chunk's P is stored but not yet announced (warp-uniform)
-    for (int ci = 0; ci < n_chunks; ++ci) {
-      const int gc = g0 + ci, pb = gc & 1, n_use = gc >> 1;
+    for (int ci = c_lo; ci < c_hi; ++ci) {
+      const int gc = g0 + ci - c_lo, pb = gc & 1, n_use = gc >> 1;
       if (gt == 0) TC_TRACE(2 + grp, ci, 0);
       if (!warp_wait(&ctl.s_full[grp], gc & 1, abort_flag)) { ok = false; break; }
       tc::tc_fence_after();
@@ -686,7 +709,7 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
             if (over) { factor = tc::ex2(ref - cm); ref = cm; }
             // every earlier PV must have completed before the accumulator rows are rewritten (ci >= 1 here: the
             // reference was set in an earlier chunk, or in this chunk's first half, whose P is not announced yet)
-            if (ci >= 1) {
+            if (ci > c_lo) {
               if (!warp_wait(&ctl.p_free[1][(gc - 1) & 1], ((gc - 1) >> 1) & 1, abort_flag)) { ok = false; break; }
               tc::tc_fence_after();
 #pragma unroll 1
@@ -731,7 +754,7 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
       }
       if (!ok) break;
       pending = true;
-      if (ci < kSlots / 2) {
+      if (ci - c_lo < kSlots / 2) {
         // while the pipeline fills (the first chunks hold the whole ring) latency counts: announce P at once, so
         // that its PV retires and the ring slots are handed to the gathers as early as possible
         tc::tmem_wait_st();
@@ -746,7 +769,7 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
       tc::tmem_wait_st();
       tc::tc_fence_before();
       __syncwarp();
-      if (lane == 0) tc::mbar_arrive(&ctl.p_full[grp][(g0 + n_chunks - 1) & 1]);
+      if (lane == 0) tc::mbar_arrive(&ctl.p_full[grp][(g0 + (c_hi - c_lo) - 1) & 1]);
     }
     // ---- epilogue ------------------------------------------------------------------------------------
     // Each group finishes 64 of the 128 head-dim columns. Its half of the O_prev tile is staged in the group's
@@ -771,37 +794,114 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
     tc::cp_async_wait<0>();
     asm volatile("bar.sync 1, 256;" ::: "memory");
     if (gt == 0) TC_TRACE(2 + grp, 61, 1);
-    const float m_i = ctl.mass[row], l_i = ctl.ell[row], ref_i = ctl.ref[row];
-    const bool acc_valid = ok && n_chunks > 0;            // warp-uniform: the tensor-memory reads below are collective
-    const bool has = acc_valid && ref_i > -INFINITY;      // per row: T_i is not empty
-    const float w = has ? m_i / l_i : 0.f;
+    float m_i = ctl.mass[row], l_i = ctl.ell[row], ref_i = ctl.ref[row];
+    const bool acc_valid = ok && c_hi > c_lo;             // warp-uniform: the tensor-memory reads below are collective
+    // ---- split problems: the CTA of the pair that finishes first leaves its partial result in the workspace, the
+    // other one adds it to its own (nobody waits for anybody: whoever finds the counter at 1 merges)
+    const float* other = nullptr;
+    float f_mine = 1.f, f_other = 0.f;
+    if (split) {
+      // counter of the pair: each CTA adds 1 when its accumulation is complete (the one that finds 0 is first), the
+      // first one adds 16 once its partial result is in the workspace; the second resets it for the next launch
+      if (tid == 0) ctl.merge_role = atomicAdd(a.part_cnt + pair, 1) & 1;
+      asm volatile("bar.sync 1, 256;" ::: "memory");
+      if (gt == 0) TC_TRACE(2 + grp, 62, 0);
+      if (ctl.merge_role == 0) {
+        float* mine = a.part_acc + ((size_t)pair * 2 + part) * kPartFloats;
 #pragma unroll 1
-    for (int hh = 0; hh < 4; ++hh) {
-      uint32_t ao[16], an[16];
-      if (acc_valid) {
-        tc::tmem_ld16(tmem + lane_base + kAccOld + grp * 64 + hh * 16, ao);
-        tc::tmem_ld16(tmem + lane_base + kAccNew + grp * 64 + hh * 16, an);
-        tc::tmem_wait_ld();
-      }
-      if (has) {
+        for (int c16 = 0; c16 < 8; ++c16) {   // acc_old columns 0-63 of the group's half, then acc_new: 16 at a time
+          uint32_t v[16];
+          const int col = (c16 >> 2) * kDH + grp * 64 + (c16 & 3) * 16;   // column of the [old | new] accumulator pair
+          if (acc_valid) {
+            tc::tmem_ld16(tmem + lane_base + kAccOld + col, v);           // kAccNew == kAccOld + kDH
+            tc::tmem_wait_ld();
+          }
 #pragma unroll
-        for (int v8 = 0; v8 < 2; ++v8) {
-          uint4* cell = reinterpret_cast<uint4*>(stage + row * 128 + (((hh * 2 + v8) ^ (row & 7)) << 4));
-          float pv[8], out[8];
-          unpack8(*cell, pv);
-#pragma unroll
-          for (int i = 0; i < 8; ++i)
-            out[i] = pv[i] - __uint_as_float(ao[v8 * 8 + i]) + w * __uint_as_float(an[v8 * 8 + i]);
-          *cell = pack8(out);
+          for (int i = 0; i < 16; ++i) mine[(col + i) * kM + row] = acc_valid ? __uint_as_float(v[i]) : 0.f;
+        }
+        if (grp == 0) mine[2 * kM * kDH + row] = acc_valid ? m_i : 0.f;
+        else {
+          mine[2 * kM * kDH + kM + row] = acc_valid ? l_i : 0.f;
+          mine[2 * kM * kDH + 2 * kM + row] = acc_valid ? ref_i : -INFINITY;
+        }
+        __threadfence();
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        if (tid == 0) atomicAdd(a.part_cnt + pair, 16);
+        if (gt == 0) TC_TRACE(2 + grp, 62, 1);
+      } else {
+        // the other CTA came first and is writing its partial result (it is resident and past its main loop: the
+        // wait is short, and bounded like every other)
+        if (tid == 0) {
+          int seen = atomicAdd(a.part_cnt + pair, 0);
+          for (int it = 0; seen < 16 && it < (1 << 16); ++it) {
+            __nanosleep(100);
+            seen = atomicAdd(a.part_cnt + pair, 0);
+          }
+          if (seen < 16) { *abort_flag = 1; ctl.merge_role = 2; }   // gave up: no output, FL_ERR_TIMEOUT
+          else a.part_cnt[pair] = 0;                                // ready for the next launch
+        }
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        if (gt == 0) TC_TRACE(2 + grp, 62, 1);
+        if (ctl.merge_role == 1) {   // CTA-uniform
+          __threadfence();
+          const float* theirs = a.part_acc + ((size_t)pair * 2 + (part ^ 1)) * kPartFloats;
+          // the other CTA's accumulators (128 KB) come into the idle ring in one round of asynchronous copies
+          static_assert(2 * kM * kDH * sizeof(float) <= (size_t)kSlots * kSlotBytes, "a partial result fits in the ring");
+#pragma unroll 1
+          for (int i = tid; i < 2 * kM * kDH / 4; i += 256) tc::cp_async16(ring + i * 16, theirs + i * 4);
+          tc::cp_async_commit();
+          other = reinterpret_cast<const float*>(ring);
+          const float m_o = __ldcg(theirs + 2 * kM * kDH + row), l_o = __ldcg(theirs + 2 * kM * kDH + kM + row);
+          const float ref_o = __ldcg(theirs + 2 * kM * kDH + 2 * kM + row);
+          const float ref_t = fmaxf(ref_i, ref_o);
+          f_mine = ref_i > -INFINITY ? tc::ex2(ref_i - ref_t) : 0.f;
+          f_other = ref_o > -INFINITY ? tc::ex2(ref_o - ref_t) : 0.f;
+          // products and sums rounded one by one (no fused multiply-add): the result must not depend on which of
+          // the two CTAs does the merging
+          m_i = __fadd_rn(m_i, m_o);
+          l_i = __fadd_rn(__fmul_rn(l_i, f_mine), __fmul_rn(l_o, f_other));
+          ref_i = ref_t;
+          tc::cp_async_wait<0>();
+          asm volatile("bar.sync 1, 256;" ::: "memory");
+          if (gt == 0) TC_TRACE(2 + grp, 62, 2);
         }
       }
     }
-    if (grp == 1 && row_ok)
+    const bool writer = !split || other != nullptr;       // CTA-uniform: this CTA produces the output rows
+    const bool has = acc_valid && ref_i > -INFINITY;      // per row: T_i is not empty
+    const float w = has ? m_i / l_i : 0.f;
+#pragma unroll 1
+    for (int c8 = 0; c8 < 8 && writer; ++c8) {   // 8 head-dim columns = one 16-byte cell of the staged row at a time
+      uint32_t ao[8], an[8];
+      const int col = grp * 64 + c8 * 8;
+      if (acc_valid) {
+        tc::tmem_ld8(tmem + lane_base + kAccOld + col, ao);
+        tc::tmem_ld8(tmem + lane_base + kAccNew + col, an);
+        tc::tmem_wait_ld();
+      }
+      if (other != nullptr) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          ao[i] = __float_as_uint(__fadd_rn(__uint_as_float(ao[i]), other[(col + i) * kM + row]));
+          an[i] = __float_as_uint(__fadd_rn(__fmul_rn(__uint_as_float(an[i]), f_mine),
+                                            __fmul_rn(other[(kDH + col + i) * kM + row], f_other)));
+        }
+      }
+      if (has) {
+        uint4* cell = reinterpret_cast<uint4*>(stage + row * 128 + ((c8 ^ (row & 7)) << 4));
+        float pv[8];
+        unpack8(*cell, pv);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) pv[i] = pv[i] - __uint_as_float(ao[i]) + w * __uint_as_float(an[i]);
+        *cell = pack8(pv);
+      }
+    }
+    if (grp == 1 && row_ok && writer)
       a.lse_out[(size_t)h * a.L + pos] = has ? (ref_i + log2f(l_i)) * kLn2 - logf(m_i) : lse2 * kLn2;
     asm volatile("bar.sync 1, 256;" ::: "memory");
     if (gt == 0) TC_TRACE(2 + grp, 61, 2);
 #pragma unroll 1
-    for (int k = 0; k < 8; ++k) {
+    for (int k = 0; k < 8 && writer; ++k) {
       const int idx = k * 128 + gt, rr = idx >> 3, cc = idx & 7;
       if (rr < n_rows) {
         const size_t dst_row = INDEXED ? (size_t)__ldg(a.active_idx + s0 + rr) : (size_t)(s0 + rr);
@@ -811,11 +911,25 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
     }
     if (gt == 0) TC_TRACE(2 + grp, 61, 3);
   }
+  if (INDEXED && split && a.q_store != nullptr) {   // CTA-uniform
+    // Both halves of a split problem gathered the previous loop's Q rows from the store; the new rows may take their
+    // place only when both are done with them, which the merging CTA knows
+    __syncthreads();
+    if (ctl.merge_role == 1 && !ctl.abort_flag) {
+#pragma unroll 1
+      for (int it = tid; it < n_rows * 16; it += kThreads) {
+        const int r = it >> 4, ch = it & 15;
+        const int pos_r = __ldg(a.active_idx + s0 + r);
+        *reinterpret_cast<uint4*>(a.q_store + (size_t)pos_r * a.d + h * kDH + ch * 8) =
+            __ldg(reinterpret_cast<const uint4*>(a.q_new + (size_t)(s0 + r) * a.d + h * kDH + ch * 8));
+      }
+    }
+  }
   // every role is done with this tile: accumulators, Q tiles and the ring bookkeeping move on together
   if (s0 + kM < q_hi) {   // CTA-uniform: another row tile of the block follows
-    g += n_chunks;
+    g += c_hi - c_lo;
     int f = fill;
-    for (int ci = 0; ci < n_chunks; ++ci) {   // replay the tile's fills (same for every role)
+    for (int ci = c_lo; ci < c_hi; ++ci) {   // replay the tile's fills (same for every role)
       const ChunkInfo ck = chunk_info(ci, n_plain, n_patch);
       const int n_slots = ck.patch ? 2 : 1;
       if (ctl.chunk_mask[ci] != 0)
@@ -849,6 +963,37 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
 }
 
 }  // namespace
+
+size_t fl_attn_workspace_bytes(const fl_ctx* ctx, const fl_shape* s) {
+  if (s->dtype != FL_BF16 || s->head_dim != kDH) return 0;
+  const int n_items = fl_n_blocks(s) * s->n_heads;
+  const int rem = n_items % ctx->sm_count;
+  if (rem == 0 || 2 * rem > ctx->sm_count || rem > kMaxSplit) return 0;
+  return (size_t)kMaxSplit * sizeof(int32_t) + (size_t)rem * 2 * kPartFloats * sizeof(float);
+}
+
+extern "C" int fl_loop_attention_workspace_bytes(fl_ctx* ctx, const fl_shape* shape, int64_t* bytes) {
+  FL_REQUIRE(ctx != nullptr && bytes != nullptr);
+  const int rc = fl_check_shape(shape);
+  if (rc != FL_OK) return rc;
+  *bytes = (int64_t)fl_attn_workspace_bytes(ctx, shape);
+  return FL_OK;
+}
+
+extern "C" int fl_set_workspace(fl_ctx* ctx, void* workspace, int64_t bytes, void* stream) {
+  FL_REQUIRE(ctx != nullptr && bytes >= 0);
+  if (workspace == nullptr || bytes < (int64_t)(kMaxSplit * sizeof(int32_t))) {
+    ctx->ws = nullptr;
+    ctx->ws_bytes = 0;
+    return workspace == nullptr ? FL_OK : FL_ERR_WORKSPACE;
+  }
+  FL_REQUIRE((reinterpret_cast<uintptr_t>(workspace) & 255u) == 0);
+  // the arrival counters at its head start at zero (every launch leaves them there)
+  FL_CHECK_CUDA(cudaMemsetAsync(workspace, 0, kMaxSplit * sizeof(int32_t), static_cast<cudaStream_t>(stream)));
+  ctx->ws = workspace;
+  ctx->ws_bytes = (size_t)bytes;
+  return FL_OK;
+}
 
 // Returns FL_ERR_UNSUPPORTED when the tensor path does not cover the request (caller falls back to the
 // SIMT kernel, which is also CUDA). indexed != 0: q_old, o_prev and o_out are position-indexed stores [L, d] and
@@ -890,7 +1035,18 @@ int fl_launch_loop_attn_tc(fl_ctx* ctx, const fl_shape* s, int loop_r, const voi
   a.lse_prev = lse_prev; a.lse_out = lse_out; a.status = status;
   a.L = s->L; a.H = s->n_heads; a.q_block = s->q_block; a.nb = fl_n_blocks(s);
   a.d = s->n_heads * s->head_dim; a.group = s->group; a.scale = s->sm_scale;
-  const dim3 grid(a.nb, s->n_heads);   // one CTA per (query block, head); it walks the block's 128-row tiles
+  // One CTA per (query block, head) problem; it walks the block's 128-row tiles. The problems are alike, so a grid
+  // that is not a multiple of the SM count ends in a partly empty wave: when at most half of the SMs would be busy in
+  // it and the caller has lent a workspace, each problem of that wave goes to a pair of CTAs (half of the chunks each).
+  const int n_items = a.nb * s->n_heads;
+  const int rem = n_items % ctx->sm_count;
+  const size_t ws_need = (size_t)kMaxSplit * sizeof(int32_t) + (size_t)rem * 2 * kPartFloats * sizeof(float);
+  const bool pairs = ctx->ws != nullptr && rem > 0 && 2 * rem <= ctx->sm_count &&
+                     rem <= kMaxSplit && ctx->ws_bytes >= ws_need;
+  a.n_full = pairs ? n_items - rem : n_items;
+  a.part_cnt = static_cast<int32_t*>(ctx->ws);
+  a.part_acc = reinterpret_cast<float*>(static_cast<uint8_t*>(ctx->ws) + kMaxSplit * sizeof(int32_t));
+  const dim3 grid(a.n_full + 2 * (n_items - a.n_full));
 #define FL_TC2(BITS, IDX)                                                                                        \
   do {                                                                                                           \
     auto kern = loop_attn_tc_kernel<BITS, IDX>;                                                                  \

@@ -68,17 +68,36 @@ def rows_workspace(dev, n: int, d: int):
     return ws
 
 
+def lend_workspace(ctx, shape, dev) -> int:
+    """Hands the context the workspace with which the attention launch splits the problems of its last, partly empty
+    wave over two CTAs each (a scheduling aid; 0 bytes when the shape cannot profit).  The tensor stays referenced
+    by the Context object.  Returns the bytes lent."""
+    need = B.fl_loop_attention_workspace_bytes(ctx, shape)
+    have = getattr(ctx, "_workspace", None)
+    if need > 0 and (have is None or have.numel() < need):
+        ws = torch.empty(need, dtype=torch.uint8, device=dev)
+        B.fl_set_workspace(ctx, ws, need)
+        ctx._workspace = ws
+    return need
+
+
 class LayerState:
     """Buffers of one layer and the calls that advance it by one loop."""
 
     def __init__(self, ctx, w: Workload, device="cuda:0", bits: Optional[int] = None, q_block: Optional[int] = None,
-                 c: Optional[int] = None):
+                 c: Optional[int] = None, split: bool = True):
         self.ctx, self.w, self.dev = ctx, w, torch.device(device)
         self.shape = shape_of(w, bits, q_block)
         self.bits = self.shape.bits
         self.c = c or w.col_budget
         self.nb = (w.L + self.shape.q_block - 1) // self.shape.q_block
         self.dt = torch_dtype(w)
+        if self.dt == torch.bfloat16:
+            if split:
+                lend_workspace(ctx, self.shape, self.dev)
+            else:   # the context's attention launches go back to one CTA per problem
+                B.fl_set_workspace(ctx, None, 0)
+                ctx._workspace = None
         self.k_streams: List[dict] = []
         self.v_streams: List[dict] = []
         self.col_idx = None

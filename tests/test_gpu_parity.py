@@ -217,18 +217,21 @@ def sets_to_arrays(w, nb, col_sets, c):
     return idx, cnt
 
 
-ROWS = pytest.mark.parametrize("rows", [True, False], ids=["materialized_rows", "rebuilt_in_kernel"])
+# rows: the columns active in the loop come from the rows the quantization kernel materialized, or are rebuilt inside
+# the attention kernel; split: the problems of the launch's last wave (here: all of them) go to two CTAs each
+ROWS = pytest.mark.parametrize("rows,split", [(True, True), (True, False), (False, True)],
+                               ids=["materialized_rows+split", "materialized_rows", "rebuilt_in_kernel+split"])
 
 
 @ROWS
-def test_loop_attention_stage_isolated(env, case, rows):
+def test_loop_attention_stage_isolated(env, case, rows, split):
     """Each loop's attention is fed the oracle's upstream state (token set, column sets, previous
     outputs and log-normalisers rounded to storage precision; the store is bit-exact anyway).  rows: the columns
     active in the loop come from the rows the quantization kernel materialized, or (without that workspace) are
     rebuilt from the residual streams inside the attention kernel."""
     B, P, ctx = env
     w, x, ref = case
-    st = P.LayerState(ctx, w)
+    st = P.LayerState(ctx, w, split=split)
     st.k_base, st.v_base = to_dev(x.K[0], w), to_dev(x.V[0], w)
     lse = ref["dense"]["lse"].astype(np.float32).copy()
     q_prev_full = x.Q[0]
@@ -362,7 +365,7 @@ def test_binary32_simt_attention_path_on_bf16_storage(env):
 
 
 @ROWS
-def test_many_patched_columns_and_wide_budgets(env, rows):
+def test_many_patched_columns_and_wide_budgets(env, rows, split):
     """Half of the rows active and a column budget of several chunks: long runs of columns that carry
     residual payloads (two ring slots per chunk) and several 128-row tiles per query block."""
     B, P, ctx = env
@@ -371,7 +374,7 @@ def test_many_patched_columns_and_wide_budgets(env, rows):
     x = workloads.make_layer_inputs(w, seed=7)
     ref = fo.LayerOracle(w.L, w.n_heads, w.head_dim, w.q_block, w.bits, w.group, w.eps, w.sm_scale,
                          storage=w.dtype).run(x.G, x.Q, x.K, x.V, [w.k_tokens] * 2, [w.col_budget] * 2)
-    st = P.LayerState(ctx, w)
+    st = P.LayerState(ctx, w, split=split)
     st.dense_loop(to_dev(x.Q[0], w), to_dev(x.K[0], w), to_dev(x.V[0], w))
     lse = ref["dense"]["lse"].astype(np.float32).copy()
     q_prev_full = x.Q[0]

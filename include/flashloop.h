@@ -217,6 +217,21 @@ FL_API int fl_loop_attention_indexed(fl_ctx* ctx, const fl_shape* shape, int loo
                               const float* lse_in, float* lse_out, const void* o_store_in, void* o_store_out,
                               float* col_scores_next, int32_t* status, void* stream);
 
+/* fl_loop_attention_indexed with the workspace of its last-wave split (see fl_set_workspace) taken from a fixed array
+ * that is part of the library's device image, for callers that cannot lend device memory; the context's own workspace,
+ * if any, is ignored by this call. The paper has no counterpart. The call allocates and frees nothing: the array's
+ * address is looked up once per device, and the arrival counters at its head are cleared on `stream` before the launch.
+ * The array holds the partial results of at most 74 split problems (half of a B200's SMs); a shape whose split needs
+ * more returns FL_ERR_WORKSPACE before anything is launched. There is one array per device: two of these calls that
+ * may overlap in time (different streams or contexts on one device) race on it and must be serialised by the caller.
+ * Arguments, results and other errors as fl_loop_attention_indexed. */
+FL_API int fl_loop_attention_indexed_static(fl_ctx* ctx, const fl_shape* shape, int loop_r, const void* q_new,
+                                     const void* q_store_in, void* q_store_out, const int32_t* active_idx,
+                                     int32_t n_active, const fl_kv_store* store, const int32_t* col_idx,
+                                     const int32_t* col_cnt, int32_t c, const float* lse_in, float* lse_out,
+                                     const void* o_store_in, void* o_store_out, float* col_scores_next,
+                                     int32_t* status, void* stream);
+
 /* KV-cache accounting (Section 1's 48 GiB example; Section 4.3): bytes held for one layer by this store
  * after n_loops loops, and by a dense looped cache of n_loops loops. Host-only, no device access.
  * share_layers = number of layers sharing each loop's slot map and index list (>= 1). */

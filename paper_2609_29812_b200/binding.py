@@ -69,6 +69,8 @@ def _load() -> C.CDLL:
                               p, p, p, p, p, p, p],
         "fl_loop_attention_indexed": [p, C.POINTER(FlShape), C.c_int, p, p, p, p, i32, C.POINTER(FlKvStore), p, p,
                                       i32, p, p, p, p, p, p, p],
+        "fl_loop_attention_indexed_static": [p, C.POINTER(FlShape), C.c_int, p, p, p, p, i32, C.POINTER(FlKvStore),
+                                             p, p, i32, p, p, p, p, p, p, p],
         "fl_kv_store_bytes": [C.POINTER(FlShape), C.POINTER(FlKvStore), C.c_int, C.c_int,
                               C.POINTER(i64), C.POINTER(i64)],
         "fl_loop_attention_workspace_bytes": [p, C.POINTER(FlShape), C.POINTER(i64)],
@@ -239,6 +241,17 @@ def fl_loop_attention_indexed(ctx, shape, loop_r, q_new, q_store_in, q_store_out
                                        int(c), _ptr(lse_in), _ptr(lse_out), _ptr(o_store_in), _ptr(o_store_out),
                                        _ptr(col_scores_next), _ptr(status), _stream(stream))
     return _check("fl_loop_attention_indexed", rc, check)
+
+
+def fl_loop_attention_indexed_static(ctx, shape, loop_r, q_new, q_store_in, q_store_out, active_idx, n_active, store,
+                                     col_idx, col_cnt, c, lse_in, lse_out, o_store_in, o_store_out,
+                                     col_scores_next=None, status=None, stream=None, check=True) -> int:
+    rc = lib.fl_loop_attention_indexed_static(_h(ctx), C.byref(shape), int(loop_r), _ptr(q_new), _ptr(q_store_in),
+                                              _ptr(q_store_out), _ptr(active_idx), int(n_active),
+                                              C.byref(store) if store is not None else None, _ptr(col_idx),
+                                              _ptr(col_cnt), int(c), _ptr(lse_in), _ptr(lse_out), _ptr(o_store_in),
+                                              _ptr(o_store_out), _ptr(col_scores_next), _ptr(status), _stream(stream))
+    return _check("fl_loop_attention_indexed_static", rc, check)
 
 
 def fl_kv_store_bytes(shape, store, n_loops, share_layers=1, check=True):

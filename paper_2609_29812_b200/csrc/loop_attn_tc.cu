@@ -57,8 +57,9 @@ constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 // A problem can be split over two CTAs, each taking half of the chunks: a CTA's partial result is both accumulators
 // (column-major, so that the row-owning threads write and read coalesced) and the three per-row statistics.
-constexpr int kPartFloats = 2 * kM * kDH + 3 * kM;
-constexpr int kMaxSplit = 256;              // counters at the head of the workspace
+constexpr int kPartFloats = kFlPartFloats;
+constexpr int kMaxSplit = kFlMaxSplit;      // counters at the head of the workspace
+static_assert(kPartFloats == 2 * kM * kDH + 3 * kM, "partial result: two accumulators and three statistics per row");
 constexpr float kRescaleThreshold = 60.f;   // in log2 units: rescale only when the reference falls this far behind
 static_assert(3 * kMaxCols * 4 <= kSlots * kSlotBytes, "prologue staging must fit in the ring");
 static_assert(kAccNew == kAccOld + kDH, "the two accumulators are adjacent in tensor memory");

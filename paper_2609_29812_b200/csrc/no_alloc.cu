@@ -1,0 +1,48 @@
+// fl_loop_attention_indexed_static: the position-indexed loop attention with the workspace of its last-wave split
+// taken from a fixed array in device memory instead of a buffer of the caller. Nothing here corresponds to anything in
+// the paper: it is a convenience for callers that cannot hand over device memory.
+#include "fl_internal.cuh"
+
+namespace {
+
+constexpr int kStaticPairs = 74;   // problems of a last wave that can be split: half of the 148 SMs of a B200
+constexpr size_t kStaticBytes =
+    (size_t)kFlMaxSplit * sizeof(int32_t) + (size_t)kStaticPairs * 2 * kFlPartFloats * sizeof(float);
+
+// The scratch itself: part of the library's device image (no allocation call ever made for it), one per device.
+static __device__ __align__(256) unsigned char g_attn_scratch[kStaticBytes];
+
+constexpr int kMaxDevices = 64;
+void* g_scratch_addr[kMaxDevices];   // device address of g_attn_scratch, looked up once per device
+
+}  // namespace
+
+extern "C" int fl_loop_attention_indexed_static(fl_ctx* ctx, const fl_shape* shape, int loop_r, const void* q_new,
+                                                const void* q_store_in, void* q_store_out, const int32_t* active_idx,
+                                                int32_t n_active, const fl_kv_store* store, const int32_t* col_idx,
+                                                const int32_t* col_cnt, int32_t c, const float* lse_in, float* lse_out,
+                                                const void* o_store_in, void* o_store_out, float* col_scores_next,
+                                                int32_t* status, void* stream) {
+  FL_REQUIRE(ctx != nullptr);
+  const int rc = fl_check_shape(shape);
+  if (rc != FL_OK) return rc;
+  FL_REQUIRE(ctx->device >= 0 && ctx->device < kMaxDevices);
+  // the split this shape would use must fit the fixed array: no silent fall-back to something else
+  const size_t need = fl_attn_workspace_bytes(ctx, shape);
+  if (need > kStaticBytes) return FL_ERR_WORKSPACE;
+  if (g_scratch_addr[ctx->device] == nullptr) {
+    void* addr = nullptr;
+    FL_CHECK_CUDA(cudaGetSymbolAddress(&addr, g_attn_scratch));
+    g_scratch_addr[ctx->device] = addr;
+  }
+  void* scratch = g_scratch_addr[ctx->device];
+  // the arrival counters at the head of the scratch must be zero when the kernel starts
+  FL_CHECK_CUDA(cudaMemsetAsync(scratch, 0, (size_t)kFlMaxSplit * sizeof(int32_t), static_cast<cudaStream_t>(stream)));
+  // a context that differs from the caller's only in its workspace (it shares the tensor-map cache and owns nothing)
+  fl_ctx with_scratch = *ctx;
+  with_scratch.ws = scratch;
+  with_scratch.ws_bytes = kStaticBytes;
+  return fl_loop_attention_indexed(&with_scratch, shape, loop_r, q_new, q_store_in, q_store_out, active_idx, n_active,
+                                   store, col_idx, col_cnt, c, lse_in, lse_out, o_store_in, o_store_out,
+                                   col_scores_next, status, stream);
+}

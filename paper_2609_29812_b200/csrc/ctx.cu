@@ -78,6 +78,10 @@ extern "C" int fl_create(fl_ctx** out, int device) {
   fl_ctx* c = new (std::nothrow) fl_ctx();
   if (c == nullptr) return FL_ERR_CUDA;
   c->device = device;
+  {
+    const char* no_pdl = std::getenv("FL_NO_PDL");
+    c->pdl = (no_pdl != nullptr && no_pdl[0] == '1') ? 0 : 1;
+  }
   if (cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess ||
       cudaDeviceGetAttribute(&c->max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device) != cudaSuccess) {
     delete c;

@@ -15,6 +15,7 @@ struct fl_ctx {
   int force_simt;  // environment FL_FORCE_SIMT=1 at fl_create: keep attention on the binary32 SIMT kernels
   void* encode_tiled;       // cuTensorMapEncodeTiled, resolved through cudaGetDriverEntryPoint (may be null)
   struct fl_tmap_cache* tmaps;  // tensor maps, keyed by (base pointer, rows, row elements, box rows)
+  int pdl;                  // launch the hot-path kernels with programmatic stream serialization (FL_NO_PDL=1: off)
   void* ws;                 // caller's workspace (fl_set_workspace), or null
   size_t ws_bytes;
 };
@@ -80,6 +81,32 @@ static inline void fl_dev_side(const fl_kv_store* st, bool is_k, DevSide* out) {
 }
 
 #ifdef __CUDACC__
+// ---- programmatic dependent launch ---------------------------------------------------------------------------
+// The kernels of the step are launched with programmatic stream serialization: the next kernel of the stream may be
+// scheduled, and run up to its fl_grid_wait(), while this one is still running. Rules every such kernel keeps:
+// fl_grid_wait() (= the previous kernel of the stream has completed and its writes are visible) comes before the
+// first access to anything an earlier kernel may still read or write, and fl_grid_release() (the next kernel may be
+// scheduled) comes after it, so that whatever runs ahead of a wait sees everything up to two kernels back.
+// Launched without the attribute both are no-ops.
+__device__ __forceinline__ void fl_grid_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void fl_grid_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t fl_launch(const fl_ctx* ctx, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                             cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = (ctx != nullptr && ctx->pdl) ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // ---- 8-element vector access in storage type ---------------------------------------------------
 template <typename T>
 __device__ __forceinline__ void load8(const T* p, float (&v)[8]);

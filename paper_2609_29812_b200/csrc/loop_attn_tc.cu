@@ -250,6 +250,8 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
   int32_t* ord_col = reinterpret_cast<int32_t*>(&ctl + 1);               // [kMaxCols] column positions, partitioned
   uint32_t* ord_mask = reinterpret_cast<uint32_t*>(ord_col + kMaxCols);  // bit s: payload in stream s
 
+  fl_grid_wait();      // nothing below runs ahead of the previous kernel of the stream
+  fl_grid_release();
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   // problem (query block b, head h) of this CTA, and for the pairs at the end of the grid which half of it
   int item = blockIdx.x, part = 0, pair = -1;
@@ -1052,7 +1054,7 @@ int fl_launch_loop_attn_tc(fl_ctx* ctx, const fl_shape* s, int loop_r, const voi
   do {                                                                                                           \
     auto kern = loop_attn_tc_kernel<BITS, IDX>;                                                                  \
     FL_CHECK_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcSmemBytes));  \
-    kern<<<grid, kThreads, kTcSmemBytes, st>>>(a);                                                               \
+    FL_CHECK_CUDA(fl_launch(ctx, kern, grid, dim3(kThreads), kTcSmemBytes, st, a));                             \
   } while (0)
 #define FL_TC(BITS)                                   \
   do {                                                \

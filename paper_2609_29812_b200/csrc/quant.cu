@@ -20,6 +20,8 @@ struct QuantArgs {
 
 template <typename T, int BITS>
 __global__ void __launch_bounds__(256) quant_residual_kernel(const __grid_constant__ QuantArgs a) {
+  fl_grid_wait();
+  fl_grid_release();
   const int t = blockIdx.x;                 // active row
   const bool is_v = blockIdx.y != 0;
   const DevSide& side = is_v ? a.v : a.k;
@@ -137,14 +139,14 @@ __global__ void __launch_bounds__(256) quant_residual_kernel(const __grid_consta
 }
 
 template <typename T>
-int launch_quant(const fl_shape* s, const QuantArgs& a, int n_active, cudaStream_t st) {
+int launch_quant(const fl_ctx* ctx, const fl_shape* s, const QuantArgs& a, int n_active, cudaStream_t st) {
   const int threads = a.d / 8 < 256 ? a.d / 8 : 256;
   dim3 grid(n_active, 2);
   switch (s->bits) {
-    case 2: quant_residual_kernel<T, 2><<<grid, threads, 0, st>>>(a); break;
-    case 4: quant_residual_kernel<T, 4><<<grid, threads, 0, st>>>(a); break;
-    case 8: quant_residual_kernel<T, 8><<<grid, threads, 0, st>>>(a); break;
-    default: quant_residual_kernel<T, 16><<<grid, threads, 0, st>>>(a); break;
+    case 2: FL_CHECK_CUDA(fl_launch(ctx, quant_residual_kernel<T, 2>, grid, dim3(threads), 0, st, a)); break;
+    case 4: FL_CHECK_CUDA(fl_launch(ctx, quant_residual_kernel<T, 4>, grid, dim3(threads), 0, st, a)); break;
+    case 8: FL_CHECK_CUDA(fl_launch(ctx, quant_residual_kernel<T, 8>, grid, dim3(threads), 0, st, a)); break;
+    default: FL_CHECK_CUDA(fl_launch(ctx, quant_residual_kernel<T, 16>, grid, dim3(threads), 0, st, a)); break;
   }
   return fl_launch_status();
 }
@@ -185,6 +187,6 @@ extern "C" int fl_quant_kv_residual(fl_ctx* ctx, const fl_shape* shape, int loop
   a.v_rows_prev = rows ? vs.rows_prev : nullptr; a.v_rows_cur = rows ? vs.rows_cur : nullptr;
   a.n_prev = loop_r - 2; a.d = d; a.group = shape->group;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  return shape->dtype == FL_F32 ? launch_quant<float>(shape, a, n_active, st)
-                                : launch_quant<__nv_bfloat16>(shape, a, n_active, st);
+  return shape->dtype == FL_F32 ? launch_quant<float>(ctx, shape, a, n_active, st)
+                                : launch_quant<__nv_bfloat16>(ctx, shape, a, n_active, st);
 }

@@ -10,6 +10,8 @@ namespace {
 template <bool GATHER>
 __global__ void __launch_bounds__(256) rows_copy_kernel(const uint4* __restrict__ src, const int32_t* __restrict__ idx,
                                                         int n, int vec_per_row, int pieces, uint4* __restrict__ dst) {
+  fl_grid_wait();
+  fl_grid_release();
   const int warps_per_block = blockDim.x >> 5;
   const int lane = threadIdx.x & 31;
   const int64_t n_work = (int64_t)n * pieces;
@@ -46,11 +48,11 @@ int rows_copy(bool gather, fl_ctx* ctx, const void* src, const int32_t* idx, int
   const int grid = (int)(grid64 > max_grid ? max_grid : grid64);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (gather)
-    rows_copy_kernel<true><<<grid, warps * 32, 0, st>>>(static_cast<const uint4*>(src), idx, n, vec_per_row, pieces,
-                                                        static_cast<uint4*>(dst));
+    FL_CHECK_CUDA(fl_launch(ctx, rows_copy_kernel<true>, dim3(grid), dim3(warps * 32), 0, st,
+                            static_cast<const uint4*>(src), idx, n, vec_per_row, pieces, static_cast<uint4*>(dst)));
   else
-    rows_copy_kernel<false><<<grid, warps * 32, 0, st>>>(static_cast<const uint4*>(src), idx, n, vec_per_row, pieces,
-                                                         static_cast<uint4*>(dst));
+    FL_CHECK_CUDA(fl_launch(ctx, rows_copy_kernel<false>, dim3(grid), dim3(warps * 32), 0, st,
+                            static_cast<const uint4*>(src), idx, n, vec_per_row, pieces, static_cast<uint4*>(dst)));
   return fl_launch_status();
 }
 

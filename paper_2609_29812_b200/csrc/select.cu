@@ -253,6 +253,8 @@ __global__ void __launch_bounds__(kSelThreads, 1) column_select_smem_kernel(cons
                                                                             int32_t* __restrict__ col_cnt) {
   extern __shared__ __align__(16) uint32_t keys[];   // [n rounded up to 4], padded with key 0 (below every real key)
   __shared__ SelectSmem2 sm;
+  fl_grid_wait();
+  fl_grid_release();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   // later blocks have more candidates (causal prefix): they are dispatched first, the short ones fill the tail
   const int h = blockIdx.x, b = gridDim.y - 1 - blockIdx.y;
@@ -569,8 +571,9 @@ extern "C" int fl_select_columns(fl_ctx* ctx, const fl_shape* shape, const float
     const int vec_ok = (fl_aligned16(col_scores) && n_cand % 4 == 0) ? 1 : 0;
     FL_CHECK_CUDA(cudaFuncSetAttribute(column_select_smem_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)key_bytes));
-    column_select_smem_kernel<<<grid, kSelThreads, key_bytes, static_cast<cudaStream_t>(stream)>>>(
-        col_scores, cand_cols, cand_cnt, n_cand, c, shape->L, shape->q_block, nb, vec_ok, col_idx, col_cnt);
+    FL_CHECK_CUDA(fl_launch(ctx, column_select_smem_kernel, grid, dim3(kSelThreads), key_bytes,
+                            static_cast<cudaStream_t>(stream), col_scores, cand_cols, cand_cnt, n_cand, c, shape->L,
+                            shape->q_block, nb, vec_ok, col_idx, col_cnt));
   } else {
     column_select_kernel<<<grid, kSelThreads, 0, static_cast<cudaStream_t>(stream)>>>(
         col_scores, cand_cols, cand_cnt, n_cand, c, shape->L, shape->q_block, nb, col_idx, col_cnt);

@@ -73,10 +73,11 @@ def lend_workspace(ctx, shape, dev) -> int:
     wave over two CTAs each (a scheduling aid; 0 bytes when the shape cannot profit).  The tensor stays referenced
     by the Context object.  Returns the bytes lent."""
     need = B.fl_loop_attention_workspace_bytes(ctx, shape)
-    have = getattr(ctx, "_workspace", None)
-    if need > 0 and (have is None or have.numel() < need):
-        ws = torch.empty(need, dtype=torch.uint8, device=dev)
-        B.fl_set_workspace(ctx, ws, need)
+    if need > 0:
+        ws = getattr(ctx, "_workspace", None)
+        if ws is None or ws.numel() < need:
+            ws = torch.empty(need, dtype=torch.uint8, device=dev)
+        B.fl_set_workspace(ctx, ws, ws.numel())
         ctx._workspace = ws
     return need
 

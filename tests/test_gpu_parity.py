@@ -339,6 +339,23 @@ def test_indexed_attention_matches_compact_path_and_oracle(env):
     assert rc == -2 and torch.equal(st32.o_store, o_before)
 
 
+def test_attention_workspace_calls(env):
+    """Size query and hand-over of the workspace that lets the attention launch split its last wave."""
+    import torch
+    B, P, ctx = env
+    sh = P.shape_of(small_bf16(L=1200))
+    need = B.fl_loop_attention_workspace_bytes(ctx, sh)
+    per_problem = 2 * 4 * (2 * 128 * 128 + 3 * 128)          # two partial results of binary32 values
+    assert need > 1024 and (need - 1024) % per_problem == 0  # counters, then a whole number of split problems
+    assert B.fl_loop_attention_workspace_bytes(ctx, P.shape_of(workloads.config1())) == 0   # f32: never split
+    buf = torch.empty(need + 512, dtype=torch.uint8, device="cuda")
+    assert B.fl_set_workspace(ctx, buf[1:], need, check=False) == B.FL_ERR_INVALID_ARG      # not 256-byte aligned
+    assert B.fl_set_workspace(ctx, buf, 512, check=False) == -3                             # too small to be of use
+    assert B.fl_set_workspace(ctx, buf, need, check=False) == 0
+    assert B.fl_set_workspace(ctx, None, 0, check=False) == 0                               # detached again
+    ctx._workspace = None
+
+
 def test_binary32_simt_attention_path_on_bf16_storage(env):
     """The SIMT attention kernels also serve bf16 storage (forced here; normally the tensor path runs)."""
     import os

@@ -18,6 +18,102 @@ struct QuantArgs {
   int d, group;
 };
 
+// Everything after the operands of 8 consecutive elements of active row t are in registers: xn = the new row,
+// xh = Xhat^(r-1) (base plus the earlier streams). Writes the codes, the group's scale and offset, and the
+// materialized rows when the caller wants them.
+template <typename T, int BITS>
+__device__ __forceinline__ void encode8(const QuantArgs& a, bool is_v, int t, int elem, int lanes_per_group,
+                                        float (&xn)[8], float (&xh)[8]) {
+  uint8_t* codes = is_v ? a.v_codes : a.k_codes;
+  __half* scale = is_v ? a.v_scale : a.k_scale;
+  __half* zero = is_v ? a.v_zero : a.k_zero;
+  T* rows_prev = static_cast<T*>(is_v ? a.v_rows_prev : a.k_rows_prev);   // null: not wanted
+  T* rows_cur = static_cast<T*>(is_v ? a.v_rows_cur : a.k_rows_cur);
+  if (rows_prev != nullptr) store8<T>(rows_prev + (size_t)t * a.d + elem, xh);
+  if (BITS == 16) {  // codec off: the stream keeps the row itself
+    store8<T>(reinterpret_cast<T*>(codes) + (size_t)t * a.d + elem, xn);
+    if (rows_cur != nullptr) store8<T>(rows_cur + (size_t)t * a.d + elem, xn);
+    return;
+  }
+  float dl[8];
+  float mn, mx;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) dl[i] = __fsub_rn(xn[i], xh[i]);
+  mn = mx = dl[0];
+#pragma unroll
+  for (int i = 1; i < 8; ++i) { mn = fminf(mn, dl[i]); mx = fmaxf(mx, dl[i]); }
+  // every lane of the warp is here: the host only launches row widths for which all threads of the
+  // block run the same number of iterations (d % 256 == 0, and d % 2048 == 0 beyond 2048)
+  for (int o = 1; o < lanes_per_group; o <<= 1) {
+    mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+  }
+  const __half zh = __float2half_rd(mn);
+  const float zf = __half2float(zh);
+  const float range = __fsub_rn(mx, zf);
+  const float qmax = (float)((1 << BITS) - 1);
+  const __half sh = range == 0.f ? __float2half_rn(0.f) : __float2half_ru(__fdiv_rn(range, qmax));
+  const float sf = __half2float(sh);
+  // Codes: round-half-even of the binary32 quotient (delta - zero) / scale. The quotient is first formed with
+  // one reciprocal per group; that estimate is within a few ulp of the correctly rounded quotient (<= 5e-5
+  // absolute for codes up to 255), so its rounding to an integer is the same unless it lies within 1e-4 of a
+  // half-integer. Only then (a few percent of the warps) the true divisions are redone.
+  float q[8];
+  bool ambiguous = false;
+  if (sf != 0.f) {
+    const float inv = __frcp_rn(sf);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const float est = __fmul_rn(__fsub_rn(dl[i], zf), inv);
+      q[i] = __fsub_rn(__fadd_rn(est, 12582912.f), 12582912.f);   // round-half-even for |est| < 2^22
+      ambiguous |= 0.5f - fabsf(est - q[i]) < 1e-4f;
+    }
+    if (__any_sync(__activemask(), ambiguous)) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) q[i] = rintf(__fdiv_rn(__fsub_rn(dl[i], zf), sf));
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) q[i] = 0.f;
+  }
+  if (rows_cur != nullptr) {
+    // the reconstruction every later reader of this stream forms: Xhat + (code * scale + zero), Eq. 8
+#pragma unroll
+    for (int i = 0; i < 8; ++i) xh[i] = __fadd_rn(xh[i], __fmaf_rn(q[i], sf, zf));
+    store8<T>(rows_cur + (size_t)t * a.d + elem, xh);
+  }
+  // The quotients are integers in [0, qmax] already: delta >= zero (the offset was rounded down) and
+  // (max - zero) / scale <= qmax (the scale was rounded up), so the oracle's clamp never acts. Four codes at a
+  // time are packed with exact binary32 arithmetic (sum of code * 2^(BITS*i) < 2^24 for BITS <= 4, two codes
+  // for 8 bits), and the integer is read from the low mantissa bits of (value + 2^23).
+  uint32_t packed_lo, packed_hi = 0;
+  if (BITS == 8) {
+    uint32_t w[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+      w[i] = __float_as_uint(__fadd_rn(__fmaf_rn(q[2 * i + 1], 256.f, q[2 * i]), 8388608.f)) & 0xFFFFu;
+    packed_lo = w[0] | (w[1] << 16);
+    packed_hi = w[2] | (w[3] << 16);
+  } else {
+    const float r1 = (float)(1 << BITS), r2 = r1 * r1, r3 = r2 * r1;
+    const float lo = __fmaf_rn(q[3], r3, __fmaf_rn(q[2], r2, __fmaf_rn(q[1], r1, q[0])));
+    const float hi = __fmaf_rn(q[7], r3, __fmaf_rn(q[6], r2, __fmaf_rn(q[5], r1, q[4])));
+    const uint32_t half_mask = (1u << (4 * BITS)) - 1u;
+    packed_lo = (__float_as_uint(__fadd_rn(lo, 8388608.f)) & half_mask) |
+                ((__float_as_uint(__fadd_rn(hi, 8388608.f)) & half_mask) << (4 * BITS));
+  }
+  uint8_t* row = codes + (size_t)t * (a.d * BITS / 8);
+  if (BITS == 8) *reinterpret_cast<uint2*>(row + elem) = make_uint2(packed_lo, packed_hi);
+  else if (BITS == 4) *reinterpret_cast<uint32_t*>(row + elem / 2) = packed_lo;
+  else *reinterpret_cast<uint16_t*>(row + elem / 4) = (uint16_t)packed_lo;
+  if (((elem >> 3) & (lanes_per_group - 1)) == 0) {
+    const int gs = 31 - __clz(a.group);   // power of two
+    const size_t gi = (size_t)t * (a.d >> gs) + (elem >> gs);
+    scale[gi] = sh;
+    zero[gi] = zh;
+  }
+}
+
 template <typename T, int BITS>
 __global__ void __launch_bounds__(256) quant_residual_kernel(const __grid_constant__ QuantArgs a) {
   fl_grid_wait();
@@ -26,11 +122,6 @@ __global__ void __launch_bounds__(256) quant_residual_kernel(const __grid_consta
   const bool is_v = blockIdx.y != 0;
   const DevSide& side = is_v ? a.v : a.k;
   const T* x_new = static_cast<const T*>(is_v ? a.v_new : a.k_new) + (size_t)t * a.d;
-  uint8_t* codes = is_v ? a.v_codes : a.k_codes;
-  __half* scale = is_v ? a.v_scale : a.k_scale;
-  __half* zero = is_v ? a.v_zero : a.k_zero;
-  T* rows_prev = static_cast<T*>(is_v ? a.v_rows_prev : a.k_rows_prev);   // null: not wanted
-  T* rows_cur = static_cast<T*>(is_v ? a.v_rows_cur : a.k_rows_cur);
   const int pos = __ldg(a.active_idx + t);
   const int lanes_per_group = a.group >> 3;  // 1, 2, 4, 8 or 16
 
@@ -52,94 +143,117 @@ __global__ void __launch_bounds__(256) quant_residual_kernel(const __grid_consta
       for (int si = 0; si < 4; ++si)
         if (sl[si] >= 0) payload_apply<T, BITS>(pl[si], xh);
     }
-    if (rows_prev != nullptr) store8<T>(rows_prev + (size_t)t * a.d + elem, xh);
-    if (BITS == 16) {  // codec off: the stream keeps the row itself
-      store8<T>(reinterpret_cast<T*>(codes) + (size_t)t * a.d + elem, xn);
-      if (rows_cur != nullptr) store8<T>(rows_cur + (size_t)t * a.d + elem, xn);
-      continue;
-    }
-    float dl[8];
-    float mn, mx;
+    encode8<T, BITS>(a, is_v, t, elem, lanes_per_group, xn, xh);
+  }
+}
+
+// The same for bf16 rows of at most 2048 elements and NP <= 3 earlier streams, as a software pipeline: a CTA walks a
+// strided set of rows, and while it encodes one row the operands of its next row (new row, base row, the earlier
+// streams' payloads), the stream rows of the one after and the position of the third are in flight. One row per
+// short-lived CTA leaves every CTA two or three dependent round trips to memory with nothing to do in between.
+template <int BITS, int NP>
+__global__ void __launch_bounds__(256) quant_residual_pipelined_kernel(const __grid_constant__ QuantArgs a, int n) {
+  using T = __nv_bfloat16;
+  fl_grid_wait();
+  fl_grid_release();
+  const bool is_v = blockIdx.y != 0;
+  const DevSide& side = is_v ? a.v : a.k;
+  const int elem = threadIdx.x * 8, G = gridDim.x;
+  const int lanes_per_group = a.group >> 3;
+  const T* x_new = static_cast<const T*>(is_v ? a.v_new : a.k_new) + elem;
+  const T* base = static_cast<const T*>(side.base) + elem;
+  int t = blockIdx.x;
+  if (t >= n) return;
+  // fill the pipeline: positions of three rows, stream rows of two, operands of one
+  int pos = __ldg(a.active_idx + t);
+  int pos1 = t + G < n ? __ldg(a.active_idx + t + G) : 0;
+  int pos2 = t + 2 * G < n ? __ldg(a.active_idx + t + 2 * G) : 0;
+  uint4 rx = __ldg(reinterpret_cast<const uint4*>(x_new + (size_t)t * a.d));
+  uint4 rh = __ldg(reinterpret_cast<const uint4*>(base + (size_t)pos * a.d));
+  int sl[NP > 0 ? NP : 1], sl1[NP > 0 ? NP : 1];
+  Payload8<T, BITS> pl[NP > 0 ? NP : 1];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) dl[i] = __fsub_rn(xn[i], xh[i]);
-    mn = mx = dl[0];
+  for (int s = 0; s < NP; ++s) {
+    sl[s] = __ldg(side.s[s].slot + pos);
+    sl1[s] = t + G < n ? __ldg(side.s[s].slot + pos1) : -1;
+  }
 #pragma unroll
-    for (int i = 1; i < 8; ++i) { mn = fminf(mn, dl[i]); mx = fmaxf(mx, dl[i]); }
-    // every lane of the warp is here: the host only launches row widths for which all threads of the
-    // block run the same number of iterations (d % 256 == 0, and d % 2048 == 0 beyond 2048)
-    for (int o = 1; o < lanes_per_group; o <<= 1) {
-      mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
-      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-    }
-    const __half zh = __float2half_rd(mn);
-    const float zf = __half2float(zh);
-    const float range = __fsub_rn(mx, zf);
-    const float qmax = (float)((1 << BITS) - 1);
-    const __half sh = range == 0.f ? __float2half_rn(0.f) : __float2half_ru(__fdiv_rn(range, qmax));
-    const float sf = __half2float(sh);
-    // Codes: round-half-even of the binary32 quotient (delta - zero) / scale. The quotient is first formed with
-    // one reciprocal per group; that estimate is within a few ulp of the correctly rounded quotient (<= 5e-5
-    // absolute for codes up to 255), so its rounding to an integer is the same unless it lies within 1e-4 of a
-    // half-integer. Only then (a few percent of the warps) the true divisions are redone.
-    float q[8];
-    bool ambiguous = false;
-    if (sf != 0.f) {
-      const float inv = __frcp_rn(sf);
+  for (int s = 0; s < NP; ++s)
+    if (sl[s] >= 0) payload_load<T, BITS>(side.s[s], sl[s], elem, a.d, a.group, pl[s]);
+  for (;;) {
+    const int t1 = t + G;
+    const bool has1 = t1 < n;
+    uint4 rx1 = rx, rh1 = rh;
+    Payload8<T, BITS> pl1[NP > 0 ? NP : 1];
+    int sl2[NP > 0 ? NP : 1];
+    int pos3 = 0;
+    if (has1) {
+      rx1 = __ldg(reinterpret_cast<const uint4*>(x_new + (size_t)t1 * a.d));
+      rh1 = __ldg(reinterpret_cast<const uint4*>(base + (size_t)pos1 * a.d));
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        const float est = __fmul_rn(__fsub_rn(dl[i], zf), inv);
-        q[i] = __fsub_rn(__fadd_rn(est, 12582912.f), 12582912.f);   // round-half-even for |est| < 2^22
-        ambiguous |= 0.5f - fabsf(est - q[i]) < 1e-4f;
+      for (int s = 0; s < NP; ++s) {
+        if (sl1[s] >= 0) payload_load<T, BITS>(side.s[s], sl1[s], elem, a.d, a.group, pl1[s]);
+        sl2[s] = t + 2 * G < n ? __ldg(side.s[s].slot + pos2) : -1;
       }
-      if (__any_sync(__activemask(), ambiguous)) {
+      if (t + 3 * G < n) pos3 = __ldg(a.active_idx + t + 3 * G);
+    }
+    // row t: Xhat^(r-1) = base plus the earlier streams in loop order, then the codec
+    float xn[8], xh[8];
+    {
+      const __nv_bfloat162* hx = reinterpret_cast<const __nv_bfloat162*>(&rx);
+      const __nv_bfloat162* hh = reinterpret_cast<const __nv_bfloat162*>(&rh);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) q[i] = rintf(__fdiv_rn(__fsub_rn(dl[i], zf), sf));
+      for (int i = 0; i < 4; ++i) {
+        const float2 fx = __bfloat1622float2(hx[i]), fh = __bfloat1622float2(hh[i]);
+        xn[2 * i] = fx.x; xn[2 * i + 1] = fx.y;
+        xh[2 * i] = fh.x; xh[2 * i + 1] = fh.y;
       }
-    } else {
+    }
 #pragma unroll
-      for (int i = 0; i < 8; ++i) q[i] = 0.f;
-    }
-    if (rows_cur != nullptr) {
-      // the reconstruction every later reader of this stream forms: Xhat + (code * scale + zero), Eq. 8
+    for (int s = 0; s < NP; ++s)
+      if (sl[s] >= 0) payload_apply<T, BITS>(pl[s], xh);
+    encode8<T, BITS>(a, is_v, t, elem, lanes_per_group, xn, xh);
+    if (!has1) break;
+    t = t1;
+    rx = rx1; rh = rh1;
+    pos1 = pos2; pos2 = pos3;
 #pragma unroll
-      for (int i = 0; i < 8; ++i) xh[i] = __fadd_rn(xh[i], __fmaf_rn(q[i], sf, zf));
-      store8<T>(rows_cur + (size_t)t * a.d + elem, xh);
-    }
-    // The quotients are integers in [0, qmax] already: delta >= zero (the offset was rounded down) and
-    // (max - zero) / scale <= qmax (the scale was rounded up), so the oracle's clamp never acts. Four codes at a
-    // time are packed with exact binary32 arithmetic (sum of code * 2^(BITS*i) < 2^24 for BITS <= 4, two codes
-    // for 8 bits), and the integer is read from the low mantissa bits of (value + 2^23).
-    uint32_t packed_lo, packed_hi = 0;
-    if (BITS == 8) {
-      uint32_t w[4];
-#pragma unroll
-      for (int i = 0; i < 4; ++i)
-        w[i] = __float_as_uint(__fadd_rn(__fmaf_rn(q[2 * i + 1], 256.f, q[2 * i]), 8388608.f)) & 0xFFFFu;
-      packed_lo = w[0] | (w[1] << 16);
-      packed_hi = w[2] | (w[3] << 16);
-    } else {
-      const float r1 = (float)(1 << BITS), r2 = r1 * r1, r3 = r2 * r1;
-      const float lo = __fmaf_rn(q[3], r3, __fmaf_rn(q[2], r2, __fmaf_rn(q[1], r1, q[0])));
-      const float hi = __fmaf_rn(q[7], r3, __fmaf_rn(q[6], r2, __fmaf_rn(q[5], r1, q[4])));
-      const uint32_t half_mask = (1u << (4 * BITS)) - 1u;
-      packed_lo = (__float_as_uint(__fadd_rn(lo, 8388608.f)) & half_mask) |
-                  ((__float_as_uint(__fadd_rn(hi, 8388608.f)) & half_mask) << (4 * BITS));
-    }
-    uint8_t* row = codes + (size_t)t * (a.d * BITS / 8);
-    if (BITS == 8) *reinterpret_cast<uint2*>(row + elem) = make_uint2(packed_lo, packed_hi);
-    else if (BITS == 4) *reinterpret_cast<uint32_t*>(row + elem / 2) = packed_lo;
-    else *reinterpret_cast<uint16_t*>(row + elem / 4) = (uint16_t)packed_lo;
-    if (((elem >> 3) & (lanes_per_group - 1)) == 0) {
-      const int gs = 31 - __clz(a.group);   // power of two
-      const size_t gi = (size_t)t * (a.d >> gs) + (elem >> gs);
-      scale[gi] = sh;
-      zero[gi] = zh;
-    }
+    for (int s = 0; s < NP; ++s) { sl[s] = sl1[s]; sl1[s] = sl2[s]; pl[s] = pl1[s]; }
+  }
+}
+
+template <int BITS, int NP>
+int launch_quant_pipelined_np(const fl_ctx* ctx, const QuantArgs& a, int n_active, cudaStream_t st) {
+  auto kern = quant_residual_pipelined_kernel<BITS, NP>;
+  const int threads = a.d / 8;
+  int per_sm = 0;   // as many CTAs as are resident at once: every one of them keeps a row in flight
+  FL_CHECK_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, threads, 0));
+  if (per_sm < 1) per_sm = 1;
+  const int resident = ctx->sm_count * per_sm / 2;   // the grid has two CTAs (K, V) per row slot
+  const int gx = n_active < resident ? n_active : (resident < 1 ? 1 : resident);
+  FL_CHECK_CUDA(fl_launch(ctx, kern, dim3(gx, 2), dim3(threads), 0, st, a, n_active));
+  return fl_launch_status();
+}
+
+template <int BITS>
+int launch_quant_pipelined(const fl_ctx* ctx, const QuantArgs& a, int n_active, cudaStream_t st) {
+  switch (a.n_prev) {
+    case 0: return launch_quant_pipelined_np<BITS, 0>(ctx, a, n_active, st);
+    case 1: return launch_quant_pipelined_np<BITS, 1>(ctx, a, n_active, st);
+    case 2: return launch_quant_pipelined_np<BITS, 2>(ctx, a, n_active, st);
+    default: return launch_quant_pipelined_np<BITS, 3>(ctx, a, n_active, st);
   }
 }
 
 template <typename T>
 int launch_quant(const fl_ctx* ctx, const fl_shape* s, const QuantArgs& a, int n_active, cudaStream_t st) {
+  if (sizeof(T) == 2 && a.d <= 2048 && a.n_prev <= 3 && s->bits != 16) {
+    switch (s->bits) {
+      case 2: return launch_quant_pipelined<2>(ctx, a, n_active, st);
+      case 4: return launch_quant_pipelined<4>(ctx, a, n_active, st);
+      default: return launch_quant_pipelined<8>(ctx, a, n_active, st);
+    }
+  }
   const int threads = a.d / 8 < 256 ? a.d / 8 : 256;
   dim3 grid(n_active, 2);
   switch (s->bits) {

@@ -152,7 +152,7 @@ __global__ void __launch_bounds__(256) quant_residual_kernel(const __grid_consta
 // streams' payloads), the stream rows of the one after and the position of the third are in flight. One row per
 // short-lived CTA leaves every CTA two or three dependent round trips to memory with nothing to do in between.
 template <int BITS, int NP>
-__global__ void __launch_bounds__(256) quant_residual_pipelined_kernel(const __grid_constant__ QuantArgs a, int n) {
+__global__ void __launch_bounds__(256, 4) quant_residual_pipelined_kernel(const __grid_constant__ QuantArgs a, int n) {
   using T = __nv_bfloat16;
   fl_grid_wait();
   fl_grid_release();

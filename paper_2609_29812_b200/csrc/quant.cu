@@ -212,7 +212,9 @@ __global__ void __launch_bounds__(256, 4) quant_residual_pipelined_kernel(const 
 #pragma unroll
     for (int s = 0; s < NP; ++s)
       if (sl[s] >= 0) payload_apply<T, BITS>(pl[s], xh);
-    encode8<T, BITS>(a, is_v, t, elem, lanes_per_group, xn, xh);
+    // the common group of 128 elements gets its own copy of the codec, with the sub-warp reduction unrolled
+    if (lanes_per_group == 16) encode8<T, BITS>(a, is_v, t, elem, 16, xn, xh);
+    else encode8<T, BITS>(a, is_v, t, elem, lanes_per_group, xn, xh);
     if (!has1) break;
     t = t1;
     rx = rx1; rh = rh1;

@@ -30,7 +30,11 @@
 // Shared memory: Q_old, Q_new tiles (64 KB) + a ring of four 32 KB operand slots (K tile | V tile); a chunk of
 // the first kind takes one slot, of the second kind two. Tensor memory (512 columns): acc_old 0-127,
 // acc_new 128-255, S_old 256-319, S_new 320-383, P_old 384-447, P_new 448-511.
-// Every mbarrier wait is bounded; on a timeout the CTA raises a flag, drains and reports FL_ERR_TIMEOUT.
+// One CTA per problem, except that the problems of a partly empty last wave are given to pairs of CTAs when the
+// caller has lent a workspace: each CTA of a pair takes half of the chunks, the one that completes first leaves its
+// accumulators and row statistics in the workspace and the other merges them into its own before the epilogue.
+// Every wait (mbarriers, the pair's counter) is bounded; on a timeout the CTA raises a flag, drains and reports
+// FL_ERR_TIMEOUT.
 #include "fl_internal.cuh"
 #include "tc_ptx.cuh"
 

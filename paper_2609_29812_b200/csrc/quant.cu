@@ -1,6 +1,10 @@
 // Stage 3: residual quantization of the active rows' K and V (Eq. 8 with the asymmetric group-wise
-// min/max quantizer of Appendix E). HBM-bound: each thread owns 8 consecutive elements (one 16-byte
-// load in bf16), group min/max by sub-warp shuffles, codes packed and stored coalesced.
+// min/max quantizer of Appendix E). Each thread owns 8 consecutive elements (one 16-byte load in bf16), group
+// min/max by sub-warp shuffles, codes packed and stored coalesced. Two kernels share the codec (encode8): a software
+// pipeline over strided rows for the common shapes (bf16 rows of up to 2048 elements, at most three earlier
+// streams), which keeps the next rows' operands in flight, and a plain one-CTA-per-row kernel for everything else.
+// Both also leave, when the caller lends the buffers, the reconstructed rows before and after the loop's residual
+// as bf16 for the attention call of the same loop.
 #include "fl_internal.cuh"
 
 namespace {

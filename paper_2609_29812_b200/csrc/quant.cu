@@ -34,87 +34,87 @@ __device__ __forceinline__ void encode8(const QuantArgs& a, bool is_v, int t, in
   T* rows_prev = static_cast<T*>(is_v ? a.v_rows_prev : a.k_rows_prev);   // null: not wanted
   T* rows_cur = static_cast<T*>(is_v ? a.v_rows_cur : a.k_rows_cur);
   if (rows_prev != nullptr) store8<T>(rows_prev + (size_t)t * a.d + elem, xh);
-  if (BITS == 16) {  // codec off: the stream keeps the row itself
+  if constexpr (BITS == 16) {  // codec off: the stream keeps the row itself
     store8<T>(reinterpret_cast<T*>(codes) + (size_t)t * a.d + elem, xn);
     if (rows_cur != nullptr) store8<T>(rows_cur + (size_t)t * a.d + elem, xn);
-    return;
-  }
-  float dl[8];
-  float mn, mx;
-#pragma unroll
-  for (int i = 0; i < 8; ++i) dl[i] = __fsub_rn(xn[i], xh[i]);
-  mn = mx = dl[0];
-#pragma unroll
-  for (int i = 1; i < 8; ++i) { mn = fminf(mn, dl[i]); mx = fmaxf(mx, dl[i]); }
-  // every lane of the warp is here: the host only launches row widths for which all threads of the
-  // block run the same number of iterations (d % 256 == 0, and d % 2048 == 0 beyond 2048)
-  for (int o = 1; o < lanes_per_group; o <<= 1) {
-    mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
-    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-  }
-  const __half zh = __float2half_rd(mn);
-  const float zf = __half2float(zh);
-  const float range = __fsub_rn(mx, zf);
-  const float qmax = (float)((1 << BITS) - 1);
-  const __half sh = range == 0.f ? __float2half_rn(0.f) : __float2half_ru(__fdiv_rn(range, qmax));
-  const float sf = __half2float(sh);
-  // Codes: round-half-even of the binary32 quotient (delta - zero) / scale. The quotient is first formed with
-  // one reciprocal per group; that estimate is within a few ulp of the correctly rounded quotient (<= 5e-5
-  // absolute for codes up to 255), so its rounding to an integer is the same unless it lies within 1e-4 of a
-  // half-integer. Only then (a few percent of the warps) the true divisions are redone.
-  float q[8];
-  bool ambiguous = false;
-  if (sf != 0.f) {
-    const float inv = __frcp_rn(sf);
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      const float est = __fmul_rn(__fsub_rn(dl[i], zf), inv);
-      q[i] = __fsub_rn(__fadd_rn(est, 12582912.f), 12582912.f);   // round-half-even for |est| < 2^22
-      ambiguous |= 0.5f - fabsf(est - q[i]) < 1e-4f;
-    }
-    if (__any_sync(__activemask(), ambiguous)) {
-#pragma unroll
-      for (int i = 0; i < 8; ++i) q[i] = rintf(__fdiv_rn(__fsub_rn(dl[i], zf), sf));
-    }
   } else {
-#pragma unroll
-    for (int i = 0; i < 8; ++i) q[i] = 0.f;
-  }
-  if (rows_cur != nullptr) {
-    // the reconstruction every later reader of this stream forms: Xhat + (code * scale + zero), Eq. 8
-#pragma unroll
-    for (int i = 0; i < 8; ++i) xh[i] = __fadd_rn(xh[i], __fmaf_rn(q[i], sf, zf));
-    store8<T>(rows_cur + (size_t)t * a.d + elem, xh);
-  }
-  // The quotients are integers in [0, qmax] already: delta >= zero (the offset was rounded down) and
-  // (max - zero) / scale <= qmax (the scale was rounded up), so the oracle's clamp never acts. Four codes at a
-  // time are packed with exact binary32 arithmetic (sum of code * 2^(BITS*i) < 2^24 for BITS <= 4, two codes
-  // for 8 bits), and the integer is read from the low mantissa bits of (value + 2^23).
-  uint32_t packed_lo, packed_hi = 0;
-  if (BITS == 8) {
-    uint32_t w[4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i)
-      w[i] = __float_as_uint(__fadd_rn(__fmaf_rn(q[2 * i + 1], 256.f, q[2 * i]), 8388608.f)) & 0xFFFFu;
-    packed_lo = w[0] | (w[1] << 16);
-    packed_hi = w[2] | (w[3] << 16);
-  } else {
-    const float r1 = (float)(1 << BITS), r2 = r1 * r1, r3 = r2 * r1;
-    const float lo = __fmaf_rn(q[3], r3, __fmaf_rn(q[2], r2, __fmaf_rn(q[1], r1, q[0])));
-    const float hi = __fmaf_rn(q[7], r3, __fmaf_rn(q[6], r2, __fmaf_rn(q[5], r1, q[4])));
-    const uint32_t half_mask = (1u << (4 * BITS)) - 1u;
-    packed_lo = (__float_as_uint(__fadd_rn(lo, 8388608.f)) & half_mask) |
-                ((__float_as_uint(__fadd_rn(hi, 8388608.f)) & half_mask) << (4 * BITS));
-  }
-  uint8_t* row = codes + (size_t)t * (a.d * BITS / 8);
-  if (BITS == 8) *reinterpret_cast<uint2*>(row + elem) = make_uint2(packed_lo, packed_hi);
-  else if (BITS == 4) *reinterpret_cast<uint32_t*>(row + elem / 2) = packed_lo;
-  else *reinterpret_cast<uint16_t*>(row + elem / 4) = (uint16_t)packed_lo;
-  if (((elem >> 3) & (lanes_per_group - 1)) == 0) {
-    const int gs = 31 - __clz(a.group);   // power of two
-    const size_t gi = (size_t)t * (a.d >> gs) + (elem >> gs);
-    scale[gi] = sh;
-    zero[gi] = zh;
+    float dl[8];
+    float mn, mx;
+  #pragma unroll
+    for (int i = 0; i < 8; ++i) dl[i] = __fsub_rn(xn[i], xh[i]);
+    mn = mx = dl[0];
+  #pragma unroll
+    for (int i = 1; i < 8; ++i) { mn = fminf(mn, dl[i]); mx = fmaxf(mx, dl[i]); }
+    // every lane of the warp is here: the host only launches row widths for which all threads of the
+    // block run the same number of iterations (d % 256 == 0, and d % 2048 == 0 beyond 2048)
+    for (int o = 1; o < lanes_per_group; o <<= 1) {
+      mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    }
+    const __half zh = __float2half_rd(mn);
+    const float zf = __half2float(zh);
+    const float range = __fsub_rn(mx, zf);
+    const float qmax = (float)((1 << BITS) - 1);
+    const __half sh = range == 0.f ? __float2half_rn(0.f) : __float2half_ru(__fdiv_rn(range, qmax));
+    const float sf = __half2float(sh);
+    // Codes: round-half-even of the binary32 quotient (delta - zero) / scale. The quotient is first formed with
+    // one reciprocal per group; that estimate is within a few ulp of the correctly rounded quotient (<= 5e-5
+    // absolute for codes up to 255), so its rounding to an integer is the same unless it lies within 1e-4 of a
+    // half-integer. Only then (a few percent of the warps) the true divisions are redone.
+    float q[8];
+    bool ambiguous = false;
+    if (sf != 0.f) {
+      const float inv = __frcp_rn(sf);
+  #pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const float est = __fmul_rn(__fsub_rn(dl[i], zf), inv);
+        q[i] = __fsub_rn(__fadd_rn(est, 12582912.f), 12582912.f);   // round-half-even for |est| < 2^22
+        ambiguous |= 0.5f - fabsf(est - q[i]) < 1e-4f;
+      }
+      if (__any_sync(__activemask(), ambiguous)) {
+  #pragma unroll
+        for (int i = 0; i < 8; ++i) q[i] = rintf(__fdiv_rn(__fsub_rn(dl[i], zf), sf));
+      }
+    } else {
+  #pragma unroll
+      for (int i = 0; i < 8; ++i) q[i] = 0.f;
+    }
+    if (rows_cur != nullptr) {
+      // the reconstruction every later reader of this stream forms: Xhat + (code * scale + zero), Eq. 8
+  #pragma unroll
+      for (int i = 0; i < 8; ++i) xh[i] = __fadd_rn(xh[i], __fmaf_rn(q[i], sf, zf));
+      store8<T>(rows_cur + (size_t)t * a.d + elem, xh);
+    }
+    // The quotients are integers in [0, qmax] already: delta >= zero (the offset was rounded down) and
+    // (max - zero) / scale <= qmax (the scale was rounded up), so the oracle's clamp never acts. Four codes at a
+    // time are packed with exact binary32 arithmetic (sum of code * 2^(BITS*i) < 2^24 for BITS <= 4, two codes
+    // for 8 bits), and the integer is read from the low mantissa bits of (value + 2^23).
+    uint32_t packed_lo, packed_hi = 0;
+    if constexpr (BITS == 8) {
+      uint32_t w[4];
+  #pragma unroll
+      for (int i = 0; i < 4; ++i)
+        w[i] = __float_as_uint(__fadd_rn(__fmaf_rn(q[2 * i + 1], 256.f, q[2 * i]), 8388608.f)) & 0xFFFFu;
+      packed_lo = w[0] | (w[1] << 16);
+      packed_hi = w[2] | (w[3] << 16);
+    } else {
+      const float r1 = (float)(1 << BITS), r2 = r1 * r1, r3 = r2 * r1;
+      const float lo = __fmaf_rn(q[3], r3, __fmaf_rn(q[2], r2, __fmaf_rn(q[1], r1, q[0])));
+      const float hi = __fmaf_rn(q[7], r3, __fmaf_rn(q[6], r2, __fmaf_rn(q[5], r1, q[4])));
+      const uint32_t half_mask = (1u << (4 * BITS)) - 1u;
+      packed_lo = (__float_as_uint(__fadd_rn(lo, 8388608.f)) & half_mask) |
+                  ((__float_as_uint(__fadd_rn(hi, 8388608.f)) & half_mask) << (4 * BITS));
+    }
+    uint8_t* row = codes + (size_t)t * (a.d * BITS / 8);
+    if (BITS == 8) *reinterpret_cast<uint2*>(row + elem) = make_uint2(packed_lo, packed_hi);
+    else if (BITS == 4) *reinterpret_cast<uint32_t*>(row + elem / 2) = packed_lo;
+    else *reinterpret_cast<uint16_t*>(row + elem / 4) = (uint16_t)packed_lo;
+    if (((elem >> 3) & (lanes_per_group - 1)) == 0) {
+      const int gs = 31 - __clz(a.group);   // power of two
+      const size_t gi = (size_t)t * (a.d >> gs) + (elem >> gs);
+      scale[gi] = sh;
+      zero[gi] = zh;
+    }
   }
 }
 

@@ -356,6 +356,34 @@ def test_attention_workspace_calls(env):
     ctx._workspace = None
 
 
+def test_programmatic_launch_off_gives_the_same_bits(env, monkeypatch):
+    """FL_NO_PDL=1 (read when a context is created) launches every kernel fully serialized: same results."""
+    import torch
+    B, P, ctx = env
+    w = small_bf16(L=1300, H=2, R=3)
+    x = workloads.make_layer_inputs(w, seed=4)
+    ref = fo.LayerOracle(w.L, w.n_heads, w.head_dim, w.q_block, w.bits, w.group, w.eps, w.sm_scale,
+                         storage=w.dtype).run(x.G, x.Q, x.K, x.V, [w.k_tokens] * 2, [w.col_budget] * 2)
+    monkeypatch.setenv("FL_NO_PDL", "1")
+    ctx_plain = B.Context(0)
+    monkeypatch.delenv("FL_NO_PDL")
+    outs = []
+    for c in (ctx, ctx_plain):
+        st = P.LayerState(c, w)
+        st.dense_loop(to_dev(x.Q[0], w), to_dev(x.K[0], w), to_dev(x.V[0], w))
+        st.select_columns_dense()
+        for r in (2, 3):
+            sel = oracle_selection(P, w, ref, r)
+            act = ref["active"][r - 2]
+            st.sparse_loop(r, to_dev(x.Q[r - 1][act], w), to_dev(x.K[r - 1][act], w), to_dev(x.V[r - 1][act], w),
+                           sel, indexed=True)
+            st.check_status()
+        outs.append((st.o_store.clone(), st.q_store.clone(), st.lse.clone(), st.col_idx.clone()))
+    for a_, b_ in zip(*outs):
+        assert torch.equal(a_, b_)
+    ctx_plain.close()
+
+
 def test_binary32_simt_attention_path_on_bf16_storage(env):
     """The SIMT attention kernels also serve bf16 storage (forced here; normally the tensor path runs)."""
     import os

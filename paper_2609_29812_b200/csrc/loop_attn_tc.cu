@@ -5,11 +5,10 @@
 // Warp roles (16 warps, 512 threads):
 //   warps 0-3   softmax of the OLD term  (fixed normaliser lse_prev: p_old = exp(s_old - lse_prev), mass m_i)
 //   warps 4-7   softmax of the NEW term  (running reference, lazy rescale of the accumulator)
-//   warps 8-11  MMA issuers, one thread each: S_old = Q_old Khat_old^T, S_new = Q_new Khat_new^T,
-//               acc_old += P_old Vhat_old, acc_new += P_new Vhat_new. A single thread issues a 128x64x16 MMA
-//               every ~60-90 cycles while the tensor pipe retires one in 48, so the four streams of MMAs are
-//               issued from four warps on four different schedulers.
-//   warps 12-15 TMA + patch: the Q tiles (two 2-D tile loads each), row gathers (cp.async.bulk.tensor
+//   warps 8-9   MMA issuers, one thread per term: S = Q Khat^T of chunk n, then acc += P Vhat of chunk n - 1. A single
+//               thread issues a 128x64x16 MMA every ~60-90 cycles while the tensor pipe retires one in 48; two threads
+//               on two schedulers keep up with a chunk period that the exponentials set
+//   warps 10-15 TMA + patch: the Q tiles (two 2-D tile loads each), row gathers (cp.async.bulk.tensor
 //               tile::gather4, 4 selected columns per copy) of bf16 K/V rows straight into 128B-swizzled
 //               operand tiles, and for columns that carry residual payloads which nobody has materialized the
 //               overwrite of the gathered base rows with the dequantize-and-add result (Eq. 8)
@@ -23,13 +22,14 @@
 // old / new tiles are plain gathers from there (indexed by the token's row in the loop's stream). Without that
 // workspace, and for columns whose only payloads are from earlier loops, the patch warps rebuild the rows here.
 //
-// Per chunk of 64 columns and per term: S (f32, 64 tensor-memory columns, ONE buffer: the softmax warps pull it
-// into registers and hand the buffer back at once, so the next chunk's QK^T runs under the current chunk's
-// exponentials), P (bf16, 32 columns, two buffers: PV of a chunk runs under the next chunk's exponentials).
+// Per chunk of 64 columns and per term: S (f32, 64 tensor-memory columns, two buffers: the next chunk's QK^T runs
+// under the current chunk's exponentials); P (bf16, 32 columns) is written over the first half of the S buffer it
+// was computed from, once those logits are in registers, so PV of a chunk runs under the next chunk's exponentials
+// and the QK^T of the chunk after that waits for it before it overwrites the buffer.
 // The two terms are independent pipelines. Epilogue: O = O_prev - acc_old + (m / l) acc_new.
 // Shared memory: Q_old, Q_new tiles (64 KB) + a ring of four 32 KB operand slots (K tile | V tile); a chunk of
 // the first kind takes one slot, of the second kind two. Tensor memory (512 columns): acc_old 0-127,
-// acc_new 128-255, S_old 256-319, S_new 320-383, P_old 384-447, P_new 448-511.
+// acc_new 128-255, S_old / P_old 256-383 (two buffers), S_new / P_new 384-511.
 // One CTA per problem, except that the problems of a partly empty last wave are given to pairs of CTAs when the
 // caller has lent a workspace: each CTA of a pair takes half of the chunks, the one that completes first leaves its
 // accumulators and row statistics in the workspace and the other merges them into its own before the epilogue.
@@ -48,15 +48,18 @@ constexpr int kTileBytes = kNC * kDH * 2;   // 16 KB
 constexpr int kSlotBytes = 2 * kTileBytes;  // K tile | V tile
 constexpr int kQTileBytes = kM * kDH * 2;   // 32 KB
 constexpr int kSoftmaxWarps = 8;
-constexpr int kIssueWarp = 8;      // warps 8..11: QK old, QK new, PV old, PV new
-constexpr int kTmaWarp = 12;       // first of the TMA / patch warps
-constexpr int kTmaWarps = 4;       // a single warp cannot issue four-row gathers fast enough; four come close
-constexpr int kWarps = kSoftmaxWarps + 4 + kTmaWarps;  // 16
+constexpr int kIssueWarp = 8;      // warps 8, 9: the MMA issuers of the old and of the new term (QK^T and PV each)
+constexpr int kIssueWarps = 2;
+constexpr int kTmaWarp = 10;       // first of the TMA / patch warps
+constexpr int kTmaWarps = 6;       // a warp's four-row gathers are taken one lane after the other (~100 cycles each):
+                                   // the 64 gathers of a ring slot need as many warps as can be had
+constexpr int kWarps = kSoftmaxWarps + kIssueWarps + kTmaWarps;  // 16
+constexpr int kSlotGathers = kSlotBytes / 512;   // 64 four-row gathers of 128-byte rows fill a slot
 constexpr int kThreads = kWarps * 32;
 constexpr int kColWarps = 14;               // warps that read the column list in the prologue (the other two search rows)
 constexpr int kMaxCols = 3072;              // column budget the shared-memory column list can hold
 constexpr int kMaxChunks = kMaxCols / kNC + 2;
-constexpr uint32_t kAccOld = 0, kAccNew = 128, kSOld = 256, kSNew = 320, kPOld = 384, kPNew = 448;
+constexpr uint32_t kAccOld = 0, kAccNew = 128, kSOld = 256, kSNew = 384;   // two S buffers of kNC columns each
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 // A problem can be split over two CTAs, each taking half of the chunks: a CTA's partial result is both accumulators
@@ -118,10 +121,9 @@ struct __align__(16) TcSmemCtl {
   uint64_t done[kSlots];     // the two PV issuers -> TMA: the MMAs that read the slot have finished (a term's PV of a chunk
                              // is issued after its softmax, hence after its QK^T of the chunk has completed)
   uint64_t q_full;           // TMA -> QK issuers: the Q tiles of the current row tile have arrived
-  uint64_t s_full[2];        // QK issuer -> softmax (per term): S of the chunk is in tensor memory
-  uint64_t s_taken[2];       // softmax -> QK issuer: S of the chunk is in registers, the buffer may be overwritten
-  uint64_t p_full[2][2];     // softmax -> PV issuer (per term, per P buffer): P of the chunk is in tensor memory
-  uint64_t p_free[2][2];     // PV issuer -> softmax: the PV MMAs that read the P buffer have finished
+  uint64_t s_full[2][2];     // QK issuer -> softmax (per term, per S buffer): S of the chunk is in tensor memory
+  uint64_t p_full[2][2];     // softmax -> PV issuer (per term, per buffer): P of the chunk is in tensor memory
+  uint64_t p_free[2][2];     // PV issuer -> QK issuer: the PV MMAs that read the buffer's P have finished
   uint64_t acc_done;         // PV issuers -> softmax: all accumulation of the tile finished
   uint32_t tmem_base;
   int abort_flag;
@@ -292,9 +294,8 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
     }
     tc::mbar_init(&ctl.q_full, 1);
     for (int t = 0; t < 2; ++t) {
-      tc::mbar_init(&ctl.s_full[t], 1);
-      tc::mbar_init(&ctl.s_taken[t], 4);
       for (int pb = 0; pb < 2; ++pb) {
+        tc::mbar_init(&ctl.s_full[t][pb], 1);
         tc::mbar_init(&ctl.p_full[t][pb], 4);
         tc::mbar_init(&ctl.p_free[t][pb], 1);
       }
@@ -442,7 +443,7 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
   }
   __syncthreads();
   if (tid == 0) TC_TRACE(0, 60, 1);
-  int g = 0;    // chunks issued so far (all tiles): one phase of s_full / s_taken per chunk, P buffer = g & 1
+  int g = 0;    // chunks issued so far (all tiles): S / P buffer = g & 1, one phase of its barriers per use
   int fill = 0; // ring slots filled so far: slot = fill % kSlots, phase = (fill / kSlots) & 1
   uint32_t dirty_par_cta = 0;  // per-slot phase parity of the patched[] barriers (they only see dirty chunks)
 
@@ -480,12 +481,15 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
   if (warp >= kTmaWarp) {
     // ========================================== TMA + patch ==========================================
     // In-order fills of the ring; the lookahead is whatever the four slots allow. The 64 four-row gathers
-    // of a slot (K: 2 slabs x 16 groups, V: the same) are split over the four warps, 16 each, one per lane;
+    // of a slot (K: 2 slabs x 16 groups, V: the same) are dealt round robin to the six warps, one per lane;
     // every warp announces its own share of the bytes on the slot's barrier. Chunks whose columns carry
-    // residual payloads are then rewritten in place by the same warps (4 columns at a time, lanes 0-15 the K
+    // residual payloads are then rewritten in place by the same warps (6 columns at a time, lanes 0-15 the K
     // row, lanes 16-31 the V row).
     const int tw = warp - kTmaWarp;
-    const int is_v = tw >> 1, slab = tw & 1, grp = lane & 15;
+    // gather `req` of a slot: tile (K, V), 64-element slab, group of four columns
+    const int req = lane * kTmaWarps + tw;
+    const int my_reqs = (kSlotGathers - 1 - tw) / kTmaWarps + 1;      // requests of this warp (lanes 0 .. my_reqs - 1)
+    const int is_v = (req >> 5) & 1, slab = (req >> 4) & 1, grp = req & 15;
     const void* map = is_v ? static_cast<const void*>(&a.v_map) : static_cast<const void*>(&a.k_map);
     const int half = lane >> 4, ch = lane & 15;
     const DevSide& side = half ? a.v : a.k;
@@ -504,12 +508,12 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
       if (!ok) break;
       if (tid == kTmaWarp * 32) TC_TRACE(0, ci, 0);
       if (lane == 0)
-        for (int k = 0; k < n_slots; ++k) tc::mbar_arrive_expect_tx(&ctl.landed[(f + k) % kSlots], kSlotBytes / kTmaWarps);
+        for (int k = 0; k < n_slots; ++k) tc::mbar_arrive_expect_tx(&ctl.landed[(f + k) % kSlots], my_reqs * 512);
       __syncwarp();
       // columns that are active in this loop come from the materialized rows (old tile: before the loop's
       // residual, new tile: after it), indexed by their row in the loop's stream; all others from the base
       const bool from_rows = ck.patch && a.use_rows;
-      if (lane < 16) {
+      if (req < kSlotGathers) {
         int y[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
@@ -568,10 +572,13 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
     }
   } else if (warp >= kIssueWarp) {
     // ========================================== MMA issuers ==========================================
-    const int role = warp - kIssueWarp;   // 0: QK old, 1: QK new, 2: PV old, 3: PV new
-    const int t = role & 1;
-    if (lane == 0 && role < 2) {
+    // One thread per term issues both kinds of MMA, in the order their operands become ready: QK^T of chunk n (its S
+    // buffer is free once PV of chunk n - 2 has retired), then PV of chunk n - 1 (its P is written while QK^T of
+    // chunk n executes).
+    const int t = warp - kIssueWarp;      // 0: old term, 1: new term
+    if (lane == 0) {
       const uint32_t idesc_qk = tc::make_idesc_bf16(kM, kNC, false);
+      const uint32_t idesc_pv = tc::make_idesc_bf16(kM, kDH, true);
       // Descriptors differ only in their start-address field (bits 0-13, units of 16 bytes): the low word
       // moves (no carry into the other fields: shared memory is < 256 KB), the high word stays.
       // K-major operands (Q, Khat): 32 bytes per 16-element K step inside a 64-element slab, then the next slab.
@@ -579,68 +586,70 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
       const uint64_t k_desc0 = tc::make_desc_sw128(tc::smem_u32(ring), 16, 1024);
       const uint32_t kq_hi = (uint32_t)(k_desc0 >> 32);
       const uint32_t q_lo_w = (uint32_t)q_desc, k_lo0 = (uint32_t)k_desc0;
-      const uint32_t s_dst = tmem + (t ? kSNew : kSOld);
-      int f = fill0;
-      uint32_t dirty_par = dirty_par0;
-#pragma unroll 1
-      for (int ci = c_lo; ci < c_hi; ++ci) {
-        const ChunkInfo ck = chunk_info(ci, n_plain, n_patch);
-        const int slot0 = f % kSlots, slot1 = (f + 1) % kSlots;
-        const int gc = g0 + ci - c_lo;
-        if (t == 0) TC_TRACE(1, ci, 0);
-        if (ci == c_lo && !tc::mbar_wait(&ctl.q_full, tile & 1, abort_flag)) break;
-        // a term reads one slot of the chunk only (the new term of a two-slot chunk the second): it starts on it
-        // without waiting for the other
-        const int my_slot = (t && ck.patch) ? slot1 : slot0, my_fill = (t && ck.patch) ? f + 1 : f;
-        if (!tc::mbar_wait(&ctl.landed[my_slot], (my_fill / kSlots) & 1, abort_flag)) break;
-        if (ctl.chunk_mask[ci] != 0) {       // residual-carrying columns are rewritten by the patch warps
-          if (!tc::mbar_wait(&ctl.patched[my_slot], (dirty_par >> my_slot) & 1, abort_flag)) break;
-          dirty_par ^= 1u << slot0;
-          if (ck.patch) dirty_par ^= 1u << slot1;
-        }
-        // the S buffer holds the previous chunk until the softmax warps have pulled it into registers
-        if (gc >= 1 && !tc::mbar_wait(&ctl.s_taken[t], (gc - 1) & 1, abort_flag)) break;
-        tc::tc_fence_after();
-        if (t == 0) TC_TRACE(1, ci, 1);
-        const uint32_t k_lo = k_lo0 + my_slot * (kSlotBytes >> 4);
-#define FL_QK(KK, ACC)                                                                                       \
-  tc::mma_ss_lo<ACC>(s_dst, q_lo_w + ((((KK) >> 2) * (kM * 128) + ((KK)&3) * 32) >> 4), kq_hi,               \
-                     k_lo + ((((KK) >> 2) * (kNC * 128) + ((KK)&3) * 32) >> 4), kq_hi, idesc_qk)
-        FL_QK(0, false); FL_QK(1, true); FL_QK(2, true); FL_QK(3, true);
-        FL_QK(4, true);  FL_QK(5, true); FL_QK(6, true); FL_QK(7, true);
-#undef FL_QK
-        tc::mma_commit(&ctl.s_full[t]);
-        f += ck.patch ? 2 : 1;
-        if (t == 0) TC_TRACE(1, ci, 2);
-      }
-    } else if (lane == 0) {
-      const uint32_t idesc_pv = tc::make_idesc_bf16(kM, kDH, true);
       // MN-major Vhat: 16 key rows = two 1024-byte row groups per K step
       const uint64_t v_desc0 = tc::make_desc_sw128(tc::smem_u32(ring) + kTileBytes, kNC * 128, 1024);
       const uint32_t v_hi = (uint32_t)(v_desc0 >> 32), v_lo0 = (uint32_t)v_desc0;
+      const uint32_t s_base = tmem + (t ? kSNew : kSOld);
       const uint32_t acc = tmem + (t ? kAccNew : kAccOld);
-      const uint32_t p_base = tmem + (t ? kPNew : kPOld);
-      int f = fill0;
+      int f = fill0;             // ring position of the chunk whose QK^T is issued next
+      int pv_slot = 0;           // slots of the chunk whose PV is issued next (the previous QK^T's)
+      int pv_slot1 = -1;
+      uint32_t dirty_par = dirty_par0;
 #pragma unroll 1
-      for (int cj = c_lo; cj < c_hi; ++cj) {
-        const ChunkInfo ck = chunk_info(cj, n_plain, n_patch);
-        const int gc = g0 + cj - c_lo, pb = gc & 1;
-        if (t == 0) TC_TRACE(4, cj, 0);
-        if (!tc::mbar_wait(&ctl.p_full[t][pb], (gc >> 1) & 1, abort_flag)) break;
-        tc::tc_fence_after();
-        if (t == 0) TC_TRACE(4, cj, 1);
-        const int slot0 = f % kSlots, slot1 = (f + 1) % kSlots;
-        const uint32_t v_lo = v_lo0 + ((t && ck.patch) ? slot1 : slot0) * (kSlotBytes >> 4);
-        const uint32_t p_src = p_base + pb * 32;
-        const uint32_t acc0 = cj > c_lo ? 1u : 0u;       // the CTA's first chunk of the tile overwrites the accumulator
+      for (int ci = c_lo; ci <= c_hi; ++ci) {
+        const int gc = g0 + ci - c_lo;
+        int qk_slot = 0, qk_slot1 = -1;
+        if (ci < c_hi) {
+          const ChunkInfo ck = chunk_info(ci, n_plain, n_patch);
+          const int slot0 = f % kSlots, slot1 = (f + 1) % kSlots;
+          if (t == 0) TC_TRACE(1, ci, 0);
+          if (ci == c_lo && !tc::mbar_wait(&ctl.q_full, tile & 1, abort_flag)) break;
+          // a term reads one slot of the chunk only (the new term of a two-slot chunk the second): it starts on it
+          // without waiting for the other
+          const int my_slot = (t && ck.patch) ? slot1 : slot0, my_fill = (t && ck.patch) ? f + 1 : f;
+          if (!tc::mbar_wait(&ctl.landed[my_slot], (my_fill / kSlots) & 1, abort_flag)) break;
+          if (ctl.chunk_mask[ci] != 0) {       // residual-carrying columns are rewritten by the patch warps
+            if (!tc::mbar_wait(&ctl.patched[my_slot], (dirty_par >> my_slot) & 1, abort_flag)) break;
+            dirty_par ^= 1u << slot0;
+            if (ck.patch) dirty_par ^= 1u << slot1;
+          }
+          // the S buffer holds P of the chunk before the previous one until its PV MMAs have read it
+          if (gc >= 2 && !tc::mbar_wait(&ctl.p_free[t][gc & 1], ((gc >> 1) - 1) & 1, abort_flag)) break;
+          const uint32_t s_dst = s_base + (gc & 1) * kNC;
+          tc::tc_fence_after();
+          if (t == 0) TC_TRACE(1, ci, 1);
+          const uint32_t k_lo = k_lo0 + my_slot * (kSlotBytes >> 4);
+#define FL_QK(KK, ACC)                                                                                       \
+  tc::mma_ss_lo<ACC>(s_dst, q_lo_w + ((((KK) >> 2) * (kM * 128) + ((KK)&3) * 32) >> 4), kq_hi,               \
+                     k_lo + ((((KK) >> 2) * (kNC * 128) + ((KK)&3) * 32) >> 4), kq_hi, idesc_qk)
+          FL_QK(0, false); FL_QK(1, true); FL_QK(2, true); FL_QK(3, true);
+          FL_QK(4, true);  FL_QK(5, true); FL_QK(6, true); FL_QK(7, true);
+#undef FL_QK
+          tc::mma_commit(&ctl.s_full[t][gc & 1]);
+          qk_slot = slot0;
+          qk_slot1 = ck.patch ? slot1 : -1;
+          f += ck.patch ? 2 : 1;
+          if (t == 0) TC_TRACE(1, ci, 2);
+        }
+        if (ci > c_lo) {
+          const int cj = ci - 1, gp = gc - 1, pb = gp & 1;
+          if (t == 0) TC_TRACE(4, cj, 0);
+          if (!tc::mbar_wait(&ctl.p_full[t][pb], (gp >> 1) & 1, abort_flag)) break;
+          tc::tc_fence_after();
+          if (t == 0) TC_TRACE(4, cj, 1);
+          const uint32_t v_lo = v_lo0 + ((t && pv_slot1 >= 0) ? pv_slot1 : pv_slot) * (kSlotBytes >> 4);
+          const uint32_t p_src = s_base + pb * kNC;
+          const uint32_t acc0 = cj > c_lo ? 1u : 0u;       // the CTA's first chunk of the tile overwrites the accumulator
 #pragma unroll
-        for (int kk = 0; kk < kNC / 16; ++kk)
-          tc::mma_ts_lo(acc, p_src + kk * 8, v_lo + kk * (2048 >> 4), v_hi, idesc_pv, kk > 0 ? 1u : acc0);
-        tc::mma_commit(&ctl.p_free[t][pb]);
-        tc::mma_commit(&ctl.done[slot0]);
-        if (ck.patch) tc::mma_commit(&ctl.done[slot1]);
-        f += ck.patch ? 2 : 1;
-        if (t == 0) TC_TRACE(4, cj, 2);
+          for (int kk = 0; kk < kNC / 16; ++kk)
+            tc::mma_ts_lo(acc, p_src + kk * 8, v_lo + kk * (2048 >> 4), v_hi, idesc_pv, kk > 0 ? 1u : acc0);
+          tc::mma_commit(&ctl.p_free[t][pb]);
+          tc::mma_commit(&ctl.done[pv_slot]);
+          if (pv_slot1 >= 0) tc::mma_commit(&ctl.done[pv_slot1]);
+          if (t == 0) TC_TRACE(4, cj, 2);
+        }
+        pv_slot = qk_slot;
+        pv_slot1 = qk_slot1;
       }
       tc::mma_commit(&ctl.acc_done);
     }
@@ -659,14 +668,12 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
     if (row_ok)
       tc::prefetch_l2(a.o_prev + (INDEXED ? (size_t)pos : (size_t)(s0 + row)) * a.d + h * kDH + grp * 64);
     const uint32_t s_addr = tmem + lane_base + (grp ? kSNew : kSOld);
-    const uint32_t p_addr = tmem + lane_base + (grp ? kPNew : kPOld);
     float mass = 0.f, ell = 0.f, ref = -INFINITY;
     bool ok = true;
-    bool pending = false;   // the previous chunk's P is stored but not yet announced (warp-uniform)
     for (int ci = c_lo; ci < c_hi; ++ci) {
       const int gc = g0 + ci - c_lo, pb = gc & 1, n_use = gc >> 1;
       if (gt == 0) TC_TRACE(2 + grp, ci, 0);
-      if (!warp_wait(&ctl.s_full[grp], gc & 1, abort_flag)) { ok = false; break; }
+      if (!warp_wait(&ctl.s_full[grp][pb], n_use & 1, abort_flag)) { ok = false; break; }
       tc::tc_fence_after();
       if (gt == 0) TC_TRACE(2 + grp, ci, 1);
       // rows of a warp that lie at or after every column of the chunk need no causal mask; rows beyond the
@@ -684,31 +691,17 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
         }
         vis = lo;
       }
-      // the P buffer is free once the PV MMAs of chunk gc - 2 have retired
-      if (n_use >= 1 && !warp_wait(&ctl.p_free[grp][pb], (n_use - 1) & 1, abort_flag)) { ok = false; break; }
+      // P goes over the first half of this S buffer (the QK^T issuer waited for the PV MMAs of chunk gc - 2 before it
+      // overwrote the buffer): the first 32 logits are in registers before columns 0-15 are stored, the second 32
+      // (columns 32-63) before columns 16-31 are
+      const uint32_t sp_addr = s_addr + pb * kNC;
       // The 64 logits of the row are taken in two halves of 32 (each its own little softmax step): 64 live logits
       // plus the pipeline's state do not fit 128 registers, and what spills lands in an L1 of ~30 KB.
 #pragma unroll 1
       for (int hf = 0; hf < 2 && ok; ++hf) {
         uint32_t r[32];
-        tc::tmem_ld32(s_addr + hf * 32, r);
+        tc::tmem_ld32(sp_addr + hf * 32, r);
         tc::tmem_wait_ld();
-        if (hf == 0) {
-          // the previous chunk's P store has had this long to land: it is announced now instead of being waited
-          // for at the end of its own iteration
-          if (pending) {
-            tc::tmem_wait_st();
-            tc::tc_fence_before();
-            __syncwarp();
-            if (lane == 0) tc::mbar_arrive(&ctl.p_full[grp][pb ^ 1]);
-            pending = false;
-          }
-        } else {
-          // S is in registers: hand the buffer back so that the next chunk's QK^T runs under the arithmetic below
-          tc::tc_fence_before();
-          __syncwarp();
-          if (lane == 0) tc::mbar_arrive(&ctl.s_taken[grp]);
-        }
         if (!unmasked) {
           const int lim = vis - hf * 32;
 #pragma unroll
@@ -749,7 +742,7 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
               // the first half of this chunk's P was formed against the old reference: bring it along
               uint32_t ph[16];
               tc::tmem_wait_st();
-              tc::tmem_ld16(p_addr + pb * 32, ph);
+              tc::tmem_ld16(sp_addr, ph);
               tc::tmem_wait_ld();
 #pragma unroll
               for (int i = 0; i < 16; ++i) {
@@ -757,7 +750,7 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
                 const float2 f = __bfloat1622float2(v);
                 ph[i] = tc::pack_bf16(f.x * factor, f.y * factor);
               }
-              tc::tmem_st16(p_addr + pb * 32, ph);
+              tc::tmem_st16(sp_addr, ph);
             }
           }
           sub = ref == -INFINITY ? 0.f : ref;
@@ -771,26 +764,16 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
           r[u >> 1] = tc::pack_bf16(p0, p1);
         }
         if (grp == 0) mass += sum; else ell += sum;
-        tc::tmem_st16(p_addr + pb * 32 + hf * 16, *reinterpret_cast<uint32_t(*)[16]>(&r[0]));
+        tc::tmem_st16(sp_addr + hf * 16, *reinterpret_cast<uint32_t(*)[16]>(&r[0]));
       }
       if (!ok) break;
-      pending = true;
-      if (ci - c_lo < kSlots / 2) {
-        // while the pipeline fills (the first chunks hold the whole ring) latency counts: announce P at once, so
-        // that its PV retires and the ring slots are handed to the gathers as early as possible
-        tc::tmem_wait_st();
-        tc::tc_fence_before();
-        __syncwarp();
-        if (lane == 0) tc::mbar_arrive(&ctl.p_full[grp][pb]);
-        pending = false;
-      }
-      if (gt == 0) TC_TRACE(2 + grp, ci, 2);
-    }
-    if (ok && pending) {   // the last chunk's P
+      // P is announced at once: its PV MMAs free both the ring slot (for the gathers) and this S buffer (for the
+      // QK^T of the chunk after the next), and both are on the critical path
       tc::tmem_wait_st();
       tc::tc_fence_before();
       __syncwarp();
-      if (lane == 0) tc::mbar_arrive(&ctl.p_full[grp][(g0 + (c_hi - c_lo) - 1) & 1]);
+      if (lane == 0) tc::mbar_arrive(&ctl.p_full[grp][pb]);
+      if (gt == 0) TC_TRACE(2 + grp, ci, 2);
     }
     // ---- epilogue ------------------------------------------------------------------------------------
     // Each group finishes 64 of the 128 head-dim columns. Its half of the O_prev tile is staged in the group's

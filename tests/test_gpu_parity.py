@@ -229,8 +229,12 @@ def test_loop_attention_stage_isolated(env, case, rows, split):
     outputs and log-normalisers rounded to storage precision; the store is bit-exact anyway).  rows: the columns
     active in the loop come from the rows the quantization kernel materialized, or (without that workspace) are
     rebuilt from the residual streams inside the attention kernel."""
-    B, P, ctx = env
     w, x, ref = case
+    run_stage_isolated(env, w, x, ref, rows, split)
+
+
+def run_stage_isolated(env, w, x, ref, rows, split):
+    B, P, ctx = env
     st = P.LayerState(ctx, w, split=split)
     st.k_base, st.v_base = to_dev(x.K[0], w), to_dev(x.V[0], w)
     lse = ref["dense"]["lse"].astype(np.float32).copy()
@@ -262,6 +266,34 @@ def test_loop_attention_stage_isolated(env, case, rows, split):
         lse[:, act] = np.where(ok, rec["lse_rows"], lse[:, act]).astype(np.float32)
         q_prev_full = q_prev_full.copy()
         q_prev_full[act] = x.Q[r - 1][act]
+
+
+@ROWS
+def test_loop_attention_with_logits_far_apart(env, rows, split):
+    """Queries scaled by 16: ordinary logits spread over tens of nats and those of the heavy key rows over more than a
+    hundred, so that for most rows a later half-chunk's maximum beats the running reference of the new term by more
+    than the rescale threshold (60 in log2 units = 41.6 nats): the accumulator rows and the half of P already
+    written are rescaled, in the first as well as in the second half of a chunk.  One loop, so the old term's
+    probabilities stay below one and the outputs O(1)."""
+    w = small_bf16(L=1500, H=2, R=2)
+    x = workloads.make_layer_inputs(w, seed=7)
+    x.Q = [workloads.round_to_bf16(q * np.float32(16.0)) for q in x.Q]
+    ref = fo.LayerOracle(w.L, w.n_heads, w.head_dim, w.q_block, w.bits, w.group, w.eps, w.sm_scale,
+                         storage=w.dtype).run(x.G, x.Q, x.K, x.V, [w.k_tokens], [w.col_budget])
+    # the premise, on the oracle's own sets: new-loop logits of a row against its selected columns
+    rec, act = ref["loops"][0], ref["loops"][0]["active"]
+    far = total = 0
+    for (h, b), S in rec["col_sets"].items():
+        rows_b = act[(act // w.q_block) == b]
+        if len(S) < 64 or len(rows_b) == 0:
+            continue
+        s_new = (x.Q[1][rows_b, h].astype(np.float64) @ x.K[1][np.asarray(S), h].astype(np.float64).T) * w.sm_scale
+        s_new = np.where(np.asarray(S)[None, :] <= rows_b[:, None], s_new, -np.inf)
+        first32 = s_new[:, :32].max(axis=1)
+        far += int(np.sum(np.isfinite(first32) & (s_new.max(axis=1) - first32 > 2 * 41.6)))
+        total += len(rows_b)
+    assert far > total // 4, (far, total)
+    run_stage_isolated(env, w, x, ref, rows, split)
 
 
 def test_chained_layer_all_on_gpu(env, case):

@@ -6,7 +6,7 @@
  *   (1) cross-loop token scoring and top-k token selection        (Section 4.1, Appendix D.1, Eq. 5)
  *   (2) column-sparse attention replacement                       (Section 4.2, Appendix D.2, Eq. 6-7)
  *   (3) quantization of the cross-loop K/V residuals              (Section 4.3, Appendix D.3, Eq. 8)
- *   (4) dequantize-and-add reconstruction of K/V inside attention (Section 4.3 "at read time", App. G)
+ *   (4) dequantize-and-add reconstruction of K/V inside attention (Section 4.3, last paragraph; App. G)
  * plus the dense source loop that produces the statistics loop 2 starts from (Eq. 2, Eq. 6 with m_C = 1).
  *
  * Conventions
@@ -124,7 +124,7 @@ FL_API int fl_select_tokens(fl_ctx* ctx, const fl_shape* shape, int loop_r, cons
                      const int32_t* cand, int32_t n_cand, int32_t k, float* scores, int32_t* active_idx,
                      int32_t* slot_of_pos, int32_t* status, void* stream);
 
-/* Active-row execution (Appendix G, "sparse execution over active tokens"):
+/* Active-row execution (Appendix G, the item on executing only the active tokens):
  * gather: dst[t, :] = src[idx[t], :];  scatter: dst[idx[t], :] = src[t, :], other rows untouched.
  * row_bytes must be a positive multiple of 16; idx ascending without repeats; n >= 0. */
 FL_API int fl_gather_rows(fl_ctx* ctx, const void* src, const int32_t* idx, int32_t n, int64_t row_bytes, void* dst,
@@ -218,13 +218,19 @@ FL_API int fl_loop_attention_indexed(fl_ctx* ctx, const fl_shape* shape, int loo
                               float* col_scores_next, int32_t* status, void* stream);
 
 /* fl_loop_attention_indexed with the workspace of its last-wave split (see fl_set_workspace) taken from a fixed array
- * that is part of the library's device image, for callers that cannot lend device memory; the context's own workspace,
- * if any, is ignored by this call. The paper has no counterpart. The call allocates and frees nothing: the array's
- * address is looked up once per device, and the arrival counters at its head are cleared on `stream` before the launch.
+ * that is part of the library's device image, for callers that cannot lend device memory (code that runs where
+ * cudaMalloc is off limits: inside a region whose memory was budgeted up front, or under an allocator the caller does
+ * not control); the context's own workspace, if any, is ignored by this call. The paper has no counterpart. The call
+ * allocates and frees nothing. The array is 19.6 MB and every device that loads the library holds its own copy until
+ * the process exits, whether this entry point is used or not. Its address is looked up on the first call per device
+ * (cudaGetSymbolAddress, which answers for the CURRENT device: that call, like every later one, must be made with the
+ * context's device current, else FL_ERR_CUDA and nothing is cached or launched); make that first call before any
+ * stream capture. The arrival counters at the head of the array are cleared on `stream` before each launch, after the
+ * arguments have passed the same host checks as fl_loop_attention_indexed (a rejected call enqueues nothing).
  * The array holds the partial results of at most 74 split problems (half of a B200's SMs); a shape whose split needs
- * more returns FL_ERR_WORKSPACE before anything is launched. There is one array per device: two of these calls that
- * may overlap in time (different streams or contexts on one device) race on it and must be serialised by the caller.
- * Arguments, results and other errors as fl_loop_attention_indexed. */
+ * more returns FL_ERR_WORKSPACE before anything is launched. There is one array per device and it keeps the last
+ * call's contents: two of these calls that may overlap in time (different streams or contexts on one device) race on
+ * it and must be serialised by the caller. Arguments, results and other errors as fl_loop_attention_indexed. */
 FL_API int fl_loop_attention_indexed_static(fl_ctx* ctx, const fl_shape* shape, int loop_r, const void* q_new,
                                      const void* q_store_in, void* q_store_out, const int32_t* active_idx,
                                      int32_t n_active, const fl_kv_store* store, const int32_t* col_idx,

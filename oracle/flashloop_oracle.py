@@ -18,8 +18,9 @@ paper's H^(r-1)):
 Functions and the passage each one follows:
   token_scores, select_tokens      Appendix D.1 (token selection equation)
   topk_ascending                   the TopK of Appendix D.1 / D.2 with a total order
-  dense_loop_attention             Section 3.2 (attention equation) + Appendix D.2
-                                   ("a dense source loop uses all causal keys, m_C = 1")
+  dense_loop_attention             Section 3.2 (attention equation) + Appendix D.2 (the
+                                   dense-source case: every causal key is a candidate and
+                                   the cached mass is one)
   select_columns                   Appendix D.2 (column selection equation)
   sparse_loop_attention            Appendix D.2 (attention replacement equation)
   quantize_groups, dequantize_groups, pack_codes, unpack_codes
@@ -288,9 +289,10 @@ def sparse_loop_attention(q_new, khat_new, vhat_new, vhat_old, o_prev, active, c
                   (zero where the column is not causal); rows must contain the block's active rows.
     kv_round  : optional rounding applied to the reconstructed K/V rows when attention consumes them.
                 The chain Xhat itself stays binary32 (the codec needs it exact); with bf16 storage the
-                reconstructed cache that attention reads is a BF16 KV cache (Appendix G: the engine runs on
-                BF16 activations and reads the packed streams "avoiding explicit reconstruction of a full BF16
-                KV cache"), so its rows are bf16 values: kv_round = round_bf16. None for binary32 storage.
+                reconstructed cache that attention reads is a BF16 KV cache (Appendix G, the items on the
+                activation type and on the kernels that consume the packed streams without first writing a
+                full-precision cache), so its rows are bf16 values: kv_round = round_bf16. None for binary32
+                storage.
     Returns dict: O [n,H,dh] fp64, mass {(h,b): m_i per active row}, probs {(h,b): (rows, P_new)},
                   col_scores {(h,b): sum over rows of P_new, per column of S},
                   lse [H, n] fp64: the one-number summary of each row's cached probabilities,
@@ -370,8 +372,8 @@ def payload_bytes_per_row(d: int, bits: int, group: int, elem_bytes: int = 2) ->
 def kv_bytes_per_token_layer(L, d, n_active_per_loop, bits, group, n_layers, elem_bytes=2):
     """(flashloop, dense) KV bytes per token per layer.
 
-    Dense looped cache: one K and one V row per loop (Section 3: "a separate pair of keys and
-    values is stored for each loop").  FlashLoop here: bf16 loop-1 base, per-loop payloads for active
+    Dense looped cache: one K and one V row per token and per loop (Section 3, first paragraph:
+    every loop keeps its own keys and values).  FlashLoop here: bf16 loop-1 base, per-loop payloads for active
     rows only, plus each loop's int32 slot map [L] and index list [n_r], shared by all layers.
     n_active_per_loop lists n_r for r = 2..R.
     """

@@ -12,6 +12,9 @@ int fl_launch_loop_attn_tc(fl_ctx* ctx, const fl_shape* s, int loop_r, const voi
                            const int32_t* col_cnt, int c, const float* lse_prev, float* lse_out, const void* o_prev,
                            void* o_out, int indexed, void* q_store, int32_t* status, cudaStream_t st);
 
+// whether the tensor-path kernel has a build for this request (storage type, head dimension, column budget, shared memory)
+bool fl_loop_attn_tc_covers(const fl_ctx* ctx, const fl_shape* s, int c);
+
 namespace {
 
 struct LoopAttnArgs {
@@ -265,12 +268,15 @@ extern "C" int fl_loop_attention(fl_ctx* ctx, const fl_shape* shape, int loop_r,
                                    col_scores_next, st);
 }
 
-extern "C" int fl_loop_attention_indexed(fl_ctx* ctx, const fl_shape* shape, int loop_r, const void* q_new,
-                                         const void* q_store_in, void* q_store_out, const int32_t* active_idx,
-                                         int32_t n_active, const fl_kv_store* store, const int32_t* col_idx,
-                                         const int32_t* col_cnt, int32_t c, const float* lse_in, float* lse_out,
-                                         const void* o_store_in, void* o_store_out, float* col_scores_next,
-                                         int32_t* status, void* stream) {
+// Host-side checks of the position-indexed form, shared with the entry point that brings its own scratch.
+// Returns FL_OK with *launch = 1 when a kernel is to be launched, FL_OK with *launch = 0 when the call has nothing
+// to compute (no active rows), or the error every caller reports before anything is enqueued.
+int fl_attn_indexed_check(const fl_ctx* ctx, const fl_shape* shape, int loop_r, const void* q_new,
+                          const void* q_store_in, const void* q_store_out, const int32_t* active_idx, int32_t n_active,
+                          const fl_kv_store* store, const int32_t* col_idx, const int32_t* col_cnt, int32_t c,
+                          const float* lse_in, const float* lse_out, const void* o_store_in, const void* o_store_out,
+                          int* launch) {
+  *launch = 0;
   FL_REQUIRE(ctx != nullptr);
   int rc = fl_check_shape(shape);
   if (rc != FL_OK) return rc;
@@ -280,18 +286,34 @@ extern "C" int fl_loop_attention_indexed(fl_ctx* ctx, const fl_shape* shape, int
   if (rc != FL_OK) return rc;
   FL_REQUIRE(col_idx != nullptr && col_cnt != nullptr && lse_in != nullptr && lse_out != nullptr);
   FL_REQUIRE(shape->n_heads <= 65535 && fl_n_blocks(shape) <= 65535);
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (n_active == 0) {
-    if (col_scores_next != nullptr)
-      FL_CHECK_CUDA(cudaMemsetAsync(col_scores_next, 0,
-                                    sizeof(float) * (size_t)shape->n_heads * fl_n_blocks(shape) * c, st));
-    return FL_OK;
-  }
+  if (n_active == 0) return FL_OK;
   FL_REQUIRE(q_new != nullptr && q_store_in != nullptr && o_store_in != nullptr && o_store_out != nullptr &&
              active_idx != nullptr);
   FL_REQUIRE(fl_aligned16(q_new) && fl_aligned16(q_store_in) && fl_aligned16(q_store_out) &&
              fl_aligned16(o_store_in) && fl_aligned16(o_store_out));
   if (ctx->force_simt) return FL_ERR_UNSUPPORTED;
+  if (!fl_loop_attn_tc_covers(ctx, shape, c)) return FL_ERR_UNSUPPORTED;
+  *launch = 1;
+  return FL_OK;
+}
+
+extern "C" int fl_loop_attention_indexed(fl_ctx* ctx, const fl_shape* shape, int loop_r, const void* q_new,
+                                         const void* q_store_in, void* q_store_out, const int32_t* active_idx,
+                                         int32_t n_active, const fl_kv_store* store, const int32_t* col_idx,
+                                         const int32_t* col_cnt, int32_t c, const float* lse_in, float* lse_out,
+                                         const void* o_store_in, void* o_store_out, float* col_scores_next,
+                                         int32_t* status, void* stream) {
+  int launch = 0;
+  int rc = fl_attn_indexed_check(ctx, shape, loop_r, q_new, q_store_in, q_store_out, active_idx, n_active, store,
+                                 col_idx, col_cnt, c, lse_in, lse_out, o_store_in, o_store_out, &launch);
+  if (rc != FL_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (!launch) {
+    if (col_scores_next != nullptr)
+      FL_CHECK_CUDA(cudaMemsetAsync(col_scores_next, 0,
+                                    sizeof(float) * (size_t)shape->n_heads * fl_n_blocks(shape) * c, st));
+    return FL_OK;
+  }
   rc = fl_launch_loop_attn_tc(ctx, shape, loop_r, q_new, q_store_in, active_idx, n_active, store, col_idx, col_cnt, c,
                               lse_in, lse_out, o_store_in, o_store_out, 1, q_store_out, status, st);
   if (rc != FL_OK || col_scores_next == nullptr) return rc;

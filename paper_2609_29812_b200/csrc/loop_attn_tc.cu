@@ -71,22 +71,6 @@ constexpr float kRescaleThreshold = 60.f;   // in log2 units: rescale only when 
 static_assert(3 * kMaxCols * 4 <= kSlots * kSlotBytes, "prologue staging must fit in the ring");
 static_assert(kAccNew == kAccOld + kDH, "the two accumulators are adjacent in tensor memory");
 
-// Optional device-side timeline for tuning (compile with -DFL_TC_TRACE): the CTA (block 1, head 0) writes
-// clock64() stamps into the buffer passed as `status` (the traced CTA can be chosen with -DFL_TC_TRACE_X/_Y): trace[(role * 64 + chunk) * 4 + event].
-#ifdef FL_TC_TRACE
-#ifndef FL_TC_TRACE_X
-#define FL_TC_TRACE_X 1
-#define FL_TC_TRACE_Y 0
-#endif
-#define TC_TRACE(role, chunk, ev)                                                                      \
-  do {                                                                                                 \
-    if (b == FL_TC_TRACE_X && h == FL_TC_TRACE_Y && part == 0 && (chunk) < 64 && a.status != nullptr) \
-      reinterpret_cast<long long*>(a.status)[((role) * 64 + (chunk)) * 4 + (ev)] = clock64();          \
-  } while (0)
-#else
-#define TC_TRACE(role, chunk, ev) do { } while (0)
-#endif
-
 struct alignas(64) TcArgs {
   CUtensorMap k_map, v_map;          // row-gather maps of the K / V base ([L, d] bf16, box 64 x 1, 128B swizzle)
   CUtensorMap k_prev_map, k_cur_map;  // use_rows: row-gather maps of the loop's materialized rows ([n_active, d] bf16):
@@ -284,7 +268,6 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
   const size_t prob = (size_t)h * a.nb + b;
   const int32_t* cols = a.col_idx + prob * a.c;
   const int cnt = min(__ldg(a.col_cnt + prob), kMaxCols);
-  if (tid == 0) TC_TRACE(0, 60, 0);
 
   if (tid == 0) {
     for (int s = 0; s < kSlots; ++s) {
@@ -442,7 +425,6 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
     }
   }
   __syncthreads();
-  if (tid == 0) TC_TRACE(0, 60, 1);
   int g = 0;    // chunks issued so far (all tiles): S / P buffer = g & 1, one phase of its barriers per use
   int fill = 0; // ring slots filled so far: slot = fill % kSlots, phase = (fill / kSlots) & 1
   uint32_t dirty_par_cta = 0;  // per-slot phase parity of the patched[] barriers (they only see dirty chunks)
@@ -476,7 +458,6 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
       tc::tma_gather4(q_old_tile + kM * 128 + lane * 512, &a.q_old_map, &ctl.q_full, h * kDH + 64, y[0], y[1], y[2], y[3]);
     }
   }
-  if (tid == 0) TC_TRACE(0, 60, 2);
 
   if (warp >= kTmaWarp) {
     // ========================================== TMA + patch ==========================================
@@ -506,7 +487,6 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
       for (int k = 0; k < n_slots && ok; ++k)
         if (f + k >= kSlots) ok = warp_wait(&ctl.done[(f + k) % kSlots], (((f + k) / kSlots) - 1) & 1, abort_flag);
       if (!ok) break;
-      if (tid == kTmaWarp * 32) TC_TRACE(0, ci, 0);
       if (lane == 0)
         for (int k = 0; k < n_slots; ++k) tc::mbar_arrive_expect_tx(&ctl.landed[(f + k) % kSlots], my_reqs * 512);
       __syncwarp();
@@ -531,7 +511,6 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
                           &ctl.landed[slot], h * kDH + slab * 64, y[0], y[1], y[2], y[3]);
         }
       }
-      if (tid == kTmaWarp * 32) TC_TRACE(0, ci, 1);
       if (dirty) {
         for (int k = 0; k < n_slots && ok; ++k)
           ok = warp_wait(&ctl.landed[(f + k) % kSlots], ((f + k) / kSlots) & 1, abort_flag);
@@ -602,7 +581,6 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
         if (ci < c_hi) {
           const ChunkInfo ck = chunk_info(ci, n_plain, n_patch);
           const int slot0 = f % kSlots, slot1 = (f + 1) % kSlots;
-          if (t == 0) TC_TRACE(1, ci, 0);
           if (ci == c_lo && !tc::mbar_wait(&ctl.q_full, tile & 1, abort_flag)) break;
           // a term reads one slot of the chunk only (the new term of a two-slot chunk the second): it starts on it
           // without waiting for the other
@@ -617,7 +595,6 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
           if (gc >= 2 && !tc::mbar_wait(&ctl.p_free[t][gc & 1], ((gc >> 1) - 1) & 1, abort_flag)) break;
           const uint32_t s_dst = s_base + (gc & 1) * kNC;
           tc::tc_fence_after();
-          if (t == 0) TC_TRACE(1, ci, 1);
           const uint32_t k_lo = k_lo0 + my_slot * (kSlotBytes >> 4);
 #define FL_QK(KK, ACC)                                                                                       \
   tc::mma_ss_lo<ACC>(s_dst, q_lo_w + ((((KK) >> 2) * (kM * 128) + ((KK)&3) * 32) >> 4), kq_hi,               \
@@ -629,14 +606,11 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
           qk_slot = slot0;
           qk_slot1 = ck.patch ? slot1 : -1;
           f += ck.patch ? 2 : 1;
-          if (t == 0) TC_TRACE(1, ci, 2);
         }
         if (ci > c_lo) {
           const int cj = ci - 1, gp = gc - 1, pb = gp & 1;
-          if (t == 0) TC_TRACE(4, cj, 0);
           if (!tc::mbar_wait(&ctl.p_full[t][pb], (gp >> 1) & 1, abort_flag)) break;
           tc::tc_fence_after();
-          if (t == 0) TC_TRACE(4, cj, 1);
           const uint32_t v_lo = v_lo0 + ((t && pv_slot1 >= 0) ? pv_slot1 : pv_slot) * (kSlotBytes >> 4);
           const uint32_t p_src = s_base + pb * kNC;
           const uint32_t acc0 = cj > c_lo ? 1u : 0u;       // the CTA's first chunk of the tile overwrites the accumulator
@@ -646,7 +620,6 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
           tc::mma_commit(&ctl.p_free[t][pb]);
           tc::mma_commit(&ctl.done[pv_slot]);
           if (pv_slot1 >= 0) tc::mma_commit(&ctl.done[pv_slot1]);
-          if (t == 0) TC_TRACE(4, cj, 2);
         }
         pv_slot = qk_slot;
         pv_slot1 = qk_slot1;
@@ -672,10 +645,8 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
     bool ok = true;
     for (int ci = c_lo; ci < c_hi; ++ci) {
       const int gc = g0 + ci - c_lo, pb = gc & 1, n_use = gc >> 1;
-      if (gt == 0) TC_TRACE(2 + grp, ci, 0);
       if (!warp_wait(&ctl.s_full[grp][pb], n_use & 1, abort_flag)) { ok = false; break; }
       tc::tc_fence_after();
-      if (gt == 0) TC_TRACE(2 + grp, ci, 1);
       // rows of a warp that lie at or after every column of the chunk need no causal mask; rows beyond the
       // tile's last (their results are never stored) must not force the masked path
       const bool unmasked = __all_sync(0xffffffffu, !row_ok || ctl.chunk_last[ci] <= pos);
@@ -773,7 +744,6 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
       tc::tc_fence_before();
       __syncwarp();
       if (lane == 0) tc::mbar_arrive(&ctl.p_full[grp][pb]);
-      if (gt == 0) TC_TRACE(2 + grp, ci, 2);
     }
     // ---- epilogue ------------------------------------------------------------------------------------
     // Each group finishes 64 of the 128 head-dim columns. Its half of the O_prev tile is staged in the group's
@@ -792,12 +762,10 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
     tc::cp_async_commit();
     if (ok) ok = warp_wait(&ctl.acc_done, tile & 1, abort_flag);
     tc::tc_fence_after();
-    if (gt == 0) TC_TRACE(2 + grp, 61, 0);
     if (grp == 0) ctl.mass[row] = mass;
     else { ctl.ell[row] = ell; ctl.ref[row] = ref; }
     tc::cp_async_wait<0>();
     asm volatile("bar.sync 1, 256;" ::: "memory");
-    if (gt == 0) TC_TRACE(2 + grp, 61, 1);
     float m_i = ctl.mass[row], l_i = ctl.ell[row], ref_i = ctl.ref[row];
     const bool acc_valid = ok && c_hi > c_lo;             // warp-uniform: the tensor-memory reads below are collective
     // ---- split problems: the CTA of the pair that finishes first leaves its partial result in the workspace, the
@@ -809,7 +777,6 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
       // first one adds 16 once its partial result is in the workspace; the second resets it for the next launch
       if (tid == 0) ctl.merge_role = atomicAdd(a.part_cnt + pair, 1) & 1;
       asm volatile("bar.sync 1, 256;" ::: "memory");
-      if (gt == 0) TC_TRACE(2 + grp, 62, 0);
       if (ctl.merge_role == 0) {
         float* mine = a.part_acc + ((size_t)pair * 2 + part) * kPartFloats;
 #pragma unroll 1
@@ -831,7 +798,6 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
         __threadfence();
         asm volatile("bar.sync 1, 256;" ::: "memory");
         if (tid == 0) atomicAdd(a.part_cnt + pair, 16);
-        if (gt == 0) TC_TRACE(2 + grp, 62, 1);
       } else {
         // the other CTA came first and is writing its partial result (it is resident and past its main loop: the
         // wait is short, and bounded like every other)
@@ -845,7 +811,6 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
           else a.part_cnt[pair] = 0;                                // ready for the next launch
         }
         asm volatile("bar.sync 1, 256;" ::: "memory");
-        if (gt == 0) TC_TRACE(2 + grp, 62, 1);
         if (ctl.merge_role == 1) {   // CTA-uniform
           __threadfence();
           const float* theirs = a.part_acc + ((size_t)pair * 2 + (part ^ 1)) * kPartFloats;
@@ -867,7 +832,6 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
           ref_i = ref_t;
           tc::cp_async_wait<0>();
           asm volatile("bar.sync 1, 256;" ::: "memory");
-          if (gt == 0) TC_TRACE(2 + grp, 62, 2);
         }
       }
     }
@@ -903,7 +867,6 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
     if (grp == 1 && row_ok && writer)
       a.lse_out[(size_t)h * a.L + pos] = has ? (ref_i + log2f(l_i)) * kLn2 - logf(m_i) : lse2 * kLn2;
     asm volatile("bar.sync 1, 256;" ::: "memory");
-    if (gt == 0) TC_TRACE(2 + grp, 61, 2);
 #pragma unroll 1
     for (int k = 0; k < 8 && writer; ++k) {
       const int idx = k * 128 + gt, rr = idx >> 3, cc = idx & 7;
@@ -913,7 +876,6 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
             *reinterpret_cast<const uint4*>(stage + rr * 128 + ((cc ^ (rr & 7)) << 4));
       }
     }
-    if (gt == 0) TC_TRACE(2 + grp, 61, 3);
   }
   if (INDEXED && split && a.q_store != nullptr) {   // CTA-uniform
     // Both halves of a split problem gathered the previous loop's Q rows from the store; the new rows may take their
@@ -961,9 +923,7 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
     tc::tc_fence_after();
     tc::tmem_dealloc(tmem, 512);
   }
-#ifndef FL_TC_TRACE
   if (tid == 0 && ctl.abort_flag && a.status != nullptr) atomicExch(a.status, (int)FL_ERR_TIMEOUT);
-#endif
 }
 
 }  // namespace
@@ -999,6 +959,11 @@ extern "C" int fl_set_workspace(fl_ctx* ctx, void* workspace, int64_t bytes, voi
   return FL_OK;
 }
 
+bool fl_loop_attn_tc_covers(const fl_ctx* ctx, const fl_shape* s, int c) {
+  return s->dtype == FL_BF16 && s->head_dim == kDH && c <= kMaxCols && (size_t)ctx->max_smem_optin >= kTcSmemBytes &&
+         ctx->encode_tiled != nullptr && ctx->tmaps != nullptr;
+}
+
 // Returns FL_ERR_UNSUPPORTED when the tensor path does not cover the request (caller falls back to the
 // SIMT kernel, which is also CUDA). indexed != 0: q_old, o_prev and o_out are position-indexed stores [L, d] and
 // q_store (may be null) receives the new Q rows.
@@ -1006,8 +971,7 @@ int fl_launch_loop_attn_tc(fl_ctx* ctx, const fl_shape* s, int loop_r, const voi
                            const int32_t* active_idx, int n_active, const fl_kv_store* store, const int32_t* col_idx,
                            const int32_t* col_cnt, int c, const float* lse_prev, float* lse_out, const void* o_prev,
                            void* o_out, int indexed, void* q_store, int32_t* status, cudaStream_t st) {
-  if (s->dtype != FL_BF16 || s->head_dim != kDH || c > kMaxCols) return FL_ERR_UNSUPPORTED;
-  if ((size_t)ctx->max_smem_optin < kTcSmemBytes) return FL_ERR_UNSUPPORTED;
+  if (!fl_loop_attn_tc_covers(ctx, s, c)) return FL_ERR_UNSUPPORTED;
   TcArgs a{};
   const int64_t d_row = (int64_t)s->n_heads * s->head_dim;
   if (!fl_tile_tmap(ctx, store->k_base, s->L, d_row, 1, &a.k_map) ||

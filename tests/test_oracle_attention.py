@@ -166,6 +166,11 @@ def test_rational_closed_form_per_position():
         # the reconstructed keys are kept in binary32, so log(weights) carry a 2^-24 rounding
         assert res["O"][i, 0, 0] == pytest.approx(float(o2), rel=1e-6, abs=1e-7)
         assert res["mass"][(0, i)][0] == pytest.approx(float(m), rel=1e-12)      # loop-1 keys are fp64
+        # the row's one-number summary: p2_j = exp(logit_j - lse) with logit_j = log w2_j, hence
+        # lse = log(sum_S w2) - log m  (a sign slip in either term moves it by 2 log m or 2 log tot2)
+        assert res["lse"][0, i] == pytest.approx(np.log(float(tot2)) - np.log(float(m)), rel=1e-6, abs=1e-6)
+        for u, j in enumerate(S):
+            assert np.exp(np.log(w2[j]) - res["lse"][0, i]) == pytest.approx(float(p2[j]), rel=1e-6)
 
 
 def test_uniform_attention_closed_form_blocks():
@@ -239,3 +244,44 @@ def test_layer_oracle_pruning_is_nested_and_error_shrinks_with_budget():
         dense = fo.dense_loop_attention(x.Q[1], k2, v2, w.sm_scale, 64)["O"]
         errs.append(np.linalg.norm(o["loops"][0]["O_full"] - dense) / np.linalg.norm(dense))
     assert errs[0] > errs[1] > errs[2] and errs[2] < 1e-9
+
+
+def test_kv_round_is_applied_to_all_three_operands_values_by_hand():
+    """One head, dh = 1, q = 1, scale = 1, two selected columns, one query: every number of the replacement equation
+    can be written down.  K and V are chosen so that bf16 rounding moves each of the three operands the attention
+    reads (Khat_new, Vhat_old, Vhat_new) by an amount that shows in the output; the expected value is computed from
+    operands rounded with torch's own bfloat16 conversion (a library routine), not with the oracle's helper.
+    Leaving any one operand unrounded fails the comparison."""
+    torch = pytest.importorskip("torch")
+    bf = lambda a: torch.tensor(np.asarray(a, dtype=np.float32)).to(torch.bfloat16).double().numpy()
+    L, S = 3, np.array([0, 1])
+    k_new = np.array([0.3, 1.7, 0.0], dtype=np.float32).reshape(L, 1, 1)          # bf16: 0.30078125, 1.703125
+    v_old = np.array([1.0 + 2.0 ** -9, -2.0 - 2.0 ** -8, 0.0], dtype=np.float32).reshape(L, 1, 1)
+    v_new = np.array([3.0 + 2.0 ** -8, 5.0 + 2.0 ** -7, 0.0], dtype=np.float32).reshape(L, 1, 1)
+    for arr in (k_new, v_old, v_new):
+        assert np.all(bf(arr)[:2] != arr[:2].astype(np.float64))                    # rounding moves every operand
+    p_old = np.array([[0.25, 0.5]])                                                # cached loop r-1 probabilities
+    o_prev = np.array([[[0.75]]])
+    active = np.array([2])
+    sets = {(0, 0): S}
+    cache = {(0, 0): (active, p_old)}
+    q = np.ones((1, 1, 1))
+    got = {}
+    for name, rd in (("rounded", fo.round_bf16), ("plain", None)):
+        got[name] = fo.sparse_loop_attention(q, k_new, v_new, v_old, o_prev, active, sets, cache, 1.0, q_block=4,
+                                             kv_round=rd)
+    m = 0.75
+    def expect(kn, vo, vn):
+        e = np.exp(kn[:2, 0, 0]); p_new = m * e / e.sum()
+        return 0.75 - p_old[0] @ vo[:2, 0, 0] + p_new @ vn[:2, 0, 0], np.log(e.sum()) - np.log(m)
+    want, want_lse = expect(bf(k_new), bf(v_old), bf(v_new))
+    assert got["rounded"]["O"][0, 0, 0] == pytest.approx(want, rel=1e-13)
+    assert got["rounded"]["lse"][0, 0] == pytest.approx(want_lse, rel=1e-13)
+    plain, _ = expect(k_new.astype(np.float64), v_old.astype(np.float64), v_new.astype(np.float64))
+    assert got["plain"]["O"][0, 0, 0] == pytest.approx(plain, rel=1e-13)
+    # each operand on its own: an implementation that forgot one of the three roundings lands on one of these
+    for miss in range(3):
+        ops = [bf(k_new), bf(v_old), bf(v_new)]
+        ops[miss] = (k_new, v_old, v_new)[miss].astype(np.float64)
+        wrong, _ = expect(*ops)
+        assert abs(wrong - want) > 1e-4 and got["rounded"]["O"][0, 0, 0] != pytest.approx(wrong, rel=1e-6)

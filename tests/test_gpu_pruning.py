@@ -1,0 +1,163 @@
+"""GPU parity with DECAYING budgets: the token set shrinks from loop to loop (nested, Appendix D.1) and the column
+set of every (head, block) is pruned inside the previous set (Appendix D.2: a sparse source loop offers its own
+selected columns as candidates, with the block sums of its new probabilities as scores).  This reaches what constant
+budgets never do: column selection over a candidate list, columns that carry a payload from an earlier loop only,
+and an old term whose columns are a strict subset of the previous loop's."""
+import dataclasses
+
+import numpy as np
+import pytest
+
+from oracle import flashloop_oracle as fo
+from paper_2609_29812_b200 import workloads
+from helpers import assert_attn_close, assert_selection_matches, storage_round, to_dev, to_np
+from test_gpu_parity import oracle_selection, sets_to_arrays, small_bf16
+
+pytestmark = pytest.mark.gpu
+torch = pytest.importorskip("torch")
+
+K_FRACS = (0.25, 0.12, 0.06)
+C_COLS = (160, 96, 48)
+
+
+@pytest.fixture(scope="module")
+def env():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2609_29812_b200 import binding, pipeline
+    ctx = binding.Context(0)
+    yield binding, pipeline, ctx
+    ctx.close()
+
+
+@pytest.fixture(scope="module")
+def decaying_case():
+    w = dataclasses.replace(small_bf16(L=2000, H=2, R=4), changed_fracs=(0.30, 0.15, 0.08))
+    x = workloads.make_layer_inputs(w, seed=13)
+    k_tok = [int(np.floor(f * w.L + 0.5)) for f in K_FRACS]
+    orc = fo.LayerOracle(w.L, w.n_heads, w.head_dim, w.q_block, w.bits, w.group, w.eps, w.sm_scale, storage=w.dtype)
+    ref = orc.run(x.G, x.Q, x.K, x.V, k_tok, list(C_COLS))
+    # the premise: sets really shrink, and loop 3+ sees columns whose only payload is from an earlier loop
+    acts = ref["active"]
+    assert len(acts[0]) > len(acts[1]) > len(acts[2])
+    stale = 0
+    for (h, b), S in ref["loops"][1]["col_sets"].items():
+        stale += int(np.sum(np.isin(S, acts[0]) & ~np.isin(S, acts[1])))
+    assert stale > 0
+    return w, x, ref, k_tok
+
+
+@pytest.mark.parametrize("rows", [True, False], ids=["materialized_rows", "rebuilt_in_kernel"])
+def test_stage_isolated_with_shrinking_token_and_column_sets(env, decaying_case, rows):
+    """Every loop is fed the oracle's upstream state; its attention output, log-normalisers and next-loop column
+    scores are checked, then fl_select_columns prunes the set over the candidate list: exact on the kernel's own
+    scores and on the oracle's, near-tie protocol against the oracle's fp64 scores."""
+    B, P, ctx = env
+    w, x, ref, k_tok = decaying_case
+    st = P.LayerState(ctx, w)
+    st.k_base, st.v_base = to_dev(x.K[0], w), to_dev(x.V[0], w)
+    lse = ref["dense"]["lse"].astype(np.float32).copy()
+    q_prev_full = x.Q[0]
+    for r in range(2, w.n_loops + 1):
+        rec = ref["loops"][r - 2]
+        act = rec["active"]
+        c_r = C_COLS[r - 2]
+        sel = oracle_selection(P, w, ref, r)
+        st.alloc_stream(sel, rows=rows)
+        st.quantize(r, to_dev(x.K[r - 1][act], w), to_dev(x.V[r - 1][act], w), sel)
+        idx, cnt = sets_to_arrays(w, st.nb, rec["col_sets"], c_r)
+        st.col_idx, st.col_cnt, st.c = torch.from_numpy(idx).cuda(), torch.from_numpy(cnt).cuda(), c_r
+        st.lse = torch.from_numpy(lse).cuda()
+        o_prev = to_dev(storage_round(rec["O_prev_rows"], w), w)
+        o_out = torch.empty_like(o_prev)
+        csn = torch.zeros(w.n_heads, st.nb, c_r, dtype=torch.float32, device="cuda")
+        st.attention(r, to_dev(x.Q[r - 1][act], w), to_dev(q_prev_full[act], w), o_prev, o_out, sel, csn)
+        st.check_status()
+        assert_attn_close(to_np(o_out), rec["O_rows"], f"loop {r} O rows (decaying budgets)")
+        got_lse = to_np(st.lse)[:, act]
+        ok = np.isfinite(rec["lse_rows"])
+        np.testing.assert_allclose(got_lse[ok], rec["lse_rows"][ok], rtol=0, atol=5e-3)
+        csn_np = to_np(csn)
+        for (h, b), s_ref in rec["col_scores_next"].items():
+            np.testing.assert_allclose(csn_np[h, b, : len(s_ref)], s_ref, rtol=2e-2, atol=2e-4)
+        if r < w.n_loops:
+            c_next = C_COLS[r - 1]
+            nxt = ref["loops"][r - 1]["col_sets"]
+            # (a) on the kernel's own scores: brute force with the total order
+            st.prune_columns(csn, c_next)
+            got_idx, got_cnt = to_np(st.col_idx), to_np(st.col_cnt)
+            n_diff = 0
+            for (h, b), S in rec["col_sets"].items():
+                k = min(c_next, len(S))
+                assert got_cnt[h, b] == k and np.all(got_idx[h, b, k:] == -1)
+                own = np.asarray(S)[fo.topk_ascending(csn_np[h, b, : len(S)], k)] if len(S) else np.zeros(0, int)
+                assert np.array_equal(got_idx[h, b, :k], own), (r, h, b)
+                if len(S):
+                    n_diff += assert_selection_matches(got_idx[h, b, :k], rec["col_scores_next"][(h, b)], S, c_next,
+                                                       f"pruned columns loop {r + 1} h{h} b{b}")
+            assert n_diff <= 0.02 * w.n_heads * st.nb * c_next
+            # (b) on the oracle's scores (binary32): the oracle's next set, bit for bit up to binary32 ties
+            s32 = np.zeros((w.n_heads, st.nb, c_r), dtype=np.float32)
+            for (h, b), s_ref in rec["col_scores_next"].items():
+                s32[h, b, : len(s_ref)] = s_ref
+            st.col_idx, st.col_cnt, st.c = torch.from_numpy(idx).cuda(), torch.from_numpy(cnt).cuda(), c_r
+            st.prune_columns(torch.from_numpy(s32).cuda(), c_next)
+            got_idx = to_np(st.col_idx)
+            for (h, b), S in rec["col_sets"].items():
+                k = min(c_next, len(S))
+                want = np.asarray(S)[fo.topk_ascending(s32[h, b, : len(S)], k)] if len(S) else np.zeros(0, int)
+                assert np.array_equal(got_idx[h, b, :k], want)
+                if len(S) and np.array_equal(want, nxt[(h, b)]):
+                    continue
+                if len(S):   # binary32 rounding of the scores made a tie the fp64 oracle does not have
+                    assert_selection_matches(want, rec["col_scores_next"][(h, b)], S, c_next, "binary32 tie")
+        lse = lse.copy()
+        lse[:, act] = np.where(ok, rec["lse_rows"], lse[:, act]).astype(np.float32)
+        q_prev_full = q_prev_full.copy()
+        q_prev_full[act] = x.Q[r - 1][act]
+
+
+@pytest.mark.parametrize("indexed", [False, True], ids=["compact_rows", "indexed_stores"])
+def test_chained_on_gpu_with_pruning(env, decaying_case, indexed):
+    """Everything on the GPU: token selection over the previous set, quantization, attention with next-loop column
+    scores, pruning.  Blocks whose column sets equal the oracle's through every loop so far (all of them unless a
+    near tie flips a column) are compared row by row."""
+    B, P, ctx = env
+    w, x, ref, k_tok = decaying_case
+    st = P.LayerState(ctx, w)
+    st.dense_loop(to_dev(x.Q[0], w), to_dev(x.K[0], w), to_dev(x.V[0], w))
+    st.select_columns_dense(C_COLS[0])
+    cand = None
+    clean = {key: True for key in ref["loops"][0]["col_sets"]}
+    tokens_equal = True
+    for r in range(2, w.n_loops + 1):
+        rec = ref["loops"][r - 2]
+        sel = P.select_tokens(ctx, st.shape, r, to_dev(x.G[r - 2], w), to_dev(x.G[r - 1], w), cand, k_tok[r - 2])
+        act = to_np(sel.active_idx).astype(np.int64)
+        cand_np = np.arange(w.L) if cand is None else to_np(cand).astype(np.int64)
+        if tokens_equal:
+            assert_selection_matches(act, ref["token_scores"][r - 2], cand_np, k_tok[r - 2], f"tokens loop {r}")
+        tokens_equal = tokens_equal and np.array_equal(act, rec["active"])
+        idx, cnt = to_np(st.col_idx), to_np(st.col_cnt)
+        for key, S in rec["col_sets"].items():
+            h, b = key
+            clean[key] = clean[key] and np.array_equal(idx[h, b, : cnt[h, b]], S)
+        o_rows, csn = st.sparse_loop(r, to_dev(x.Q[r - 1][act], w), to_dev(x.K[r - 1][act], w),
+                                     to_dev(x.V[r - 1][act], w), sel, want_col_scores_next=r < w.n_loops,
+                                     indexed=indexed)
+        st.check_status()
+        if tokens_equal:
+            o_np = to_np(o_rows)
+            blk = act // w.q_block
+            n_cmp = 0
+            for (h, b), is_clean in clean.items():
+                t_idx = np.nonzero(blk == b)[0]
+                if is_clean and len(t_idx):
+                    assert_attn_close(o_np[t_idx, h], rec["O_rows"][t_idx, h], f"chained loop {r} h{h} b{b}",
+                                      loops=r - 1)
+                    n_cmp += 1
+            assert n_cmp >= 0.8 * len(clean)
+        if r < w.n_loops:
+            st.prune_columns(csn, C_COLS[r - 1])
+        cand = sel.active_idx
+    assert sum(clean.values()) >= 0.8 * len(clean)

@@ -32,11 +32,26 @@ def attn_errors(got, ref):
     return rel, float(np.max(np.abs(got - ref))) if got.size else 0.0
 
 
-def assert_attn_close(got, ref, what="", loops=1):
-    """One loop: the stated tolerance.  `loops` chained loops: max-abs scales with the number of loops
-    (each adds a storage rounding of the carried output), relative L2 stays as stated."""
+ERROR_LOG = []   # (what, carried roundings, relative L2, max abs, max-abs bound) of every attention comparison of the session
+
+
+def half_ulp_storage(ref, bf16=True):
+    """Largest rounding error of one store of a value as large as max|ref| in the storage type."""
+    if not bf16:
+        return 0.0
+    mag = float(np.max(np.abs(ref))) if np.size(ref) else 0.0
+    return 0.0 if mag == 0.0 else 2.0 ** (np.floor(np.log2(mag)) - 8)
+
+
+def assert_attn_close(got, ref, what="", carried=0, bf16=True):
+    """Relative L2 <= 1e-2 and max-abs <= 3e-2 (the stated tolerance) when both sides start from the same stored
+    inputs.  `carried`: how many times the output carried into this comparison was rounded to the storage type on the
+    GPU side only (the oracle carries fp64 between loops): the max-abs bound grows by half a storage ulp of the
+    largest reference value per such rounding; the relative L2 bound stays as stated."""
     rel, mx = attn_errors(got, ref)
-    assert rel <= REL_L2_TOL and mx <= MAX_ABS_TOL * loops, f"{what}: rel L2 {rel:.3e}, max abs {mx:.3e}"
+    bound = MAX_ABS_TOL + carried * half_ulp_storage(ref, bf16)
+    ERROR_LOG.append((what, carried, float(rel), float(mx), float(bound)))
+    assert rel <= REL_L2_TOL and mx <= bound, f"{what}: rel L2 {rel:.3e}, max abs {mx:.3e} (bound {bound:.3e})"
     return rel, mx
 
 

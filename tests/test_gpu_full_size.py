@@ -12,7 +12,9 @@ from helpers import assert_attn_close, assert_selection_matches, to_np
 
 pytestmark = pytest.mark.gpu
 
-SAMPLES = [(0, 0), (3, 7), (9, 20), (15, 31)]     # (head, query block): first, middle and last blocks
+# (head, query block): first, early, middle and last blocks (every block of this workload holds 84-120 active rows,
+# i.e. one 128-row tile)
+SAMPLES = [(0, 0), (5, 1), (3, 7), (12, 13), (9, 20), (6, 26), (1, 30), (15, 31)]
 
 
 def test_full_size_layer_loops_2_and_3_sampled_against_oracle():
@@ -57,7 +59,9 @@ def test_full_size_layer_loops_2_and_3_sampled_against_oracle():
                       k_codes=to_np(st.k_streams[-1]["codes"]).reshape(len(act), w.n_heads, -1),
                       v_codes=to_np(st.v_streams[-1]["codes"]).reshape(len(act), w.n_heads, -1),
                       k_scale=to_np(st.k_streams[-1]["scale"]).view(np.uint16).reshape(len(act), w.n_heads, -1),
-                      k_zero=to_np(st.k_streams[-1]["zero"]).view(np.uint16).reshape(len(act), w.n_heads, -1))
+                      k_zero=to_np(st.k_streams[-1]["zero"]).view(np.uint16).reshape(len(act), w.n_heads, -1),
+                      v_scale=to_np(st.v_streams[-1]["scale"]).view(np.uint16).reshape(len(act), w.n_heads, -1),
+                      v_zero=to_np(st.v_streams[-1]["zero"]).view(np.uint16).reshape(len(act), w.n_heads, -1))
         cand = sel.active_idx
 
     # ---- the oracle, on its own, for sampled (head, block) pairs -------------------------------------------
@@ -90,6 +94,8 @@ def test_full_size_layer_loops_2_and_3_sampled_against_oracle():
             assert np.array_equal(g["v_codes"][:, h], vpay["packed"][:, 0]), (r, h, "V codes")
             assert np.array_equal(g["k_scale"][:, h], kpay["scale"][:, 0].view(np.uint16)), (r, h, "K scale")
             assert np.array_equal(g["k_zero"][:, h], kpay["zero"][:, 0].view(np.uint16)), (r, h, "K offset")
+            assert np.array_equal(g["v_scale"][:, h], vpay["scale"][:, 0].view(np.uint16)), (r, h, "V scale")
+            assert np.array_equal(g["v_zero"][:, h], vpay["zero"][:, 0].view(np.uint16)), (r, h, "V offset")
             # attention replacement of the block's active rows (Eq. 7) over the GPU's column set
             res = fo.sparse_loop_attention(to_np(g["q"][:, hs, :]), khat_new, vhat_new, vhat, o_full[act], act, sets,
                                            cache, w.sm_scale, w.q_block, head_list=[0], block_list=[b],
@@ -97,10 +103,56 @@ def test_full_size_layer_loops_2_and_3_sampled_against_oracle():
             in_block = np.nonzero(act // w.q_block == b)[0]
             assert len(in_block) > 0
             assert_attn_close(g["o"][act[in_block], h], res["O"][in_block, 0],
-                              f"O rows of loop {r}, head {h}, block {b}", loops=r - 1)
+                              f"O rows of loop {r}, head {h}, block {b}", carried=r - 1)
             np.testing.assert_allclose(g["lse"][h, act[in_block]], res["lse"][0, in_block], rtol=0, atol=5e-3 * (r - 1))
             o_full = o_full.copy()
             o_full[act] = res["O"]
             cache = {key: (res["probs"][key] if key[1] == b else cache[key]) for key in cache}
             khat, vhat = khat_new, vhat_new
+    ctx.close()
+
+
+def test_config2_full_size_chained_on_gpu_against_the_full_oracle():
+    """One layer at L = 8192 with all 16 heads, loops 2-4 chained on the GPU through the indexed entry point, against
+    the oracle run in full on the same inputs: token sets, codes of every head, O rows of every loop and the final
+    O store."""
+    import torch
+    from paper_2609_29812_b200 import binding as B, pipeline as P
+    from helpers import to_dev
+    w = workloads.config2()
+    x = workloads.make_layer_inputs(w, seed=0)
+    ref = fo.LayerOracle(w.L, w.n_heads, w.head_dim, w.q_block, w.bits, w.group, w.eps, w.sm_scale,
+                         storage=w.dtype).run(x.G, x.Q, x.K, x.V, [w.k_tokens] * 3, [w.col_budget] * 3)
+    ctx = B.Context(0)
+    st = P.LayerState(ctx, w)
+    st.dense_loop(to_dev(x.Q[0], w), to_dev(x.K[0], w), to_dev(x.V[0], w))
+    st.select_columns_dense()
+    assert_attn_close(to_np(st.o_store), ref["dense"]["O"], "config 2 dense source O")
+    idx, cnt = to_np(st.col_idx), to_np(st.col_cnt)
+    n_diff = 0
+    for (h, b), S in ref["loops"][0]["col_sets"].items():
+        end = min(w.L, (b + 1) * w.q_block)
+        n_diff += assert_selection_matches(idx[h, b, : cnt[h, b]], ref["dense"]["col_scores"][h, b, :end],
+                                           np.arange(end), w.col_budget, f"config 2 columns h{h} b{b}")
+    assert n_diff <= 0.01 * w.n_heads * st.nb * w.col_budget
+    cand = None
+    for r in range(2, w.n_loops + 1):
+        rec = ref["loops"][r - 2]
+        sel = P.select_tokens(ctx, st.shape, r, to_dev(x.G[r - 2], w), to_dev(x.G[r - 1], w), cand, w.k_tokens)
+        act = to_np(sel.active_idx).astype(np.int64)
+        assert np.array_equal(act, rec["active"]), f"token set of loop {r}"
+        o_rows, _ = st.sparse_loop(r, to_dev(x.Q[r - 1][act], w), to_dev(x.K[r - 1][act], w),
+                                   to_dev(x.V[r - 1][act], w), sel, indexed=True)
+        st.check_status()
+        for side, streams in (("k_payload", st.k_streams), ("v_payload", st.v_streams)):
+            pay, got = rec[side], streams[-1]
+            assert np.array_equal(to_np(got["codes"]).reshape(len(act), w.n_heads, -1), pay["packed"]), (r, side)
+            assert np.array_equal(to_np(got["scale"]).view(np.uint16).reshape(pay["scale"].shape),
+                                  pay["scale"].view(np.uint16)), (r, side)
+            assert np.array_equal(to_np(got["zero"]).view(np.uint16).reshape(pay["zero"].shape),
+                                  pay["zero"].view(np.uint16)), (r, side)
+        assert_attn_close(to_np(o_rows), rec["O_rows"], f"config 2 chained loop {r} O rows", carried=r - 1)
+        cand = sel.active_idx
+    assert_attn_close(to_np(st.o_store), ref["loops"][-1]["O_full"], "config 2 chained final O store",
+                      carried=w.n_loops - 1)
     ctx.close()

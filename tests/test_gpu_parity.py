@@ -310,12 +310,14 @@ def test_chained_layer_all_on_gpu(env, case):
                                    to_dev(x.V[r - 1][act], w), sel)
         cand = sel.active_idx
         st.check_status()
-        # The GPU carries O between loops in storage precision (the oracle carries fp64), so every chained
-        # loop adds one storage rounding of O on top of that loop's own attention error: the max-abs bound
-        # grows linearly with the number of chained loops; the relative L2 bound is kept as stated.
+        # The GPU carries O between loops in storage precision (the oracle carries fp64): the output entering
+        # loop r has been rounded r - 1 times on the GPU side only (loops 1 .. r-1), each by up to half a storage
+        # ulp, on top of this loop's own error; the relative L2 bound is kept as stated.
         if np.array_equal(act, ref["active"][r - 2]):
-            assert_attn_close(to_np(o_rows), ref["loops"][r - 2]["O_rows"], f"chained loop {r}", loops=r - 1)
-    assert_attn_close(to_np(st.o_store), ref["loops"][-1]["O_full"], "chained final O store", loops=w.n_loops - 1)
+            assert_attn_close(to_np(o_rows), ref["loops"][r - 2]["O_rows"], f"chained loop {r}", carried=r - 1,
+                              bf16=w.dtype == "bf16")
+    assert_attn_close(to_np(st.o_store), ref["loops"][-1]["O_full"], "chained final O store", carried=w.n_loops - 1,
+                      bf16=w.dtype == "bf16")
     # KV accounting of the real store
     fl, dense = B.fl_kv_store_bytes(sh, st.store, w.n_loops, 1)
     n_r = [len(a) for a in ref["active"]]
@@ -351,7 +353,7 @@ def test_indexed_attention_matches_compact_path_and_oracle(env):
     assert torch.equal(a.o_store, b.o_store)
     assert torch.equal(a.q_store, b.q_store)
     assert torch.equal(a.lse, b.lse)
-    assert_attn_close(to_np(b.o_store), ref["loops"][-1]["O_full"], "indexed final O store", loops=2)
+    assert_attn_close(to_np(b.o_store), ref["loops"][-1]["O_full"], "indexed final O store", carried=2)
     touched = np.zeros(w.L, dtype=bool)
     touched[ref["active"][0]] = True
     assert torch.equal(b.q_store[torch.from_numpy(~touched).to(b.q_store.device)],
@@ -437,7 +439,7 @@ def test_binary32_simt_attention_path_on_bf16_storage(env):
         act = ref["active"][r - 2]
         o_rows, _ = st.sparse_loop(r, to_dev(x.Q[r - 1][act], w), to_dev(x.K[r - 1][act], w),
                                    to_dev(x.V[r - 1][act], w), sel)
-    assert_attn_close(to_np(st.o_store), ref["loops"][-1]["O_full"], "SIMT path final O store", loops=2)
+    assert_attn_close(to_np(st.o_store), ref["loops"][-1]["O_full"], "SIMT path final O store", carried=2)
     ctx.close()
 
 

@@ -154,7 +154,7 @@ def test_chained_on_gpu_with_pruning(env, decaying_case, indexed):
                 t_idx = np.nonzero(blk == b)[0]
                 if is_clean and len(t_idx):
                     assert_attn_close(o_np[t_idx, h], rec["O_rows"][t_idx, h], f"chained loop {r} h{h} b{b}",
-                                      loops=r - 1)
+                                      carried=r - 1)
                     n_cmp += 1
             assert n_cmp >= 0.8 * len(clean)
         if r < w.n_loops:

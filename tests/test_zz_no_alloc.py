@@ -49,7 +49,7 @@ def test_static_scratch_entry_point_matches_the_workspace_one_twice_in_a_row():
             assert torch.equal(got, want), (r, name)
         st.q_store, st.o_store, st.lse = outs[1][0], outs[1][1], outs[1][2]
     # and the result is the method's (not merely the same as the other entry point's): two chained loops
-    assert_attn_close(to_np(st.o_store), ref["loops"][-1]["O_full"], "final O store", loops=2)
+    assert_attn_close(to_np(st.o_store), ref["loops"][-1]["O_full"], "final O store", carried=2)
     # a second pass over the same state with the static entry point alone: its counters were left at zero
     q, o, lse = st.q_store.clone(), st.o_store.clone(), st.lse.clone()
     sel = oracle_selection(P, w, ref, 3)

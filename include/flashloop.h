@@ -217,11 +217,46 @@ FL_API int fl_loop_attention_indexed(fl_ctx* ctx, const fl_shape* shape, int loo
                               const float* lse_in, float* lse_out, const void* o_store_in, void* o_store_out,
                               float* col_scores_next, int32_t* status, void* stream);
 
+/* Old-term economy for fl_loop_attention_indexed (Eq. 7 against Eq. 3: the old term of loop r is the cached
+ * p^(r-1) Vhat^(r-1) over the selected columns, which is loop r-1's NEW term whenever the column set of the row's
+ * (head, block) is unchanged since loop r-1 and the row was active in it; Eq. 6's cached mass m_i then carries over
+ * unchanged too). With
+ *   B_i = o^(w-1)_i - sum_{T_i} p_old_j Vhat^(w-1)_j      (the row's background, fixed at the last loop w that
+ *                                                          recomputed the old term)
+ * every later loop over the same sets is  o^(r)_i = B_i + sum_{T_i} p_new_j Vhat^(r)_j,  p_new = m_i softmax_{T_i}(.).
+ *   bg_store [L, H, dh] storage type, by position; mass f32 [H, L] by position. Caller-owned, 16-byte aligned,
+ *   distinct from the O stores; only rows / entries of active positions are touched.
+ *   reuse == 0: the call computes what fl_loop_attention_indexed computes and also WRITES, for every active row,
+ *               B_i (rounded once to the storage type) and m_i (0 for a row with empty T_i, whose B_i is o_prev_i).
+ *   reuse != 0: the call READS B_i and m_i and computes the new term only: q_store_in, o_store_in and lse_in are not
+ *               read (they may be NULL). Rows with m_i == 0 get o_out = B_i; their lse_out entry is copied from
+ *               lse_in when that is given and left alone otherwise.
+ * The caller guarantees, for a reuse call: col_idx / col_cnt are those of the call that wrote the buffers, and every
+ * active row was active in that call (nested token sets, Appendix D.1). After the column sets are pruned the next
+ * call must recompute (reuse == 0). The result differs from the recomputing form only by rounding (B is rounded to
+ * the storage type once instead of the output of every loop). */
+typedef struct {
+  void* bg_store;
+  float* mass;
+  int32_t reuse;
+  int32_t reserved_;
+} fl_attn_carry;
+
+/* fl_loop_attention_indexed with the carried old term; carry == NULL makes it that call exactly. Arguments, results
+ * and errors otherwise as fl_loop_attention_indexed; additionally FL_ERR_INVALID_ARG when a buffer of `carry` is NULL,
+ * misaligned or one of the O stores. */
+FL_API int fl_loop_attention_indexed_carry(fl_ctx* ctx, const fl_shape* shape, int loop_r, const void* q_new,
+                                    const void* q_store_in, void* q_store_out, const int32_t* active_idx,
+                                    int32_t n_active, const fl_kv_store* store, const int32_t* col_idx,
+                                    const int32_t* col_cnt, int32_t c, const float* lse_in, float* lse_out,
+                                    const void* o_store_in, void* o_store_out, const fl_attn_carry* carry /* host */,
+                                    float* col_scores_next, int32_t* status, void* stream);
+
 /* fl_loop_attention_indexed with the workspace of its last-wave split (see fl_set_workspace) taken from a fixed array
  * that is part of the library's device image, for callers that cannot lend device memory (code that runs where
  * cudaMalloc is off limits: inside a region whose memory was budgeted up front, or under an allocator the caller does
  * not control); the context's own workspace, if any, is ignored by this call. The paper has no counterpart. The call
- * allocates and frees nothing. The array is 19.6 MB and every device that loads the library holds its own copy until
+ * allocates and frees nothing. The array is 19.7 MB and every device that loads the library holds its own copy until
  * the process exits, whether this entry point is used or not. Its address is looked up on the first call per device
  * (cudaGetSymbolAddress, which answers for the CURRENT device: that call, like every later one, must be made with the
  * context's device current, else FL_ERR_CUDA and nothing is cached or launched); make that first call before any

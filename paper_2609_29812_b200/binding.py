@@ -42,6 +42,10 @@ class FlKvStore(C.Structure):
                 ("n_streams", C.c_int32), ("reserved_", C.c_int32)]
 
 
+class FlAttnCarry(C.Structure):
+    _fields_ = [("bg_store", C.c_void_p), ("mass", C.c_void_p), ("reuse", C.c_int32), ("reserved_", C.c_int32)]
+
+
 class FlashLoopError(RuntimeError):
     def __init__(self, call: str, status: int):
         self.status = status
@@ -69,6 +73,8 @@ def _load() -> C.CDLL:
                               p, p, p, p, p, p, p],
         "fl_loop_attention_indexed": [p, C.POINTER(FlShape), C.c_int, p, p, p, p, i32, C.POINTER(FlKvStore), p, p,
                                       i32, p, p, p, p, p, p, p],
+        "fl_loop_attention_indexed_carry": [p, C.POINTER(FlShape), C.c_int, p, p, p, p, i32, C.POINTER(FlKvStore), p, p,
+                                            i32, p, p, p, p, C.POINTER(FlAttnCarry), p, p, p],
         "fl_loop_attention_indexed_static": [p, C.POINTER(FlShape), C.c_int, p, p, p, p, i32, C.POINTER(FlKvStore),
                                              p, p, i32, p, p, p, p, p, p, p],
         "fl_kv_store_bytes": [C.POINTER(FlShape), C.POINTER(FlKvStore), C.c_int, C.c_int,
@@ -241,6 +247,24 @@ def fl_loop_attention_indexed(ctx, shape, loop_r, q_new, q_store_in, q_store_out
                                        int(c), _ptr(lse_in), _ptr(lse_out), _ptr(o_store_in), _ptr(o_store_out),
                                        _ptr(col_scores_next), _ptr(status), _stream(stream))
     return _check("fl_loop_attention_indexed", rc, check)
+
+
+def make_carry(bg_store, mass, reuse: bool) -> FlAttnCarry:
+    """Host struct of the old-term economy: background rows [L, H, dh], mass [H, L], and whether the call reuses
+    them (True) or recomputes the old term and writes them (False).  The caller keeps the tensors alive."""
+    return FlAttnCarry(_ptr(bg_store), _ptr(mass), 1 if reuse else 0, 0)
+
+
+def fl_loop_attention_indexed_carry(ctx, shape, loop_r, q_new, q_store_in, q_store_out, active_idx, n_active, store,
+                                    col_idx, col_cnt, c, lse_in, lse_out, o_store_in, o_store_out, carry,
+                                    col_scores_next=None, status=None, stream=None, check=True) -> int:
+    rc = lib.fl_loop_attention_indexed_carry(_h(ctx), C.byref(shape), int(loop_r), _ptr(q_new), _ptr(q_store_in),
+                                             _ptr(q_store_out), _ptr(active_idx), int(n_active),
+                                             C.byref(store) if store is not None else None, _ptr(col_idx),
+                                             _ptr(col_cnt), int(c), _ptr(lse_in), _ptr(lse_out), _ptr(o_store_in),
+                                             _ptr(o_store_out), C.byref(carry) if carry is not None else None,
+                                             _ptr(col_scores_next), _ptr(status), _stream(stream))
+    return _check("fl_loop_attention_indexed_carry", rc, check)
 
 
 def fl_loop_attention_indexed_static(ctx, shape, loop_r, q_new, q_store_in, q_store_out, active_idx, n_active, store,

@@ -21,8 +21,8 @@ struct fl_ctx {
 };
 
 // Layout of the loop-attention workspace: kFlMaxSplit int32 arrival counters, then per split problem two partial
-// results of kFlPartFloats binary32 values (both 128 x 128 accumulators and three statistics per row).
-constexpr int kFlPartFloats = 2 * 128 * 128 + 3 * 128;
+// results of kFlPartFloats binary32 values (both 128 x 128 accumulators and four statistics per row).
+constexpr int kFlPartFloats = 2 * 128 * 128 + 4 * 128;
 constexpr int kFlMaxSplit = 256;
 
 // Bytes of workspace with which the loop-attention launch can split the problems of its last wave (0: never useful).

@@ -10,7 +10,8 @@ int fl_launch_sparse_colscore(const fl_shape* s, const void* q_new, const int32_
 int fl_launch_loop_attn_tc(fl_ctx* ctx, const fl_shape* s, int loop_r, const void* q_new, const void* q_old,
                            const int32_t* active_idx, int n_active, const fl_kv_store* store, const int32_t* col_idx,
                            const int32_t* col_cnt, int c, const float* lse_prev, float* lse_out, const void* o_prev,
-                           void* o_out, int indexed, void* q_store, int32_t* status, cudaStream_t st);
+                           void* o_out, int indexed, void* q_store, const fl_attn_carry* carry, int32_t* status,
+                           cudaStream_t st);
 
 // whether the tensor-path kernel has a build for this request (storage type, head dimension, column budget, shared memory)
 bool fl_loop_attn_tc_covers(const fl_ctx* ctx, const fl_shape* s, int c);
@@ -236,7 +237,7 @@ extern "C" int fl_loop_attention(fl_ctx* ctx, const fl_shape* shape, int loop_r,
   if (!ctx->force_simt) {
     // tensor path (bf16 storage, head_dim 128); anything else runs on the binary32 SIMT kernel below
     rc = fl_launch_loop_attn_tc(ctx, shape, loop_r, q_new, q_old, active_idx, n_active, store, col_idx, col_cnt, c,
-                                lse_prev, lse_out, o_prev, o_out, 0, nullptr, status, st);
+                                lse_prev, lse_out, o_prev, o_out, 0, nullptr, nullptr, status, st);
     if (rc == FL_OK) {
       if (col_scores_next == nullptr) return FL_OK;
       return fl_launch_sparse_colscore(shape, q_new, active_idx, n_active, kside, loop_r - 1, col_idx, col_cnt, c,
@@ -275,7 +276,7 @@ int fl_attn_indexed_check(const fl_ctx* ctx, const fl_shape* shape, int loop_r, 
                           const void* q_store_in, const void* q_store_out, const int32_t* active_idx, int32_t n_active,
                           const fl_kv_store* store, const int32_t* col_idx, const int32_t* col_cnt, int32_t c,
                           const float* lse_in, const float* lse_out, const void* o_store_in, const void* o_store_out,
-                          int* launch) {
+                          const fl_attn_carry* carry, int* launch) {
   *launch = 0;
   FL_REQUIRE(ctx != nullptr);
   int rc = fl_check_shape(shape);
@@ -284,11 +285,17 @@ int fl_attn_indexed_check(const fl_ctx* ctx, const fl_shape* shape, int loop_r, 
   FL_REQUIRE(n_active >= 0 && n_active <= shape->L && c >= 1);
   rc = fl_check_store(shape, store, loop_r - 1);
   if (rc != FL_OK) return rc;
-  FL_REQUIRE(col_idx != nullptr && col_cnt != nullptr && lse_in != nullptr && lse_out != nullptr);
+  // a call that reuses the carried old term reads neither the previous loop's Q and O rows nor its log-normalisers
+  const bool reuse = carry != nullptr && carry->reuse != 0;
+  FL_REQUIRE(col_idx != nullptr && col_cnt != nullptr && lse_out != nullptr && (reuse || lse_in != nullptr));
   FL_REQUIRE(shape->n_heads <= 65535 && fl_n_blocks(shape) <= 65535);
+  if (carry != nullptr) {
+    FL_REQUIRE(carry->bg_store != nullptr && carry->mass != nullptr && fl_aligned16(carry->bg_store));
+    FL_REQUIRE(carry->bg_store != o_store_out && carry->bg_store != o_store_in);
+  }
   if (n_active == 0) return FL_OK;
-  FL_REQUIRE(q_new != nullptr && q_store_in != nullptr && o_store_in != nullptr && o_store_out != nullptr &&
-             active_idx != nullptr);
+  FL_REQUIRE(q_new != nullptr && o_store_out != nullptr && active_idx != nullptr);
+  FL_REQUIRE(reuse || (q_store_in != nullptr && o_store_in != nullptr));
   FL_REQUIRE(fl_aligned16(q_new) && fl_aligned16(q_store_in) && fl_aligned16(q_store_out) &&
              fl_aligned16(o_store_in) && fl_aligned16(o_store_out));
   if (ctx->force_simt) return FL_ERR_UNSUPPORTED;
@@ -297,15 +304,15 @@ int fl_attn_indexed_check(const fl_ctx* ctx, const fl_shape* shape, int loop_r, 
   return FL_OK;
 }
 
-extern "C" int fl_loop_attention_indexed(fl_ctx* ctx, const fl_shape* shape, int loop_r, const void* q_new,
-                                         const void* q_store_in, void* q_store_out, const int32_t* active_idx,
-                                         int32_t n_active, const fl_kv_store* store, const int32_t* col_idx,
-                                         const int32_t* col_cnt, int32_t c, const float* lse_in, float* lse_out,
-                                         const void* o_store_in, void* o_store_out, float* col_scores_next,
-                                         int32_t* status, void* stream) {
+extern "C" int fl_loop_attention_indexed_carry(fl_ctx* ctx, const fl_shape* shape, int loop_r, const void* q_new,
+                                               const void* q_store_in, void* q_store_out, const int32_t* active_idx,
+                                               int32_t n_active, const fl_kv_store* store, const int32_t* col_idx,
+                                               const int32_t* col_cnt, int32_t c, const float* lse_in, float* lse_out,
+                                               const void* o_store_in, void* o_store_out, const fl_attn_carry* carry,
+                                               float* col_scores_next, int32_t* status, void* stream) {
   int launch = 0;
   int rc = fl_attn_indexed_check(ctx, shape, loop_r, q_new, q_store_in, q_store_out, active_idx, n_active, store,
-                                 col_idx, col_cnt, c, lse_in, lse_out, o_store_in, o_store_out, &launch);
+                                 col_idx, col_cnt, c, lse_in, lse_out, o_store_in, o_store_out, carry, &launch);
   if (rc != FL_OK) return rc;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (!launch) {
@@ -315,10 +322,21 @@ extern "C" int fl_loop_attention_indexed(fl_ctx* ctx, const fl_shape* shape, int
     return FL_OK;
   }
   rc = fl_launch_loop_attn_tc(ctx, shape, loop_r, q_new, q_store_in, active_idx, n_active, store, col_idx, col_cnt, c,
-                              lse_in, lse_out, o_store_in, o_store_out, 1, q_store_out, status, st);
+                              lse_in, lse_out, o_store_in, o_store_out, 1, q_store_out, carry, status, st);
   if (rc != FL_OK || col_scores_next == nullptr) return rc;
   DevSide kside;
   fl_dev_side(store, true, &kside);
   return fl_launch_sparse_colscore(shape, q_new, active_idx, n_active, kside, loop_r - 1, col_idx, col_cnt, c, lse_out,
                                    col_scores_next, st);
+}
+
+extern "C" int fl_loop_attention_indexed(fl_ctx* ctx, const fl_shape* shape, int loop_r, const void* q_new,
+                                         const void* q_store_in, void* q_store_out, const int32_t* active_idx,
+                                         int32_t n_active, const fl_kv_store* store, const int32_t* col_idx,
+                                         const int32_t* col_cnt, int32_t c, const float* lse_in, float* lse_out,
+                                         const void* o_store_in, void* o_store_out, float* col_scores_next,
+                                         int32_t* status, void* stream) {
+  return fl_loop_attention_indexed_carry(ctx, shape, loop_r, q_new, q_store_in, q_store_out, active_idx, n_active,
+                                         store, col_idx, col_cnt, c, lse_in, lse_out, o_store_in, o_store_out, nullptr,
+                                         col_scores_next, status, stream);
 }

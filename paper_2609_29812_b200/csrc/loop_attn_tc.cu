@@ -35,6 +35,15 @@
 // accumulators and row statistics in the workspace and the other merges them into its own before the epilogue.
 // Every wait (mbarriers, the pair's counter) is bounded; on a timeout the CTA raises a flag, drains and reports
 // FL_ERR_TIMEOUT.
+//
+// Old-term economy (template parameter ECON). When the column sets of a (head, block) are the ones of the loop
+// before and the row was active in it, the old term of Eq. 7 is that loop's new term, so
+//   O^(r) = B + new^(r),   B = O^(w-1) - old^(w)   of the last loop w that recomputed the old term,
+// and the cached mass m_i is the one of loop w (Eq. 6: it does not change while the set does not). A recomputing
+// launch can leave B (storage type, by position) and m_i (binary32, [H, L]) in buffers of the caller; an ECON launch
+// reads them and computes the new term only. Its two pipelines then are two STREAMS of the new term (even and odd
+// chunks of the column list, an accumulator, a running reference and a row sum each), merged in the epilogue like the
+// two halves of a split problem; the previous loop's Q rows, O rows and log-normalisers are not read.
 #include "fl_internal.cuh"
 #include "tc_ptx.cuh"
 
@@ -66,7 +75,7 @@ constexpr float kLn2 = 0.6931471805599453f;
 // (column-major, so that the row-owning threads write and read coalesced) and the three per-row statistics.
 constexpr int kPartFloats = kFlPartFloats;
 constexpr int kMaxSplit = kFlMaxSplit;      // counters at the head of the workspace
-static_assert(kPartFloats == 2 * kM * kDH + 3 * kM, "partial result: two accumulators and three statistics per row");
+static_assert(kPartFloats == 2 * kM * kDH + 4 * kM, "partial result: two accumulators and four statistics per row");
 constexpr float kRescaleThreshold = 60.f;   // in log2 units: rescale only when the reference falls this far behind
 static_assert(3 * kMaxCols * 4 <= kSlots * kSlotBytes, "prologue staging must fit in the ring");
 static_assert(kAccNew == kAccOld + kDH, "the two accumulators are adjacent in tensor memory");
@@ -79,6 +88,9 @@ struct alignas(64) TcArgs {
                                      // indexed form q_old_map is a row-gather map of the Q store ([L, d], box 64 x 1)
   const __nv_bfloat16* o_prev;       // compact rows; in the indexed form the O stores [L, d] (may be the same)
   __nv_bfloat16* o_out;
+  const __nv_bfloat16* bg_in;        // ECON: the rows' background B [L, d] by position (read instead of o_prev)
+  __nv_bfloat16* bg_out;             // recomputing launch: receives B = o_prev - old term [L, d] by position, or null
+  float* mass;                       // [H, L] by position: read by an ECON launch, written with bg_out otherwise
   const __nv_bfloat16* q_new;        // indexed form only: compact new Q rows, copied into q_store at the end
   __nv_bfloat16* q_store;            // indexed form only: Q store [L, d] that receives them, or null
   const int32_t* active_idx;
@@ -118,9 +130,10 @@ struct __align__(16) TcSmemCtl {
   int warp_cnt[kWarps][2];
   int chunk_last[kMaxChunks];       // largest column position of the chunk, INT32_MAX if the chunk is padded
   uint32_t chunk_mask[kMaxChunks];  // OR of the stream masks of the chunk's columns (0: plain gather only)
-  float mass[kM];
+  float mass[kM];            // ECON: row sums of stream 0
   float ell[kM];
   float ref[kM];
+  float ref0[kM];            // ECON: running references of stream 0
 };
 
 constexpr size_t kTcSmemBytes = 1024 /* alignment slack */ + 2 * kQTileBytes + kSlots * kSlotBytes + sizeof(TcSmemCtl) +
@@ -229,7 +242,8 @@ __device__ __forceinline__ ChunkInfo chunk_info(int ci, int n_plain, int n_patch
 
 // INDEXED: the previous loop's Q and O rows are read from, and the new O rows written to, position-indexed
 // stores (row active_idx[t] for compact row t) instead of compact buffers.
-template <int BITS, bool INDEXED>
+// ECON: the old term is not recomputed (see the head of this file); the two pipelines are two streams of the new term.
+template <int BITS, bool INDEXED, bool ECON>
 __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_constant__ TcArgs a) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -273,7 +287,7 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
     for (int s = 0; s < kSlots; ++s) {
       tc::mbar_init(&ctl.landed[s], kTmaWarps);
       tc::mbar_init(&ctl.patched[s], kTmaWarps);
-      tc::mbar_init(&ctl.done[s], 2);
+      tc::mbar_init(&ctl.done[s], ECON ? 1 : 2);   // ECON: a slot is read by one stream only
     }
     tc::mbar_init(&ctl.q_full, 1);
     for (int t = 0; t < 2; ++t) {
@@ -426,26 +440,27 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
   }
   __syncthreads();
   int g = 0;    // chunks issued so far (all tiles): S / P buffer = g & 1, one phase of its barriers per use
+  int g1 = 0;   // ECON: the same count for stream 1 (g counts stream 0): a stream takes every other chunk
   int fill = 0; // ring slots filled so far: slot = fill % kSlots, phase = (fill / kSlots) & 1
   uint32_t dirty_par_cta = 0;  // per-slot phase parity of the patched[] barriers (they only see dirty chunks)
 
   for (int s0 = q_lo, tile = 0; s0 < q_hi && !(pair >= 0 && part == 1 && !split); s0 += kM, ++tile) {
   const int n_rows = min(kM, q_hi - s0);
-  const int g0 = g, fill0 = fill;
+  const int g0 = g, g0_1 = g1, fill0 = fill;
   const uint32_t dirty_par0 = dirty_par_cta;
   if (warp == kTmaWarp) {
     // Q tiles of this row tile: two 64-element slabs each; rows past the compact list read as zero, rows of the
     // next block (past n_rows) are computed and dropped
     if (lane == 0) {
-      tc::mbar_arrive_expect_tx(&ctl.q_full, 2 * kQTileBytes);
+      tc::mbar_arrive_expect_tx(&ctl.q_full, ECON ? kQTileBytes : 2 * kQTileBytes);
       tc::tma_tile2d(q_new_tile, &a.q_new_map, &ctl.q_full, h * kDH, s0);
       tc::tma_tile2d(q_new_tile + kM * 128, &a.q_new_map, &ctl.q_full, h * kDH + 64, s0);
-      if (!INDEXED) {
+      if (!INDEXED && !ECON) {
         tc::tma_tile2d(q_old_tile, &a.q_old_map, &ctl.q_full, h * kDH, s0);
         tc::tma_tile2d(q_old_tile + kM * 128, &a.q_old_map, &ctl.q_full, h * kDH + 64, s0);
       }
     }
-    if (INDEXED) {
+    if (INDEXED && !ECON) {
       // the previous loop's Q rows come from the store: four-row gathers by position, one group of rows per lane
       __syncwarp();
       int y[4];
@@ -482,7 +497,7 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
 #pragma unroll 1
     for (int ci = c_lo; ci < c_hi && ok; ++ci) {
       const ChunkInfo ck = chunk_info(ci, n_plain, n_patch);
-      const int n_slots = ck.patch ? 2 : 1;
+      const int n_slots = (ck.patch && !ECON) ? 2 : 1;    // ECON: only the tiles after the loop's residual are needed
       const bool dirty = ctl.chunk_mask[ci] != 0;
       for (int k = 0; k < n_slots && ok; ++k)
         if (f + k >= kSlots) ok = warp_wait(&ctl.done[(f + k) % kSlots], (((f + k) / kSlots) - 1) & 1, abort_flag);
@@ -505,7 +520,7 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
         for (int k = 0; k < n_slots; ++k) {
           const int slot = (f + k) % kSlots;
           const void* src = !from_rows ? map
-                            : (k == 0 ? (is_v ? static_cast<const void*>(&a.v_prev_map) : static_cast<const void*>(&a.k_prev_map))
+                            : ((k == 0 && !ECON) ? (is_v ? static_cast<const void*>(&a.v_prev_map) : static_cast<const void*>(&a.k_prev_map))
                                       : (is_v ? static_cast<const void*>(&a.v_cur_map) : static_cast<const void*>(&a.k_cur_map)));
           tc::tma_gather4(ring + slot * kSlotBytes + is_v * kTileBytes + slab * (kNC * 128) + grp * 512, src,
                           &ctl.landed[slot], h * kDH + slab * 64, y[0], y[1], y[2], y[3]);
@@ -526,8 +541,12 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
           uint4 v_old, v_new;
           patch_piece<BITS>(side, a.n_old, mask, j, elem, a.d, a.group, base16, v_old, v_new);
           const uint32_t off = tc::sw128_offset(u, ch & 7);
-          if (mask & ((1u << a.n_old) - 1u)) *reinterpret_cast<uint4*>(t_old + off) = v_old;
-          if (ck.patch) *reinterpret_cast<uint4*>(t_new + off) = v_new;
+          if (ECON) {
+            *reinterpret_cast<uint4*>(t_old + off) = v_new;     // the chunk's only slot holds Xhat^(r)
+          } else {
+            if (mask & ((1u << a.n_old) - 1u)) *reinterpret_cast<uint4*>(t_old + off) = v_old;
+            if (ck.patch) *reinterpret_cast<uint4*>(t_new + off) = v_new;
+          }
         }
         tc::fence_proxy_async_smem();
         __syncwarp();
@@ -554,14 +573,14 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
     // One thread per term issues both kinds of MMA, in the order their operands become ready: QK^T of chunk n (its S
     // buffer is free once PV of chunk n - 2 has retired), then PV of chunk n - 1 (its P is written while QK^T of
     // chunk n executes).
-    const int t = warp - kIssueWarp;      // 0: old term, 1: new term
+    const int t = warp - kIssueWarp;      // 0: old term, 1: new term (ECON: streams 0 and 1 of the new term)
     if (lane == 0) {
       const uint32_t idesc_qk = tc::make_idesc_bf16(kM, kNC, false);
       const uint32_t idesc_pv = tc::make_idesc_bf16(kM, kDH, true);
       // Descriptors differ only in their start-address field (bits 0-13, units of 16 bytes): the low word
       // moves (no carry into the other fields: shared memory is < 256 KB), the high word stays.
       // K-major operands (Q, Khat): 32 bytes per 16-element K step inside a 64-element slab, then the next slab.
-      const uint64_t q_desc = tc::make_desc_sw128(tc::smem_u32(t ? q_new_tile : q_old_tile), 16, 1024);
+      const uint64_t q_desc = tc::make_desc_sw128(tc::smem_u32((t || ECON) ? q_new_tile : q_old_tile), 16, 1024);
       const uint64_t k_desc0 = tc::make_desc_sw128(tc::smem_u32(ring), 16, 1024);
       const uint32_t kq_hi = (uint32_t)(k_desc0 >> 32);
       const uint32_t q_lo_w = (uint32_t)q_desc, k_lo0 = (uint32_t)k_desc0;
@@ -574,22 +593,32 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
       int pv_slot = 0;           // slots of the chunk whose PV is issued next (the previous QK^T's)
       int pv_slot1 = -1;
       uint32_t dirty_par = dirty_par0;
+      // the chunks this thread issues: all of them, or (ECON) every other one starting at the stream's number
+      constexpr int kStep = ECON ? 2 : 1;
+      const int first = c_lo + (ECON ? t : 0);
+      const int n_mine = first < c_hi ? (c_hi - first + kStep - 1) / kStep : 0;
+      const int gbase = (ECON && t) ? g0_1 : g0;
 #pragma unroll 1
-      for (int ci = c_lo; ci <= c_hi; ++ci) {
-        const int gc = g0 + ci - c_lo;
+      for (int n = 0; n <= n_mine; ++n) {
+        const int ci = first + n * kStep;
+        const int gc = gbase + n;
         int qk_slot = 0, qk_slot1 = -1;
-        if (ci < c_hi) {
+        if (n < n_mine) {
           const ChunkInfo ck = chunk_info(ci, n_plain, n_patch);
+          if (ECON) f = fill0 + (ci - c_lo);    // one slot per chunk, filled in chunk order
+          const bool two = ck.patch && !ECON;
           const int slot0 = f % kSlots, slot1 = (f + 1) % kSlots;
-          if (ci == c_lo && !tc::mbar_wait(&ctl.q_full, tile & 1, abort_flag)) break;
+          if (n == 0 && !tc::mbar_wait(&ctl.q_full, tile & 1, abort_flag)) break;
           // a term reads one slot of the chunk only (the new term of a two-slot chunk the second): it starts on it
           // without waiting for the other
-          const int my_slot = (t && ck.patch) ? slot1 : slot0, my_fill = (t && ck.patch) ? f + 1 : f;
+          const int my_slot = (t && two) ? slot1 : slot0, my_fill = (t && two) ? f + 1 : f;
           if (!tc::mbar_wait(&ctl.landed[my_slot], (my_fill / kSlots) & 1, abort_flag)) break;
           if (ctl.chunk_mask[ci] != 0) {       // residual-carrying columns are rewritten by the patch warps
+            // (ECON: the ring has an even number of slots and the streams alternate, so within a row tile a slot
+            // always serves the same stream, which therefore sees every phase of the slot's barrier)
             if (!tc::mbar_wait(&ctl.patched[my_slot], (dirty_par >> my_slot) & 1, abort_flag)) break;
             dirty_par ^= 1u << slot0;
-            if (ck.patch) dirty_par ^= 1u << slot1;
+            if (two) dirty_par ^= 1u << slot1;
           }
           // the S buffer holds P of the chunk before the previous one until its PV MMAs have read it
           if (gc >= 2 && !tc::mbar_wait(&ctl.p_free[t][gc & 1], ((gc >> 1) - 1) & 1, abort_flag)) break;
@@ -604,16 +633,16 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
 #undef FL_QK
           tc::mma_commit(&ctl.s_full[t][gc & 1]);
           qk_slot = slot0;
-          qk_slot1 = ck.patch ? slot1 : -1;
-          f += ck.patch ? 2 : 1;
+          qk_slot1 = two ? slot1 : -1;
+          f += two ? 2 : 1;
         }
-        if (ci > c_lo) {
-          const int cj = ci - 1, gp = gc - 1, pb = gp & 1;
+        if (n > 0) {
+          const int gp = gc - 1, pb = gp & 1;
           if (!tc::mbar_wait(&ctl.p_full[t][pb], (gp >> 1) & 1, abort_flag)) break;
           tc::tc_fence_after();
           const uint32_t v_lo = v_lo0 + ((t && pv_slot1 >= 0) ? pv_slot1 : pv_slot) * (kSlotBytes >> 4);
           const uint32_t p_src = s_base + pb * kNC;
-          const uint32_t acc0 = cj > c_lo ? 1u : 0u;       // the CTA's first chunk of the tile overwrites the accumulator
+          const uint32_t acc0 = n > 1 ? 1u : 0u;           // the thread's first chunk of the tile overwrites the accumulator
 #pragma unroll
           for (int kk = 0; kk < kNC / 16; ++kk)
             tc::mma_ts_lo(acc, p_src + kk * 8, v_lo + kk * (2048 >> 4), v_hi, idesc_pv, kk > 0 ? 1u : acc0);
@@ -629,22 +658,26 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
     __syncwarp();
   } else {
     // ============================================ softmax ============================================
-    const int grp = warp >> 2;                    // 0: old term, 1: new term
+    const int grp = warp >> 2;                    // 0: old term, 1: new term (ECON: streams 0 and 1 of the new term)
     const int gt = tid & 127;                     // thread inside the term's group of four warps
     const int row = (warp & 3) * 32 + lane;
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
     const bool row_ok = row < n_rows;
     const int pos = row_ok ? __ldg(a.active_idx + s0 + row) : -1;
     const float c2 = a.scale * kLog2e;
-    const float lse2 = (row_ok ? a.lse_prev[(size_t)h * a.L + pos] : 0.f) * kLog2e;
-    // the epilogue reads the row's previous output: have it in L2 by then (each group asks for its 128-byte half)
+    const float lse2 = ((row_ok && !ECON) ? a.lse_prev[(size_t)h * a.L + pos] : 0.f) * kLog2e;
+    // the epilogue reads the row's previous output (ECON: its background): have it in L2 by then (each group asks
+    // for its 128-byte half)
+    const __nv_bfloat16* prev_rows = ECON ? a.bg_in : a.o_prev;
     if (row_ok)
-      tc::prefetch_l2(a.o_prev + (INDEXED ? (size_t)pos : (size_t)(s0 + row)) * a.d + h * kDH + grp * 64);
+      tc::prefetch_l2(prev_rows + (INDEXED ? (size_t)pos : (size_t)(s0 + row)) * a.d + h * kDH + grp * 64);
     const uint32_t s_addr = tmem + lane_base + (grp ? kSNew : kSOld);
     float mass = 0.f, ell = 0.f, ref = -INFINITY;
     bool ok = true;
-    for (int ci = c_lo; ci < c_hi; ++ci) {
-      const int gc = g0 + ci - c_lo, pb = gc & 1, n_use = gc >> 1;
+    constexpr int kStep = ECON ? 2 : 1;           // ECON: a group's stream takes every other chunk
+    const int gbase = (ECON && grp) ? g0_1 : g0;
+    for (int ci = c_lo + (ECON ? grp : 0), n = 0; ci < c_hi; ci += kStep, ++n) {
+      const int gc = gbase + n, pb = gc & 1, n_use = gc >> 1;
       if (!warp_wait(&ctl.s_full[grp][pb], n_use & 1, abort_flag)) { ok = false; break; }
       tc::tc_fence_after();
       // rows of a warp that lie at or after every column of the chunk need no causal mask; rows beyond the
@@ -679,7 +712,7 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
           for (int u = 0; u < 32; ++u) r[u] = u < lim ? r[u] : 0xff800000u;
         }
         float sub = lse2;
-        if (grp == 1) {
+        if (ECON || grp == 1) {
           // running reference of the new term: taken from the first columns that show a finite logit and moved
           // (with a rescale of the accumulator row) only when a maximum beats it by more than the threshold
           float cm = -INFINITY;
@@ -692,19 +725,20 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
           if (__any_sync(0xffffffffu, over)) {
             float factor = 1.f;
             if (over) { factor = tc::ex2(ref - cm); ref = cm; }
-            // every earlier PV must have completed before the accumulator rows are rewritten (ci >= 1 here: the
+            // every earlier PV must have completed before the accumulator rows are rewritten (n >= 1 here: the
             // reference was set in an earlier chunk, or in this chunk's first half, whose P is not announced yet)
-            if (ci > c_lo) {
-              if (!warp_wait(&ctl.p_free[1][(gc - 1) & 1], ((gc - 1) >> 1) & 1, abort_flag)) { ok = false; break; }
+            if (n > 0) {
+              if (!warp_wait(&ctl.p_free[grp][(gc - 1) & 1], ((gc - 1) >> 1) & 1, abort_flag)) { ok = false; break; }
               tc::tc_fence_after();
+              const uint32_t acc_col = grp ? kAccNew : kAccOld;    // the group's own accumulator
 #pragma unroll 1
               for (int q4 = 0; q4 < 8; ++q4) {
                 uint32_t acc[16];
-                tc::tmem_ld16(tmem + lane_base + kAccNew + q4 * 16, acc);
+                tc::tmem_ld16(tmem + lane_base + acc_col + q4 * 16, acc);
                 tc::tmem_wait_ld();
 #pragma unroll
                 for (int i = 0; i < 16; ++i) acc[i] = __float_as_uint(__uint_as_float(acc[i]) * factor);
-                tc::tmem_st16(tmem + lane_base + kAccNew + q4 * 16, acc);
+                tc::tmem_st16(tmem + lane_base + acc_col + q4 * 16, acc);
               }
               tc::tmem_wait_st();
             }
@@ -734,7 +768,7 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
           sum += p0 + p1;
           r[u >> 1] = tc::pack_bf16(p0, p1);
         }
-        if (grp == 0) mass += sum; else ell += sum;
+        if (!ECON && grp == 0) mass += sum; else ell += sum;
         tc::tmem_st16(sp_addr + hf * 16, *reinterpret_cast<uint32_t(*)[16]>(&r[0]));
       }
       if (!ok) break;
@@ -746,32 +780,52 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
       if (lane == 0) tc::mbar_arrive(&ctl.p_full[grp][pb]);
     }
     // ---- epilogue ------------------------------------------------------------------------------------
-    // Each group finishes 64 of the 128 head-dim columns. Its half of the O_prev tile is staged in the group's
-    // own Q tile (the QK^T MMAs of the group's term have all retired once its last S arrived) with coalesced
-    // asynchronous copies, combined in place by the row-owning threads, and written out coalesced again.
-    uint8_t* stage = grp ? q_new_tile : q_old_tile;          // [128 rows][8 x 16 B], 16-byte chunks XOR-swizzled by row
+    // Each group finishes 64 of the 128 head-dim columns. Its half of the O_prev tile (ECON: of the background rows) is
+    // staged in shared memory with coalesced asynchronous copies, combined in place by the row-owning threads, and
+    // written out coalesced again. The staging area is the first half of the group's own Q tile (the QK^T MMAs of
+    // the group's term have all retired once its last S arrived); the second half takes the background rows a
+    // recomputing launch leaves for later loops. In ECON both streams read the new Q tile until the very end and the
+    // old one is never loaded: the groups stage in its two halves.
+    uint8_t* stage = ECON ? q_old_tile + grp * (kM * 128)    // [128 rows][8 x 16 B], 16-byte chunks XOR-swizzled by row
+                          : (grp ? q_new_tile : q_old_tile);
+    uint8_t* stage_bg = stage + kM * 128;                    // recomputing launch with bg_out only
+    const bool write_bg = !ECON && INDEXED && a.bg_out != nullptr;   // CTA-uniform
     const size_t o_col0 = (size_t)h * kDH + grp * 64;
+    // a tile without a single chunk (empty column set): no issuer has waited for the Q tiles, which are still on
+    // their way into the very memory the rows are staged in
+    if (ok && c_hi == c_lo) ok = warp_wait(&ctl.q_full, tile & 1, abort_flag);
 #pragma unroll 1
     for (int k = 0; k < 8; ++k) {
       const int idx = k * 128 + gt, rr = idx >> 3, cc = idx & 7;
       if (rr < n_rows) {
         const size_t src_row = INDEXED ? (size_t)__ldg(a.active_idx + s0 + rr) : (size_t)(s0 + rr);
-        tc::cp_async16(stage + rr * 128 + ((cc ^ (rr & 7)) << 4), a.o_prev + src_row * a.d + o_col0 + cc * 8);
+        tc::cp_async16(stage + rr * 128 + ((cc ^ (rr & 7)) << 4), prev_rows + src_row * a.d + o_col0 + cc * 8);
       }
     }
     tc::cp_async_commit();
     if (ok) ok = warp_wait(&ctl.acc_done, tile & 1, abort_flag);
     tc::tc_fence_after();
-    if (grp == 0) ctl.mass[row] = mass;
-    else { ctl.ell[row] = ell; ctl.ref[row] = ref; }
+    if (ECON) {
+      if (grp == 0) { ctl.mass[row] = ell; ctl.ref0[row] = ref; }
+      else { ctl.ell[row] = ell; ctl.ref[row] = ref; }
+    } else {
+      if (grp == 0) ctl.mass[row] = mass;
+      else { ctl.ell[row] = ell; ctl.ref[row] = ref; }
+    }
     tc::cp_async_wait<0>();
     asm volatile("bar.sync 1, 256;" ::: "memory");
-    float m_i = ctl.mass[row], l_i = ctl.ell[row], ref_i = ctl.ref[row];
-    const bool acc_valid = ok && c_hi > c_lo;             // warp-uniform: the tensor-memory reads below are collective
+    // per-row statistics. Accumulator A (tensor-memory columns 0-127) is the old term's, B (128-255) the new term's;
+    // in ECON they are streams 0 and 1 of the new term, each with its own row sum and reference.
+    float m_i = ECON ? (row_ok ? a.mass[(size_t)h * a.L + pos] : 0.f) : ctl.mass[row];
+    float l_a = ECON ? ctl.mass[row] : 0.f, ref_a = ECON ? ctl.ref0[row] : -INFINITY;
+    float l_i = ctl.ell[row], ref_i = ctl.ref[row];
+    // warp-uniform: the tensor-memory reads below are collective
+    const bool valid_a = ok && c_hi > c_lo;
+    const bool valid_b = ok && (ECON ? c_hi > c_lo + 1 : c_hi > c_lo);
     // ---- split problems: the CTA of the pair that finishes first leaves its partial result in the workspace, the
     // other one adds it to its own (nobody waits for anybody: whoever finds the counter at 1 merges)
     const float* other = nullptr;
-    float f_mine = 1.f, f_other = 0.f;
+    float f_a = 0.f, f_b = 1.f, f_oa = 0.f, f_ob = 0.f;   // factors of accumulators A and B, own and other CTA's
     if (split) {
       // counter of the pair: each CTA adds 1 when its accumulation is complete (the one that finds 0 is first), the
       // first one adds 16 once its partial result is in the workspace; the second resets it for the next launch
@@ -780,20 +834,23 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
       if (ctl.merge_role == 0) {
         float* mine = a.part_acc + ((size_t)pair * 2 + part) * kPartFloats;
 #pragma unroll 1
-        for (int c16 = 0; c16 < 8; ++c16) {   // acc_old columns 0-63 of the group's half, then acc_new: 16 at a time
+        for (int c16 = 0; c16 < 8; ++c16) {   // accumulator A columns 0-63 of the group's half, then B: 16 at a time
           uint32_t v[16];
-          const int col = (c16 >> 2) * kDH + grp * 64 + (c16 & 3) * 16;   // column of the [old | new] accumulator pair
-          if (acc_valid) {
+          const int col = (c16 >> 2) * kDH + grp * 64 + (c16 & 3) * 16;   // column of the [A | B] accumulator pair
+          const bool valid = (c16 >> 2) ? valid_b : valid_a;
+          if (valid) {
             tc::tmem_ld16(tmem + lane_base + kAccOld + col, v);           // kAccNew == kAccOld + kDH
             tc::tmem_wait_ld();
           }
 #pragma unroll
-          for (int i = 0; i < 16; ++i) mine[(col + i) * kM + row] = acc_valid ? __uint_as_float(v[i]) : 0.f;
+          for (int i = 0; i < 16; ++i) mine[(col + i) * kM + row] = valid ? __uint_as_float(v[i]) : 0.f;
         }
-        if (grp == 0) mine[2 * kM * kDH + row] = acc_valid ? m_i : 0.f;
-        else {
-          mine[2 * kM * kDH + kM + row] = acc_valid ? l_i : 0.f;
-          mine[2 * kM * kDH + 2 * kM + row] = acc_valid ? ref_i : -INFINITY;
+        if (grp == 0) {
+          mine[2 * kM * kDH + row] = ECON ? (valid_a ? l_a : 0.f) : (valid_a ? m_i : 0.f);
+          mine[2 * kM * kDH + 3 * kM + row] = (ECON && valid_a) ? ref_a : -INFINITY;
+        } else {
+          mine[2 * kM * kDH + kM + row] = valid_b ? l_i : 0.f;
+          mine[2 * kM * kDH + 2 * kM + row] = valid_b ? ref_i : -INFINITY;
         }
         __threadfence();
         asm volatile("bar.sync 1, 256;" ::: "memory");
@@ -808,7 +865,7 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
             seen = atomicAdd(a.part_cnt + pair, 0);
           }
           if (seen < 16) { *abort_flag = 1; ctl.merge_role = 2; }   // gave up: no output, FL_ERR_TIMEOUT
-          else a.part_cnt[pair] = 0;                                // ready for the next launch
+          a.part_cnt[pair] = 0;                                     // ready for the next launch either way
         }
         asm volatile("bar.sync 1, 256;" ::: "memory");
         if (ctl.merge_role == 1) {   // CTA-uniform
@@ -820,52 +877,96 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
           for (int i = tid; i < 2 * kM * kDH / 4; i += 256) tc::cp_async16(ring + i * 16, theirs + i * 4);
           tc::cp_async_commit();
           other = reinterpret_cast<const float*>(ring);
-          const float m_o = __ldcg(theirs + 2 * kM * kDH + row), l_o = __ldcg(theirs + 2 * kM * kDH + kM + row);
+          const float s0_o = __ldcg(theirs + 2 * kM * kDH + row), l_o = __ldcg(theirs + 2 * kM * kDH + kM + row);
           const float ref_o = __ldcg(theirs + 2 * kM * kDH + 2 * kM + row);
-          const float ref_t = fmaxf(ref_i, ref_o);
-          f_mine = ref_i > -INFINITY ? tc::ex2(ref_i - ref_t) : 0.f;
-          f_other = ref_o > -INFINITY ? tc::ex2(ref_o - ref_t) : 0.f;
-          // products and sums rounded one by one (no fused multiply-add): the result must not depend on which of
-          // the two CTAs does the merging
-          m_i = __fadd_rn(m_i, m_o);
-          l_i = __fadd_rn(__fmul_rn(l_i, f_mine), __fmul_rn(l_o, f_other));
-          ref_i = ref_t;
+          const float ref_oa = __ldcg(theirs + 2 * kM * kDH + 3 * kM + row);
+          // products and sums rounded one by one (no fused multiply-add), the two CTAs' contributions joined by one
+          // commutative addition: the result must not depend on which of the two does the merging
+          if (ECON) {
+            const float ref_t = fmaxf(fmaxf(ref_a, ref_i), fmaxf(ref_oa, ref_o));
+            f_a = ref_a > -INFINITY ? tc::ex2(ref_a - ref_t) : 0.f;
+            f_b = ref_i > -INFINITY ? tc::ex2(ref_i - ref_t) : 0.f;
+            f_oa = ref_oa > -INFINITY ? tc::ex2(ref_oa - ref_t) : 0.f;
+            f_ob = ref_o > -INFINITY ? tc::ex2(ref_o - ref_t) : 0.f;
+            l_i = __fadd_rn(__fadd_rn(__fmul_rn(l_a, f_a), __fmul_rn(l_i, f_b)),
+                            __fadd_rn(__fmul_rn(s0_o, f_oa), __fmul_rn(l_o, f_ob)));
+            ref_i = ref_t;
+          } else {
+            const float ref_t = fmaxf(ref_i, ref_o);
+            f_b = ref_i > -INFINITY ? tc::ex2(ref_i - ref_t) : 0.f;
+            f_ob = ref_o > -INFINITY ? tc::ex2(ref_o - ref_t) : 0.f;
+            m_i = __fadd_rn(m_i, s0_o);
+            l_i = __fadd_rn(__fmul_rn(l_i, f_b), __fmul_rn(l_o, f_ob));
+            ref_i = ref_t;
+          }
           tc::cp_async_wait<0>();
           asm volatile("bar.sync 1, 256;" ::: "memory");
         }
       }
     }
+    if (ECON && other == nullptr) {   // the CTA's own two streams on a common reference
+      const float ref_t = fmaxf(ref_a, ref_i);
+      f_a = ref_a > -INFINITY ? tc::ex2(ref_a - ref_t) : 0.f;
+      f_b = ref_i > -INFINITY ? tc::ex2(ref_i - ref_t) : 0.f;
+      l_i = __fadd_rn(__fmul_rn(l_a, f_a), __fmul_rn(l_i, f_b));
+      ref_i = ref_t;
+    }
     const bool writer = !split || other != nullptr;       // CTA-uniform: this CTA produces the output rows
-    const bool has = acc_valid && ref_i > -INFINITY;      // per row: T_i is not empty
+    const bool has = valid_a && ref_i > -INFINITY && (!ECON || m_i > 0.f);   // per row: T_i is not empty
     const float w = has ? m_i / l_i : 0.f;
 #pragma unroll 1
     for (int c8 = 0; c8 < 8 && writer; ++c8) {   // 8 head-dim columns = one 16-byte cell of the staged row at a time
       uint32_t ao[8], an[8];
       const int col = grp * 64 + c8 * 8;
-      if (acc_valid) {
-        tc::tmem_ld8(tmem + lane_base + kAccOld + col, ao);
-        tc::tmem_ld8(tmem + lane_base + kAccNew + col, an);
-        tc::tmem_wait_ld();
+      if (valid_a) tc::tmem_ld8(tmem + lane_base + kAccOld + col, ao);
+      if (valid_b) tc::tmem_ld8(tmem + lane_base + kAccNew + col, an);
+      tc::tmem_wait_ld();
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        if (!valid_a) ao[i] = 0u;
+        if (!valid_b) an[i] = 0u;
       }
-      if (other != nullptr) {
+      if (ECON) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          float v = __fadd_rn(__fmul_rn(__uint_as_float(ao[i]), f_a), __fmul_rn(__uint_as_float(an[i]), f_b));
+          if (other != nullptr)
+            v = __fadd_rn(v, __fadd_rn(__fmul_rn(other[(col + i) * kM + row], f_oa),
+                                       __fmul_rn(other[(kDH + col + i) * kM + row], f_ob)));
+          an[i] = __float_as_uint(v);
+        }
+      } else if (other != nullptr) {
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
           ao[i] = __float_as_uint(__fadd_rn(__uint_as_float(ao[i]), other[(col + i) * kM + row]));
-          an[i] = __float_as_uint(__fadd_rn(__fmul_rn(__uint_as_float(an[i]), f_mine),
-                                            __fmul_rn(other[(kDH + col + i) * kM + row], f_other)));
+          an[i] = __float_as_uint(__fadd_rn(__fmul_rn(__uint_as_float(an[i]), f_b),
+                                            __fmul_rn(other[(kDH + col + i) * kM + row], f_ob)));
         }
       }
+      uint4* cell = reinterpret_cast<uint4*>(stage + row * 128 + ((c8 ^ (row & 7)) << 4));
+      uint4* cell_bg = reinterpret_cast<uint4*>(stage_bg + row * 128 + ((c8 ^ (row & 7)) << 4));
       if (has) {
-        uint4* cell = reinterpret_cast<uint4*>(stage + row * 128 + ((c8 ^ (row & 7)) << 4));
         float pv[8];
         unpack8(*cell, pv);
+        if (!ECON) {
+          // background of the row: what stays of its previous output once the old term is taken out
 #pragma unroll
-        for (int i = 0; i < 8; ++i) pv[i] = pv[i] - __uint_as_float(ao[i]) + w * __uint_as_float(an[i]);
+          for (int i = 0; i < 8; ++i) pv[i] = pv[i] - __uint_as_float(ao[i]);
+          if (write_bg) *cell_bg = pack8(pv);
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) pv[i] = pv[i] + w * __uint_as_float(an[i]);
         *cell = pack8(pv);
+      } else if (write_bg) {
+        *cell_bg = *cell;                                   // empty T_i: the row itself is its background
       }
     }
-    if (grp == 1 && row_ok && writer)
-      a.lse_out[(size_t)h * a.L + pos] = has ? (ref_i + log2f(l_i)) * kLn2 - logf(m_i) : lse2 * kLn2;
+    if (grp == 1 && row_ok && writer) {
+      if (has) a.lse_out[(size_t)h * a.L + pos] = (ref_i + log2f(l_i)) * kLn2 - logf(m_i);
+      else if (!ECON) a.lse_out[(size_t)h * a.L + pos] = lse2 * kLn2;
+      else if (a.lse_prev != nullptr) a.lse_out[(size_t)h * a.L + pos] = a.lse_prev[(size_t)h * a.L + pos];
+    }
+    if (write_bg && grp == 0 && row_ok && writer) a.mass[(size_t)h * a.L + pos] = has ? m_i : 0.f;
     asm volatile("bar.sync 1, 256;" ::: "memory");
 #pragma unroll 1
     for (int k = 0; k < 8 && writer; ++k) {
@@ -874,6 +975,9 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
         const size_t dst_row = INDEXED ? (size_t)__ldg(a.active_idx + s0 + rr) : (size_t)(s0 + rr);
         *reinterpret_cast<uint4*>(a.o_out + dst_row * a.d + o_col0 + cc * 8) =
             *reinterpret_cast<const uint4*>(stage + rr * 128 + ((cc ^ (rr & 7)) << 4));
+        if (write_bg)
+          *reinterpret_cast<uint4*>(a.bg_out + dst_row * a.d + o_col0 + cc * 8) =
+              *reinterpret_cast<const uint4*>(stage_bg + rr * 128 + ((cc ^ (rr & 7)) << 4));
       }
     }
   }
@@ -893,11 +997,12 @@ __global__ void __launch_bounds__(kThreads, 1) loop_attn_tc_kernel(const __grid_
   }
   // every role is done with this tile: accumulators, Q tiles and the ring bookkeeping move on together
   if (s0 + kM < q_hi) {   // CTA-uniform: another row tile of the block follows
-    g += c_hi - c_lo;
+    if (ECON) { g += (c_hi - c_lo + 1) >> 1; g1 += (c_hi - c_lo) >> 1; }
+    else g += c_hi - c_lo;
     int f = fill;
     for (int ci = c_lo; ci < c_hi; ++ci) {   // replay the tile's fills (same for every role)
       const ChunkInfo ck = chunk_info(ci, n_plain, n_patch);
-      const int n_slots = ck.patch ? 2 : 1;
+      const int n_slots = (ck.patch && !ECON) ? 2 : 1;
       if (ctl.chunk_mask[ci] != 0)
         for (int k = 0; k < n_slots; ++k) dirty_par_cta ^= 1u << ((f + k) % kSlots);
       f += n_slots;
@@ -966,11 +1071,13 @@ bool fl_loop_attn_tc_covers(const fl_ctx* ctx, const fl_shape* s, int c) {
 
 // Returns FL_ERR_UNSUPPORTED when the tensor path does not cover the request (caller falls back to the
 // SIMT kernel, which is also CUDA). indexed != 0: q_old, o_prev and o_out are position-indexed stores [L, d] and
-// q_store (may be null) receives the new Q rows.
+// q_store (may be null) receives the new Q rows. carry (indexed form only, may be null): the old-term economy's
+// buffers; carry->reuse != 0 launches the ECON kernel, which reads them instead of q_old, o_prev and lse_prev.
 int fl_launch_loop_attn_tc(fl_ctx* ctx, const fl_shape* s, int loop_r, const void* q_new, const void* q_old,
                            const int32_t* active_idx, int n_active, const fl_kv_store* store, const int32_t* col_idx,
                            const int32_t* col_cnt, int c, const float* lse_prev, float* lse_out, const void* o_prev,
-                           void* o_out, int indexed, void* q_store, int32_t* status, cudaStream_t st) {
+                           void* o_out, int indexed, void* q_store, const fl_attn_carry* carry, int32_t* status,
+                           cudaStream_t st) {
   if (!fl_loop_attn_tc_covers(ctx, s, c)) return FL_ERR_UNSUPPORTED;
   TcArgs a{};
   const int64_t d_row = (int64_t)s->n_heads * s->head_dim;
@@ -978,9 +1085,15 @@ int fl_launch_loop_attn_tc(fl_ctx* ctx, const fl_shape* s, int loop_r, const voi
       !fl_tile_tmap(ctx, store->v_base, s->L, d_row, 1, &a.v_map) ||
       !fl_tile_tmap(ctx, q_new, n_active, d_row, kM, &a.q_new_map))
     return FL_ERR_UNSUPPORTED;
-  if (indexed ? !fl_tile_tmap(ctx, q_old, s->L, d_row, 1, &a.q_old_map)
-              : !fl_tile_tmap(ctx, q_old, n_active, d_row, kM, &a.q_old_map))
+  const bool econ = indexed && carry != nullptr && carry->reuse != 0;
+  if (!econ && (indexed ? !fl_tile_tmap(ctx, q_old, s->L, d_row, 1, &a.q_old_map)
+                        : !fl_tile_tmap(ctx, q_old, n_active, d_row, kM, &a.q_old_map)))
     return FL_ERR_UNSUPPORTED;
+  if (indexed && carry != nullptr) {
+    a.bg_in = econ ? static_cast<const __nv_bfloat16*>(carry->bg_store) : nullptr;
+    a.bg_out = econ ? nullptr : static_cast<__nv_bfloat16*>(carry->bg_store);
+    a.mass = carry->mass;
+  }
   a.o_prev = static_cast<const __nv_bfloat16*>(o_prev);
   a.o_out = static_cast<__nv_bfloat16*>(o_out);
   a.q_new = static_cast<const __nv_bfloat16*>(q_new);
@@ -1015,15 +1128,17 @@ int fl_launch_loop_attn_tc(fl_ctx* ctx, const fl_shape* s, int loop_r, const voi
   a.part_cnt = static_cast<int32_t*>(ctx->ws);
   a.part_acc = reinterpret_cast<float*>(static_cast<uint8_t*>(ctx->ws) + kMaxSplit * sizeof(int32_t));
   const dim3 grid(a.n_full + 2 * (n_items - a.n_full));
-#define FL_TC2(BITS, IDX)                                                                                        \
+#define FL_TC2(BITS, IDX, ECON)                                                                                  \
   do {                                                                                                           \
-    auto kern = loop_attn_tc_kernel<BITS, IDX>;                                                                  \
+    auto kern = loop_attn_tc_kernel<BITS, IDX, ECON>;                                                            \
     FL_CHECK_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcSmemBytes));  \
     FL_CHECK_CUDA(fl_launch(ctx, kern, grid, dim3(kThreads), kTcSmemBytes, st, a));                             \
   } while (0)
 #define FL_TC(BITS)                                   \
   do {                                                \
-    if (indexed) FL_TC2(BITS, true); else FL_TC2(BITS, false); \
+    if (econ) FL_TC2(BITS, true, true);               \
+    else if (indexed) FL_TC2(BITS, true, false);      \
+    else FL_TC2(BITS, false, false);                  \
   } while (0)
   switch (s->bits) {
     case 2: FL_TC(2); break;

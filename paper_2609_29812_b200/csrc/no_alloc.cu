@@ -7,7 +7,7 @@ int fl_attn_indexed_check(const fl_ctx* ctx, const fl_shape* shape, int loop_r, 
                           const void* q_store_in, const void* q_store_out, const int32_t* active_idx, int32_t n_active,
                           const fl_kv_store* store, const int32_t* col_idx, const int32_t* col_cnt, int32_t c,
                           const float* lse_in, const float* lse_out, const void* o_store_in, const void* o_store_out,
-                          int* launch);
+                          const fl_attn_carry* carry, int* launch);
 
 namespace {
 
@@ -16,7 +16,7 @@ constexpr size_t kStaticBytes =
     (size_t)kFlMaxSplit * sizeof(int32_t) + (size_t)kStaticPairs * 2 * kFlPartFloats * sizeof(float);
 
 // The scratch itself: part of the library's device image (no allocation call ever made for it). Every device that
-// loads the library holds its own copy of these 19.6 MB until the process exits, whether this entry point is used
+// loads the library holds its own copy of these 19.7 MB until the process exits, whether this entry point is used
 // or not.
 static __device__ __align__(256) unsigned char g_attn_scratch[kStaticBytes];
 
@@ -34,7 +34,7 @@ extern "C" int fl_loop_attention_indexed_static(fl_ctx* ctx, const fl_shape* sha
   // the same host checks as the workspace form, before anything is enqueued
   int launch = 0;
   const int rc = fl_attn_indexed_check(ctx, shape, loop_r, q_new, q_store_in, q_store_out, active_idx, n_active, store,
-                                       col_idx, col_cnt, c, lse_in, lse_out, o_store_in, o_store_out, &launch);
+                                       col_idx, col_cnt, c, lse_in, lse_out, o_store_in, o_store_out, nullptr, &launch);
   if (rc != FL_OK) return rc;
   FL_REQUIRE(ctx->device >= 0 && ctx->device < kMaxDevices);
   // the split this shape would use must fit the fixed array: no silent fall-back to something else

@@ -188,13 +188,31 @@ class LayerState:
                             self.col_idx, self.col_cnt, self.c, self.lse, self.lse, o_prev, o_out,
                             col_scores_next, status=self.status)   # lse updated in place (active rows only)
 
-    def attention_indexed(self, loop_r, q_new, sel: TokenSelection, col_scores_next=None, check=True) -> int:
+    def carry_buffers(self):
+        """Buffers of the old-term economy, allocated on first use: background rows [L, H, dh] and mass [H, L]."""
+        if getattr(self, "bg_store", None) is None:
+            self.bg_store = torch.zeros_like(self.o_store)
+            self.mass = torch.zeros(self.w.n_heads, self.w.L, dtype=torch.float32, device=self.dev)
+        return self.bg_store, self.mass
+
+    def attention_indexed(self, loop_r, q_new, sel: TokenSelection, col_scores_next=None, check=True,
+                          carry: Optional[str] = None) -> int:
         """Same step on the position-indexed Q / O stores, updated in place (no gathers or scatters around it);
-        returns the status code, FL_ERR_UNSUPPORTED when the shape is outside the tensor path."""
-        return B.fl_loop_attention_indexed(self.ctx, self.shape, loop_r, q_new, self.q_store, self.q_store,
-                                           sel.active_idx, sel.n, self.store, self.col_idx, self.col_cnt, self.c,
-                                           self.lse, self.lse, self.o_store, self.o_store, col_scores_next,
-                                           status=self.status, check=check)
+        returns the status code, FL_ERR_UNSUPPORTED when the shape is outside the tensor path.
+        carry: None (plain call), "write" (recompute the old term and leave background rows and masses for later
+        loops) or "reuse" (take the old term from them: valid while the column sets are unchanged and the token sets
+        nested)."""
+        if carry is None:
+            return B.fl_loop_attention_indexed(self.ctx, self.shape, loop_r, q_new, self.q_store, self.q_store,
+                                               sel.active_idx, sel.n, self.store, self.col_idx, self.col_cnt, self.c,
+                                               self.lse, self.lse, self.o_store, self.o_store, col_scores_next,
+                                               status=self.status, check=check)
+        bg, mass = self.carry_buffers()
+        cs = B.make_carry(bg, mass, carry == "reuse")
+        return B.fl_loop_attention_indexed_carry(self.ctx, self.shape, loop_r, q_new, self.q_store, self.q_store,
+                                                 sel.active_idx, sel.n, self.store, self.col_idx, self.col_cnt,
+                                                 self.c, self.lse, self.lse, self.o_store, self.o_store, cs,
+                                                 col_scores_next, status=self.status, check=check)
 
     def check_status(self):
         """Synchronises and raises if a kernel reported an asynchronous error (e.g. a bounded wait ran out)."""
@@ -203,17 +221,17 @@ class LayerState:
             raise B.FlashLoopError("device status", code)
 
     def sparse_loop(self, loop_r, q_new, k_new, v_new, sel: TokenSelection, want_col_scores_next=False,
-                    indexed=False):
+                    indexed=False, carry: Optional[str] = None, rows: bool = True):
         """One loop r >= 2 for this layer: store residuals, gather the carried rows, attend, scatter back
         (indexed=True: one call on the stores instead).  q_new, k_new, v_new: [n, H, dh] rows of the active tokens.
         Returns (o_rows, col_scores_next)."""
-        self.alloc_stream(sel)
+        self.alloc_stream(sel, rows=rows)
         self.quantize(loop_r, k_new, v_new, sel)
         if indexed:
             csn = None
             if want_col_scores_next:
                 csn = torch.zeros(self.w.n_heads, self.nb, self.c, dtype=torch.float32, device=self.dev)
-            self.attention_indexed(loop_r, q_new, sel, csn)
+            self.attention_indexed(loop_r, q_new, sel, csn, carry=carry)
             return self.gather(self.o_store, sel), csn
         q_old = self.gather(self.q_store, sel)
         o_prev = self.gather(self.o_store, sel)

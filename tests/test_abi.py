@@ -95,6 +95,17 @@ def test_argument_validation_happens_before_any_launch(B):
                                           P, P, P, P, None, **call)
     assert la(r=1) == INV and la(c=0) == INV and la(q=None) == INV and la(ci=None) == INV
     assert la(r=3) == INV and la(st=None) == INV and la(n=-1) == INV and la(n=4096) == INV
+    # the carried old term of the indexed form
+    idx = lambda carry, **kw: B.fl_loop_attention_indexed_carry(
+        ctx, sh, 2, P, kw.get("qs", P), P, P, 16, st, P, P, 64, kw.get("lse", P), P, kw.get("o", P + 0x1000),
+        P + 0x2000, carry, None, **call)
+    assert idx(B.make_carry(None, P, False)) == INV and idx(B.make_carry(P + 0x4000, None, True)) == INV
+    assert idx(B.make_carry(P + 0x2000, P, False)) == INV                                      # background = O store
+    assert idx(B.make_carry(P + 0x4004, P, False)) == INV                                      # misaligned
+    assert idx(B.make_carry(P + 0x4000, P, False), qs=None) == INV         # recomputing needs the previous Q rows
+    # a reusing call needs none of the previous loop's rows: the checks pass and the stand-in context, which has no
+    # tensor path, answers "unsupported"
+    assert idx(B.make_carry(P + 0x4000, P, True), qs=None, lse=None, o=None) == UNS
     # accounting
     rc = B.lib.fl_kv_store_bytes(C.byref(sh), C.byref(st), 3, 1, C.byref(C.c_int64()), C.byref(C.c_int64()))
     assert rc == INV                                                                          # only one stream

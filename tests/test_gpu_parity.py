@@ -379,7 +379,7 @@ def test_attention_workspace_calls(env):
     B, P, ctx = env
     sh = P.shape_of(small_bf16(L=1200))
     need = B.fl_loop_attention_workspace_bytes(ctx, sh)
-    per_problem = 2 * 4 * (2 * 128 * 128 + 3 * 128)          # two partial results of binary32 values
+    per_problem = 2 * 4 * (2 * 128 * 128 + 4 * 128)          # two partial results of binary32 values
     assert need > 1024 and (need - 1024) % per_problem == 0  # counters, then a whole number of split problems
     assert B.fl_loop_attention_workspace_bytes(ctx, P.shape_of(workloads.config1())) == 0   # f32: never split
     buf = torch.empty(need + 512, dtype=torch.uint8, device="cuda")

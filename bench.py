@@ -2,11 +2,18 @@
 """Benchmark of the FlashLoop loop-r prefill hot path on B200.
 
 One "step" = one pass of the whole hot path over one synthetic prompt: for every sparse loop
-r = 2..R, one token selection, then for every layer: gather of the active hidden rows, column
-selection (loop 2 only, from the dense source loop's statistics), K/V residual quantization,
-gathers of the carried Q / O rows, loop attention (column-sparse delta with in-kernel
-dequantize-and-add), scatters of the new O / Q rows; and one hidden-state scatter per loop.
-The dense source loop (loop 1) and the Q/K/V projections are set-up, outside the timed region.
+r = 2..R, one token selection, then for every layer: gather of the active hidden rows (input of
+the projections, which are scaffolding outside the library), column selection (loop 2 only, from
+the dense source loop's statistics), K/V residual quantization (which also leaves the active
+rows' reconstructed K/V as bf16 rows in a transient workspace), and the loop attention on the
+position-indexed stores (it reads the carried rows and writes the new O / Q rows itself: no
+gathers or scatters around it); and one hidden-state scatter per loop.  Loop 2 recomputes the old
+term of the replacement equation and leaves each row's background and mass; loops 3.. reuse them
+(constant column budget) and compute the new term only.  A second timed variant runs the same
+step without the materialized rows: every residual-carrying column is dequantized and added
+inside the attention kernel (reported under "variants").
+The dense source loop (loop 1) and the Q/K/V/O projections are outside the timed region; their
+times are printed separately ("setup_ms", "scaffold_ms").
 
 Metric: prompt tokens per second of the loop-r prefill, L / (time of one step).
 Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead.
@@ -33,9 +40,12 @@ METRIC = "loop_r_prefill_tokens_per_s"
 UNIT = "tokens/s"
 
 
-# DRAM bytes one attention launch of the default workload moves, from one ncu capture of exactly that launch shape
-# (one layer of the 48: every layer launches the same grid); the live timing of this file cannot measure it.
-NCU_ATTN_TRAFFIC_BYTES = 158.8e6
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) one attention launch moves, from ncu captures of exactly
+# these launch shapes (one layer: every layer launches the same grid); the live timing of this file cannot measure
+# it, so the bench line says "not measured in this run".  Keyed by (workload, L, layers-independent) and loop kind;
+# a shape that is not listed reports null.
+NCU_ATTN_TRAFFIC_BYTES = {
+}
 
 
 def parse_args():
@@ -44,7 +54,13 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c3", choices=["c2", "c3"])
+    ap.add_argument("--workload", default="c3", choices=["c2", "c3", "c4", "c5"],
+                    help="c3: the 48-layer stack at 32K (default, the metric's configuration); c2: one layer at 8K; "
+                         "c5: the 128K memory configuration (prefill part; 24 layers resident unless --layers); "
+                         "c4: the sparsity / depth sweep (one layer at 8K, a table of points)")
+    ap.add_argument("--sweep", default="subset", choices=["subset", "full"], help="c4: which points to run")
+    ap.add_argument("--no-economy", action="store_true", help="recompute the old term in every loop")
+    ap.add_argument("--no-variants", action="store_true", help="skip the in-kernel dequantization variant")
     ap.add_argument("--layers", type=int, default=0, help="override the number of layers (development)")
     ap.add_argument("--L", type=int, default=0, help="override the context length (development / profiling)")
     ap.add_argument("--no-e2e", action="store_true")
@@ -58,6 +74,8 @@ def get_workload(args):
     if args.workload == "c2":
         w = workloads.config2()
         w = workloads.replace(w, rmsnorm=False)
+    elif args.workload == "c5":
+        w = workloads.config5(n_layers=args.layers or 24)
     else:
         w = workloads.config3()
     if args.L:
@@ -125,7 +143,7 @@ class ClockSampler:
 # the CUDA arm
 # ------------------------------------------------------------------------------------------------
 class Bench:
-    def __init__(self, args, w, device):
+    def __init__(self, args, w, device, economy=True):
         import torch
         from paper_2609_29812_b200 import binding as B, pipeline as P, workloads
         self.torch, self.B, self.P, self.w, self.dev = torch, B, P, w, device
@@ -134,22 +152,22 @@ class Bench:
         self.R, self.NL, self.H, self.dh, self.L, self.d = w.n_loops, w.n_layers, w.n_heads, w.head_dim, w.L, w.d
         self.nb = (w.L + w.q_block - 1) // w.q_block
         self.c = w.col_budget
+        self.economy = economy
         self.stream = torch.cuda.Stream(device=device)
         self.sp = int(self.stream.cuda_stream)
-        self.calls = []          # (tag, fn, args)
-        self.launches_per_step = 0
-        self.keep = []           # keeps tensors alive
-        self.attn_flops, self.attn_bytes = [], []
+        self.keep = []           # keeps tensors and host structs alive
+        self.attn_flops_min, self.attn_flops_exec, self.attn_bytes = {}, {}, {}   # per loop r: lists over layers
+        self.setup_ms = {}
         self._setup(workloads)
 
     # -- set-up: dense source loop per layer, token sets, buffers ------------------------------------
     def _setup(self, workloads):
         torch, B, P, w = self.torch, self.B, self.P, self.w
         dev, ctx, sh = self.dev, self.ctx, self.shape
-        e = 2
         stack = workloads.DeviceStack(w, seed=0, device=dev)
         self.G = stack.stack_hidden()
         k_tok = w.k_tokens
+        dense_ms = []
         with torch.cuda.stream(self.stream):
             self.sels, cand = [], None
             for r in range(2, self.R + 1):
@@ -168,26 +186,61 @@ class Bench:
                 gen = stack.layer(l)
                 q1, k1, v1 = gen.qkv1()
                 st = P.LayerState(ctx, w, dev)
+                e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+                e0.record(self.stream)
                 st.dense_loop(q1, k1, v1)
+                e1.record(self.stream)
                 st.select_columns_dense()
                 st.hidden = gen.hidden(self.R)
                 st.lse1 = st.lse
                 st.lse_work = st.lse.clone()
                 st.q_work, st.o_work = st.q_store.clone(), st.o_store.clone()
+                st.carry_buffers()
                 st.rows = {}
                 for r in range(2, self.R + 1):
                     sel = self.sels[r - 2]
                     st.rows[r] = gen.rows(r, sel.active_idx)
                     st.alloc_stream(sel)
+                # the same store without the transient rows: the attention kernel then rebuilds every
+                # residual-carrying column itself (dequantize-and-add inside the kernel)
+                strip = lambda streams: [{k: v for k, v in s_.items() if not k.startswith("rows_")} for s_ in streams]
+                st.store_plain = B.make_store(st.k_base, st.v_base, strip(st.k_streams), strip(st.v_streams))
                 gen.release()
                 self.stream.synchronize()
-                self._account(st)
+                dense_ms.append(e0.elapsed_time(e1))
+                if l == 0 or w.name.startswith("c4"):
+                    self._account(st)
                 self.layers.append(st)
         torch.cuda.synchronize()
-        self._plan()
+        self.setup_ms["dense_source_loop_per_layer"] = statistics.median(dense_ms)
+        self.setup_ms["dense_source_loop_all_layers"] = sum(dense_ms)
+        self._scaffold()
+        self.plans = {}
+
+    def _scaffold(self):
+        """Times the projections around the hot path (cuBLAS through torch; scaffolding, not part of the metric):
+        [n, d] x [d, 3d] for Q/K/V and [n, d] x [d, d] for the output projection, per layer and loop."""
+        torch = self.torch
+        n = self.sels[0].n
+        x = torch.randn(n, self.d, device=self.dev, dtype=torch.bfloat16)
+        wqkv = torch.randn(self.d, 3 * self.d, device=self.dev, dtype=torch.bfloat16)
+        wo = torch.randn(self.d, self.d, device=self.dev, dtype=torch.bfloat16)
+        out = {}
+        for name, wt in (("qkv_projection", wqkv), ("o_projection", wo)):
+            for _ in range(3):
+                x @ wt
+            e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(10):
+                x @ wt
+            e1.record(); torch.cuda.synchronize()
+            out[name + "_per_layer_loop"] = e0.elapsed_time(e1) / 10
+        out["per_step"] = (out["qkv_projection_per_layer_loop"] + out["o_projection_per_layer_loop"]) * self.NL * (self.R - 1)
+        self.scaffold_ms = out
 
     def _account(self, st):
-        """Algorithmic FLOPs and bytes of each loop's attention launch for this layer (from the index sets)."""
+        """Algorithmic FLOPs and bytes of each loop's attention launch for one layer, from the index sets (every
+        layer of the stack has the same token sets; its column sets differ but not their sizes)."""
         torch, w = self.torch, self.w
         e, H, dh, d, c, L = 2, self.H, self.dh, self.d, self.c, self.L
         col = st.col_idx.long()                                 # [H, nb, c], -1 padded
@@ -203,7 +256,12 @@ class Bench:
             for h in range(H):
                 rows_cols = col[h][blk]                         # [n, c]
                 pairs += int(((rows_cols >= 0) & (rows_cols <= act[:, None])).sum().item())
-            flops = 4.0 * dh * pairs * 2.0                      # QK^T and PV, old term and new term
+            one_term = 4.0 * dh * pairs                         # QK^T and PV of one term over the kept (row, column) pairs
+            # minimum the method needs: the old term is recomputed only after a dense source loop (loop 2) or a
+            # pruned set; otherwise it is the previous loop's new term
+            need_old = r == 2
+            self.attn_flops_min.setdefault(r, []).append(one_term * (2.0 if need_old else 1.0))
+            self.attn_flops_exec.setdefault(r, []).append(one_term * (2.0 if (need_old or not self.economy) else 1.0))
             byt = 0.0
             for h in range(H):
                 byt += float(len(uniq[h])) * 2 * dh * e         # K and V base rows of the selected columns
@@ -211,11 +269,15 @@ class Bench:
                     slot = self.sels[rr - 2].slot_of_pos.long()
                     byt += float((slot[uniq[h]] >= 0).sum().item()) * pay_col_head
             byt += 4.0 * sel.n * d * e + 8.0 * H * sel.n + 4.0 * H * self.nb * (c + 1) + 4.0 * L * (r - 1)
-            self.attn_flops.append(flops)
-            self.attn_bytes.append(byt)
+            self.attn_bytes.setdefault(r, []).append(byt)
 
     # -- the step as a flat list of C-ABI calls ---------------------------------------------------------
-    def _plan(self):
+    def plan(self, rows=True):
+        """The step as a list of (tag, function, arguments, loop).  rows: the attention gathers the loop's active
+        columns from the rows the quantization kernel materialized (True) or rebuilds them itself (False)."""
+        key = bool(rows)
+        if key in self.plans:
+            return self.plans[key]
         B, lib, w = self.B, self.B.lib, self.w
         ctx, shp, sp = self.ctx.handle, C.byref(self.shape), self.sp
         p = lambda t: C.c_void_p(int(t.data_ptr())) if t is not None else None
@@ -223,7 +285,7 @@ class Bench:
         row_bytes = self.d * e
         calls, launches = [], 0
         # per-step algorithmic bytes of the memory-bound stages (for the whole-step roofline)
-        self.stage_bytes = {"select_tokens": 0.0, "gather_scatter": 0.0, "quant": 0.0, "select_columns": 0.0}
+        stage_bytes = {"select_tokens": 0.0, "gather_scatter": 0.0, "quant": 0.0, "select_columns": 0.0}
         pay_row = 2 * (self.d * w.bits // 8 + 4 * (self.d // w.group)) if w.bits != 16 else 2 * self.d * e
         for r in range(2, self.R + 1):
             sel = self.sels[r - 2]
@@ -232,91 +294,192 @@ class Bench:
             cand = prev.active_idx if prev is not None else None
             calls.append(("select_tokens", lib.fl_select_tokens,
                           (ctx, shp, r, p(self.G[r - 2]), p(self.G[r - 1]), p(cand), n_cand, w.k_tokens,
-                           p(sel.scores), p(sel.active_idx), p(sel.slot_of_pos), None, sp)))
+                           p(sel.scores), p(sel.active_idx), p(sel.slot_of_pos), None, sp), r))
             launches += 2
-            self.stage_bytes["select_tokens"] += 2.0 * n_cand * self.d * e + 8.0 * n_cand + 4.0 * sel.n + 4.0 * self.L
+            stage_bytes["select_tokens"] += 2.0 * n_cand * self.d * e + 8.0 * n_cand + 4.0 * sel.n + 4.0 * self.L
             n = sel.n
             for st in self.layers:
-                store = st.store
+                store = st.store if rows else st.store_plain
                 self.keep.append(store)
                 calls.append(("gather", lib.fl_gather_rows, (ctx, p(st.hidden), p(sel.active_idx), n, row_bytes,
-                                                             p(self.xbuf), sp)))
+                                                             p(self.xbuf), sp), r))
                 if r == 2:
                     calls.append(("select_columns", lib.fl_select_columns,
                                   (ctx, shp, p(st.col_scores), None, None, self.L, self.c, p(st.col_idx),
-                                   p(st.col_cnt), None, sp)))
+                                   p(st.col_cnt), None, sp), r))
                     launches += 1
                     tri = sum(min(self.L, (b + 1) * w.q_block) for b in range(self.nb))
-                    self.stage_bytes["select_columns"] += 4.0 * self.H * (tri + self.nb * (self.c + 1))
+                    stage_bytes["select_columns"] += 4.0 * self.H * (tri + self.nb * (self.c + 1))
                 q_new, k_new, v_new = st.rows[r]
                 calls.append(("quant", lib.fl_quant_kv_residual,
-                              (ctx, shp, r, p(k_new), p(v_new), p(sel.active_idx), n, C.byref(store), None, sp)))
+                              (ctx, shp, r, p(k_new), p(v_new), p(sel.active_idx), n, C.byref(store), None, sp), r))
                 # Q^(r-1), O^(r-1) are read from and O^(r), Q^(r) written to position-indexed stores by the attention
                 # call itself; loop 2 reads the pristine loop-1 stores and writes the work stores, so that every
                 # step starts from the same state
                 q_src = st.q_store if r == 2 else st.q_work
                 o_src = st.o_store if r == 2 else st.o_work
                 lse_prev = st.lse1 if r == 2 else st.lse_work
-                calls.append(("attention", lib.fl_loop_attention_indexed,
-                              (ctx, shp, r, p(q_new), p(q_src), p(st.q_work), p(sel.active_idx), n, C.byref(store),
-                               p(st.col_idx), p(st.col_cnt), self.c, p(lse_prev), p(st.lse_work),
-                               p(o_src), p(st.o_work), None, None, sp)))
+                if self.economy:
+                    carry = B.make_carry(st.bg_store, st.mass, r > 2)
+                    self.keep.append(carry)
+                    calls.append(("attention", lib.fl_loop_attention_indexed_carry,
+                                  (ctx, shp, r, p(q_new), p(q_src), p(st.q_work), p(sel.active_idx), n,
+                                   C.byref(store), p(st.col_idx), p(st.col_cnt), self.c, p(lse_prev), p(st.lse_work),
+                                   p(o_src), p(st.o_work), C.byref(carry), None, None, sp), r))
+                else:
+                    calls.append(("attention", lib.fl_loop_attention_indexed,
+                                  (ctx, shp, r, p(q_new), p(q_src), p(st.q_work), p(sel.active_idx), n,
+                                   C.byref(store), p(st.col_idx), p(st.col_cnt), self.c, p(lse_prev), p(st.lse_work),
+                                   p(o_src), p(st.o_work), None, None, sp), r))
                 launches += 3
-                self.stage_bytes["gather_scatter"] += 2.0 * n * row_bytes
-                self.stage_bytes["quant"] += 4.0 * n * self.d * e + n * pay_row * (r - 1)
+                stage_bytes["gather_scatter"] += 2.0 * n * row_bytes
+                stage_bytes["quant"] += 4.0 * n * self.d * e + n * pay_row * (r - 1)
             calls.append(("scatter", lib.fl_scatter_update, (ctx, p(self.xbuf), p(sel.active_idx), n, row_bytes,
-                                                             p(self.g_work), sp)))
+                                                             p(self.g_work), sp), r))
             launches += 1
-            self.stage_bytes["gather_scatter"] += 2.0 * n * row_bytes
-        self.calls, self.launches_per_step = calls, launches
-        self.n_attn = sum(1 for c_ in calls if c_[0] == "attention")
+            stage_bytes["gather_scatter"] += 2.0 * n * row_bytes
+        self.plans[key] = (calls, launches, stage_bytes)
+        return self.plans[key]
 
-    def run_step(self, attn_events=None, before_call=None):
-        """Issue one step on self.stream.  attn_events: list to which (start, end) event pairs are appended."""
+    def run_step(self, rows=True, attn_events=None):
+        """Issue one step on self.stream.  attn_events: list to which (loop, start, end) events are appended."""
         torch = self.torch
+        calls = self.plan(rows)[0]
         bad = 0
-        for i, (tag, fn, a) in enumerate(self.calls):
-            if before_call is not None:
-                before_call(i, tag)
+        for tag, fn, a, r in calls:
             if attn_events is not None and tag == "attention":
                 e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
                 e0.record(self.stream)
                 bad |= fn(*a)
                 e1.record(self.stream)
-                attn_events.append((e0, e1))
+                attn_events.append((r, e0, e1))
             else:
                 bad |= fn(*a)
         if bad:
             raise RuntimeError("a C-ABI call failed inside the step")
 
-    def breakdown(self):
-        """One untimed-for-the-metric pass with events around every call: per-stage GPU time (ms) and the time of
-        each loop r (select_tokens of loop r up to the call before loop r + 1)."""
+    def breakdown(self, rows=True):
+        """One untimed-for-the-metric pass with events around every call: per-stage GPU time (ms), per stage and
+        loop, and the time of each loop r (select_tokens of loop r up to the call before loop r + 1)."""
         torch = self.torch
         evs = []
         with torch.cuda.stream(self.stream):
-            for tag, fn, a in self.calls:
+            for tag, fn, a, r in self.plan(rows)[0]:
                 e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
                 e0.record(self.stream); rc = fn(*a); e1.record(self.stream)
                 assert rc == 0
-                evs.append((tag, e0, e1))
+                evs.append((tag, e0, e1, r))
         self.stream.synchronize()
-        out = {}
-        for tag, e0, e1 in evs:
-            out[tag] = out.get(tag, 0.0) + e0.elapsed_time(e1)
-        starts = [i for i, (tag, _, _) in enumerate(evs) if tag == "select_tokens"] + [len(evs)]
+        out, by_loop = {}, {}
+        for tag, e0, e1, r in evs:
+            ms = e0.elapsed_time(e1)
+            out[tag] = out.get(tag, 0.0) + ms
+            d = by_loop.setdefault(f"loop_{r}", {})
+            d[tag] = d.get(tag, 0.0) + ms
+        starts = [i for i, (tag, _, _, _) in enumerate(evs) if tag == "select_tokens"] + [len(evs)]
         per_loop = {}
         for li in range(len(starts) - 1):
             ms = evs[starts[li]][1].elapsed_time(evs[starts[li + 1] - 1][2])
-            per_loop[f"loop_{li + 2}"] = {"ms": round(ms, 4), "tokens_per_s": round(self.L / (ms * 1e-3), 1)}
+            per_loop[f"loop_{li + 2}"] = {"ms": round(ms, 4), "tokens_per_s": round(self.L / (ms * 1e-3), 1),
+                                          "stages_ms": {k: round(v, 4) for k, v in by_loop[f"loop_{li + 2}"].items()}}
         self.per_loop = per_loop
         return {k: round(v, 4) for k, v in out.items()}
+
+    def time_graph(self, rows, steps, barrier):
+        """Captures one step into a CUDA graph and times `steps` replays with CUDA events on the stream."""
+        torch = self.torch
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=self.stream):
+            self.run_step(rows)
+        with torch.cuda.stream(self.stream):
+            for _ in range(2):
+                graph.replay()
+        barrier()
+        t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+        host_t0 = time.perf_counter()
+        with torch.cuda.stream(self.stream):
+            t0.record(self.stream)
+            for _ in range(steps):
+                graph.replay()
+            t1.record(self.stream)
+        host_issue_ms = (time.perf_counter() - host_t0) * 1e3 / steps
+        barrier()
+        return t0.elapsed_time(t1) / steps, host_issue_ms
 
 
 def kv_bytes_per_token(bench):
     B, w = bench.B, bench.w
     fl, dense = B.fl_kv_store_bytes(bench.shape, bench.layers[0].store, w.n_loops, w.n_layers)
     return fl / w.L, dense / w.L
+
+
+def attention_roofline(bench, attn_events, steps, peaks, workload_key):
+    """Roofline of the attention launches (the dominant kernel) from the live event timings: the whole set and per
+    loop.  FLOPs are the minimum the method needs (old term counted only where it must be recomputed: loop 2); the
+    count the kernel executes is printed beside it."""
+    P_tc, BW = peaks["bf16_tflops"] * 1e12, peaks["hbm_gbs"] * 1e9
+    per_loop, tot_ms, tot_fmin, tot_fexec, tot_b, tot_roof = {}, 0.0, 0.0, 0.0, 0.0, 0.0
+    n_launch = 0
+    for r in sorted(bench.attn_flops_min):
+        ms = [a.elapsed_time(b) for rr, a, b in attn_events if rr == r]
+        if not ms:
+            continue
+        avg = sum(ms) / len(ms)
+        fmin = sum(bench.attn_flops_min[r]) / len(bench.attn_flops_min[r])
+        fexec = sum(bench.attn_flops_exec[r]) / len(bench.attn_flops_exec[r])
+        byt = sum(bench.attn_bytes[r]) / len(bench.attn_bytes[r])
+        t_roof = max(fmin / P_tc, byt / BW)
+        traffic = NCU_ATTN_TRAFFIC_BYTES.get((workload_key, "recompute" if fexec > 1.5 * fmin or r == 2 else "economy"))
+        per_loop[f"loop_{r}"] = {"avg_launch_ms": avg, "launches_per_step": len(ms) // steps, "flops_min": fmin,
+                                 "flops_executed": fexec, "bytes": byt, "t_roof_us": t_roof * 1e6,
+                                 "bound": "tensor" if fmin / P_tc >= byt / BW else "hbm",
+                                 "frac": t_roof / (avg * 1e-3), "tflops_min": fmin / (avg * 1e-3) / 1e12,
+                                 "traffic": traffic}
+        k = len(ms)
+        tot_ms += sum(ms); tot_fmin += fmin * k; tot_fexec += fexec * k; tot_b += byt * k; tot_roof += t_roof * k
+        n_launch += k
+    avg_ms = tot_ms / n_launch
+    flops, byt = tot_fmin / n_launch, tot_b / n_launch
+    if tot_fmin / P_tc >= tot_b / BW:
+        roof = {"bound": "tensor", "achieved": flops / (avg_ms * 1e-3) / 1e12, "peak": peaks["bf16_tflops"],
+                "unit": "TFLOP/s"}
+    else:
+        roof = {"bound": "hbm", "achieved": byt / (avg_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    traffics = [v["traffic"] for v in per_loop.values()]
+    roof.update({"kernel": "fl_loop_attention_indexed_carry", "kernel_name": "loop_attn_tc_kernel",
+                 "avg_launch_ms": avg_ms, "launches": n_launch // steps,
+                 "flops_per_launch": flops, "flops_executed_per_launch": tot_fexec / n_launch,
+                 "bytes_per_launch": byt,
+                 "flop_count": "minimum the method needs: both terms in loop 2 (dense source), the new term only in "
+                               "later loops over unchanged column sets; flops_executed is what the kernel ran",
+                 "frac_per_launch_roofs": tot_roof / (tot_ms * 1e-3),
+                 "traffic": (sum(t * v["launches_per_step"] for t, v in zip(traffics, per_loop.values())) /
+                             sum(v["launches_per_step"] for v in per_loop.values())) if all(t is not None for t in traffics) else None,
+                 "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum per launch of this shape, from the "
+                                   "captures summarised under profiles/; not measured in this run",
+                 "peak_source": peaks["source"],
+                 "avg_launch_ms_source": "CUDA events around every attention launch of K steps issued call by call on "
+                                         "the timed stream, right after the timed graph replays",
+                 "per_loop": per_loop})
+    return roof
+
+
+def step_roofline(bench, stage_bytes, peaks, ms):
+    """The benchmark spec's definition for the whole step: the slower of (all kept FLOPs at the tensor peak) and (all
+    algorithmic bytes at the HBM bandwidth); the sum of per-stage maxima is printed beside it for diagnosis."""
+    P_tc, BW = peaks["bf16_tflops"] * 1e12, peaks["hbm_gbs"] * 1e9
+    NL = bench.NL
+    F = sum(sum(v) / len(v) * NL for v in bench.attn_flops_min.values())
+    Bt = sum(sum(v) / len(v) * NL for v in bench.attn_bytes.values()) + sum(stage_bytes.values())
+    t_roof = max(F / P_tc, Bt / BW)
+    t_sum = sum(max(sum(bench.attn_flops_min[r]) / len(bench.attn_flops_min[r]) / P_tc,
+                    sum(bench.attn_bytes[r]) / len(bench.attn_bytes[r]) / BW) * NL for r in bench.attn_flops_min)
+    t_sum += sum(stage_bytes.values()) / BW
+    return {"t_roof_ms": t_roof * 1e3, "frac": t_roof * 1e3 / ms, "flops": F, "bytes": Bt,
+            "t_flops_ms": F / P_tc * 1e3, "t_bytes_ms": Bt / BW * 1e3,
+            "definition": "max(sum of kept FLOPs / bf16 peak, sum of algorithmic bytes / HBM copy bandwidth) over the step",
+            "sum_of_stage_maxima_ms": t_sum * 1e3, "frac_sum_of_stage_maxima": t_sum * 1e3 / ms}
 
 
 def run_ours(args):
@@ -328,9 +491,14 @@ def run_ours(args):
     device = f"cuda:{local}"
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device(device))
+    if args.workload == "c4":
+        run_sweep(args, device, rank)
+        if world > 1:
+            dist.destroy_process_group()
+        return
     w = get_workload(args)
     peaks = load_peaks()
-    bench = Bench(args, w, device)
+    bench = Bench(args, w, device, economy=not args.no_economy)
     stream = bench.stream
 
     def barrier():
@@ -339,74 +507,38 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
+    calls, launches_per_step, stage_bytes = bench.plan(True)
     with torch.cuda.stream(stream):
         for _ in range(max(args.warmup, 3)):
             bench.run_step()
     barrier()
     sampler = ClockSampler(local)
     sampler.start()
-    # The step (489 dependent launches at the default workload) is captured once into a CUDA graph; the timed region
-    # replays it K times. Events cannot sit between the kernels of a replay, so the attention launches are timed in a
-    # second pass of K steps issued call by call on the same stream, whose step time is reported next to the graph's.
-    graph = None
+    # The step (a few hundred dependent launches) is captured once into a CUDA graph; the timed region replays it K
+    # times. Events cannot sit between the kernels of a replay, so the attention launches are timed in a second pass
+    # of K steps issued call by call on the same stream, whose step time is reported next to the graph's.
+    host_issue_ms = None
+    ms_graph = None
     if not args.no_graph:
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph, stream=stream):
-            bench.run_step()
-        with torch.cuda.stream(stream):
-            for _ in range(2):
-                graph.replay()
-        barrier()
+        ms_graph, host_issue_ms = bench.time_graph(True, args.steps, barrier)
     attn_events = []
-    t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
     e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
-    host_t0 = time.perf_counter()
     with torch.cuda.stream(stream):
-        if graph is not None:
-            t0.record(stream)
-            for _ in range(args.steps):
-                graph.replay()
-            t1.record(stream)
-        host_issue_ms = (time.perf_counter() - host_t0) * 1e3 / args.steps
         e0.record(stream)
         for _ in range(args.steps):
-            bench.run_step(attn_events)
+            bench.run_step(True, attn_events)
         e1.record(stream)
     barrier()
     clocks = sampler.stop()
     ms_evented = e0.elapsed_time(e1) / args.steps
-    ms = t0.elapsed_time(t1) / args.steps if graph is not None else ms_evented
+    ms = ms_graph if ms_graph is not None else ms_evented
     ms = replicas.max_over_ranks(ms, world, device)
     value = replicas.job_throughput(w.L, world, ms)
 
-    # dominant kernel: loop attention
-    attn_ms = [a.elapsed_time(b) for a, b in attn_events]
-    avg_attn_ms = sum(attn_ms) / len(attn_ms)
-    flops = sum(bench.attn_flops) / len(bench.attn_flops)
-    byt = sum(bench.attn_bytes) / len(bench.attn_bytes)
-    t_tc = flops / (peaks["bf16_tflops"] * 1e12); t_hbm = byt / (peaks["hbm_gbs"] * 1e9)
-    if t_tc >= t_hbm:
-        roof = {"bound": "tensor", "achieved": flops / (avg_attn_ms * 1e-3) / 1e12, "peak": peaks["bf16_tflops"],
-                "unit": "TFLOP/s"}
-    else:
-        roof = {"bound": "hbm", "achieved": byt / (avg_attn_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
-                "unit": "GB/s"}
-    roof["frac"] = roof["achieved"] / roof["peak"]
-    roof.update({"kernel": "fl_loop_attention", "avg_launch_ms": avg_attn_ms, "launches": len(attn_ms) // args.steps,
-                 "flops_per_launch": flops, "bytes_per_launch": byt,
-                 "traffic": NCU_ATTN_TRAFFIC_BYTES if (args.workload == "c3" and not args.L) else None,
-                 "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum per launch of this shape, mean of "
-                                   "loops 2-4 (one capture, summary under profiles/)",
-                 "kernel_name": "loop_attn_tc_kernel", "peak_source": peaks["source"],
-                 "avg_launch_ms_source": "CUDA events around every attention launch of K steps issued call by call on "
-                                         "the timed stream, right after the timed graph replays",
-                 "share_of_step": sum(attn_ms) / args.steps / ms_evented})
-    # whole-step roofline: sum over stages of max(flops / tensor peak, bytes / HBM bandwidth)
-    t_roof = sum(max(f / (peaks["bf16_tflops"] * 1e12), b / (peaks["hbm_gbs"] * 1e9))
-                 for f, b in zip(bench.attn_flops, bench.attn_bytes))
-    t_roof += sum(bench.stage_bytes.values()) / (peaks["hbm_gbs"] * 1e9)
-    step_roof = {"t_roof_ms": t_roof * 1e3, "frac": t_roof * 1e3 / ms,
-                 "definition": "sum over stages of max(kept FLOPs / bf16 peak, algorithmic bytes / HBM copy bandwidth)"}
+    wl_key = f"{args.workload}:L={w.L}"
+    roof = attention_roofline(bench, attn_events, args.steps, peaks, wl_key)
+    roof["share_of_step"] = sum(a.elapsed_time(b) for _, a, b in attn_events) / args.steps / ms_evented
+    step_roof = step_roofline(bench, stage_bytes, peaks, ms)
 
     out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
            "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
@@ -414,19 +546,44 @@ def run_ours(args):
            "config": {"workload": f"{w.name}: L={w.L}, {w.n_layers} layers, d={w.d}, {w.n_heads}x{w.head_dim} MHA, "
                                   f"R={w.n_loops}, token budget {w.k_tokens} rows, column budget {w.col_budget}, "
                                   f"q_block {w.q_block}, int{w.bits} g{w.group} residuals",
+                      "old_term": ("recomputed in loop 2, carried (background rows + mass) in later loops"
+                                   if bench.economy else "recomputed in every loop"),
                       "parallelism": "replicas only" if world > 1 else "single GPU",
                       "l2": "inputs exceed L2 (each step streams the per-layer stores, far above 126 MB)"},
-           "gpu_launches": bench.launches_per_step * args.steps, "host_issue_ms_per_step": host_issue_ms,
-           "launch_mode": ("CUDA graph of one step, replayed" if graph is not None else "call by call"),
+           "gpu_launches": launches_per_step * args.steps, "host_issue_ms_per_step": host_issue_ms,
+           "launch_mode": ("CUDA graph of one step, replayed" if ms_graph is not None else "call by call"),
            "ms_per_step_call_by_call_with_events": ms_evented,
            "clocks": clocks, "roofline": roof,
-           "step_roofline": step_roof}
+           "step_roofline": step_roof,
+           "setup_ms": {k: round(v, 3) for k, v in bench.setup_ms.items()},
+           "scaffold_ms": {k: round(v, 4) for k, v in bench.scaffold_ms.items()}}
     fl_b, dense_b = kv_bytes_per_token(bench)
     out["kv_bytes_per_token"] = {"flashloop": fl_b * w.n_layers, "dense_looped": dense_b * w.n_layers,
                                  "ratio": dense_b / fl_b, "per": "token, all layers"}
     if rank == 0:
         out["breakdown_ms"] = bench.breakdown()
         out["per_loop"] = bench.per_loop
+    if not args.no_variants and not args.no_graph:
+        # stage (4) as the paper words it: the packed residual streams are read, dequantized and added inside the
+        # attention kernel (no materialized rows); same step otherwise
+        with torch.cuda.stream(stream):
+            for _ in range(3):
+                bench.run_step(False)
+        barrier()
+        ms_b, _ = bench.time_graph(False, args.steps, barrier)
+        ev_b = []
+        with torch.cuda.stream(stream):
+            bench.run_step(False, ev_b)
+        barrier()
+        ms_b = replicas.max_over_ranks(ms_b, world, device)
+        out["variants"] = {"in_kernel_dequantize_and_add": {
+            "ms_per_step": ms_b, "value": replicas.job_throughput(w.L, world, ms_b), "unit": UNIT,
+            "attention_avg_launch_ms": {f"loop_{r}": (lambda v: sum(v) / len(v))([a.elapsed_time(b) for rr, a, b in ev_b if rr == r])
+                                        for r in sorted(set(rr for rr, _, _ in ev_b))},
+            "note": "fl_quant_kv_residual writes no rows; the attention kernel rebuilds every selected column that is "
+                    "active in the loop from base + residual streams (Eq. 8) on its way into shared memory"}}
+        if rank == 0:
+            out["variants"]["in_kernel_dequantize_and_add"]["breakdown_ms"] = bench.breakdown(False)
     if not args.no_e2e:
         out["e2e"] = run_e2e(bench, args, world, barrier)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -435,6 +592,46 @@ def run_ours(args):
         print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()
+
+
+SWEEP_SUBSET = [(R, t, c, b) for R in (2, 4, 8, 16) for t in (0.10,) for c in (512,) for b in (4,)] + \
+               [(4, t, 512, 4) for t in (0.05, 0.25, 0.50)] + [(4, 0.10, c, 4) for c in (128, 2048)] + \
+               [(4, 0.10, 512, b) for b in (2, 8)]
+
+
+def run_sweep(args, device, rank):
+    """Config 4: one layer at L = 8192; R x token budget x column budget x bit width.  Each point: the step as a
+    CUDA graph, K replays timed with CUDA events.  Prints one JSON line holding the table."""
+    import torch
+    from paper_2609_29812_b200 import workloads
+    pts = SWEEP_SUBSET if args.sweep == "subset" else \
+        [(R, t, c, b) for R in (2, 4, 8, 16) for t in (0.05, 0.10, 0.25, 0.50) for c in (128, 512, 2048) for b in (2, 4, 8)]
+    peaks = load_peaks()
+    rows = []
+    barrier = torch.cuda.synchronize
+    for (R, t, c, b) in pts:
+        w = workloads.replace(workloads.sweep_point(R, t, c, b, L=args.L or 8192), rmsnorm=False)
+        bench = Bench(args, w, device, economy=not args.no_economy)
+        calls, launches, stage_bytes = bench.plan(True)
+        with torch.cuda.stream(bench.stream):
+            for _ in range(3):
+                bench.run_step()
+        barrier()
+        ms, _ = bench.time_graph(True, args.steps, barrier)
+        sr = step_roofline(bench, stage_bytes, peaks, ms)
+        fl_b, dense_b = kv_bytes_per_token(bench)
+        rows.append({"R": R, "token_frac": t, "c": c, "bits": b, "ms_per_step": round(ms, 4),
+                     "tokens_per_s": round(w.L / (ms * 1e-3), 1), "step_roofline_frac": round(sr["frac"], 4),
+                     "kv_ratio": round(dense_b / fl_b, 3), "launches": launches})
+        del bench
+        torch.cuda.empty_cache()
+    if rank == 0:
+        print(json.dumps({"metric": METRIC, "unit": UNIT, "n_gpus": 1, "steps": args.steps, "warmup": 3,
+                          "higher_is_better": True, "dtype": "bf16", "data": "synthetic",
+                          "config": {"workload": f"c4 sweep ({args.sweep}): one layer, L={args.L or 8192}, "
+                                                 "d=2048, 16x128 MHA, g128 residuals"},
+                          "value": statistics.median([r_["tokens_per_s"] for r_ in rows]),
+                          "sweep": rows}))
 
 
 def run_e2e(bench, args, world, barrier):
@@ -455,19 +652,14 @@ def run_e2e(bench, args, world, barrier):
     out_host = torch.empty_like(bench.o_out_buf, device="cpu").pin_memory()
     d2h = out_host.numel() * out_host.element_size() * (bench.R - 1)
     # which call index starts each (loop) and each (layer, loop)
+    calls = bench.plan(True)[0]
     marks = {}
-    li, r = -1, 1
-    for i, (tag, fn, a) in enumerate(bench.calls):
+    li = -1
+    for i, (tag, fn, a, r) in enumerate(calls):
         if tag == "select_tokens":
-            r += 1; li = -1; marks[i] = ("G", r)
+            li = -1; marks[i] = ("G", r)
         elif tag == "quant":
             li += 1; marks[i] = (li, r)
-
-    loop_of_call, r_cur = {}, 1
-    for i, (tag, fn, a) in enumerate(bench.calls):
-        if tag == "select_tokens":
-            r_cur += 1
-        loop_of_call[i] = r_cur
 
     def one_step():
         events = {}
@@ -481,16 +673,16 @@ def run_e2e(bench, args, world, barrier):
                     for j, t in enumerate(bench.layers[key[0]].rows[key[1]]):
                         t.copy_(host[(key[0], key[1], j)], non_blocking=True)
                 ev = torch.cuda.Event(); ev.record(copy_stream); events[i] = ev
-        n_calls = len(bench.calls)
+        n_calls = len(calls)
         with torch.cuda.stream(bench.stream):
-            for i, (tag, fn, a) in enumerate(bench.calls):
+            for i, (tag, fn, a, r) in enumerate(calls):
                 if i in events:
                     bench.stream.wait_event(events[i])
                 rc = fn(*a)
                 assert rc == 0
-                end_of_loop = i == n_calls - 1 or bench.calls[i + 1][0] == "select_tokens"
+                end_of_loop = i == n_calls - 1 or calls[i + 1][0] == "select_tokens"
                 if end_of_loop:                        # result of the loop: the last layer's new attention rows
-                    sel = bench.sels[loop_of_call[i] - 2]
+                    sel = bench.sels[r - 2]
                     rc = bench.B.fl_gather_rows(bench.ctx, bench.layers[-1].o_work, sel.active_idx, sel.n,
                                                 bench.d * 2, bench.o_out_buf, stream=bench.sp)
                     out_host.copy_(bench.o_out_buf, non_blocking=True)

@@ -331,7 +331,9 @@ class Bench:
                                   (ctx, shp, r, p(q_new), p(q_src), p(st.q_work), p(sel.active_idx), n,
                                    C.byref(store), p(st.col_idx), p(st.col_cnt), self.c, p(lse_prev), p(st.lse_work),
                                    p(o_src), p(st.o_work), None, None, sp), r))
-                launches += 3
+                # gather, quantization, attention; with the carried old term and the materialized rows the recomputing
+                # call of loop 2 is two launches (old-term pass, new-term pass)
+                launches += 3 + (1 if (self.economy and rows and r == 2) else 0)
                 stage_bytes["gather_scatter"] += 2.0 * n * row_bytes
                 stage_bytes["quant"] += 4.0 * n * self.d * e + n * pay_row * (r - 1)
             calls.append(("scatter", lib.fl_scatter_update, (ctx, p(self.xbuf), p(sel.active_idx), n, row_bytes,

@@ -89,6 +89,8 @@ extern "C" int fl_create(fl_ctx** out, int device) {
   }
   const char* env = std::getenv("FL_FORCE_SIMT");
   c->force_simt = (env != nullptr && env[0] == '1') ? 1 : 0;
+  const char* fused = std::getenv("FL_FUSED_ATTN");
+  c->fused_attn = (fused != nullptr && fused[0] == '1') ? 1 : 0;
   c->encode_tiled = nullptr;
   {
     void* fn = nullptr;

@@ -13,6 +13,13 @@ int fl_launch_loop_attn_tc(fl_ctx* ctx, const fl_shape* s, int loop_r, const voi
                            void* o_out, int indexed, void* q_store, const fl_attn_carry* carry, int32_t* status,
                            cudaStream_t st);
 
+// the same call as one or two single-term launches (needs the loop's materialized rows and the carried buffers)
+int fl_launch_loop_attn_stream(fl_ctx* ctx, const fl_shape* s, int loop_r, const void* q_new, const void* q_store_in,
+                               void* q_store_out, const int32_t* active_idx, int n_active, const fl_kv_store* store,
+                               const int32_t* col_idx, const int32_t* col_cnt, int c, const float* lse_in,
+                               float* lse_out, const void* o_store_in, void* o_store_out, const fl_attn_carry* carry,
+                               int32_t* status, cudaStream_t st);
+
 // whether the tensor-path kernel has a build for this request (storage type, head dimension, column budget, shared memory)
 bool fl_loop_attn_tc_covers(const fl_ctx* ctx, const fl_shape* s, int c);
 
@@ -321,8 +328,15 @@ extern "C" int fl_loop_attention_indexed_carry(fl_ctx* ctx, const fl_shape* shap
                                     sizeof(float) * (size_t)shape->n_heads * fl_n_blocks(shape) * c, st));
     return FL_OK;
   }
-  rc = fl_launch_loop_attn_tc(ctx, shape, loop_r, q_new, q_store_in, active_idx, n_active, store, col_idx, col_cnt, c,
-                              lse_in, lse_out, o_store_in, o_store_out, 1, q_store_out, carry, status, st);
+  // With the carried buffers and the loop's materialized rows the two terms run as single-term launches (two CTAs
+  // per SM); everything else takes the fused kernel.
+  rc = FL_ERR_UNSUPPORTED;
+  if (carry != nullptr && !ctx->fused_attn)
+    rc = fl_launch_loop_attn_stream(ctx, shape, loop_r, q_new, q_store_in, q_store_out, active_idx, n_active, store,
+                                    col_idx, col_cnt, c, lse_in, lse_out, o_store_in, o_store_out, carry, status, st);
+  if (rc == FL_ERR_UNSUPPORTED)
+    rc = fl_launch_loop_attn_tc(ctx, shape, loop_r, q_new, q_store_in, active_idx, n_active, store, col_idx, col_cnt,
+                                c, lse_in, lse_out, o_store_in, o_store_out, 1, q_store_out, carry, status, st);
   if (rc != FL_OK || col_scores_next == nullptr) return rc;
   DevSide kside;
   fl_dev_side(store, true, &kside);

@@ -91,6 +91,8 @@ extern "C" int fl_create(fl_ctx** out, int device) {
   c->force_simt = (env != nullptr && env[0] == '1') ? 1 : 0;
   const char* fused = std::getenv("FL_FUSED_ATTN");
   c->fused_attn = (fused != nullptr && fused[0] == '1') ? 1 : 0;
+  const char* two_pass = std::getenv("FL_TWO_PASS");
+  c->two_pass = (two_pass != nullptr && two_pass[0] == '1') ? 1 : 0;
   c->encode_tiled = nullptr;
   {
     void* fn = nullptr;

@@ -328,10 +328,12 @@ extern "C" int fl_loop_attention_indexed_carry(fl_ctx* ctx, const fl_shape* shap
                                     sizeof(float) * (size_t)shape->n_heads * fl_n_blocks(shape) * c, st));
     return FL_OK;
   }
-  // With the carried buffers and the loop's materialized rows the two terms run as single-term launches (two CTAs
-  // per SM); everything else takes the fused kernel.
+  // With the carried buffers and the loop's materialized rows a call that reuses the old term runs the single-term
+  // kernel (new term only, two CTAs per SM). A recomputing call stays on the fused kernel, whose two terms share the
+  // gathered tiles of every column without a payload in this loop (the gathers are what bounds these kernels);
+  // FL_TWO_PASS=1 at fl_create sends it through the single-term kernel twice instead (old-term pass, new-term pass).
   rc = FL_ERR_UNSUPPORTED;
-  if (carry != nullptr && !ctx->fused_attn)
+  if (carry != nullptr && !ctx->fused_attn && (carry->reuse != 0 || ctx->two_pass))
     rc = fl_launch_loop_attn_stream(ctx, shape, loop_r, q_new, q_store_in, q_store_out, active_idx, n_active, store,
                                     col_idx, col_cnt, c, lse_in, lse_out, o_store_in, o_store_out, carry, status, st);
   if (rc == FL_ERR_UNSUPPORTED)

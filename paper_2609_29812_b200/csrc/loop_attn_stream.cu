@@ -14,9 +14,11 @@
 // A CTA computes one (query block, head) problem with ONE pipeline, which leaves room for two CTAs per SM (half the
 // shared memory, half the tensor memory, 256 threads each): the second CTA's gathers, MMAs and exponentials fill the
 // gaps that the dependent chain  QK^T -> exponentials -> PV  leaves in the first one's, and one CTA's prologue and
-// epilogue run under the other's main loop.
+// epilogue run under the other's main loop. (cudaOccupancyMaxActiveBlocksPerMultiprocessor answers 1 for any kernel
+// that allocates tensor memory; two CTAs of 256 columns each do run side by side.) What bounds the pair is the rate
+// at which an SM's TMA unit takes four-row gathers: a 32 KB chunk per ~1.3 k cycles with eight issuing warps.
 //
-// Warp roles (8 warps): 0-3 softmax (one row of the 128-row tile per thread), 4 the MMA issuer (one thread), 5-7 TMA:
+// Warp roles (9 warps): 0-3 softmax (one row of the 128-row tile per thread), 4 the MMA issuer (one thread), 5-8 TMA:
 // the Q tile, then per chunk of 64 columns the K tile and the V tile, each gathered four rows per copy
 // (cp.async.bulk.tensor tile::gather4) into 128B-swizzled operand tiles. K and V have rings of their own (two tiles
 // each): a K tile is free again as soon as its QK^T has completed, long before the chunk's PV.
@@ -35,10 +37,10 @@ using namespace fl_tc;
 constexpr int kSmWarps = 4;
 constexpr int kIssueWarp = 4;
 constexpr int kTmaWarp = 5;
-constexpr int kTmaWarps = 3;
-constexpr int kWarps = 8;
+constexpr int kTmaWarps = 4;
+constexpr int kWarps = 9;
 constexpr int kThreads = kWarps * 32;
-constexpr int kColWarps = 6;                   // warps that read the column list in the prologue (the other two search rows)
+constexpr int kColWarps = 7;                   // warps that read the column list in the prologue (the other two search rows)
 constexpr int kMaxCols = 3072;
 constexpr int kMaxChunks = kMaxCols / kNC + 2;
 constexpr int kTileGathers = kTileBytes / 512; // 32 four-row gathers of 128-byte rows fill a K or V tile
@@ -638,6 +640,9 @@ int launch_mode(fl_ctx* ctx, int bits, dim3 grid, const StArgs& a, cudaStream_t 
   do {                                                                                                           \
     auto kern = loop_attn_stream_kernel<BITS, MODE>;                                                             \
     FL_CHECK_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kStSmemBytes));  \
+    /* two CTAs per SM need the SM's whole shared memory: ask for the largest carve-out */                      \
+    FL_CHECK_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout,                    \
+                                       (int)cudaSharedmemCarveoutMaxShared));                                   \
     FL_CHECK_CUDA(fl_launch(ctx, kern, grid, dim3(kThreads), kStSmemBytes, st, a));                             \
   } while (0)
   switch (bits) {

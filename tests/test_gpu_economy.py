@@ -236,3 +236,33 @@ def test_empty_column_sets_and_no_active_rows(env):
                                            st.col_cnt, st.c, None, st.lse, None, st.o_store,
                                            B.make_carry(st.bg_store, st.mass, True), None, status=st.status)
     assert rc == 0
+
+
+def test_two_pass_recompute_matches_oracle(env, monkeypatch):
+    """FL_TWO_PASS=1 (read when a context is created): a recomputing call with carried buffers runs as an old-term
+    launch followed by a new-term launch of the single-term kernel; constant budgets, then shrinking token sets
+    (stale columns are rebuilt inside both passes)."""
+    B, P, _ = env
+    monkeypatch.setenv("FL_TWO_PASS", "1")
+    ctx = B.Context(0)
+    monkeypatch.delenv("FL_TWO_PASS")
+    for seed, k_tok in ((31, None), (32, [500, 240, 120])):
+        w = dataclasses.replace(small_bf16(L=2000, H=2, R=4), changed_fracs=(0.30, 0.15, 0.08))
+        x = workloads.make_layer_inputs(w, seed=seed)
+        ref = run_oracle(w, x, k_tok=k_tok)
+        st = P.LayerState(ctx, w)
+        st.dense_loop(to_dev(x.Q[0], w), to_dev(x.K[0], w), to_dev(x.V[0], w))
+        st.select_columns_dense()
+        for r in range(2, w.n_loops + 1):
+            rec = ref["loops"][r - 2]
+            sel = oracle_selection(P, w, ref, r)
+            act = rec["active"]
+            # every loop recomputes (two passes each): the old-term pass of loops 3, 4 reads what the new-term pass of
+            # the loop before wrote
+            o_rows, _ = st.sparse_loop(r, to_dev(x.Q[r - 1][act], w), to_dev(x.K[r - 1][act], w),
+                                       to_dev(x.V[r - 1][act], w), sel, indexed=True, carry="write")
+            st.check_status()
+            assert_attn_close(to_np(o_rows), rec["O_rows"], f"two-pass loop {r} O rows", carried=r)
+            ok = np.isfinite(rec["lse_rows"])
+            np.testing.assert_allclose(to_np(st.lse)[:, act][ok], rec["lse_rows"][ok], rtol=0, atol=5e-3 * (r - 1))
+    ctx.close()

@@ -3,6 +3,8 @@
 // reduction). Selection is an exact radix select on the order-preserving integer image of the float
 // scores, followed by an index-ordered compaction, so the result equals a full sort with the total
 // order (score descending, index ascending) and comes out ascending.
+#include <cstdlib>
+
 #include "fl_internal.cuh"
 
 namespace {
@@ -492,6 +494,247 @@ __global__ void __launch_bounds__(kSelThreads, 1) column_select_smem_kernel(cons
   }
 }
 
+// ------------------------------------------------------------------------------------------
+// Selection by a sampled pre-threshold (the common case: k much smaller than n, few exact ties at the boundary).
+// A regular sample of the keys gives a value that, with a margin of several standard deviations, lies below the
+// k-th largest key and above all but a few thousand keys. One coalesced pass over the scores collects every key at
+// or above it (key and position) in shared memory; the exact k-th largest and the tie break by position are then
+// found inside that short list, the winners are marked in a bit map over the positions, and the bit map is read
+// out in position order. Every decision is exact: the list is a superset of the top k whenever it holds at least k
+// keys, and whenever it does not (or is too long, or too many keys tie with the threshold) the CTA falls back to
+// the radix select over all keys.
+// ------------------------------------------------------------------------------------------
+constexpr int kCandCap = 6144;         // keys the candidate list can hold
+constexpr int kSample = 1024;          // one sampled key per thread
+constexpr int kTieCap = 1024;          // ties with the threshold that are ranked by position here
+constexpr int kBitmapWords = 8192;     // positions a problem may have: 32 * kBitmapWords
+
+struct SampledSmem {
+  SelectSmem generic;                  // fallback: radix select over all keys
+  uint32_t hist[256];
+  uint32_t prefix, rank, n_eq;
+  uint32_t n_cand, n_tie;
+  uint32_t warp_sum[32];
+  int32_t tie_idx[kTieCap];
+};
+
+// `rank`-th largest (1-based) of the keys the threads hold (KPT per thread, `valid` marks the real ones), by four
+// 8-bit radix passes with warp-aggregated shared-memory histograms. Returns the key; *rank_in_eq = how many of the
+// keys equal to it belong to the `rank` largest, *n_eq = how many keys equal it. All kSelThreads threads call it.
+template <int KPT>
+__device__ uint32_t block_kth_largest(const uint32_t (&key)[KPT], const bool (&valid)[KPT], uint32_t rank, SampledSmem& sm,
+                                      uint32_t* rank_in_eq, uint32_t* n_eq) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  uint32_t prefix = 0;
+  for (int shift = 24; shift >= 0; shift -= 8) {
+    for (int i = tid; i < 256; i += kSelThreads) sm.hist[i] = 0;
+    __syncthreads();
+    const uint32_t hi_mask = shift == 24 ? 0u : (0xFFFFFFFFu << (shift + 8));
+#pragma unroll
+    for (int q = 0; q < KPT; ++q) {
+      const bool on = valid[q] && (key[q] & hi_mask) == prefix;
+      const uint32_t digit = (key[q] >> shift) & 0xFFu;
+      const uint32_t active = __ballot_sync(0xffffffffu, on);
+      if (on) {
+        const uint32_t peers = __match_any_sync(active, digit);
+        if ((peers & ((1u << lane) - 1)) == 0) atomicAdd(&sm.hist[digit], (uint32_t)__popc(peers));
+      }
+    }
+    __syncthreads();
+    if (warp == 0) {
+      uint32_t local[8], sum = 0;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) { local[j] = sm.hist[lane * 8 + j]; sum += local[j]; }
+      uint32_t incl = sum;                    // inclusive suffix sum over the lanes (higher lanes = larger digits)
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t v = __shfl_down_sync(0xffffffffu, incl, o);
+        if (lane + o < 32) incl += v;
+      }
+      const uint32_t above = incl - sum;
+      if (above < rank && rank <= above + sum) {
+        uint32_t acc = above;
+        for (int j = 7; j >= 0; --j) {
+          if (rank <= acc + local[j]) {
+            sm.prefix = prefix | ((uint32_t)(lane * 8 + j) << shift);
+            sm.rank = rank - acc;
+            sm.n_eq = local[j];
+            break;
+          }
+          acc += local[j];
+        }
+      }
+    }
+    __syncthreads();
+    prefix = sm.prefix;
+    rank = sm.rank;
+  }
+  *rank_in_eq = rank;
+  *n_eq = sm.n_eq;
+  __syncthreads();
+  return prefix;
+}
+
+__global__ void __launch_bounds__(kSelThreads, 2) column_select_sampled_kernel(const float* __restrict__ col_scores,
+                                                                               const int32_t* __restrict__ cand_cols,
+                                                                               const int32_t* __restrict__ cand_cnt,
+                                                                               int stride, int c, int L, int q_block, int nb,
+                                                                               int vec_ok, int32_t* __restrict__ col_idx,
+                                                                               int32_t* __restrict__ col_cnt) {
+  // dynamic shared memory: the candidate list (keys, positions), then one bit per position of the problem
+  extern __shared__ __align__(16) uint32_t dyn_smem[];
+  uint32_t* cand_key = dyn_smem;
+  int32_t* cand_idx = reinterpret_cast<int32_t*>(dyn_smem + kCandCap);
+  uint32_t* bitmap = dyn_smem + 2 * kCandCap;
+  __shared__ SampledSmem sm;
+  fl_grid_wait();
+  fl_grid_release();
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  // later blocks have more candidates (causal prefix): they are dispatched first, the short ones fill the tail
+  const int h = blockIdx.x, b = gridDim.y - 1 - blockIdx.y;
+  const size_t prob = (size_t)h * nb + b;
+  const float* vals = col_scores + prob * stride;
+  const int32_t* cols = cand_cols != nullptr ? cand_cols + prob * stride : nullptr;
+  int n = cand_cols != nullptr ? __ldg(cand_cnt + prob) : min(L, (b + 1) * q_block);
+  n = max(0, min(n, stride));
+  const int k = min(c, n);
+  int32_t* out = col_idx + prob * c;
+  for (int i = k + tid; i < c; i += kSelThreads) out[i] = -1;
+  if (tid == 0) col_cnt[prob] = k;
+  if (k == 0) return;
+  if (k >= n) {   // everything is selected
+    for (int i = tid; i < n; i += kSelThreads) out[i] = cols != nullptr ? __ldg(cols + i) : i;
+    return;
+  }
+  // ---- a value below the k-th largest key: from a regular sample when the problem is too long to list whole ----
+  uint32_t thr_lo = 0;                                  // n <= kCandCap: every key is a candidate
+  if (n > kCandCap) {
+    const uint32_t skey[1] = {ordered_key(__ldg(vals + (size_t)tid * n / kSample))};
+    const bool sval[1] = {true};
+    // aim at population rank k + k/2 + 256: the count of keys above the sample's r-th largest has mean r n/m and
+    // standard deviation ~sqrt(r) n/m; the margin is several of those for the sizes this is used at, and a miss
+    // only costs the fallback
+    const uint64_t target = (uint64_t)k + (uint64_t)k / 2 + 256;
+    uint32_t r_s = (uint32_t)((target * kSample + n - 1) / n);
+    r_s = min(max(r_s, 1u), (uint32_t)kSample);
+    uint32_t dummy0, dummy1;
+    thr_lo = block_kth_largest<1>(skey, sval, r_s, sm, &dummy0, &dummy1);
+  }
+  if (tid == 0) { sm.n_cand = 0; sm.n_tie = 0; }
+  const int n_words = (n + 31) >> 5;
+  for (int i = tid; i < n_words; i += kSelThreads) bitmap[i] = 0u;
+  __syncthreads();
+  // ---- one pass over the scores: keys at or above the pre-threshold go to the list (any order) ---------------
+  {
+    const float4* v4 = reinterpret_cast<const float4*>(vals);
+    const int n4 = (n + 3) >> 2;
+    for (int base = 0; base < n4; base += kSelThreads) {
+      const int i = base + tid;
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (i < n4) {
+        if (vec_ok && i * 4 + 3 < n) v = __ldg(v4 + i);
+        else {
+          if (i * 4 + 0 < n) v.x = __ldg(vals + i * 4 + 0);
+          if (i * 4 + 1 < n) v.y = __ldg(vals + i * 4 + 1);
+          if (i * 4 + 2 < n) v.z = __ldg(vals + i * 4 + 2);
+          if (i * 4 + 3 < n) v.w = __ldg(vals + i * 4 + 3);
+        }
+      }
+      const uint32_t kk[4] = {ordered_key(v.x), ordered_key(v.y), ordered_key(v.z), ordered_key(v.w)};
+      bool on[4];
+      int mine = 0;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) { on[e] = i < n4 && i * 4 + e < n && kk[e] >= thr_lo; mine += on[e] ? 1 : 0; }
+      // one atomic per warp and step: lanes take consecutive places behind it
+      int incl = mine;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+      }
+      const int total = __shfl_sync(0xffffffffu, incl, 31);
+      if (total == 0) continue;
+      uint32_t at = 0;
+      if (lane == 31) at = atomicAdd(&sm.n_cand, (uint32_t)total);
+      at = __shfl_sync(0xffffffffu, at, 31) + (uint32_t)(incl - mine);
+#pragma unroll
+      for (int e = 0; e < 4; ++e)
+        if (on[e]) {
+          if (at < (uint32_t)kCandCap) { cand_key[at] = kk[e]; cand_idx[at] = i * 4 + e; }
+          ++at;
+        }
+    }
+  }
+  __syncthreads();
+  const uint32_t n_cand = sm.n_cand;
+  bool fallback = n_cand < (uint32_t)k || n_cand > (uint32_t)kCandCap;    // CTA-uniform
+  uint32_t thr = 0, take_eq = 0;
+  if (!fallback) {
+    // ---- the exact k-th largest inside the list ---------------------------------------------------------------
+    constexpr int KPT = kCandCap / kSelThreads;
+    uint32_t key[KPT];
+    bool valid[KPT];
+#pragma unroll
+    for (int q = 0; q < KPT; ++q) {
+      const uint32_t u = (uint32_t)(q * kSelThreads + tid);
+      valid[q] = u < n_cand;
+      key[q] = valid[q] ? cand_key[u] : 0u;
+    }
+    uint32_t n_eq;
+    thr = block_kth_largest<KPT>(key, valid, (uint32_t)k, sm, &take_eq, &n_eq);
+    // ties with the threshold: all of them, or the take_eq lowest positions
+    const bool rank_ties = take_eq < n_eq;
+    if (rank_ties && n_eq > (uint32_t)kTieCap) fallback = true;            // CTA-uniform (n_eq is)
+    if (!fallback) {
+#pragma unroll
+      for (int q = 0; q < KPT; ++q) {
+        if (!valid[q]) continue;
+        const int idx = cand_idx[q * kSelThreads + tid];
+        if (key[q] > thr || (key[q] == thr && !rank_ties)) atomicOr(&bitmap[idx >> 5], 1u << (idx & 31));
+        else if (key[q] == thr) sm.tie_idx[atomicAdd(&sm.n_tie, 1u)] = idx;
+      }
+      __syncthreads();
+      if (rank_ties) {
+        // a tie is taken when fewer than take_eq ties lie at lower positions
+        for (uint32_t t = tid; t < n_eq; t += kSelThreads) {
+          const int mine = sm.tie_idx[t];
+          uint32_t lower = 0;
+          for (uint32_t u = 0; u < n_eq; ++u) lower += sm.tie_idx[u] < mine ? 1u : 0u;
+          if (lower < take_eq) atomicOr(&bitmap[mine >> 5], 1u << (mine & 31));
+        }
+      }
+      __syncthreads();
+      // ---- read the bit map out in position order: every thread owns a run of words ----------------------------
+      const int per = (n_words + kSelThreads - 1) / kSelThreads;
+      const int w0 = tid * per, w1 = min(n_words, w0 + per);
+      uint32_t cnt = 0;
+      for (int w = w0; w < w1; ++w) cnt += __popc(bitmap[w]);
+      uint32_t incl = cnt;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+      }
+      if (lane == 31) sm.warp_sum[warp] = incl;
+      __syncthreads();
+      uint32_t before = incl - cnt;
+      for (int w = 0; w < warp; ++w) before += sm.warp_sum[w];
+      for (int w = w0; w < w1; ++w) {
+        uint32_t bits = bitmap[w];
+        while (bits) {
+          const int bit = __ffs(bits) - 1;
+          bits &= bits - 1;
+          const int i = w * 32 + bit;
+          out[before++] = cols != nullptr ? __ldg(cols + i) : i;
+        }
+      }
+      return;
+    }
+  }
+  // ---- fallback: the radix select over all keys (exact for every input) -------------------------------------
+  block_topk_ascending(vals, n, k, sm.generic, [&](int rank, int i) { out[rank] = cols != nullptr ? __ldg(cols + i) : i; });
+}
+
 // one block per (head, query block)
 __global__ void __launch_bounds__(kSelThreads) column_select_kernel(const float* __restrict__ col_scores,
                                                                     const int32_t* __restrict__ cand_cols,
@@ -566,9 +809,18 @@ extern "C" int fl_select_columns(fl_ctx* ctx, const fl_shape* shape, const float
   FL_REQUIRE(nb <= 65535);
   dim3 grid(shape->n_heads, nb);
   const size_t key_bytes = sizeof(uint32_t) * (((size_t)n_cand + 3) & ~(size_t)3);
-  if (n_cand <= kSelCap && key_bytes + 32768 <= (size_t)ctx->max_smem_optin) {
+  const int vec_ok = (fl_aligned16(col_scores) && n_cand % 4 == 0) ? 1 : 0;
+  const char* staged = std::getenv("FL_SELECT_STAGED");
+  if (n_cand <= 32 * kBitmapWords && !(staged != nullptr && staged[0] == '1')) {
+    // sampled pre-threshold, candidate list, bit map over the positions (exact; falls back inside the kernel)
+    const size_t dyn_bytes = sizeof(uint32_t) * (2 * (size_t)kCandCap + ((size_t)n_cand + 31) / 32);
+    FL_CHECK_CUDA(cudaFuncSetAttribute(column_select_sampled_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)dyn_bytes));
+    FL_CHECK_CUDA(fl_launch(ctx, column_select_sampled_kernel, grid, dim3(kSelThreads), dyn_bytes,
+                            static_cast<cudaStream_t>(stream), col_scores, cand_cols, cand_cnt, n_cand, c, shape->L,
+                            shape->q_block, nb, vec_ok, col_idx, col_cnt));
+  } else if (n_cand <= kSelCap && key_bytes + 32768 <= (size_t)ctx->max_smem_optin) {
     // keys staged in shared memory: the scores are read from global memory once
-    const int vec_ok = (fl_aligned16(col_scores) && n_cand % 4 == 0) ? 1 : 0;
     FL_CHECK_CUDA(cudaFuncSetAttribute(column_select_smem_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)key_bytes));
     FL_CHECK_CUDA(fl_launch(ctx, column_select_smem_kernel, grid, dim3(kSelThreads), key_bytes,

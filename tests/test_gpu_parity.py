@@ -474,3 +474,62 @@ def test_many_patched_columns_and_wide_budgets(env, rows, split):
         ok = np.isfinite(rec["lse_rows"])
         lse = lse.copy(); lse[:, act] = np.where(ok, rec["lse_rows"], lse[:, act]).astype(np.float32)
         q_prev_full = q_prev_full.copy(); q_prev_full[act] = x.Q[r - 1][act]
+
+
+def test_column_selection_exact_on_long_problems(env):
+    """fl_select_columns on problems too long to list whole (a sampled pre-threshold, a candidate list, the bit map
+    read-out) against brute force with the total order, for score distributions that stress every branch: heavy
+    tails, a plateau of exact ties across the boundary, all zeros (the in-kernel fallback), a budget too wide for
+    the candidate list, and a sparse source with a candidate list of columns."""
+    B, P, ctx = env
+    rng = np.random.default_rng(5)
+    L, q_block, H = 24576, 8192, 2
+    w = dataclasses.replace(workloads.config2(L=L, n_heads=H), q_block=q_block)
+    sh = P.shape_of(w)
+    nb = 3
+    def scores(kind):
+        s = np.zeros((H, nb, L), dtype=np.float32)
+        for h in range(H):
+            for b in range(nb):
+                if kind == "lognormal":
+                    v = np.exp(rng.standard_normal(L) * 3.0 - 6.0)
+                elif kind == "plateau":
+                    v = np.exp(rng.standard_normal(L) * 2.0 - 8.0)
+                    v[rng.permutation(L)[: L // 8]] = 0.125          # thousands of exact ties, some across the boundary
+                elif kind == "few_levels":
+                    v = rng.integers(0, 4, L).astype(np.float64)     # four values only: ties everywhere
+                else:
+                    v = np.zeros(L)
+                s[h, b] = v.astype(np.float32)
+        return s
+    for kind in ("lognormal", "plateau", "few_levels", "zeros"):
+        cs = scores(kind)
+        for c in (1, 300, 1024, 5000):
+            col_idx = torch.empty(H, nb, c, dtype=torch.int32, device="cuda")
+            col_cnt = torch.empty(H, nb, dtype=torch.int32, device="cuda")
+            B.fl_select_columns(ctx, sh, torch.from_numpy(cs).cuda(), None, None, L, c, col_idx, col_cnt)
+            idx, cnt = to_np(col_idx), to_np(col_cnt)
+            for h in range(H):
+                for b in range(nb):
+                    end = min(L, (b + 1) * q_block)
+                    k = min(c, end)
+                    assert cnt[h, b] == k and np.all(idx[h, b, k:] == -1)
+                    assert np.array_equal(idx[h, b, :k], fo.topk_ascending(cs[h, b, :end], k)), (kind, c, h, b)
+    # sparse source: candidates are a subset of the columns (ascending), scores aligned with the list
+    n_cand = 20000
+    cand = np.sort(rng.permutation(L)[:n_cand]).astype(np.int32)
+    cand_cols = np.broadcast_to(cand, (H, nb, n_cand)).copy()
+    cand_cnt = np.array([[n_cand, 9000, 0]] * H, dtype=np.int32)
+    cs = np.exp(rng.standard_normal((H, nb, n_cand)) * 3.0).astype(np.float32)
+    for c in (700, 10000):
+        col_idx = torch.empty(H, nb, c, dtype=torch.int32, device="cuda")
+        col_cnt = torch.empty(H, nb, dtype=torch.int32, device="cuda")
+        B.fl_select_columns(ctx, sh, torch.from_numpy(cs).cuda(), torch.from_numpy(cand_cols).cuda(),
+                            torch.from_numpy(cand_cnt).cuda(), n_cand, c, col_idx, col_cnt)
+        idx, cnt = to_np(col_idx), to_np(col_cnt)
+        for h in range(H):
+            for b in range(nb):
+                n = cand_cnt[h, b]
+                k = min(c, n)
+                assert cnt[h, b] == k and np.all(idx[h, b, k:] == -1)
+                assert np.array_equal(idx[h, b, :k], cand[fo.topk_ascending(cs[h, b, :n], k)]), (c, h, b)

@@ -282,9 +282,11 @@ int fl_launch_sparse_colscore(const fl_shape* s, const void* q_new, const int32_
   return fl_launch_status();
 }
 
+int fl_launch_dense_tc(fl_ctx* ctx, const fl_shape* s, const void* q, const void* k, const void* v, void* o, float* lse,
+                       float* col_scores, int32_t* status, cudaStream_t st);
+
 extern "C" int fl_dense_loop_attention(fl_ctx* ctx, const fl_shape* shape, const void* q, const void* k, const void* v,
                                        void* o, float* lse, float* col_scores, int32_t* status, void* stream) {
-  (void)status;
   FL_REQUIRE(ctx != nullptr);
   int rc = fl_check_shape(shape);
   if (rc != FL_OK) return rc;
@@ -293,6 +295,9 @@ extern "C" int fl_dense_loop_attention(fl_ctx* ctx, const fl_shape* shape, const
   FL_REQUIRE(col_scores == nullptr || lse != nullptr);
   FL_REQUIRE(shape->n_heads <= 65535 && fl_n_blocks(shape) <= 65535);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // tensor path (bf16 storage, head dimension 128); everything else runs on the binary32 kernels below
+  rc = fl_launch_dense_tc(ctx, shape, q, k, v, o, lse, col_scores, status, st);
+  if (rc != FL_ERR_UNSUPPORTED) return rc;
   if (shape->dtype == FL_F32)
     return shape->head_dim == 64 ? launch_dense<float, 64>(shape, q, k, v, o, lse, col_scores, st)
                                  : launch_dense<float, 128>(shape, q, k, v, o, lse, col_scores, st);

@@ -54,10 +54,13 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c3", choices=["c2", "c3", "c4", "c5"],
+    ap.add_argument("--loops", type=int, default=0, help="sched: number of loops R (default 8)")
+    ap.add_argument("--workload", default="c3", choices=["c2", "c3", "c4", "c5", "sched"],
                     help="c3: the 48-layer stack at 32K (default, the metric's configuration); c2: one layer at 8K; "
                          "c5: the 128K memory configuration (prefill part; 24 layers resident unless --layers); "
-                         "c4: the sparsity / depth sweep (one layer at 8K, a table of points)")
+                         "c4: the sparsity / depth sweep (one layer at 8K, a table of points); "
+                         "sched: budgets that decay from loop to loop with real column pruning (Table 6's deep "
+                         "schedule: tokens 90% -> 20%, columns pruned inside the previous set every loop)")
     ap.add_argument("--sweep", default="subset", choices=["subset", "full"], help="c4: which points to run")
     ap.add_argument("--no-economy", action="store_true", help="recompute the old term in every loop")
     ap.add_argument("--no-variants", action="store_true", help="skip the in-kernel dequantization variant")
@@ -493,8 +496,8 @@ def run_ours(args):
     device = f"cuda:{local}"
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device(device))
-    if args.workload == "c4":
-        run_sweep(args, device, rank)
+    if args.workload in ("c4", "sched"):
+        (run_sweep if args.workload == "c4" else run_schedule)(args, device, rank)
         if world > 1:
             dist.destroy_process_group()
         return
@@ -594,6 +597,134 @@ def run_ours(args):
         print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()
+
+
+def run_schedule(args, device, rank):
+    """Decaying schedule (Appendix E, Table 6, the deep model's row): the token budget falls linearly from 90% to 20%
+    of the prompt over loops 2..R and every loop prunes the column sets inside the previous ones (Appendix D.2, a
+    sparse source loop), from 2048 down to 256 columns per block.  The old term is recomputed in every loop (the
+    sets change), next-loop column scores are emitted by the attention call and fl_select_columns runs on candidate
+    lists.  Prints one JSON line: step time, tokens/s and the per-stage breakdown."""
+    import torch
+    from paper_2609_29812_b200 import binding as B, pipeline as P, workloads
+    L, R, NL = args.L or 8192, args.loops or 8, args.layers or 4
+    lin = lambda a, b: [a + (b - a) * i / max(R - 2, 1) for i in range(R - 1)]
+    tok_frac = lin(0.90, 0.20)
+    c_cols = [max(64, int(round(x / 64.0)) * 64) for x in lin(2048, 256)]
+    w = workloads.replace(workloads.sweep_point(R, tok_frac[0], c_cols[0], 4, L=L), name=f"sched_R{R}", rmsnorm=False,
+                          n_layers=NL, changed_fracs=tuple(tok_frac))
+    k_tok = [int(f * L + 0.5) for f in tok_frac]
+    ctx = B.Context(torch.device(device).index or 0)
+    sh = P.shape_of(w)
+    stream = torch.cuda.Stream(device=device)
+    sp = int(stream.cuda_stream)
+    stack = workloads.DeviceStack(w, seed=0, device=device)
+    G = stack.stack_hidden()
+    H, dh, d = w.n_heads, w.head_dim, w.d
+    nb = (L + w.q_block - 1) // w.q_block
+    lib = B.lib
+    p = lambda t: C.c_void_p(int(t.data_ptr())) if t is not None else None
+    calls, keep = [], []
+    with torch.cuda.stream(stream):
+        sels, cand = [], None
+        for r in range(2, R + 1):
+            sel = P.select_tokens(ctx, sh, r, G[r - 2], G[r - 1], cand, k_tok[r - 2])
+            sels.append(sel); cand = sel.active_idx
+        stream.synchronize()
+        xbuf = torch.empty(sels[0].n, d, dtype=torch.bfloat16, device=device)
+        g_work = G[0].clone()
+        layers = []
+        for l in range(NL):
+            gen = stack.layer(l)
+            st = P.LayerState(ctx, w, device)
+            st.dense_loop(*gen.qkv1())
+            st.hidden = gen.hidden(R)
+            st.lse1, st.lse_work = st.lse, st.lse.clone()
+            st.q_work, st.o_work = st.q_store.clone(), st.o_store.clone()
+            st.rows = {r: gen.rows(r, sels[r - 2].active_idx) for r in range(2, R + 1)}
+            for r in range(2, R + 1):
+                st.alloc_stream(sels[r - 2])
+            st.cols = {r: (torch.empty(H, nb, c_cols[r - 2], dtype=torch.int32, device=device),
+                           torch.empty(H, nb, dtype=torch.int32, device=device),
+                           torch.zeros(H, nb, c_cols[r - 2], dtype=torch.float32, device=device)) for r in range(2, R + 1)}
+            gen.release()
+            layers.append(st)
+        stream.synchronize()
+    launches = 0
+    for r in range(2, R + 1):
+        sel, prev = sels[r - 2], (sels[r - 3] if r > 2 else None)
+        n_cand = prev.n if prev is not None else L
+        calls.append(("select_tokens", lib.fl_select_tokens,
+                      (ctx.handle, C.byref(sh), r, p(G[r - 2]), p(G[r - 1]), p(prev.active_idx) if prev else None, n_cand,
+                       k_tok[r - 2], p(sel.scores), p(sel.active_idx), p(sel.slot_of_pos), None, sp)))
+        launches += 2
+        for st in layers:
+            ci, cc, cs = st.cols[r]
+            calls.append(("gather", lib.fl_gather_rows, (ctx.handle, p(st.hidden), p(sel.active_idx), sel.n, d * 2, p(xbuf), sp)))
+            if r == 2:
+                calls.append(("select_columns", lib.fl_select_columns,
+                              (ctx.handle, C.byref(sh), p(st.col_scores), None, None, L, c_cols[0], p(ci), p(cc), None, sp)))
+                launches += 1
+            q_new, k_new, v_new = st.rows[r]
+            keep.append(st.store)
+            calls.append(("quant", lib.fl_quant_kv_residual,
+                          (ctx.handle, C.byref(sh), r, p(k_new), p(v_new), p(sel.active_idx), sel.n, C.byref(st.store), None, sp)))
+            q_src, o_src, lse_prev = (st.q_store, st.o_store, st.lse1) if r == 2 else (st.q_work, st.o_work, st.lse_work)
+            last = r == R
+            calls.append(("attention", lib.fl_loop_attention_indexed,
+                          (ctx.handle, C.byref(sh), r, p(q_new), p(q_src), p(st.q_work), p(sel.active_idx), sel.n,
+                           C.byref(st.store), p(ci), p(cc), c_cols[r - 2], p(lse_prev), p(st.lse_work), p(o_src),
+                           p(st.o_work), None if last else p(cs), None, sp)))
+            launches += 3 + (0 if last else 1)
+            if not last:
+                ni, nc, _ = st.cols[r + 1]
+                calls.append(("prune_columns", lib.fl_select_columns,
+                              (ctx.handle, C.byref(sh), p(cs), p(ci), p(cc), c_cols[r - 2], c_cols[r - 1], p(ni), p(nc), None, sp)))
+                launches += 1
+        calls.append(("scatter", lib.fl_scatter_update, (ctx.handle, p(xbuf), p(sel.active_idx), sel.n, d * 2, p(g_work), sp)))
+        launches += 1
+
+    def step():
+        for tag, fn, a in calls:
+            assert fn(*a) == 0
+    with torch.cuda.stream(stream):
+        for _ in range(3):
+            step()
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=stream):
+        step()
+    with torch.cuda.stream(stream):
+        graph.replay()
+    torch.cuda.synchronize()
+    t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+    with torch.cuda.stream(stream):
+        t0.record(stream)
+        for _ in range(args.steps):
+            graph.replay()
+        t1.record(stream)
+    torch.cuda.synchronize()
+    ms = t0.elapsed_time(t1) / args.steps
+    evs = []
+    with torch.cuda.stream(stream):
+        for tag, fn, a in calls:
+            e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+            e0.record(stream); assert fn(*a) == 0; e1.record(stream)
+            evs.append((tag, e0, e1))
+    torch.cuda.synchronize()
+    brk = {}
+    for tag, e0, e1 in evs:
+        brk[tag] = brk.get(tag, 0.0) + e0.elapsed_time(e1)
+    fl_b, dense_b = B.fl_kv_store_bytes(sh, layers[0].store, R, NL)
+    if rank == 0:
+        print(json.dumps({"metric": METRIC, "value": L / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+                          "warmup": 3, "ms_per_step": ms, "higher_is_better": True, "dtype": "bf16", "data": "synthetic",
+                          "config": {"workload": f"decaying schedule: L={L}, {NL} layers, R={R}, token budgets {k_tok}, "
+                                                 f"column budgets {c_cols} (pruned inside the previous set), int4 g128"},
+                          "gpu_launches": launches * args.steps, "launch_mode": "CUDA graph of one step, replayed",
+                          "breakdown_ms": {k: round(v, 4) for k, v in brk.items()},
+                          "kv_bytes_per_token": {"flashloop": fl_b / L * NL, "dense_looped": dense_b / L * NL,
+                                                 "ratio": dense_b / fl_b}}))
 
 
 SWEEP_SUBSET = [(R, t, c, b) for R in (2, 4, 8, 16) for t in (0.10,) for c in (512,) for b in (4,)] + \

@@ -119,7 +119,9 @@ typedef struct {
  * h_prev, h_cur : [L, d] storage type.  cand: ascending positions [n_cand], or NULL for all L rows
  * (then n_cand must equal L).  Outputs: scores f32 [n_cand] (aligned with cand), active_idx int32
  * [min(k, n_cand)] ascending, slot_of_pos int32 [L] (rank in active_idx, or -1).
- * Inputs must be finite. Errors: null pointers, k < 1, n_cand < 1 or > L, loop_r < 2. */
+ * Inputs must be finite. Errors: null pointers, k < 1, n_cand < 1 or > L, loop_r < 2; FL_ERR_UNSUPPORTED unless
+ * d = H*dh is a multiple of 256 (a warp reads a row in 256-element steps). `status` is accepted for symmetry and never
+ * written: this call has no bounded device wait and checks nothing on the device. */
 FL_API int fl_select_tokens(fl_ctx* ctx, const fl_shape* shape, int loop_r, const void* h_prev, const void* h_cur,
                      const int32_t* cand, int32_t n_cand, int32_t k, float* scores, int32_t* active_idx,
                      int32_t* slot_of_pos, int32_t* status, void* stream);
@@ -144,7 +146,9 @@ FL_API int fl_scatter_update(fl_ctx* ctx, const void* src, const int32_t* idx, i
  * Xhat^(r-1)_i and Xhat^(r)_i = Xhat^(r-1)_i + (code * scale + zero), each rounded once to bf16.
  * k_new, v_new: [n_active, H, dh] storage type. store is a host struct; store->n_streams must be
  * >= loop_r - 1 (the stream being written counts). Errors: loop_r < 2 or > FL_MAX_LOOPS+1, bad bits or
- * group, null buffers, n_rows mismatch. n_active == 0 is a no-op. */
+ * group, null buffers, n_rows mismatch; FL_ERR_UNSUPPORTED unless d = H*dh is a multiple of 256, and of 2048 beyond
+ * 2048 (whole warps must walk a row together: the group reductions are sub-warp shuffles). n_active == 0 is a no-op.
+ * `status` is accepted for symmetry and never written. */
 FL_API int fl_quant_kv_residual(fl_ctx* ctx, const fl_shape* shape, int loop_r, const void* k_new, const void* v_new,
                          const int32_t* active_idx, int32_t n_active, const fl_kv_store* store,
                          int32_t* status, void* stream);
@@ -162,7 +166,8 @@ FL_API int fl_dense_loop_attention(fl_ctx* ctx, const fl_shape* shape, const voi
  *   cand_cols != NULL : sparse source. cand_cols int32 [H, nb, n_cand] ascending with cand_cnt[H, nb] valid
  *                       entries each; col_scores is [H, nb, n_cand], aligned with cand_cols.
  * Outputs: col_idx int32 [H, nb, c] ascending, padded with -1; col_cnt int32 [H, nb] = min(c, candidates).
- * n_cand is the row stride of the candidate arrays (L for a dense source). */
+ * n_cand is the row stride of the candidate arrays (L for a dense source). `status` is accepted for symmetry and never
+ * written. */
 FL_API int fl_select_columns(fl_ctx* ctx, const fl_shape* shape, const float* col_scores, const int32_t* cand_cols,
                       const int32_t* cand_cnt, int32_t n_cand, int32_t c, int32_t* col_idx, int32_t* col_cnt,
                       int32_t* status, void* stream);
@@ -174,8 +179,9 @@ FL_API int fl_select_columns(fl_ctx* ctx, const fl_shape* shape, const float* co
  * split cannot help the shape), the problems of that last wave are given to two CTAs each; the one that finishes
  * first leaves its partial accumulators there and the other adds them to its own, so the result does not depend on
  * which came first beyond the rounding order of that one addition. fl_set_workspace clears the arrival counters at the
- * head of the buffer on `stream` (every launch leaves them cleared); the buffer must stay valid until fl_destroy or
- * the next fl_set_workspace (NULL detaches it). Attention calls of one context that may overlap in time (different
+ * head of the buffer on `stream` (every launch leaves them cleared, also one that reported FL_ERR_TIMEOUT through the
+ * status word; the outputs of such a launch are undefined); the buffer must stay valid until fl_destroy or the next
+ * fl_set_workspace (NULL detaches it). Attention calls of one context that may overlap in time (different
  * streams) must not share a workspace. */
 FL_API int fl_loop_attention_workspace_bytes(fl_ctx* ctx, const fl_shape* shape, int64_t* bytes /* host */);
 FL_API int fl_set_workspace(fl_ctx* ctx, void* workspace /* device */, int64_t bytes, void* stream);

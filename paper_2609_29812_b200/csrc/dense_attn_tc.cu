@@ -430,6 +430,225 @@ __global__ void __launch_bounds__(kThreads, 2) dense_colsum_kernel(const __grid_
   if (tid == 0 && ctl.abort_flag && a.status != nullptr) atomicExch(a.status, (int)FL_ERR_TIMEOUT);
 }
 
+// ------------------------------------------------------------------------------------------------------------
+// Next-loop column scores of a SPARSE loop (Appendix D.2: a sparse source loop offers its own selected columns as
+// candidates, scored by the block sums of its new probabilities): the same K Q^T tiles, with the 128 keys of a tile
+// gathered by position from the base (four rows per TMA copy) and the columns that carry residual payloads rebuilt
+// in place (Eq. 8 chain up to the loop itself), and the queries taken from the compact rows of the block's active
+// tokens. col_scores_next[h, b, u] = sum over the block's active rows i >= S[u] of exp(s_iu - lse_i), lse the loop's
+// new log-normaliser.
+// ------------------------------------------------------------------------------------------------------------
+struct alignas(64) SpArgs {
+  CUtensorMap k_map;      // K base [L, d], box 64 x 1 (row gathers)
+  CUtensorMap q_map;      // compact new Q rows [n_active, d], box 64 x 128
+  DevSide k;
+  int n_use;              // residual streams contained in Khat^(r): loop_r - 1
+  const int32_t* active_idx;
+  int n_active;
+  const int32_t* col_idx;
+  const int32_t* col_cnt;
+  int c;
+  const float* lse;       // [H, L]: the loop's new log-normalisers
+  float* out;             // [H, nb, c]
+  int32_t* status;
+  int L, H, d, q_block, nb, group;
+  float scale;
+};
+
+struct __align__(16) SpColsumCtl {
+  uint64_t k_full, k_ready, q_full[2], d_full[2], d_free[2];
+  uint32_t tmem_base;
+  int abort_flag;
+  int q_lo, q_hi;
+  float lse2[2][kM];
+  int pos[2][kM];
+};
+constexpr size_t kSpColsumSmem = 1024 + 3 * kQTileBytes + sizeof(SpColsumCtl);
+
+template <int BITS>
+__global__ void __launch_bounds__(kThreads, 2) sparse_colsum_kernel(const __grid_constant__ SpArgs a) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* k_tile = smem;
+  uint8_t* q_ring = smem + kQTileBytes;
+  SpColsumCtl& ctl = *reinterpret_cast<SpColsumCtl*>(q_ring + 2 * kQTileBytes);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int kc = blockIdx.x, b = blockIdx.y, h = blockIdx.z;
+  const size_t prob = (size_t)h * a.nb + b;
+  const int cnt = min(__ldg(a.col_cnt + prob), a.c);
+  const int u0 = kc * kM;
+  if (u0 >= cnt) return;
+  const int32_t* cols = a.col_idx + prob * a.c;
+  if (warp < 2) {
+    const int target = warp == 0 ? b * a.q_block : min(a.L, (b + 1) * a.q_block);
+    int below;
+    const int r = lower_bound_warp(a.active_idx, a.n_active, target, lane, &below);
+    if (lane == 0) { if (warp == 0) ctl.q_lo = r; else ctl.q_hi = r; }
+  }
+  if (tid == 0) {
+    tc::mbar_init(&ctl.k_full, 1);
+    tc::mbar_init(&ctl.k_ready, 4);
+    for (int s = 0; s < 2; ++s) {
+      tc::mbar_init(&ctl.q_full[s], 2);
+      tc::mbar_init(&ctl.d_full[s], 1);
+      tc::mbar_init(&ctl.d_free[s], 4);
+    }
+    ctl.abort_flag = 0;
+    tc::fence_barrier_init();
+  }
+  __syncthreads();
+  const int q_lo = ctl.q_lo, q_hi = ctl.q_hi;
+  if (q_hi <= q_lo) {   // no active row in the block: every score is zero
+    for (int u = u0 + tid; u < min(cnt, u0 + kM); u += kThreads) a.out[prob * a.c + u] = 0.f;
+    return;
+  }
+  if (warp == kIssueWarp) {
+    tc::tmem_alloc(&ctl.tmem_base, kTmemCols);
+    tc::tmem_relinquish();
+  }
+  tc::tc_fence_before();
+  __syncthreads();
+  tc::tc_fence_after();
+  const uint32_t tmem = ctl.tmem_base;
+  volatile int* abort_flag = &ctl.abort_flag;
+  const int n_tiles = (q_hi - q_lo + kM - 1) / kM;
+
+  if (warp == kTmaWarp) {
+    // the tile's 128 selected columns: base rows by position, four per copy; positions past the count read as zero
+    if (lane == 0) tc::mbar_arrive_expect_tx(&ctl.k_full, kQTileBytes);
+    __syncwarp();
+    {
+      int y[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int u = u0 + lane * 4 + i;
+        y[i] = u < cnt ? __ldg(cols + u) : a.L;
+      }
+      tc::tma_gather4(k_tile + lane * 512, &a.k_map, &ctl.k_full, h * kDH, y[0], y[1], y[2], y[3]);
+      tc::tma_gather4(k_tile + kM * 128 + lane * 512, &a.k_map, &ctl.k_full, h * kDH + 64, y[0], y[1], y[2], y[3]);
+    }
+    bool ok = true;
+    for (int t = 0; t < n_tiles && ok; ++t) {
+      const int sl = t & 1, s0 = q_lo + t * kM;
+      if (t >= 2) ok = warp_wait(&ctl.d_full[sl], ((t >> 1) - 1) & 1, abort_flag) &&
+                       warp_wait(&ctl.d_free[sl], ((t >> 1) - 1) & 1, abort_flag);
+      if (!ok) break;
+      if (lane == 0) {
+        tc::mbar_arrive_expect_tx(&ctl.q_full[sl], kQTileBytes);
+        tc::tma_tile2d(q_ring + sl * kQTileBytes, &a.q_map, &ctl.q_full[sl], h * kDH, s0);
+        tc::tma_tile2d(q_ring + sl * kQTileBytes + kM * 128, &a.q_map, &ctl.q_full[sl], h * kDH + 64, s0);
+      }
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int i = s0 + q * 32 + lane;
+        const int pos = i < q_hi ? __ldg(a.active_idx + i) : -1;
+        ctl.pos[sl][q * 32 + lane] = pos;
+        ctl.lse2[sl][q * 32 + lane] = pos >= 0 ? __ldg(a.lse + (size_t)h * a.L + pos) * kLog2e : INFINITY;
+      }
+      __syncwarp();
+      if (lane == 0) tc::mbar_arrive(&ctl.q_full[sl]);
+    }
+  } else if (warp == kIssueWarp) {
+    if (lane == 0) {
+      const uint32_t idesc = tc::make_idesc_bf16(kM, kM, false);
+      const uint64_t k_desc = tc::make_desc_sw128(tc::smem_u32(k_tile), 16, 1024);
+      const uint64_t q_desc0 = tc::make_desc_sw128(tc::smem_u32(q_ring), 16, 1024);
+      const uint32_t hi = (uint32_t)(k_desc >> 32);
+      const uint32_t k_lo_w = (uint32_t)k_desc, q_lo0 = (uint32_t)q_desc0;
+      for (int t = 0; t < n_tiles; ++t) {
+        const int sl = t & 1;
+        if (t == 0 && !tc::mbar_wait(&ctl.k_ready, 0, abort_flag)) break;
+        if (!tc::mbar_wait(&ctl.q_full[sl], (t >> 1) & 1, abort_flag)) break;
+        if (t >= 2 && !tc::mbar_wait(&ctl.d_free[sl], ((t >> 1) - 1) & 1, abort_flag)) break;
+        tc::tc_fence_after();
+        const uint32_t d_dst = tmem + sl * kM;
+        const uint32_t q_lo_w = q_lo0 + sl * (kQTileBytes >> 4);
+#define FL_KQ(KK, ACC)                                                                                       \
+  tc::mma_ss_lo<ACC>(d_dst, k_lo_w + ((((KK) >> 2) * (kM * 128) + ((KK)&3) * 32) >> 4), hi,                  \
+                     q_lo_w + ((((KK) >> 2) * (kM * 128) + ((KK)&3) * 32) >> 4), hi, idesc)
+        FL_KQ(0, false); FL_KQ(1, true); FL_KQ(2, true); FL_KQ(3, true);
+        FL_KQ(4, true);  FL_KQ(5, true); FL_KQ(6, true); FL_KQ(7, true);
+#undef FL_KQ
+        tc::mma_commit(&ctl.d_full[sl]);
+      }
+    }
+    __syncwarp();
+  } else {
+    // ---- the four epilogue warps first rebuild the columns that carry residual payloads (Eq. 8 chain) ----------
+    bool ok = warp_wait(&ctl.k_full, 0, abort_flag);
+    if (ok) {
+      const int ch = tid & 15;                        // 16-byte piece of the row
+      const int elem = h * kDH + ch * 8;
+      const __nv_bfloat16* base_rows = static_cast<const __nv_bfloat16*>(a.k.base) + elem;
+#pragma unroll 1
+      for (int u = tid >> 4; u < kM; u += 8) {
+        if (u0 + u >= cnt) break;
+        const int j = __ldg(cols + u0 + u);
+        float x[8];
+        unpack8(__ldg(reinterpret_cast<const uint4*>(base_rows + (size_t)j * a.d)), x);
+        bool any = false;
+#pragma unroll 1
+        for (int s = 0; s < a.n_use; ++s) any |= apply_stream8<__nv_bfloat16, BITS>(a.k.s[s], j, elem, a.d, a.group, x);
+        if (any) *reinterpret_cast<uint4*>(k_tile + (ch >> 3) * (kM * 128) + tc::sw128_offset(u, ch & 7)) = pack8(x);
+      }
+      tc::fence_proxy_async_smem();
+    }
+    __syncwarp();
+    if (lane == 0) tc::mbar_arrive(&ctl.k_ready);
+    // ---- then sum the tiles: the thread of lane u owns selected column u0 + u -----------------------------------
+    const int ur = warp * 32 + lane;
+    const int jpos = u0 + ur < cnt ? __ldg(cols + u0 + ur) : INT32_MAX;
+    const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+    const float c2 = a.scale * kLog2e;
+    float sum = 0.f;
+    for (int t = 0; t < n_tiles && ok; ++t) {
+      const int sl = t & 1;
+      if (!warp_wait(&ctl.q_full[sl], (t >> 1) & 1, abort_flag)) { ok = false; break; }
+      if (!warp_wait(&ctl.d_full[sl], (t >> 1) & 1, abort_flag)) { ok = false; break; }
+      tc::tc_fence_after();
+      // the active rows ascend: when the tile's first row lies at or after every column of the warp nothing is masked
+      const int pos_first = ctl.pos[sl][0];
+      const bool all_visible = __all_sync(0xffffffffu, jpos == INT32_MAX || jpos <= pos_first);
+#pragma unroll 1
+      for (int q = 0; q < 4; ++q) {
+        uint32_t r[32];
+        tc::tmem_ld32(tmem + lane_base + sl * kM + q * 32, r);
+        tc::tmem_wait_ld();
+        const float* l2 = ctl.lse2[sl] + q * 32;
+        float part = 0.f;
+        if (all_visible) {
+#pragma unroll
+          for (int u = 0; u < 32; ++u) part += tc::ex2(fmaf(__uint_as_float(r[u]), c2, -l2[u]));
+        } else {
+          const int* ps = ctl.pos[sl] + q * 32;
+#pragma unroll
+          for (int u = 0; u < 32; ++u) {
+            const float p = tc::ex2(fmaf(__uint_as_float(r[u]), c2, -l2[u]));
+            part += ps[u] >= jpos ? p : 0.f;
+          }
+        }
+        sum += part;
+      }
+      tc::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) tc::mbar_arrive(&ctl.d_free[sl]);
+    }
+    if (ok && u0 + ur < cnt) a.out[prob * a.c + u0 + ur] = sum;
+  }
+  tc::tc_fence_before();
+  __syncthreads();
+  if (warp == kIssueWarp) {
+    if (ctl.abort_flag) {
+      if (lane == 0) tc::mma_commit(&ctl.d_full[0]);
+      __syncwarp();
+      for (int it = 0; it < (1 << 16); ++it) __nanosleep(256);
+    }
+    tc::tc_fence_after();
+    tc::tmem_dealloc(tmem, kTmemCols);
+  }
+  if (tid == 0 && ctl.abort_flag && a.status != nullptr) atomicExch(a.status, (int)FL_ERR_TIMEOUT);
+}
+
 }  // namespace
 
 // Returns FL_ERR_UNSUPPORTED when the tensor path does not cover the request (the caller then runs the binary32
@@ -462,5 +681,43 @@ int fl_launch_dense_tc(fl_ctx* ctx, const fl_shape* s, const void* q, const void
   FL_CHECK_CUDA(cudaFuncSetAttribute(dense_colsum_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
                                      (int)cudaSharedmemCarveoutMaxShared));
   dense_colsum_kernel<<<dim3(n_tiles, a.nb, s->n_heads), kThreads, kColsumSmem, st>>>(a);
+  return fl_launch_status();
+}
+
+// Next-loop column scores of a sparse loop on the tensor path; FL_ERR_UNSUPPORTED when it does not cover the request.
+int fl_launch_sparse_colsum_tc(fl_ctx* ctx, const fl_shape* s, int loop_r, const void* q_new, const int32_t* active_idx,
+                               int n_active, const fl_kv_store* store, const int32_t* col_idx, const int32_t* col_cnt,
+                               int c, const float* lse, float* out, int32_t* status, cudaStream_t st) {
+  if (s->dtype != FL_BF16 || s->head_dim != kDH || ctx->force_simt || n_active < 1) return FL_ERR_UNSUPPORTED;
+  if ((size_t)ctx->max_smem_optin < kSpColsumSmem || ctx->encode_tiled == nullptr || ctx->tmaps == nullptr)
+    return FL_ERR_UNSUPPORTED;
+  SpArgs a{};
+  const int64_t d_row = (int64_t)s->n_heads * s->head_dim;
+  if (!fl_tile_tmap(ctx, store->k_base, s->L, d_row, 1, &a.k_map) ||
+      !fl_tile_tmap(ctx, q_new, n_active, d_row, kM, &a.q_map))
+    return FL_ERR_UNSUPPORTED;
+  fl_dev_side(store, true, &a.k);
+  a.n_use = loop_r - 1;
+  a.active_idx = active_idx; a.n_active = n_active;
+  a.col_idx = col_idx; a.col_cnt = col_cnt; a.c = c;
+  a.lse = lse; a.out = out; a.status = status;
+  a.L = s->L; a.H = s->n_heads; a.d = (int)d_row; a.q_block = s->q_block; a.nb = fl_n_blocks(s); a.group = s->group;
+  a.scale = s->sm_scale;
+  const dim3 grid((c + kM - 1) / kM, a.nb, s->n_heads);
+#define FL_SC(BITS)                                                                                               \
+  do {                                                                                                            \
+    auto kern = sparse_colsum_kernel<BITS>;                                                                       \
+    FL_CHECK_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSpColsumSmem));  \
+    FL_CHECK_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout,                     \
+                                       (int)cudaSharedmemCarveoutMaxShared));                                    \
+    kern<<<grid, kThreads, kSpColsumSmem, st>>>(a);                                                               \
+  } while (0)
+  switch (s->bits) {
+    case 2: FL_SC(2); break;
+    case 4: FL_SC(4); break;
+    case 8: FL_SC(8); break;
+    default: FL_SC(16); break;
+  }
+#undef FL_SC
   return fl_launch_status();
 }

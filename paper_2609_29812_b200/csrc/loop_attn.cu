@@ -7,6 +7,15 @@ int fl_launch_sparse_colscore(const fl_shape* s, const void* q_new, const int32_
                               const DevSide& kside, int n_use, const int32_t* col_idx, const int32_t* col_cnt, int c,
                               const float* lse, float* out, cudaStream_t st);
 
+int fl_launch_sparse_colsum_tc(fl_ctx* ctx, const fl_shape* s, int loop_r, const void* q_new, const int32_t* active_idx,
+                               int n_active, const fl_kv_store* store, const int32_t* col_idx, const int32_t* col_cnt,
+                               int c, const float* lse, float* out, int32_t* status, cudaStream_t st);
+
+// next-loop column scores: tensor path when it covers the request, the binary32 kernel otherwise
+static int fl_next_col_scores(fl_ctx* ctx, const fl_shape* s, int loop_r, const void* q_new, const int32_t* active_idx,
+                              int n_active, const fl_kv_store* store, const int32_t* col_idx, const int32_t* col_cnt,
+                              int c, const float* lse, float* out, int32_t* status, cudaStream_t st);
+
 int fl_launch_loop_attn_tc(fl_ctx* ctx, const fl_shape* s, int loop_r, const void* q_new, const void* q_old,
                            const int32_t* active_idx, int n_active, const fl_kv_store* store, const int32_t* col_idx,
                            const int32_t* col_cnt, int c, const float* lse_prev, float* lse_out, const void* o_prev,
@@ -247,8 +256,8 @@ extern "C" int fl_loop_attention(fl_ctx* ctx, const fl_shape* shape, int loop_r,
                                 lse_prev, lse_out, o_prev, o_out, 0, nullptr, nullptr, status, st);
     if (rc == FL_OK) {
       if (col_scores_next == nullptr) return FL_OK;
-      return fl_launch_sparse_colscore(shape, q_new, active_idx, n_active, kside, loop_r - 1, col_idx, col_cnt, c,
-                                       lse_out, col_scores_next, st);
+      return fl_next_col_scores(ctx, shape, loop_r, q_new, active_idx, n_active, store, col_idx, col_cnt, c, lse_out,
+                                col_scores_next, status, st);
     }
     if (rc != FL_ERR_UNSUPPORTED) return rc;
   }
@@ -272,8 +281,8 @@ extern "C" int fl_loop_attention(fl_ctx* ctx, const fl_shape* shape, int loop_r,
                                : launch_loop<__nv_bfloat16, 128>(shape, a, max_tiles, st);
   if (rc != FL_OK || col_scores_next == nullptr) return rc;
   // column scores that prepare a pruned selection for loop r+1 (Eq. 6 with a sparse source loop)
-  return fl_launch_sparse_colscore(shape, q_new, active_idx, n_active, a.k, loop_r - 1, col_idx, col_cnt, c, lse_out,
-                                   col_scores_next, st);
+  return fl_next_col_scores(ctx, shape, loop_r, q_new, active_idx, n_active, store, col_idx, col_cnt, c, lse_out,
+                            col_scores_next, status, st);
 }
 
 // Host-side checks of the position-indexed form, shared with the entry point that brings its own scratch.
@@ -340,10 +349,8 @@ extern "C" int fl_loop_attention_indexed_carry(fl_ctx* ctx, const fl_shape* shap
     rc = fl_launch_loop_attn_tc(ctx, shape, loop_r, q_new, q_store_in, active_idx, n_active, store, col_idx, col_cnt,
                                 c, lse_in, lse_out, o_store_in, o_store_out, 1, q_store_out, carry, status, st);
   if (rc != FL_OK || col_scores_next == nullptr) return rc;
-  DevSide kside;
-  fl_dev_side(store, true, &kside);
-  return fl_launch_sparse_colscore(shape, q_new, active_idx, n_active, kside, loop_r - 1, col_idx, col_cnt, c, lse_out,
-                                   col_scores_next, st);
+  return fl_next_col_scores(ctx, shape, loop_r, q_new, active_idx, n_active, store, col_idx, col_cnt, c, lse_out,
+                            col_scores_next, status, st);
 }
 
 extern "C" int fl_loop_attention_indexed(fl_ctx* ctx, const fl_shape* shape, int loop_r, const void* q_new,
@@ -355,4 +362,15 @@ extern "C" int fl_loop_attention_indexed(fl_ctx* ctx, const fl_shape* shape, int
   return fl_loop_attention_indexed_carry(ctx, shape, loop_r, q_new, q_store_in, q_store_out, active_idx, n_active,
                                          store, col_idx, col_cnt, c, lse_in, lse_out, o_store_in, o_store_out, nullptr,
                                          col_scores_next, status, stream);
+}
+
+static int fl_next_col_scores(fl_ctx* ctx, const fl_shape* s, int loop_r, const void* q_new, const int32_t* active_idx,
+                              int n_active, const fl_kv_store* store, const int32_t* col_idx, const int32_t* col_cnt,
+                              int c, const float* lse, float* out, int32_t* status, cudaStream_t st) {
+  const int rc = fl_launch_sparse_colsum_tc(ctx, s, loop_r, q_new, active_idx, n_active, store, col_idx, col_cnt, c, lse,
+                                            out, status, st);
+  if (rc != FL_ERR_UNSUPPORTED) return rc;
+  DevSide kside;
+  fl_dev_side(store, true, &kside);
+  return fl_launch_sparse_colscore(s, q_new, active_idx, n_active, kside, loop_r - 1, col_idx, col_cnt, c, lse, out, st);
 }

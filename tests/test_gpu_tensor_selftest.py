@@ -66,3 +66,23 @@ def test_tma_row_gather_feeds_the_tensor_core():
             kg[t] = base[j].double().cpu()
     s_ref = q.double().cpu() @ kg.T
     np.testing.assert_allclose(s_out.cpu().numpy(), s_ref.numpy(), rtol=1e-4, atol=1e-3)
+
+
+def test_bounded_wait_runs_out_and_reports_a_timeout():
+    """A wait on a barrier that nothing completes gives up after its poll limit, the kernel reports FL_ERR_TIMEOUT
+    through the status word and returns; the context stays usable (a normal launch right after works)."""
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2609_29812_b200 import binding as B, build
+    lib = C.CDLL(build.SELFTEST_LIB_PATH)
+    lib.fl_selftest_timeout.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
+    lib.fl_selftest_timeout.restype = C.c_int
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    gave_up = torch.zeros(1, dtype=torch.int32, device="cuda")
+    assert lib.fl_selftest_timeout(status.data_ptr(), gave_up.data_ptr(), None) == 0
+    torch.cuda.synchronize()
+    assert int(gave_up.item()) == 1
+    assert int(status.item()) == B.FL_ERR_TIMEOUT
+    assert "wait" in B.status_string(int(status.item()))
+    x = torch.arange(8, device="cuda")
+    assert int((x + 1).sum().item()) == 36

@@ -23,6 +23,7 @@ Functions and the passage each one follows:
                                    the cached mass is one)
   select_columns                   Appendix D.2 (column selection equation)
   sparse_loop_attention            Appendix D.2 (attention replacement equation)
+  decode_sparse_attention          Appendix D.2 as written, for decode positions (per-position sets)
   quantize_groups, dequantize_groups, pack_codes, unpack_codes
                                    Appendix E "Quantization Setting" (asymmetric,
                                    group-wise, scale and offset from min / max)
@@ -342,6 +343,43 @@ def sparse_loop_attention(q_new, khat_new, vhat_new, vhat_old, o_prev, active, c
             with np.errstate(divide="ignore", invalid="ignore"):
                 lse[h, t_idx] = np.where(has, mx + np.log(np.where(den > 0, den, 1.0)) - np.log(m), np.nan)
     return {"O": O, "mass": mass, "probs": probs, "col_scores": scores, "lse": lse}
+
+
+def decode_sparse_attention(q_new, khat_new, vhat_new, vhat_old, o_prev, col_sets, p_old, sm_scale, kv_round=None):
+    """Appendix D.2 literally: one decode position per query, its own selected subset S and cached probabilities.
+
+    q_new  : [B, H, dh] current queries of loop r (decode positions follow every cached key: no causal cut)
+    khat_new, vhat_new : [L, H, dh] reconstructed K, V of loop r;  vhat_old : [L, H, dh] reconstructed V of loop r-1
+    o_prev : [B, H, dh] fp64 outputs of loop r-1
+    col_sets : {(t, h): ascending column ids S};  p_old : {(t, h): cached loop r-1 probabilities over S}
+    Returns dict O [B,H,dh] fp64, p_new {(t,h): probabilities over S}, mass [B,H], lse [B,H] with
+    p_new_j = exp(logit_j - lse) (NaN for an empty S, whose output row is o_prev unchanged).
+    """
+    q_new = np.asarray(q_new)
+    Bq, H, dh = q_new.shape
+    rd = (lambda x: x) if kv_round is None else kv_round
+    O = np.array(o_prev, dtype=F64, copy=True)
+    mass = np.zeros((Bq, H))
+    lse = np.full((Bq, H), np.nan)
+    p_out = {}
+    for t in range(Bq):
+        for h in range(H):
+            S = np.asarray(col_sets[(t, h)], dtype=np.int64)
+            po = np.asarray(p_old[(t, h)], dtype=F64)
+            if len(S) == 0:
+                p_out[(t, h)] = np.zeros(0)
+                continue
+            m = po.sum()                                           # cached global mass of the subset
+            logits = (rd(khat_new[S, h, :]).astype(F64) @ q_new[t, h, :].astype(F64)) * F64(sm_scale)
+            mx = logits.max()
+            e = np.exp(logits - mx)
+            pn = m * e / e.sum()                                   # m * softmax over S
+            O[t, h, :] = O[t, h, :] - po @ rd(vhat_old[S, h, :]).astype(F64) + pn @ rd(vhat_new[S, h, :]).astype(F64)
+            mass[t, h] = m
+            with np.errstate(divide="ignore"):
+                lse[t, h] = mx + np.log(e.sum()) - np.log(m)
+            p_out[(t, h)] = pn
+    return {"O": O, "p_new": p_out, "mass": mass, "lse": lse}
 
 
 def old_term_local_softmax(q_old, khat_old, vhat_old, rows, S, m, sm_scale, head):

@@ -285,3 +285,60 @@ def test_kv_round_is_applied_to_all_three_operands_values_by_hand():
         ops[miss] = (k_new, v_old, v_new)[miss].astype(np.float64)
         wrong, _ = expect(*ops)
         assert abs(wrong - want) > 1e-4 and got["rounded"]["O"][0, 0, 0] != pytest.approx(wrong, rel=1e-6)
+
+
+def test_decode_oracle_pins():
+    """decode_sparse_attention: (i) all keys selected with mass 1 = textbook softmax attention over the new K/V
+    (library routine); (ii) unchanged query, keys and values leave the output where it was, for any subset;
+    (iii) it is the per-position case (q_block = 1) of the prefill replacement, so the two must agree on a position
+    appended after the prompt; (iv) hand values for one query, two columns."""
+    torch = pytest.importorskip("torch")
+    rng = np.random.default_rng(11)
+    L, H, dh, Bq = 30, 2, 8, 3
+    k1, v1, k2, v2 = [f32r(rng.standard_normal((L, H, dh))) for _ in range(4)]
+    q1, q2 = [f32r(rng.standard_normal((Bq, H, dh))) for _ in range(2)]
+    scale = dh ** -0.5
+    def dense(q, k, v):
+        out = torch.nn.functional.scaled_dot_product_attention(
+            torch.from_numpy(q).permute(1, 0, 2)[None], torch.from_numpy(k).permute(1, 0, 2)[None],
+            torch.from_numpy(v).permute(1, 0, 2)[None])[0].permute(1, 0, 2).numpy()
+        logits = np.einsum("thd,lhd->thl", q, k) * scale
+        p = np.exp(logits - logits.max(axis=2, keepdims=True)); p /= p.sum(axis=2, keepdims=True)
+        return out, p
+    o1, p1 = dense(q1, k1, v1)
+    # (i) full sets: loop 2 equals dense attention over loop-2 K/V
+    full = {(t, h): np.arange(L) for t in range(Bq) for h in range(H)}
+    res = fo.decode_sparse_attention(q2, k2.astype(np.float32), v2.astype(np.float32), v1.astype(np.float32), o1, full,
+                                     {(t, h): p1[t, h] for t in range(Bq) for h in range(H)}, scale)
+    o2, p2 = dense(q2, k2, v2)
+    np.testing.assert_allclose(res["O"], o2, rtol=1e-9, atol=1e-11)
+    np.testing.assert_allclose(res["mass"], 1.0, rtol=1e-12)
+    for t in range(Bq):
+        for h in range(H):
+            np.testing.assert_allclose(res["p_new"][(t, h)], p2[t, h], rtol=1e-9)
+    # (ii) fixed point for arbitrary subsets
+    sets = {(t, h): np.sort(rng.permutation(L)[: 1 + 3 * t + h]) for t in range(Bq) for h in range(H)}
+    pold = {key: p1[key[0], key[1]][S] for key, S in sets.items()}
+    same = fo.decode_sparse_attention(q1, k1.astype(np.float32), v1.astype(np.float32), v1.astype(np.float32), o1, sets,
+                                      pold, scale)
+    np.testing.assert_allclose(same["O"], o1, rtol=1e-12, atol=1e-13)
+    # (iii) against the prefill form with one position per block: the decode position is row L of an extended prompt
+    t, h = 1, 0
+    ext = lambda a: np.concatenate([a, np.zeros((1, H, dh))], axis=0).astype(np.float32)
+    S = sets[(t, h)]
+    pre = fo.sparse_loop_attention(q2[t:t + 1], ext(k2), ext(v2), ext(v1), o1[t:t + 1], np.array([L]), {(h, L): S},
+                                   {(h, L): (np.array([L]), pold[(t, h)][None, :])}, scale, q_block=1, head_list=[h],
+                                   block_list=[L])
+    dec = fo.decode_sparse_attention(q2, k2.astype(np.float32), v2.astype(np.float32), v1.astype(np.float32), o1, sets,
+                                     pold, scale)
+    np.testing.assert_allclose(dec["O"][t, h], pre["O"][0, h], rtol=1e-12, atol=1e-14)
+    assert dec["lse"][t, h] == pytest.approx(pre["lse"][h, 0], rel=1e-12)
+    # (iv) by hand: dh = 1, q = 1, scale = 1, keys log 2 and log 6, cached p = (1/4, 1/2): m = 3/4,
+    # p_new = 3/4 * (2/8, 6/8) = (3/16, 9/16); o = 1 - (1/4 * 4 + 1/2 * (-2)) + (3/16 * 8 + 9/16 * 16) = 1 + 10.5
+    one = fo.decode_sparse_attention(np.ones((1, 1, 1)), np.log(np.array([2.0, 6.0], dtype=np.float32)).reshape(2, 1, 1),
+                                     np.array([8.0, 16.0], dtype=np.float32).reshape(2, 1, 1),
+                                     np.array([4.0, -2.0], dtype=np.float32).reshape(2, 1, 1), np.ones((1, 1, 1)),
+                                     {(0, 0): np.array([0, 1])}, {(0, 0): np.array([0.25, 0.5])}, 1.0)
+    assert one["O"][0, 0, 0] == pytest.approx(11.5, rel=1e-6)
+    np.testing.assert_allclose(one["p_new"][(0, 0)], [3 / 16, 9 / 16], rtol=1e-6)
+    assert one["lse"][0, 0] == pytest.approx(np.log(8.0) - np.log(0.75), rel=1e-6)

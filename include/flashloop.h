@@ -279,6 +279,25 @@ FL_API int fl_loop_attention_indexed_static(fl_ctx* ctx, const fl_shape* shape, 
                                      const void* o_store_in, void* o_store_out, float* col_scores_next,
                                      int32_t* status, void* stream);
 
+/* Sparse decode attention -- Eq. 6-7 as Appendix D.2 writes them, for decode positions (Appendix G, the item on
+ * sparse decode kernels): loop r >= 2 of n_queries single-token queries that follow the prompt, over the prompt's
+ * store. Query t, head h has its OWN selected subset S = col_idx[t, h, :col_cnt[t, h]] (ascending positions of the
+ * prompt, padded with -1; every one of them is causal for a decode position) and log-normaliser lse_prev[t, h] with
+ * p_old_j = exp(sm_scale q_old . Khat^(r-1)_j - lse_prev) (a dense source loop gives lse_prev = logsumexp over all keys):
+ *   m = sum_S p_old_j;  p_new_j = m softmax_S(sm_scale q_new . Khat^(r)_j);
+ *   o_out = o_prev - sum_S p_old_j Vhat^(r-1)_j + sum_S p_new_j Vhat^(r)_j;  lse_out = logsumexp_S - log m;
+ *   p_new_out[t, h, u] = p_new of column S[u] (the scores from which the next loop's subset is pruned; 0 beyond the
+ *   count), or NULL.
+ * K/V of the selected columns are rebuilt inside the kernel from the base and the residual streams (Eq. 8), rounded
+ * to the storage type where attention consumes them. q_new, q_old, o_prev, o_out: [n_queries, H, dh] storage type
+ * (o_out may alias o_prev); lse_prev, lse_out: f32 [n_queries, H] (may alias). A query with an empty subset keeps its
+ * output and log-normaliser. The decode tokens' own K/V (the short full-precision tail of Appendix E) are not part of
+ * this call. `status` is accepted for symmetry and never written. */
+FL_API int fl_decode_attention(fl_ctx* ctx, const fl_shape* shape, int loop_r, const void* q_new, const void* q_old,
+                        int32_t n_queries, const fl_kv_store* store, const int32_t* col_idx, const int32_t* col_cnt,
+                        int32_t c, const float* lse_prev, float* lse_out, const void* o_prev, void* o_out,
+                        float* p_new_out, int32_t* status, void* stream);
+
 /* KV-cache accounting (Section 1's 48 GiB example; Section 4.3): bytes held for one layer by this store
  * after n_loops loops, and by a dense looped cache of n_loops loops. Host-only, no device access.
  * share_layers = number of layers sharing each loop's slot map and index list (>= 1). */

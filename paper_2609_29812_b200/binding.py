@@ -77,6 +77,8 @@ def _load() -> C.CDLL:
                                             i32, p, p, p, p, C.POINTER(FlAttnCarry), p, p, p],
         "fl_loop_attention_indexed_static": [p, C.POINTER(FlShape), C.c_int, p, p, p, p, i32, C.POINTER(FlKvStore),
                                              p, p, i32, p, p, p, p, p, p, p],
+        "fl_decode_attention": [p, C.POINTER(FlShape), C.c_int, p, p, i32, C.POINTER(FlKvStore), p, p, i32, p, p, p, p, p,
+                                p, p],
         "fl_kv_store_bytes": [C.POINTER(FlShape), C.POINTER(FlKvStore), C.c_int, C.c_int,
                               C.POINTER(i64), C.POINTER(i64)],
         "fl_loop_attention_workspace_bytes": [p, C.POINTER(FlShape), C.POINTER(i64)],
@@ -276,6 +278,15 @@ def fl_loop_attention_indexed_static(ctx, shape, loop_r, q_new, q_store_in, q_st
                                               _ptr(col_cnt), int(c), _ptr(lse_in), _ptr(lse_out), _ptr(o_store_in),
                                               _ptr(o_store_out), _ptr(col_scores_next), _ptr(status), _stream(stream))
     return _check("fl_loop_attention_indexed_static", rc, check)
+
+
+def fl_decode_attention(ctx, shape, loop_r, q_new, q_old, n_queries, store, col_idx, col_cnt, c, lse_prev, lse_out,
+                        o_prev, o_out, p_new_out=None, status=None, stream=None, check=True) -> int:
+    rc = lib.fl_decode_attention(_h(ctx), C.byref(shape), int(loop_r), _ptr(q_new), _ptr(q_old), int(n_queries),
+                                 C.byref(store) if store is not None else None, _ptr(col_idx), _ptr(col_cnt), int(c),
+                                 _ptr(lse_prev), _ptr(lse_out), _ptr(o_prev), _ptr(o_out), _ptr(p_new_out),
+                                 _ptr(status), _stream(stream))
+    return _check("fl_decode_attention", rc, check)
 
 
 def fl_kv_store_bytes(shape, store, n_loops, share_layers=1, check=True):

@@ -106,6 +106,11 @@ def test_argument_validation_happens_before_any_launch(B):
     # a reusing call needs none of the previous loop's rows: the checks pass and the stand-in context, which has no
     # tensor path, answers "unsupported"
     assert idx(B.make_carry(P + 0x4000, P, True), qs=None, lse=None, o=None) == UNS
+    # sparse decode attention
+    dec = lambda **kw: B.fl_decode_attention(ctx, sh, kw.get("r", 2), kw.get("q", P), P, kw.get("n", 4), kw.get("st", st),
+                                             kw.get("ci", P), P, kw.get("c", 64), P, P, P, P, None, **call)
+    assert dec(r=1) == INV and dec(c=0) == INV and dec(q=None) == INV and dec(ci=None) == INV and dec(st=None) == INV
+    assert dec(n=-1) == INV and dec(r=3) == INV and dec(n=0) == B.FL_OK
     # accounting
     rc = B.lib.fl_kv_store_bytes(C.byref(sh), C.byref(st), 3, 1, C.byref(C.c_int64()), C.byref(C.c_int64()))
     assert rc == INV                                                                          # only one stream

@@ -55,10 +55,12 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--loops", type=int, default=0, help="sched: number of loops R (default 8)")
-    ap.add_argument("--workload", default="c3", choices=["c2", "c3", "c4", "c5", "sched"],
+    ap.add_argument("--workload", default="c3", choices=["c2", "c3", "c4", "c5", "sched", "decode"],
                     help="c3: the 48-layer stack at 32K (default, the metric's configuration); c2: one layer at 8K; "
                          "c5: the 128K memory configuration (prefill part; 24 layers resident unless --layers); "
                          "c4: the sparsity / depth sweep (one layer at 8K, a table of points); "
+                         "decode: config 5's second phase, 32 single-token queries over the 4-loop store (sparse decode "
+                         "attention, loops 2-4; a separate metric); "
                          "sched: budgets that decay from loop to loop with real column pruning (Table 6's deep "
                          "schedule: tokens 90% -> 20%, columns pruned inside the previous set every loop)")
     ap.add_argument("--sweep", default="subset", choices=["subset", "full"], help="c4: which points to run")
@@ -496,8 +498,8 @@ def run_ours(args):
     device = f"cuda:{local}"
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device(device))
-    if args.workload in ("c4", "sched"):
-        (run_sweep if args.workload == "c4" else run_schedule)(args, device, rank)
+    if args.workload in ("c4", "sched", "decode"):
+        {"c4": run_sweep, "sched": run_schedule, "decode": run_decode}[args.workload](args, device, rank)
         if world > 1:
             dist.destroy_process_group()
         return
@@ -597,6 +599,89 @@ def run_ours(args):
         print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()
+
+
+def run_decode(args, device, rank):
+    """Config 5's decode phase on the hot path's side of it: a batch of 32 single-token queries runs loops 2..4 of the
+    sparse decode attention over the store the prefill left (bf16 base + int4 residual streams), column budget 2048
+    per (query, head), every layer.  Column subsets are random ascending subsets of the prompt (what they are does not
+    change the traffic); K/V of the selected columns are rebuilt in registers.  HBM-bound: the roofline is the bytes
+    of the selected base rows and payloads.  Prints one JSON line (a metric of its own, not the prefill metric)."""
+    import torch
+    from paper_2609_29812_b200 import binding as B, pipeline as P, workloads
+    L, NL, Bq = args.L or 131072, args.layers or 8, 32
+    w = workloads.config5(L=L, n_layers=NL)
+    c = w.col_budget
+    peaks = load_peaks()
+    ctx = B.Context(torch.device(device).index or 0)
+    sh = P.shape_of(w)
+    stack = workloads.DeviceStack(w, seed=0, device=device)
+    G = stack.stack_hidden()
+    H, dh, R = w.n_heads, w.head_dim, w.n_loops
+    sels, cand = [], None
+    for r in range(2, R + 1):
+        sel = P.select_tokens(ctx, sh, r, G[r - 2], G[r - 1], cand, w.k_tokens)
+        sels.append(sel); cand = sel.active_idx
+    layers = []
+    for l in range(NL):
+        gen = stack.layer(l)
+        st = P.LayerState(ctx, w, device)
+        _, k1, v1 = gen.qkv1()
+        st.k_base, st.v_base = k1, v1
+        for r in range(2, R + 1):
+            sel = sels[r - 2]
+            st.alloc_stream(sel, rows=False)
+            _, kr, vr = gen.rows(r, sel.active_idx)
+            st.quantize(r, kr, vr, sel)
+        gen.release()
+        layers.append(st)
+    g = torch.Generator(device=device); g.manual_seed(7)
+    col_idx = torch.stack([torch.sort(torch.randperm(L, device=device, generator=g)[:c])[0]
+                           for _ in range(Bq * H)]).to(torch.int32).view(Bq, H, c).contiguous()
+    col_cnt = torch.full((Bq, H), c, dtype=torch.int32, device=device)
+    mk = lambda: (torch.randn(Bq, H, dh, device=device, generator=g) * 0.5).to(torch.bfloat16)
+    q = [mk() for _ in range(R)]
+    o = mk(); lse = torch.full((Bq, H), 12.0, dtype=torch.float32, device=device)
+    stream = torch.cuda.Stream(device=device)
+    def step():
+        for st in layers:
+            for r in range(2, R + 1):
+                B.fl_decode_attention(ctx, sh, r, q[r - 1], q[r - 2], Bq, st.store, col_idx, col_cnt, c, lse, lse, o, o,
+                                      None, stream=stream)
+    with torch.cuda.stream(stream):
+        for _ in range(3):
+            step()
+    torch.cuda.synchronize()
+    t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+    with torch.cuda.stream(stream):
+        t0.record(stream)
+        for _ in range(args.steps):
+            step()
+        t1.record(stream)
+    torch.cuda.synchronize()
+    ms = t0.elapsed_time(t1) / args.steps
+    n_calls = NL * (R - 1)
+    # bytes per call: base K and V rows of every selected column, plus the payloads those columns carry
+    pay = 2 * (dh * w.bits // 8 + 4 * (dh // w.group))
+    byt = 0.0
+    flat = col_idx.long().view(-1)
+    for r in range(2, R + 1):
+        b_r = float(flat.numel()) * 2 * dh * 2
+        for rr in range(2, r + 1):
+            b_r += float((sels[rr - 2].slot_of_pos.long()[flat] >= 0).sum().item()) * pay
+        byt += b_r
+    byt *= NL
+    if rank == 0:
+        print(json.dumps({"metric": "sparse_decode_attention_ms_per_step", "value": ms, "unit": "ms", "n_gpus": 1,
+                          "steps": args.steps, "warmup": 3, "higher_is_better": False, "dtype": "f32",
+                          "data": "synthetic",
+                          "config": {"workload": f"decode over the 4-loop store: L={L}, {NL} layers, batch {Bq} single-token "
+                                                 f"queries, {H}x{dh} heads, column budget {c}, loops 2..{R}, int4 g128"},
+                          "gpu_launches": n_calls * args.steps, "ms_per_layer_loop": ms / n_calls,
+                          "roofline": {"bound": "hbm", "achieved": byt / (ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
+                                       "unit": "GB/s", "frac": byt / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                                       "bytes_per_step": byt, "traffic": None, "peak_source": peaks["source"]},
+                          "scaled_to_48_layers_ms": ms * 48 / NL}))
 
 
 def run_schedule(args, device, rank):

@@ -45,6 +45,8 @@ UNIT = "tokens/s"
 # it, so the bench line says "not measured in this run".  Keyed by (workload, L, layers-independent) and loop kind;
 # a shape that is not listed reports null.
 NCU_ATTN_TRAFFIC_BYTES = {
+    ("c3:L=32768", "recompute"): 170.9e6,   # loop 2: loop_attn_tc_kernel<4,1,0> (144.0 MB read + 26.8 MB written)
+    ("c3:L=32768", "economy"): 132.6e6,     # loops 3, 4: loop_attn_stream_kernel<4,1> (mean of 134.0 and 131.2 MB)
 }
 
 

@@ -28,6 +28,8 @@ Functions and the passage each one follows:
                                    Appendix E "Quantization Setting" (asymmetric,
                                    group-wise, scale and offset from min / max)
   residual_update                  Section 4.3 / Appendix D.3 (masked residual codec)
+  project_rows                     Section 4.4 / Appendix G (only the selected token rows pass through
+                                   the projections; results return to their positions)
   kv_bytes_per_token_layer         Section 1 (48 GiB example) and Section 4.3 accounting
   LayerOracle                      the steps above in the order of Appendix D
 
@@ -394,6 +396,29 @@ def old_term_local_softmax(q_old, khat_old, vhat_old, rows, S, m, sm_scale, head
         logit = (khat_old[T, head, :].astype(F64) @ q_old[t].astype(F64)) * F64(sm_scale)
         e = np.exp(logit - logit.max())
         out[t] = m[t] * (e / e.sum()) @ vhat_old[T, head, :].astype(F64)
+    return out
+
+
+# --------------------------------------------------------------------------------------
+# Section 4.4 / Appendix G: projections of the active rows only.
+# --------------------------------------------------------------------------------------
+def project_rows(x, src_idx, w, y, dst_idx, accumulate):
+    """y[dst(t), :] (+)= x[src(t), :] @ w.T for t = 0..n-1, in fp64; other rows of y are left as they are.
+
+    src(t) = src_idx[t] (or t when src_idx is None), dst(t) = dst_idx[t] (or t).  w is [d_out, d_in] (the layout
+    of a linear layer's weight).  With accumulate the product is added to the row that is there (the residual
+    add of the output projection); without, it replaces it.  Returns the new y (fp64); the caller applies the
+    storage rounding.
+    """
+    x = np.asarray(x, dtype=F64)
+    w = np.asarray(w, dtype=F64)
+    out = np.array(y, dtype=F64, copy=True)
+    n = len(src_idx) if src_idx is not None else (len(dst_idx) if dst_idx is not None else x.shape[0])
+    for t in range(n):
+        s = int(src_idx[t]) if src_idx is not None else t
+        d = int(dst_idx[t]) if dst_idx is not None else t
+        row = w @ x[s]
+        out[d] = out[d] + row if accumulate else row
     return out
 
 

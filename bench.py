@@ -57,12 +57,14 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--loops", type=int, default=0, help="sched: number of loops R (default 8)")
-    ap.add_argument("--workload", default="c3", choices=["c2", "c3", "c4", "c5", "sched", "decode"],
+    ap.add_argument("--workload", default="c3", choices=["c2", "c3", "c4", "c5", "sched", "decode", "proj"],
                     help="c3: the 48-layer stack at 32K (default, the metric's configuration); c2: one layer at 8K; "
                          "c5: the 128K memory configuration (prefill part; 24 layers resident unless --layers); "
                          "c4: the sparsity / depth sweep (one layer at 8K, a table of points); "
                          "decode: config 5's second phase, 32 single-token queries over the 4-loop store (sparse decode "
                          "attention, loops 2-4; a separate metric); "
+                         "proj: the projections of the active rows as one gathered / scattering tensor-core GEMM "
+                         "(fl_project_rows) beside row copies + library GEMMs (a separate line, not the metric); "
                          "sched: budgets that decay from loop to loop with real column pruning (Table 6's deep "
                          "schedule: tokens 90% -> 20%, columns pruned inside the previous set every loop)")
     ap.add_argument("--sweep", default="subset", choices=["subset", "full"], help="c4: which points to run")
@@ -500,8 +502,9 @@ def run_ours(args):
     device = f"cuda:{local}"
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device(device))
-    if args.workload in ("c4", "sched", "decode"):
-        {"c4": run_sweep, "sched": run_schedule, "decode": run_decode}[args.workload](args, device, rank)
+    if args.workload in ("c4", "sched", "decode", "proj"):
+        {"c4": run_sweep, "sched": run_schedule, "decode": run_decode, "proj": run_projection}[args.workload](
+            args, device, rank)
         if world > 1:
             dist.destroy_process_group()
         return
@@ -684,6 +687,88 @@ def run_decode(args, device, rank):
                                        "unit": "GB/s", "frac": byt / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
                                        "bytes_per_step": byt, "traffic": None, "peak_source": peaks["source"]},
                           "scaled_to_48_layers_ms": ms * 48 / NL}))
+
+
+def run_projection(args, device, rank):
+    """The projections around the hot path at the benchmark shape (3277 active rows of 32768, d = 2048), per layer and
+    loop: Q/K/V ([n, d] x [d, 3d]) from rows gathered out of the hidden store, and the output projection ([n, d] x
+    [d, d]) added into the rows of the hidden store.  Two arms on the same buffers: fl_project_rows (one kernel each:
+    the gather is the GEMM's A-operand load, the scatter-add its epilogue) and row copies + library GEMMs
+    (fl_gather_rows + cuBLAS through torch; cuBLAS + torch's index_add_).  Eight layers' stores and weights are used in
+    turn (1.3 GB: each call finds its inputs in HBM, not in L2).  Prints one JSON line, a metric of its own."""
+    import torch
+    from paper_2609_29812_b200 import binding as B
+    L, d, NL = args.L or 32768, 2048, args.layers or 8
+    n = max(1, L // 10)
+    peaks = load_peaks()
+    ctx = B.Context(torch.device(device).index or 0)
+    g = torch.Generator(device=device); g.manual_seed(3)
+    bf = torch.bfloat16
+    hid = [(torch.randn(L, d, device=device, generator=g)).to(bf) for _ in range(NL)]
+    wqkv = [(torch.randn(3 * d, d, device=device, generator=g) / d ** 0.5).to(bf) for _ in range(NL)]
+    wo = [(torch.randn(d, d, device=device, generator=g) / d ** 0.5).to(bf) for _ in range(NL)]
+    idx = torch.sort(torch.randperm(L, device=device, generator=g)[:n])[0].to(torch.int32)
+    idx64 = idx.long()
+    qkv = torch.empty(n, 3 * d, device=device, dtype=bf)
+    rows = torch.empty(n, d, device=device, dtype=bf)
+    attn_out = (torch.randn(n, d, device=device, generator=g)).to(bf)
+    status = torch.zeros(1, dtype=torch.int32, device=device)
+    stream = torch.cuda.Stream(device=device)
+
+    def timed(fn, reps):
+        with torch.cuda.stream(stream):
+            for l in range(3):
+                fn(l % NL)
+        torch.cuda.synchronize()
+        t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(stream):
+            t0.record(stream)
+            for it in range(reps):
+                fn(it % NL)
+            t1.record(stream)
+        torch.cuda.synchronize()
+        return t0.elapsed_time(t1) / reps
+
+    reps = max(8, args.steps * NL)
+    fused_qkv = lambda l: B.fl_project_rows(ctx, hid[l], L, idx, n, d, wqkv[l], 3 * d, qkv, n, None, 0, status, stream=stream)
+    fused_o = lambda l: B.fl_project_rows(ctx, attn_out, n, None, n, d, wo[l], d, hid[l], L, idx, 1, status, stream=stream)
+    fused_qkv_compact = lambda l: B.fl_project_rows(ctx, rows, n, None, n, d, wqkv[l], 3 * d, qkv, n, None, 0, status, stream=stream)
+    lib_gather = lambda l: B.fl_gather_rows(ctx, hid[l], idx, n, d * 2, rows, stream=stream)
+    lib_qkv = lambda l: torch.matmul(rows, wqkv[l].t(), out=qkv)
+    o_tmp = torch.empty(n, d, device=device, dtype=bf)
+    lib_o = lambda l: torch.matmul(attn_out, wo[l].t(), out=o_tmp)
+    lib_add = lambda l: hid[l].index_add_(0, idx64, o_tmp)
+    def lib_qkv_both(l):
+        lib_gather(l); lib_qkv(l)
+    def lib_o_both(l):
+        lib_o(l); lib_add(l)
+    sampler = ClockSampler(torch.device(device).index or 0)
+    sampler.start()
+    res = {"fused_qkv": timed(fused_qkv, reps), "fused_o": timed(fused_o, reps),
+           "same_kernel_qkv_on_compact_rows": timed(fused_qkv_compact, reps),
+           "library_qkv": timed(lib_qkv_both, reps), "library_o": timed(lib_o_both, reps),
+           "library_gather_alone": timed(lib_gather, reps), "library_qkv_gemm_alone": timed(lib_qkv, reps),
+           "library_o_gemm_alone": timed(lib_o, reps), "library_index_add_alone": timed(lib_add, reps)}
+    clocks = sampler.stop()
+    assert int(status.item()) == 0, "a bounded wait ran out inside fl_project_rows"
+    fl_qkv, fl_o = 2.0 * n * d * 3 * d, 2.0 * n * d * d
+    ms = res["fused_qkv"] + res["fused_o"]
+    if rank == 0:
+        print(json.dumps({"metric": "active_row_projection_ms_per_layer_loop", "value": ms, "unit": "ms", "n_gpus": 1,
+                          "steps": reps, "warmup": 3, "higher_is_better": False, "dtype": "bf16", "data": "synthetic",
+                          "config": {"workload": f"projections of the active rows: L={L}, n={n}, d={d}, Q/K/V + output "
+                                                 f"projection with scattered residual add; {NL} layers' stores and "
+                                                 "weights in turn (inputs exceed L2)"},
+                          "gpu_launches": 2 * reps, "ms": {k: round(v, 5) for k, v in res.items()},
+                          "library_ms_per_layer_loop": res["library_qkv"] + res["library_o"],
+                          "roofline": {"bound": "tensor", "achieved": (fl_qkv + fl_o) / (ms * 1e-3) / 1e12,
+                                       "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                                       "frac": (fl_qkv + fl_o) / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                                       "qkv_tflops": fl_qkv / (res["fused_qkv"] * 1e-3) / 1e12,
+                                       "o_tflops": fl_o / (res["fused_o"] * 1e-3) / 1e12,
+                                       "library_qkv_gemm_tflops": fl_qkv / (res["library_qkv_gemm_alone"] * 1e-3) / 1e12,
+                                       "traffic": None, "peak_source": peaks["source"]},
+                          "clocks": clocks}))
 
 
 def run_schedule(args, device, rank):

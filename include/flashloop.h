@@ -134,6 +134,27 @@ FL_API int fl_gather_rows(fl_ctx* ctx, const void* src, const int32_t* idx, int3
 FL_API int fl_scatter_update(fl_ctx* ctx, const void* src, const int32_t* idx, int32_t n, int64_t row_bytes,
                       void* dst, void* stream);
 
+/* Projection of the active rows (Section 4.4 and Appendix G: the selected token rows are gathered so that the
+ * projections remain regular GEMMs, and results return to their positions). One tensor-core GEMM whose A operand is
+ * gathered by row index and whose epilogue writes or adds into indexed rows:
+ *   for t in [0, n):  y[dst(t), :] = (accumulate ? y[dst(t), :] : 0) + x[src(t), :] . w^T
+ * with src(t) = src_idx[t] (or t when src_idx is NULL) and dst(t) = dst_idx[t] (or t when dst_idx is NULL).
+ * x: bf16 [x_rows, d_in]; w: bf16 [d_out, d_in] (a linear layer's weight, e.g. the stacked Q, K, V weights);
+ * y: bf16 [y_rows, d_out]; all row-major, device memory, 16-byte aligned, owned by the caller; y must not overlap
+ * x or w. Products accumulate in binary32 over d_in; each output element is rounded to bf16 once (after the add
+ * when accumulate = 1). Index lists: device int32 [n], values inside their matrix, dst_idx without repeats; rows of y
+ * that are not listed are left untouched. With src_idx = the active list this replaces fl_gather_rows + a GEMM on the
+ * compact rows; with dst_idx = the active list and accumulate = 1 it is the output projection with the residual add
+ * scattered back.
+ * Errors: FL_ERR_INVALID_ARG for null or misaligned pointers, n < 0, n beyond a matrix that has no index list,
+ * accumulate not 0 or 1, y aliasing an input; FL_ERR_UNSUPPORTED unless d_in is a multiple of 64 and d_out a multiple
+ * of 8, or when the device offers no tensor maps (nothing is launched). n = 0 returns FL_OK without a launch.
+ * `status` (device int32, may be NULL) receives FL_ERR_TIMEOUT if a bounded wait inside the kernel ran out; y is then
+ * undefined. */
+FL_API int fl_project_rows(fl_ctx* ctx, const void* x, int64_t x_rows, const int32_t* src_idx, int32_t n, int32_t d_in,
+                    const void* w, int32_t d_out, void* y, int64_t y_rows, const int32_t* dst_idx,
+                    int32_t accumulate, int32_t* status, void* stream);
+
 /* Stage 3 -- Eq. 8 with the quantizer of Appendix E (asymmetric, group-wise, min/max).
  * For each active row i = active_idx[t], X in {K, V}, head, group of `group` elements, in binary32:
  *   delta = X^(r)_i - Xhat^(r-1)_i            (Xhat^(r-1) rebuilt from base + streams of loops < r)

@@ -66,6 +66,7 @@ def _load() -> C.CDLL:
         "fl_select_tokens": [p, C.POINTER(FlShape), C.c_int, p, p, p, i32, i32, p, p, p, p, p],
         "fl_gather_rows": [p, p, p, i32, i64, p, p],
         "fl_scatter_update": [p, p, p, i32, i64, p, p],
+        "fl_project_rows": [p, p, i64, p, i32, i32, p, i32, p, i64, p, i32, p, p],
         "fl_quant_kv_residual": [p, C.POINTER(FlShape), C.c_int, p, p, p, i32, C.POINTER(FlKvStore), p, p],
         "fl_dense_loop_attention": [p, C.POINTER(FlShape), p, p, p, p, p, p, p, p],
         "fl_select_columns": [p, C.POINTER(FlShape), p, p, p, i32, i32, p, p, p, p],
@@ -207,6 +208,13 @@ def fl_gather_rows(ctx, src, idx, n, row_bytes, dst, stream=None, check=True) ->
 def fl_scatter_update(ctx, src, idx, n, row_bytes, dst, stream=None, check=True) -> int:
     rc = lib.fl_scatter_update(_h(ctx), _ptr(src), _ptr(idx), int(n), int(row_bytes), _ptr(dst), _stream(stream))
     return _check("fl_scatter_update", rc, check)
+
+
+def fl_project_rows(ctx, x, x_rows, src_idx, n, d_in, w, d_out, y, y_rows, dst_idx, accumulate, status=None,
+                    stream=None, check=True) -> int:
+    rc = lib.fl_project_rows(_h(ctx), _ptr(x), int(x_rows), _ptr(src_idx), int(n), int(d_in), _ptr(w), int(d_out),
+                             _ptr(y), int(y_rows), _ptr(dst_idx), int(accumulate), _ptr(status), _stream(stream))
+    return _check("fl_project_rows", rc, check)
 
 
 def fl_quant_kv_residual(ctx, shape, loop_r, k_new, v_new, active_idx, n_active, store, status=None, stream=None,

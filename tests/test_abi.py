@@ -72,6 +72,17 @@ def test_argument_validation_happens_before_any_launch(B):
     assert B.fl_gather_rows(ctx, None, P, 4, 64, P, **call) == INV
     assert B.fl_scatter_update(ctx, P, P, 4, 64, P + 8, **call) == INV
     assert B.fl_gather_rows(ctx, P, P, 0, 64, P, **call) == B.FL_OK                            # empty is a no-op
+    # projection of the active rows
+    pr = lambda **kw: B.fl_project_rows(ctx, kw.get("x", P), kw.get("xr", 1024), kw.get("si", P), kw.get("n", 16),
+                                        kw.get("din", 256), kw.get("w", P + 0x100000), kw.get("dout", 512),
+                                        kw.get("y", P + 0x200000), kw.get("yr", 1024), kw.get("di", None),
+                                        kw.get("acc", 0), **call)
+    assert pr(x=None) == INV and pr(w=None) == INV and pr(y=None) == INV and pr(n=-1) == INV and pr(acc=2) == INV
+    assert pr(x=P + 4) == INV and pr(y=P) == INV                         # misaligned; y aliases x
+    assert pr(si=None, n=2000) == INV and pr(di=None, n=2000, yr=100) == INV   # no index list: n must fit the matrix
+    assert pr(din=100) == UNS and pr(dout=100) == UNS
+    assert pr(n=0) == B.FL_OK
+    assert pr() == UNS                                                   # the stand-in context has no tensor path
     # quantizer
     st = fake_store(B)
     assert B.fl_quant_kv_residual(ctx, sh, 1, P, P, P, 16, st, **call) == INV                  # loop_r < 2

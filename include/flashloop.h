@@ -319,6 +319,16 @@ FL_API int fl_decode_attention(fl_ctx* ctx, const fl_shape* shape, int loop_r, c
                         int32_t c, const float* lse_prev, float* lse_out, const void* o_prev, void* o_out,
                         float* p_new_out, int32_t* status, void* stream);
 
+/* The checked build (libflashloop_debug.so, compiled with -DFL_DEBUG_BOUNDS) validates, before every launch, the
+ * index arrays the call is about to trust: row lists (range, strictly ascending), column lists against their counts
+ * (range, ascending, counts within [0, c]), candidate lists, and the slot maps of the residual streams the call reads
+ * (each value -1 or a row of its stream). A small kernel reads the arrays (never what they point to), the host waits for
+ * its verdict, and on a violation the call returns FL_ERR_INVALID_ARG, writes that code to `status` when one was given
+ * (also in the calls whose normal build never writes it) and launches nothing else. Nothing traps. The wait makes the
+ * checked build slow and unusable inside a stream capture: it is for tests and debugging. Returns 1 in the checked
+ * build, 0 otherwise. */
+FL_API int fl_debug_bounds_enabled(void);
+
 /* KV-cache accounting (Section 1's 48 GiB example; Section 4.3): bytes held for one layer by this store
  * after n_loops loops, and by a dense looped cache of n_loops loops. Host-only, no device access.
  * share_layers = number of layers sharing each loop's slot map and index list (>= 1). */

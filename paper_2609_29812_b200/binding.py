@@ -63,6 +63,7 @@ def _load() -> C.CDLL:
         "fl_create": [C.POINTER(C.c_void_p), C.c_int],
         "fl_destroy": [p],
         "fl_version": [],
+        "fl_debug_bounds_enabled": [],
         "fl_select_tokens": [p, C.POINTER(FlShape), C.c_int, p, p, p, i32, i32, p, p, p, p, p],
         "fl_gather_rows": [p, p, p, i32, i64, p, p],
         "fl_scatter_update": [p, p, p, i32, i64, p, p],

@@ -14,6 +14,7 @@ CSRC = os.path.join(PKG, "csrc")
 OBJ_DIR = os.path.join(PKG, "build")
 LIB_PATH = os.path.join(PKG, "libflashloop.so")
 SELFTEST_LIB_PATH = os.path.join(PKG, "libflashloop_selftest.so")
+DEBUG_LIB_PATH = os.path.join(PKG, "libflashloop_debug.so")   # the checked build (-DFL_DEBUG_BOUNDS)
 
 NVCC_FLAGS = [
     "-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
@@ -74,6 +75,17 @@ def build(force: bool = False, verbose: bool = False) -> str:
     r = subprocess.run(cmd, capture_output=True, text=True)
     if r.returncode != 0:
         raise RuntimeError(f"link failed:\n{r.stdout}\n{r.stderr}")
+    # the checked build: the same objects, with the index validator compiled in
+    dbg_obj = os.path.join(OBJ_DIR, "debug_bounds.checked.o")
+    r = subprocess.run([nvcc, *NVCC_FLAGS, "-DFL_DEBUG_BOUNDS", "-c", os.path.join(CSRC, "debug_bounds.cu"), "-o", dbg_obj],
+                       capture_output=True, text=True)
+    if r.returncode != 0:
+        raise RuntimeError(f"nvcc failed on the checked build of debug_bounds.cu:\n{r.stdout}\n{r.stderr}")
+    dbg_objs = [dbg_obj if os.path.basename(o) == "debug_bounds.o" else o for o in objs]
+    r = subprocess.run([nvcc, "-shared", "-o", DEBUG_LIB_PATH, *dbg_objs, "-gencode", "arch=compute_100a,code=sm_100a"],
+                       capture_output=True, text=True)
+    if r.returncode != 0:
+        raise RuntimeError(f"link of the checked build failed:\n{r.stdout}\n{r.stderr}")
     # tensor-path self-test kernels: a library of their own, loaded only by a GPU test
     st_dir = os.path.join(CSRC, "selftest")
     st_srcs = sorted(os.path.join(st_dir, f) for f in os.listdir(st_dir) if f.endswith(".cu"))

@@ -93,6 +93,7 @@ extern "C" int fl_create(fl_ctx** out, int device) {
   c->fused_attn = (fused != nullptr && fused[0] == '1') ? 1 : 0;
   const char* two_pass = std::getenv("FL_TWO_PASS");
   c->two_pass = (two_pass != nullptr && two_pass[0] == '1') ? 1 : 0;
+  c->dbg_flag = nullptr;
   c->encode_tiled = nullptr;
   {
     void* fn = nullptr;
@@ -107,12 +108,18 @@ extern "C" int fl_create(fl_ctx** out, int device) {
     delete c;
     return FL_ERR_CUDA;
   }
+  if (fl_debug_init(c) != FL_OK) {
+    delete c->tmaps;
+    delete c;
+    return FL_ERR_CUDA;
+  }
   *out = c;
   return FL_OK;
 }
 
 extern "C" int fl_destroy(fl_ctx* ctx) {
   if (ctx == nullptr) return FL_ERR_INVALID_ARG;
+  if (ctx->dbg_flag != nullptr) (void)cudaFree(ctx->dbg_flag);
   delete ctx->tmaps;
   delete ctx;
   return FL_OK;

@@ -328,7 +328,6 @@ extern "C" int fl_decode_attention(fl_ctx* ctx, const fl_shape* shape, int loop_
                                    int32_t n_queries, const fl_kv_store* store, const int32_t* col_idx,
                                    const int32_t* col_cnt, int32_t c, const float* lse_prev, float* lse_out,
                                    const void* o_prev, void* o_out, float* p_new_out, int32_t* status, void* stream) {
-  (void)status;
   FL_REQUIRE(ctx != nullptr);
   int rc = fl_check_shape(shape);
   if (rc != FL_OK) return rc;
@@ -343,6 +342,9 @@ extern "C" int fl_decode_attention(fl_ctx* ctx, const fl_shape* shape, int loop_
   FL_REQUIRE(fl_aligned16(q_new) && fl_aligned16(q_old) && fl_aligned16(o_prev) && fl_aligned16(o_out));
   const size_t smem = shape->head_dim == 64 ? decode_smem<64>(c) : decode_smem<128>(c);
   if (smem > (size_t)ctx->max_smem_optin) return FL_ERR_UNSUPPORTED;
+  rc = fl_debug_check_attn(ctx, shape, loop_r - 1, nullptr, 0, store, col_idx, col_cnt, c,
+                           (int64_t)n_queries * shape->n_heads, status, stream);
+  if (rc != FL_OK) return rc;
   DecodeArgs a{};
   a.q_new = q_new; a.q_old = q_old; a.o_prev = o_prev; a.o_out = o_out;
   fl_dev_side(store, true, &a.k);

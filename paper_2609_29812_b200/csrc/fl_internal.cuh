@@ -20,7 +20,30 @@ struct fl_ctx {
   int pdl;                  // launch the hot-path kernels with programmatic stream serialization (FL_NO_PDL=1: off)
   void* ws;                 // caller's workspace (fl_set_workspace), or null
   size_t ws_bytes;
+  void* dbg_flag;           // checked build only: device word of the index validator (allocated on first use)
 };
+
+// Index validation of the checked build (debug_bounds.cu; an empty stub otherwise). One entry per array:
+// values a[0..n) must lie in [lo, hi]; with seg > 0 the array is a sequence of segments of seg entries, of which
+// only the first cnt[segment] count (cnt null: all of them; a count outside [0, seg] is itself a violation);
+// ascending: strictly increasing inside a segment (the whole array when seg = 0).
+struct fl_idx_check {
+  const int32_t* a;
+  int64_t n;
+  int64_t seg;
+  const int32_t* cnt;
+  int32_t lo, hi;
+  int ascending;
+};
+// Returns FL_OK, or FL_ERR_INVALID_ARG (also written to *status, if given) when an index is out of range; the caller
+// must then launch nothing. Synchronises the stream in the checked build.
+int fl_debug_check(fl_ctx* ctx, const fl_idx_check* checks, int n_checks, int32_t* status, void* stream);
+int fl_debug_init(fl_ctx* ctx);   // allocates the validator's device word (checked build); FL_OK or FL_ERR_CUDA
+// The index inputs of an attention call: the active list, the column lists with their counts (n_segments lists of c
+// entries) and the slot maps of the first n_streams residual streams.
+int fl_debug_check_attn(fl_ctx* ctx, const fl_shape* s, int n_streams, const int32_t* active_idx, int32_t n_active,
+                        const fl_kv_store* store, const int32_t* col_idx, const int32_t* col_cnt, int32_t c,
+                        int64_t n_segments, int32_t* status, void* stream);
 
 // Layout of the loop-attention workspace: kFlMaxSplit int32 arrival counters, then per split problem two partial
 // results of kFlPartFloats binary32 values (both 128 x 128 accumulators and four statistics per row).

@@ -228,7 +228,6 @@ extern "C" int fl_loop_attention(fl_ctx* ctx, const fl_shape* shape, int loop_r,
                                  const int32_t* col_idx, const int32_t* col_cnt, int32_t c, const float* lse_prev,
                                  float* lse_out, const void* o_prev, void* o_out, float* col_scores_next,
                                  int32_t* status, void* stream) {
-  (void)status;
   FL_REQUIRE(ctx != nullptr);
   int rc = fl_check_shape(shape);
   if (rc != FL_OK) return rc;
@@ -247,6 +246,9 @@ extern "C" int fl_loop_attention(fl_ctx* ctx, const fl_shape* shape, int loop_r,
   }
   FL_REQUIRE(q_new != nullptr && q_old != nullptr && o_prev != nullptr && o_out != nullptr && active_idx != nullptr);
   FL_REQUIRE(fl_aligned16(q_new) && fl_aligned16(q_old) && fl_aligned16(o_prev) && fl_aligned16(o_out));
+  rc = fl_debug_check_attn(ctx, shape, loop_r - 1, active_idx, n_active, store, col_idx, col_cnt, c,
+                           (int64_t)shape->n_heads * fl_n_blocks(shape), status, stream);
+  if (rc != FL_OK) return rc;
 
   DevSide kside;
   fl_dev_side(store, true, &kside);
@@ -337,6 +339,9 @@ extern "C" int fl_loop_attention_indexed_carry(fl_ctx* ctx, const fl_shape* shap
                                     sizeof(float) * (size_t)shape->n_heads * fl_n_blocks(shape) * c, st));
     return FL_OK;
   }
+  rc = fl_debug_check_attn(ctx, shape, loop_r - 1, active_idx, n_active, store, col_idx, col_cnt, c,
+                           (int64_t)shape->n_heads * fl_n_blocks(shape), status, stream);
+  if (rc != FL_OK) return rc;
   // With the carried buffers and the loop's materialized rows a call that reuses the old term runs the single-term
   // kernel (new term only, two CTAs per SM). A recomputing call stays on the fused kernel, whose two terms share the
   // gathered tiles of every column without a payload in this loop (the gathers are what bounds these kernels);

@@ -250,6 +250,12 @@ extern "C" int fl_project_rows(fl_ctx* ctx, const void* x, int64_t x_rows, const
   FL_REQUIRE(x != y && w != y);
   if ((size_t)ctx->max_smem_optin < kProjSmem || ctx->encode_tiled == nullptr || ctx->tmaps == nullptr)
     return FL_ERR_UNSUPPORTED;
+  {
+    const fl_idx_check ck[2] = {{src_idx, n, 0, nullptr, 0, (int32_t)x_rows - 1, 0},
+                                {dst_idx, n, 0, nullptr, 0, (int32_t)y_rows - 1, 1}};
+    const int rc = fl_debug_check(ctx, ck, 2, status, stream);
+    if (rc != FL_OK) return rc;
+  }
   ProjArgs a;
   const bool gather = src_idx != nullptr;
   a.m_tiles = (n + kBM - 1) / kBM;

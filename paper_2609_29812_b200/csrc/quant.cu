@@ -276,7 +276,6 @@ int launch_quant(const fl_ctx* ctx, const fl_shape* s, const QuantArgs& a, int n
 extern "C" int fl_quant_kv_residual(fl_ctx* ctx, const fl_shape* shape, int loop_r, const void* k_new,
                                     const void* v_new, const int32_t* active_idx, int32_t n_active,
                                     const fl_kv_store* store, int32_t* status, void* stream) {
-  (void)status;
   FL_REQUIRE(ctx != nullptr);
   int rc = fl_check_shape(shape);
   if (rc != FL_OK) return rc;
@@ -293,6 +292,17 @@ extern "C" int fl_quant_kv_residual(fl_ctx* ctx, const fl_shape* shape, int loop
   const int d = shape->n_heads * shape->head_dim;
   // whole warps must enter or leave the element loop together (sub-warp shuffles inside)
   if (d % 256 != 0 || (d > 2048 && d % 2048 != 0)) return FL_ERR_UNSUPPORTED;
+  {
+    fl_idx_check ck[1 + 2 * FL_MAX_LOOPS];
+    int n = 0;
+    ck[n++] = {active_idx, n_active, 0, nullptr, 0, shape->L - 1, 1};
+    for (int i = 0; i < loop_r - 2; ++i) {   // the earlier streams' slot maps: the chain is rebuilt through them
+      ck[n++] = {store->k_res[i].slot_of_pos, shape->L, 0, nullptr, -1, store->k_res[i].n_rows - 1, 0};
+      ck[n++] = {store->v_res[i].slot_of_pos, shape->L, 0, nullptr, -1, store->v_res[i].n_rows - 1, 0};
+    }
+    rc = fl_debug_check(ctx, ck, n, status, stream);
+    if (rc != FL_OK) return rc;
+  }
 
   QuantArgs a;
   fl_dev_side(store, true, &a.k);

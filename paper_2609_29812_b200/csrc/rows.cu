@@ -40,6 +40,12 @@ int rows_copy(bool gather, fl_ctx* ctx, const void* src, const int32_t* idx, int
   if (n == 0) return FL_OK;
   FL_REQUIRE(src != nullptr && dst != nullptr && idx != nullptr);
   FL_REQUIRE(fl_aligned16(src) && fl_aligned16(dst));
+  {
+    // the row count of the indexed matrix is not part of this call: only sign and order can be checked
+    const fl_idx_check ck = {idx, n, 0, nullptr, 0, INT32_MAX, 1};
+    const int rc = fl_debug_check(ctx, &ck, 1, nullptr, stream);
+    if (rc != FL_OK) return rc;
+  }
   const int warps = 8;
   const int vec_per_row = (int)(row_bytes / 16);
   const int pieces = (vec_per_row + 127) / 128;

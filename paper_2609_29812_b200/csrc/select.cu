@@ -763,7 +763,6 @@ __global__ void __launch_bounds__(kSelThreads) column_select_kernel(const float*
 extern "C" int fl_select_tokens(fl_ctx* ctx, const fl_shape* shape, int loop_r, const void* h_prev, const void* h_cur,
                                 const int32_t* cand, int32_t n_cand, int32_t k, float* scores, int32_t* active_idx,
                                 int32_t* slot_of_pos, int32_t* status, void* stream) {
-  (void)status;
   FL_REQUIRE(ctx != nullptr);
   int rc = fl_check_shape(shape);
   if (rc != FL_OK) return rc;
@@ -775,6 +774,11 @@ extern "C" int fl_select_tokens(fl_ctx* ctx, const fl_shape* shape, int loop_r, 
   FL_REQUIRE(cand != nullptr || n_cand == shape->L);
   const int d = shape->n_heads * shape->head_dim;
   if (d % 256 != 0) return FL_ERR_UNSUPPORTED;
+  {
+    const fl_idx_check ck = {cand, n_cand, 0, nullptr, 0, shape->L - 1, 1};
+    rc = fl_debug_check(ctx, &ck, 1, status, stream);
+    if (rc != FL_OK) return rc;
+  }
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int warps = 8;
   const int grid = (n_cand + warps - 1) / warps;
@@ -797,7 +801,6 @@ extern "C" int fl_select_tokens(fl_ctx* ctx, const fl_shape* shape, int loop_r, 
 extern "C" int fl_select_columns(fl_ctx* ctx, const fl_shape* shape, const float* col_scores, const int32_t* cand_cols,
                                  const int32_t* cand_cnt, int32_t n_cand, int32_t c, int32_t* col_idx, int32_t* col_cnt,
                                  int32_t* status, void* stream) {
-  (void)status;
   FL_REQUIRE(ctx != nullptr);
   int rc = fl_check_shape(shape);
   if (rc != FL_OK) return rc;
@@ -807,6 +810,11 @@ extern "C" int fl_select_columns(fl_ctx* ctx, const fl_shape* shape, const float
   else FL_REQUIRE(cand_cnt != nullptr);
   const int nb = fl_n_blocks(shape);
   FL_REQUIRE(nb <= 65535);
+  {
+    const fl_idx_check ck = {cand_cols, (int64_t)shape->n_heads * nb * n_cand, n_cand, cand_cnt, 0, shape->L - 1, 0};
+    rc = fl_debug_check(ctx, &ck, 1, status, stream);
+    if (rc != FL_OK) return rc;
+  }
   dim3 grid(shape->n_heads, nb);
   const size_t key_bytes = sizeof(uint32_t) * (((size_t)n_cand + 3) & ~(size_t)3);
   const int vec_ok = (fl_aligned16(col_scores) && n_cand % 4 == 0) ? 1 : 0;

@@ -28,6 +28,8 @@ Functions and the passage each one follows:
                                    Appendix E "Quantization Setting" (asymmetric,
                                    group-wise, scale and offset from min / max)
   residual_update                  Section 4.3 / Appendix D.3 (masked residual codec)
+  quantize_base, base_q_bytes      Appendix E "Quantization Setting" (the loop-1 base: keys per channel,
+                                   values per token, the most recent tokens kept unquantized)
   project_rows                     Section 4.4 / Appendix G (only the selected token rows pass through
                                    the projections; results return to their positions)
   kv_bytes_per_token_layer         Section 1 (48 GiB example) and Section 4.3 accounting
@@ -265,6 +267,60 @@ def residual_update(x_new_rows, xhat_prev, active, bits, group):
     deq = dequantize_groups(codes, scale, zero, group)
     xhat_new[active] = (xhat_prev[active] + deq).astype(F32)      # binary32 addition
     return xhat_new, {"codes": codes, "packed": pack_codes(codes, bits), "scale": scale, "zero": zero}
+
+
+# --------------------------------------------------------------------------------------
+# Appendix E "Quantization Setting", the base states: the same asymmetric min/max quantizer, with the keys
+# grouped per channel (a group = `group` consecutive tokens of ONE channel) and the values per token (a group =
+# `group` consecutive channels of ONE token); the most recent `tail` tokens stay in the storage type.
+# --------------------------------------------------------------------------------------
+def quantize_base(k, v, bits, group, tail, storage_round=None):
+    """Quantizes the loop-1 K and V of one layer and returns what every later reader sees in their place.
+
+    k, v: [L, H, dh] (or [L, d]) storage-precision values.  Positions [0, Lq), Lq = max(0, L - tail), are
+    quantized; the last `tail` positions are kept as they are.  K: for every channel, groups of `group`
+    consecutive positions (the last group of the quantized range may be shorter).  V: for every position, groups
+    of `group` consecutive channels.  The dequantized value code * scale + offset is formed with one binary32
+    rounding and then rounded to the storage type by `storage_round` (None: binary32 storage).
+    Returns a dict: khat, vhat [L, d] float32 (the base as read back), k_codes, v_codes uint8 [Lq, d],
+    k_scale, k_zero fp16 [ceil(Lq / group), d], v_scale, v_zero fp16 [Lq, d / group], k_tail, v_tail [min(tail, L), d].
+    """
+    L = k.shape[0]
+    k2 = np.asarray(k).reshape(L, -1).astype(F32)
+    v2 = np.asarray(v).reshape(L, -1).astype(F32)
+    d = k2.shape[1]
+    Lq = max(0, L - tail)
+    n_tg = (Lq + group - 1) // group
+    rnd = storage_round if storage_round is not None else (lambda a: a)
+    khat, vhat = k2.copy(), v2.copy()
+    k_codes = np.zeros((Lq, d), dtype=np.uint8)
+    k_scale = np.zeros((n_tg, d), dtype=np.float16)
+    k_zero = np.zeros((n_tg, d), dtype=np.float16)
+    for g in range(n_tg):                                   # keys: one group = one channel over up to `group` tokens
+        lo, hi = g * group, min(Lq, (g + 1) * group)
+        chan_major = np.ascontiguousarray(k2[lo:hi].T)      # [d, tokens of the group]
+        c, s, z = quantize_groups(chan_major, bits, hi - lo)
+        k_codes[lo:hi] = c.T
+        k_scale[g], k_zero[g] = s[:, 0], z[:, 0]
+        khat[lo:hi] = rnd(dequantize_groups(c, s, z, hi - lo).T)
+    v_codes = np.zeros((Lq, d), dtype=np.uint8)
+    v_scale = np.zeros((Lq, d // group), dtype=np.float16)
+    v_zero = np.zeros((Lq, d // group), dtype=np.float16)
+    if Lq > 0:                                              # values: one group = one token over `group` channels
+        v_codes, v_scale, v_zero = quantize_groups(np.ascontiguousarray(v2[:Lq]), bits, group)
+        vhat[:Lq] = rnd(dequantize_groups(v_codes, v_scale, v_zero, group))
+    return {"khat": khat, "vhat": vhat, "k_codes": k_codes, "k_scale": k_scale, "k_zero": k_zero,
+            "v_codes": v_codes, "v_scale": v_scale, "v_zero": v_zero, "k_tail": k2[Lq:].copy(), "v_tail": v2[Lq:].copy()}
+
+
+def base_q_bytes(L, d, bits, group, tail, elem_bytes=2):
+    """Bytes of one layer's quantized base, K and V together: packed codes of the quantized positions, fp16 scale
+    and offset per group (keys: per channel and token group; values: per token and channel group), the tail rows."""
+    Lq = max(0, L - tail)
+    n_tg = (Lq + group - 1) // group
+    codes = 2 * Lq * (d * bits // 8)
+    meta = 2 * 2 * (n_tg * d) + 2 * 2 * (Lq * (d // group))
+    return codes + meta + 2 * (L - Lq) * d * elem_bytes
 
 
 # --------------------------------------------------------------------------------------

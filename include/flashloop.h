@@ -319,6 +319,38 @@ FL_API int fl_decode_attention(fl_ctx* ctx, const fl_shape* shape, int loop_r, c
                         int32_t c, const float* lse_prev, float* lse_out, const void* o_prev, void* o_out,
                         float* p_new_out, int32_t* status, void* stream);
 
+/* Quantized loop-1 base (Appendix E, "Quantization Setting"): the quantizer of the residual streams (asymmetric,
+ * scale and offset from the group's minimum and maximum, shape->bits bits) applied to the base K and V of a layer, the
+ * keys grouped PER CHANNEL (a group = `group` consecutive positions of one channel) and the values PER TOKEN (a group =
+ * `group` consecutive channels of one position); the most recent `tail` positions stay in the storage type.
+ * With Lq = max(0, L - tail), d = H*dh, all device buffers owned by the caller, 16-byte aligned:
+ *   k_codes, v_codes : uint8 [Lq, d*bits/8]  packed like the residual codes (little-endian inside a byte)
+ *   k_scale, k_zero  : fp16  [ceil(Lq/group), d]      (the last token group may be shorter)
+ *   v_scale, v_zero  : fp16  [Lq, d/group]
+ *   k_tail, v_tail   : storage type [L - Lq, d]        rows Lq .. L-1 as they are */
+typedef struct {
+  void* k_codes; void* k_scale; void* k_zero;
+  void* v_codes; void* v_scale; void* v_zero;
+  void* k_tail;  void* v_tail;
+  int32_t group; /* 32, 64 or 128; must divide d */
+  int32_t tail;  /* >= 0 */
+} fl_kv_base_q; /* host struct holding device pointers */
+
+/* Packs k, v ([L, H, dh] storage type) into `base`. Arithmetic as in fl_quant_kv_residual, in binary32:
+ *   zero = fp16 round-down(min);  scale = fp16 round-up((max - zero) / (2^bits - 1)), 0 for a constant group;
+ *   code = clamp(round-half-even((x - zero) / scale), 0, 2^bits - 1).
+ * fl_dequant_kv_base writes all L rows of k_out, v_out ([L, H, dh] storage type): rows below Lq as
+ * storage-round(fma(code, scale, zero)), the tail rows copied back. The sparse loops then run on k_out / v_out as
+ * their base: the packed form is what stays resident, the rebuilt rows are a transient copy of one layer.
+ * Errors: FL_ERR_INVALID_ARG for null or misaligned buffers, a group other than 32 / 64 / 128, tail < 0;
+ * FL_ERR_UNSUPPORTED when shape->bits is 16, or d is not a multiple of 256 and of the group. `status` is never
+ * written. fl_kv_base_q_bytes returns the bytes of the packed form (codes, metadata and tail, K and V). */
+FL_API int fl_quant_kv_base(fl_ctx* ctx, const fl_shape* shape, const void* k, const void* v, const fl_kv_base_q* base,
+                     int32_t* status, void* stream);
+FL_API int fl_dequant_kv_base(fl_ctx* ctx, const fl_shape* shape, const fl_kv_base_q* base, void* k_out, void* v_out,
+                       int32_t* status, void* stream);
+FL_API int fl_kv_base_q_bytes(const fl_shape* shape, int32_t group, int32_t tail, int64_t* bytes);
+
 /* The checked build (libflashloop_debug.so, compiled with -DFL_DEBUG_BOUNDS) validates, before every launch, the
  * index arrays the call is about to trust: row lists (range, strictly ascending), column lists against their counts
  * (range, ascending, counts within [0, c]), candidate lists, and the slot maps of the residual streams the call reads

@@ -24,6 +24,12 @@ FL_F32 = 1
 FL_MAX_LOOPS = 32
 
 
+class FlKvBaseQ(C.Structure):
+    _fields_ = [("k_codes", C.c_void_p), ("k_scale", C.c_void_p), ("k_zero", C.c_void_p),
+                ("v_codes", C.c_void_p), ("v_scale", C.c_void_p), ("v_zero", C.c_void_p),
+                ("k_tail", C.c_void_p), ("v_tail", C.c_void_p), ("group", C.c_int32), ("tail", C.c_int32)]
+
+
 class FlShape(C.Structure):
     _fields_ = [("L", C.c_int32), ("n_heads", C.c_int32), ("head_dim", C.c_int32), ("dtype", C.c_int32),
                 ("q_block", C.c_int32), ("bits", C.c_int32), ("group", C.c_int32),
@@ -81,6 +87,9 @@ def _load() -> C.CDLL:
                                              p, p, i32, p, p, p, p, p, p, p],
         "fl_decode_attention": [p, C.POINTER(FlShape), C.c_int, p, p, i32, C.POINTER(FlKvStore), p, p, i32, p, p, p, p, p,
                                 p, p],
+        "fl_quant_kv_base": [p, C.POINTER(FlShape), p, p, C.POINTER(FlKvBaseQ), p, p],
+        "fl_dequant_kv_base": [p, C.POINTER(FlShape), C.POINTER(FlKvBaseQ), p, p, p, p],
+        "fl_kv_base_q_bytes": [C.POINTER(FlShape), i32, i32, C.POINTER(i64)],
         "fl_kv_store_bytes": [C.POINTER(FlShape), C.POINTER(FlKvStore), C.c_int, C.c_int,
                               C.POINTER(i64), C.POINTER(i64)],
         "fl_loop_attention_workspace_bytes": [p, C.POINTER(FlShape), C.POINTER(i64)],
@@ -216,6 +225,34 @@ def fl_project_rows(ctx, x, x_rows, src_idx, n, d_in, w, d_out, y, y_rows, dst_i
     rc = lib.fl_project_rows(_h(ctx), _ptr(x), int(x_rows), _ptr(src_idx), int(n), int(d_in), _ptr(w), int(d_out),
                              _ptr(y), int(y_rows), _ptr(dst_idx), int(accumulate), _ptr(status), _stream(stream))
     return _check("fl_project_rows", rc, check)
+
+
+def make_base_q(k_codes, k_scale, k_zero, v_codes, v_scale, v_zero, k_tail, v_tail, group, tail) -> FlKvBaseQ:
+    """Host struct of a quantized base; the tensors (or raw addresses) must outlive every call that uses it."""
+    q = FlKvBaseQ()
+    for name, t in (("k_codes", k_codes), ("k_scale", k_scale), ("k_zero", k_zero), ("v_codes", v_codes),
+                    ("v_scale", v_scale), ("v_zero", v_zero), ("k_tail", k_tail), ("v_tail", v_tail)):
+        setattr(q, name, _ptr(t))
+    q.group, q.tail = int(group), int(tail)
+    return q
+
+
+def fl_quant_kv_base(ctx, shape, k, v, base, status=None, stream=None, check=True) -> int:
+    rc = lib.fl_quant_kv_base(_h(ctx), C.byref(shape), _ptr(k), _ptr(v), C.byref(base) if base is not None else None,
+                              _ptr(status), _stream(stream))
+    return _check("fl_quant_kv_base", rc, check)
+
+
+def fl_dequant_kv_base(ctx, shape, base, k_out, v_out, status=None, stream=None, check=True) -> int:
+    rc = lib.fl_dequant_kv_base(_h(ctx), C.byref(shape), C.byref(base) if base is not None else None, _ptr(k_out),
+                                _ptr(v_out), _ptr(status), _stream(stream))
+    return _check("fl_dequant_kv_base", rc, check)
+
+
+def fl_kv_base_q_bytes(shape, group, tail) -> int:
+    out = C.c_int64()
+    _check("fl_kv_base_q_bytes", lib.fl_kv_base_q_bytes(C.byref(shape), int(group), int(tail), C.byref(out)), True)
+    return out.value
 
 
 def fl_quant_kv_residual(ctx, shape, loop_r, k_new, v_new, active_idx, n_active, store, status=None, stream=None,

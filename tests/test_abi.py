@@ -122,6 +122,19 @@ def test_argument_validation_happens_before_any_launch(B):
                                              kw.get("ci", P), P, kw.get("c", 64), P, P, P, P, None, **call)
     assert dec(r=1) == INV and dec(c=0) == INV and dec(q=None) == INV and dec(ci=None) == INV and dec(st=None) == INV
     assert dec(n=-1) == INV and dec(r=3) == INV and dec(n=0) == B.FL_OK
+    # quantized base
+    bq = lambda **kw: B.make_base_q(kw.get("kc", P), P, P, P, P, P, kw.get("kt", P), P, kw.get("g", 64), kw.get("t", 64))
+    qb = lambda base, k=P: B.fl_quant_kv_base(ctx, kw_sh.get("sh", sh), k, P, base, **call)
+    kw_sh = {}
+    assert qb(bq(g=48)) == INV and qb(bq(t=-1)) == INV and qb(bq(kc=None)) == INV and qb(bq(kt=None)) == INV
+    assert qb(bq(kc=P + 4)) == INV and qb(None) == INV and qb(bq(), k=None) == INV
+    kw_sh["sh"] = good_shape(B, bits=16)
+    assert qb(bq()) == UNS
+    kw_sh["sh"] = good_shape(B, n_heads=1)
+    assert qb(bq()) == UNS                                                                     # d = 128
+    assert B.fl_dequant_kv_base(ctx, sh, bq(), None, P, **call) == INV
+    assert B.fl_kv_base_q_bytes(good_shape(B, L=192, n_heads=2, head_dim=64, group=64), 64, 64) == \
+        2 * 128 * 64 + 2 * 128 * 4 + 128 * 2 * 4 + 2 * 64 * 128 * 2
     # accounting
     rc = B.lib.fl_kv_store_bytes(C.byref(sh), C.byref(st), 3, 1, C.byref(C.c_int64()), C.byref(C.c_int64()))
     assert rc == INV                                                                          # only one stream

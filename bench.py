@@ -68,6 +68,10 @@ def parse_args():
                          "sched: budgets that decay from loop to loop with real column pruning (Table 6's deep "
                          "schedule: tokens 90% -> 20%, columns pruned inside the previous set every loop)")
     ap.add_argument("--sweep", default="subset", choices=["subset", "full"], help="c4: which points to run")
+    ap.add_argument("--int4-base", action="store_true",
+                    help="keep every layer's loop-1 K/V packed (Appendix E: int4, keys per channel, values per token, "
+                         "groups of 64, last 64 positions unquantized) and rebuild one layer's rows into a transient "
+                         "buffer before each layer's work in each loop (fl_dequant_kv_base, inside the timed step)")
     ap.add_argument("--no-economy", action="store_true", help="recompute the old term in every loop")
     ap.add_argument("--no-variants", action="store_true", help="skip the in-kernel dequantization variant")
     ap.add_argument("--layers", type=int, default=0, help="override the number of layers (development)")
@@ -162,6 +166,8 @@ class Bench:
         self.nb = (w.L + w.q_block - 1) // w.q_block
         self.c = w.col_budget
         self.economy = economy
+        self.int4_base = bool(getattr(args, "int4_base", False))
+        self.base_group, self.base_tail = 64, 64
         self.stream = torch.cuda.Stream(device=device)
         self.sp = int(self.stream.cuda_stream)
         self.keep = []           # keeps tensors and host structs alive
@@ -191,10 +197,30 @@ class Bench:
             self.xbuf = torch.empty(n_max, self.d, dtype=torch.bfloat16, device=dev)
             self.o_out_buf = mkrows()      # end-to-end arm: the last layer's new O rows, gathered for the read-back
             self.layers = []
+            if self.int4_base:
+                # one transient copy of a layer's rebuilt base for the whole stack; the packed form is what stays
+                self.k_transient = torch.empty(self.L, self.H, self.dh, dtype=torch.bfloat16, device=dev)
+                self.v_transient = torch.empty_like(self.k_transient)
             for l in range(self.NL):
                 gen = stack.layer(l)
                 q1, k1, v1 = gen.qkv1()
                 st = P.LayerState(ctx, w, dev)
+                if self.int4_base:
+                    g_, t_ = self.base_group, self.base_tail
+                    Lq = max(0, self.L - t_)
+                    n_tg = (Lq + g_ - 1) // g_
+                    u8 = lambda *s_: torch.empty(s_, dtype=torch.uint8, device=dev)
+                    f16 = lambda *s_: torch.empty(s_, dtype=torch.float16, device=dev)
+                    st.base_tensors = [u8(Lq, self.d * w.bits // 8), f16(n_tg, self.d), f16(n_tg, self.d),
+                                       u8(Lq, self.d * w.bits // 8), f16(Lq, self.d // g_), f16(Lq, self.d // g_),
+                                       torch.empty(self.L - Lq, self.d, dtype=torch.bfloat16, device=dev),
+                                       torch.empty(self.L - Lq, self.d, dtype=torch.bfloat16, device=dev)]
+                    st.base_q = B.make_base_q(*st.base_tensors, g_, t_)
+                    st.row_mask = torch.zeros(self.H, (self.L + 31) // 32, dtype=torch.int32, device=dev)
+                    B.fl_quant_kv_base(ctx, sh, k1, v1, st.base_q)
+                    B.fl_dequant_kv_base(ctx, sh, st.base_q, self.k_transient, self.v_transient)
+                    # every loop of the layer, the dense one included, reads the base as it is stored
+                    k1, v1 = self.k_transient, self.v_transient
                 e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
                 e0.record(self.stream)
                 st.dense_loop(q1, k1, v1)
@@ -295,6 +321,18 @@ class Bench:
         calls, launches = [], 0
         # per-step algorithmic bytes of the memory-bound stages (for the whole-step roofline)
         stage_bytes = {"select_tokens": 0.0, "gather_scatter": 0.0, "quant": 0.0, "select_columns": 0.0}
+        if self.int4_base:
+            stage_bytes["dequant_base"] = 0.0
+            base_q_bytes = B.fl_kv_base_q_bytes(self.shape, self.base_group, self.base_tail)
+            if not hasattr(self, "base_share"):
+                # share of a layer's (head, position) pairs its sparse loops read, measured on layer 0
+                st0, sel0 = self.layers[0], self.sels[0]
+                B.fl_mark_base_rows(self.ctx, self.shape, st0.col_idx, st0.col_cnt, self.c, sel0.active_idx, sel0.n,
+                                    st0.row_mask, stream=self.stream)
+                self.stream.synchronize()
+                m = st0.row_mask.view(self.torch.uint8)
+                lut = self.torch.tensor([bin(i).count("1") for i in range(256)], device=m.device)
+                self.base_share = float(lut[m.long()].sum().item()) / (self.H * self.L)
         pay_row = 2 * (self.d * w.bits // 8 + 4 * (self.d // w.group)) if w.bits != 16 else 2 * self.d * e
         for r in range(2, self.R + 1):
             sel = self.sels[r - 2]
@@ -319,6 +357,22 @@ class Bench:
                     launches += 1
                     tri = sum(min(self.L, (b + 1) * w.q_block) for b in range(self.nb))
                     stage_bytes["select_columns"] += 4.0 * self.H * (tri + self.nb * (self.c + 1))
+                if self.int4_base:
+                    # the rows this layer's sparse loops read (selected columns per head, active positions) are marked
+                    # once, in loop 2 (later active sets are nested in loop 2's, the column lists stay), and only they
+                    # are rebuilt into the transient buffer before the layer's work in every loop
+                    if r == 2:
+                        calls.append(("dequant_base", lib.fl_mark_base_rows,
+                                      (ctx, shp, p(st.col_idx), p(st.col_cnt), self.c, p(sel.active_idx), n,
+                                       p(st.row_mask), None, sp), r))
+                        launches += 1
+                        stage_bytes["dequant_base"] += 4.0 * self.H * self.nb * (self.c + 1) + 4.0 * n
+                    calls.append(("dequant_base", lib.fl_dequant_kv_base,
+                                  (ctx, shp, C.byref(st.base_q), p(st.row_mask), p(self.k_transient),
+                                   p(self.v_transient), None, sp), r))
+                    launches += 1
+                    # algorithmic bytes: packed codes + metadata in, rows out, for the marked share of the rows
+                    stage_bytes["dequant_base"] += self.base_share * (base_q_bytes + 2.0 * self.L * self.d * e)
                 q_new, k_new, v_new = st.rows[r]
                 calls.append(("quant", lib.fl_quant_kv_residual,
                               (ctx, shp, r, p(k_new), p(v_new), p(sel.active_idx), n, C.byref(store), None, sp), r))
@@ -421,6 +475,9 @@ class Bench:
 def kv_bytes_per_token(bench):
     B, w = bench.B, bench.w
     fl, dense = B.fl_kv_store_bytes(bench.shape, bench.layers[0].store, w.n_loops, w.n_layers)
+    if bench.int4_base:   # the packed base replaces the bf16 rows; the transient copy of one layer is shared by the stack
+        fl += B.fl_kv_base_q_bytes(bench.shape, bench.base_group, bench.base_tail) - 2 * w.L * w.d * 2
+        fl += 2 * w.L * w.d * 2 / w.n_layers
     return fl / w.L, dense / w.L
 
 
@@ -558,6 +615,9 @@ def run_ours(args):
            "config": {"workload": f"{w.name}: L={w.L}, {w.n_layers} layers, d={w.d}, {w.n_heads}x{w.head_dim} MHA, "
                                   f"R={w.n_loops}, token budget {w.k_tokens} rows, column budget {w.col_budget}, "
                                   f"q_block {w.q_block}, int{w.bits} g{w.group} residuals",
+                      "base": ("int4 per-channel K / per-token V, groups of 64, last 64 positions bf16; one layer's rows "
+                               "rebuilt into a transient buffer per layer and loop inside the step"
+                               if bench.int4_base else "bf16 rows resident"),
                       "old_term": ("recomputed in loop 2, carried (background rows + mass) in later loops"
                                    if bench.economy else "recomputed in every loop"),
                       "parallelism": "replicas only" if world > 1 else "single GPU",

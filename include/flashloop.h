@@ -339,16 +339,25 @@ typedef struct {
 /* Packs k, v ([L, H, dh] storage type) into `base`. Arithmetic as in fl_quant_kv_residual, in binary32:
  *   zero = fp16 round-down(min);  scale = fp16 round-up((max - zero) / (2^bits - 1)), 0 for a constant group;
  *   code = clamp(round-half-even((x - zero) / scale), 0, 2^bits - 1).
- * fl_dequant_kv_base writes all L rows of k_out, v_out ([L, H, dh] storage type): rows below Lq as
- * storage-round(fma(code, scale, zero)), the tail rows copied back. The sparse loops then run on k_out / v_out as
- * their base: the packed form is what stays resident, the rebuilt rows are a transient copy of one layer.
+ * fl_dequant_kv_base writes rows of k_out, v_out ([L, H, dh] storage type): rows below Lq as
+ * storage-round(fma(code, scale, zero)), the tail rows copied back. row_mask = NULL rebuilds every row; otherwise
+ * (device uint32 [H, ceil(L/32)], bit t%32 of word [h][t/32]) only the (head, position) pairs whose bit is set, and
+ * the rest of k_out / v_out is left untouched (the tail rows are always copied). The sparse loops then run on
+ * k_out / v_out as their base: the packed form is what stays resident, the rebuilt rows are a transient copy of one
+ * layer. fl_mark_base_rows fills such a mask with what the sparse loops of a layer read (Appendix D.2: attention
+ * touches the selected columns only; Eq. 8: the residual chain starts from the base rows of the active positions):
+ * for every head the first col_cnt[h, b] entries of col_idx[h, b, :] of all its blocks, plus active_idx[0..n_active).
+ * It clears the mask first. A mask made with the active set of loop r also serves every later loop whose active set
+ * is nested in it and whose column lists are subsets.
  * Errors: FL_ERR_INVALID_ARG for null or misaligned buffers, a group other than 32 / 64 / 128, tail < 0;
  * FL_ERR_UNSUPPORTED when shape->bits is 16, or d is not a multiple of 256 and of the group. `status` is never
  * written. fl_kv_base_q_bytes returns the bytes of the packed form (codes, metadata and tail, K and V). */
 FL_API int fl_quant_kv_base(fl_ctx* ctx, const fl_shape* shape, const void* k, const void* v, const fl_kv_base_q* base,
                      int32_t* status, void* stream);
-FL_API int fl_dequant_kv_base(fl_ctx* ctx, const fl_shape* shape, const fl_kv_base_q* base, void* k_out, void* v_out,
-                       int32_t* status, void* stream);
+FL_API int fl_dequant_kv_base(fl_ctx* ctx, const fl_shape* shape, const fl_kv_base_q* base, const uint32_t* row_mask,
+                       void* k_out, void* v_out, int32_t* status, void* stream);
+FL_API int fl_mark_base_rows(fl_ctx* ctx, const fl_shape* shape, const int32_t* col_idx, const int32_t* col_cnt, int32_t c,
+                      const int32_t* active_idx, int32_t n_active, uint32_t* row_mask, int32_t* status, void* stream);
 FL_API int fl_kv_base_q_bytes(const fl_shape* shape, int32_t group, int32_t tail, int64_t* bytes);
 
 /* The checked build (libflashloop_debug.so, compiled with -DFL_DEBUG_BOUNDS) validates, before every launch, the

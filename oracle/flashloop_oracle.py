@@ -30,6 +30,7 @@ Functions and the passage each one follows:
   residual_update                  Section 4.3 / Appendix D.3 (masked residual codec)
   quantize_base, base_q_bytes      Appendix E "Quantization Setting" (the loop-1 base: keys per channel,
                                    values per token, the most recent tokens kept unquantized)
+  base_rows_needed                 Appendix D.2 / D.3 (which base rows a layer's sparse loops read)
   project_rows                     Section 4.4 / Appendix G (only the selected token rows pass through
                                    the projections; results return to their positions)
   kv_bytes_per_token_layer         Section 1 (48 GiB example) and Section 4.3 accounting
@@ -311,6 +312,19 @@ def quantize_base(k, v, bits, group, tail, storage_round=None):
         vhat[:Lq] = rnd(dequantize_groups(v_codes, v_scale, v_zero, group))
     return {"khat": khat, "vhat": vhat, "k_codes": k_codes, "k_scale": k_scale, "k_zero": k_zero,
             "v_codes": v_codes, "v_scale": v_scale, "v_zero": v_zero, "k_tail": k2[Lq:].copy(), "v_tail": v2[Lq:].copy()}
+
+
+def base_rows_needed(col_sets, active, H, L):
+    """[H, L] booleans: the base rows of head h that a layer's sparse loops read.  The attention of Appendix D.2
+    touches, for head h, only the columns of its blocks' selected sets; the residual codec of Appendix D.3 starts the
+    chain of every active position from its base row (all heads)."""
+    need = np.zeros((H, L), dtype=bool)
+    for (h, _b), S in col_sets.items():
+        for j in S:
+            need[h, int(j)] = True
+    for i in active:
+        need[:, int(i)] = True
+    return need
 
 
 def base_q_bytes(L, d, bits, group, tail, elem_bytes=2):

@@ -88,7 +88,8 @@ def _load() -> C.CDLL:
         "fl_decode_attention": [p, C.POINTER(FlShape), C.c_int, p, p, i32, C.POINTER(FlKvStore), p, p, i32, p, p, p, p, p,
                                 p, p],
         "fl_quant_kv_base": [p, C.POINTER(FlShape), p, p, C.POINTER(FlKvBaseQ), p, p],
-        "fl_dequant_kv_base": [p, C.POINTER(FlShape), C.POINTER(FlKvBaseQ), p, p, p, p],
+        "fl_dequant_kv_base": [p, C.POINTER(FlShape), C.POINTER(FlKvBaseQ), p, p, p, p, p],
+        "fl_mark_base_rows": [p, C.POINTER(FlShape), p, p, i32, p, i32, p, p, p],
         "fl_kv_base_q_bytes": [C.POINTER(FlShape), i32, i32, C.POINTER(i64)],
         "fl_kv_store_bytes": [C.POINTER(FlShape), C.POINTER(FlKvStore), C.c_int, C.c_int,
                               C.POINTER(i64), C.POINTER(i64)],
@@ -243,10 +244,17 @@ def fl_quant_kv_base(ctx, shape, k, v, base, status=None, stream=None, check=Tru
     return _check("fl_quant_kv_base", rc, check)
 
 
-def fl_dequant_kv_base(ctx, shape, base, k_out, v_out, status=None, stream=None, check=True) -> int:
-    rc = lib.fl_dequant_kv_base(_h(ctx), C.byref(shape), C.byref(base) if base is not None else None, _ptr(k_out),
-                                _ptr(v_out), _ptr(status), _stream(stream))
+def fl_dequant_kv_base(ctx, shape, base, k_out, v_out, row_mask=None, status=None, stream=None, check=True) -> int:
+    rc = lib.fl_dequant_kv_base(_h(ctx), C.byref(shape), C.byref(base) if base is not None else None, _ptr(row_mask),
+                                _ptr(k_out), _ptr(v_out), _ptr(status), _stream(stream))
     return _check("fl_dequant_kv_base", rc, check)
+
+
+def fl_mark_base_rows(ctx, shape, col_idx, col_cnt, c, active_idx, n_active, row_mask, status=None, stream=None,
+                      check=True) -> int:
+    rc = lib.fl_mark_base_rows(_h(ctx), C.byref(shape), _ptr(col_idx), _ptr(col_cnt), int(c), _ptr(active_idx),
+                               int(n_active), _ptr(row_mask), _ptr(status), _stream(stream))
+    return _check("fl_mark_base_rows", rc, check)
 
 
 def fl_kv_base_q_bytes(shape, group, tail) -> int:

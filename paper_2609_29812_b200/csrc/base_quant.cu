@@ -12,9 +12,12 @@ namespace {
 struct BaseArgs {
   const void* k; const void* v;        // quantize: inputs [L, d]; dequantize: unused
   void* k_out; void* v_out;            // dequantize: outputs [L, d]; quantize: unused
+  const void* k_tail; const void* v_tail;   // dequantize: rows Lq .. L-1 in the storage type
+  int L;
   uint8_t* k_codes; __half* k_scale; __half* k_zero;
   uint8_t* v_codes; __half* v_scale; __half* v_zero;
-  int Lq, d, group;
+  const uint32_t* row_mask;            // dequantize: bit t of word [h][t / 32] set = rebuild row t of head h; null = all rows
+  int Lq, d, group, dh, mask_words;
 };
 
 template <int BITS>
@@ -127,7 +130,9 @@ __global__ void __launch_bounds__(256) base_quant_v_kernel(const __grid_constant
 }
 
 // Rebuild rows [0, Lq) of K and V in the storage type: blockIdx.y = 0 keys (metadata per token group and channel),
-// 1 values (metadata per token and channel group).
+// 1 values (metadata per token and channel group). One thread per 8 channels of a position, four positions per
+// thread and pass so that their loads are in flight together. With a row mask only the (head, position) pairs whose
+// bit is set are rebuilt; everything else of the output is left as it is.
 template <typename T, int BITS>
 __global__ void __launch_bounds__(256) base_dequant_kernel(const __grid_constant__ BaseArgs a) {
   fl_grid_wait();
@@ -135,29 +140,104 @@ __global__ void __launch_bounds__(256) base_dequant_kernel(const __grid_constant
   const bool is_v = blockIdx.y != 0;
   const int per_row = a.d >> 3;
   const int gs = 31 - __clz(a.group);
-  const int64_t total = (int64_t)a.Lq * per_row;
   const uint8_t* codes = is_v ? a.v_codes : a.k_codes;
+  const __half* scale = is_v ? a.v_scale : a.k_scale;
+  const __half* zero = is_v ? a.v_zero : a.k_zero;
   T* out = static_cast<T*>(is_v ? a.v_out : a.k_out);
-  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
-    const int t = (int)(i / per_row), elem = (int)(i - (int64_t)t * per_row) * 8;
-    uint32_t c[8];
-    load_codes8<BITS>(codes + (size_t)t * (a.d * BITS / 8), elem, c);
-    float x[8];
-    if (is_v) {
-      const size_t gi = (size_t)t * (a.d >> gs) + (elem >> gs);
-      const float sc = __half2float(a.v_scale[gi]), zr = __half2float(a.v_zero[gi]);
+  constexpr int U = 4;
+  // the unquantized tail rows, copied as they are (always: they are few)
+  {
+    const T* tail = static_cast<const T*>(is_v ? a.v_tail : a.k_tail);
+    const int n_vec = (a.L - a.Lq) * per_row * (int)(sizeof(T) * 8 / 16);
+    const uint4* src = reinterpret_cast<const uint4*>(tail);
+    uint4* dst = reinterpret_cast<uint4*>(out + (size_t)a.Lq * a.d);
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n_vec; i += gridDim.x * blockDim.x) dst[i] = __ldg(src + i);
+  }
+  // a CTA walks rows blockIdx.x, blockIdx.x + gridDim.x, ...; its threads cover a row in steps of blockDim.x vectors
+  for (int v0 = threadIdx.x; v0 < per_row; v0 += blockDim.x)
+  for (int t0 = blockIdx.x; t0 < a.Lq; t0 += U * gridDim.x) {
+    int t[U], elem[U];
+    bool on[U];
+    uint32_t raw[U][2];
+    uint4 sraw[U], zraw[U];
+    const int head = (v0 * 8) / a.dh;
 #pragma unroll
-      for (int u = 0; u < 8; ++u) x[u] = __fmaf_rn((float)c[u], sc, zr);
-    } else {
-      const size_t mi = (size_t)(t >> gs) * a.d + elem;
-      const uint4 sraw = *reinterpret_cast<const uint4*>(a.k_scale + mi);
-      const uint4 zraw = *reinterpret_cast<const uint4*>(a.k_zero + mi);
-      const __half* sh = reinterpret_cast<const __half*>(&sraw);
-      const __half* zh = reinterpret_cast<const __half*>(&zraw);
-#pragma unroll
-      for (int u = 0; u < 8; ++u) x[u] = __fmaf_rn((float)c[u], __half2float(sh[u]), __half2float(zh[u]));
+    for (int u = 0; u < U; ++u) {
+      t[u] = t0 + u * gridDim.x;
+      elem[u] = v0 * 8;
+      on[u] = t[u] < a.Lq;
+      if (on[u] && a.row_mask != nullptr)
+        on[u] = (__ldg(a.row_mask + (size_t)head * a.mask_words + (t[u] >> 5)) >> (t[u] & 31)) & 1u;
     }
-    store8<T>(out + (size_t)t * a.d + elem, x);
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      if (!on[u]) continue;
+      const uint8_t* row = codes + (size_t)t[u] * (a.d * BITS / 8);
+      if (BITS == 8) {
+        const uint2 r2 = __ldg(reinterpret_cast<const uint2*>(row + elem[u]));
+        raw[u][0] = r2.x; raw[u][1] = r2.y;
+      } else if (BITS == 4) {
+        raw[u][0] = __ldg(reinterpret_cast<const uint32_t*>(row + elem[u] / 2));
+      } else {
+        raw[u][0] = __ldg(reinterpret_cast<const uint16_t*>(row + elem[u] / 4));
+      }
+      if (is_v) {
+        const size_t gi = (size_t)t[u] * (a.d >> gs) + (elem[u] >> gs);
+        sraw[u].x = __half_as_ushort(__ldg(scale + gi));
+        zraw[u].x = __half_as_ushort(__ldg(zero + gi));
+      } else {
+        const size_t mi = (size_t)(t[u] >> gs) * a.d + elem[u];
+        sraw[u] = __ldg(reinterpret_cast<const uint4*>(scale + mi));
+        zraw[u] = __ldg(reinterpret_cast<const uint4*>(zero + mi));
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      if (!on[u]) continue;
+      float x[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        uint32_t c;
+        if (BITS == 8) c = (raw[u][e >> 2] >> (8 * (e & 3))) & 0xFFu;
+        else if (BITS == 4) c = (raw[u][0] >> (4 * e)) & 0xFu;
+        else c = (raw[u][0] >> (2 * e)) & 0x3u;
+        float sc, zr;
+        if (is_v) {
+          sc = __half2float(__ushort_as_half((unsigned short)sraw[u].x));
+          zr = __half2float(__ushort_as_half((unsigned short)zraw[u].x));
+        } else {
+          sc = __half2float(reinterpret_cast<const __half*>(&sraw[u])[e]);
+          zr = __half2float(reinterpret_cast<const __half*>(&zraw[u])[e]);
+        }
+        x[e] = __fmaf_rn((float)c, sc, zr);
+      }
+      store8<T>(out + (size_t)t[u] * a.d + elem[u], x);
+    }
+  }
+}
+
+// Marks the base rows a layer's sparse loops read: for every head the columns of its blocks' lists (attention) and
+// the active positions (the residual chain of the quantizer starts from their base rows). Bits are only ever set.
+__global__ void __launch_bounds__(256) mark_base_rows_kernel(const int32_t* __restrict__ col_idx,
+                                                             const int32_t* __restrict__ col_cnt, int c, int nb, int H,
+                                                             const int32_t* __restrict__ active_idx, int n_active,
+                                                             uint32_t* __restrict__ mask, int mask_words) {
+  fl_grid_wait();
+  fl_grid_release();
+  const int64_t n_col = (int64_t)H * nb * c, total = n_col + (int64_t)H * n_active;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    int h, t;
+    if (i < n_col) {
+      const int64_t list = i / c;
+      if ((int)(i - list * c) >= __ldg(col_cnt + list)) continue;
+      h = (int)(list / nb);
+      t = __ldg(col_idx + i);
+    } else {
+      const int64_t k = i - n_col;
+      h = (int)(k / n_active);
+      t = __ldg(active_idx + (k - (int64_t)h * n_active));
+    }
+    atomicOr(mask + (size_t)h * mask_words + (t >> 5), 1u << (t & 31));
   }
 }
 
@@ -176,7 +256,7 @@ int check_base(const fl_ctx* ctx, const fl_shape* s, const fl_kv_base_q* q) {
     FL_REQUIRE(fl_aligned16(q->k_codes) && fl_aligned16(q->k_scale) && fl_aligned16(q->k_zero) &&
                fl_aligned16(q->v_codes) && fl_aligned16(q->v_scale) && fl_aligned16(q->v_zero));
   }
-  if (Lq < s->L) FL_REQUIRE(q->k_tail != nullptr && q->v_tail != nullptr);
+  if (Lq < s->L) FL_REQUIRE(q->k_tail != nullptr && q->v_tail != nullptr && fl_aligned16(q->k_tail) && fl_aligned16(q->v_tail));
   return FL_OK;
 }
 
@@ -189,6 +269,12 @@ BaseArgs base_args(const fl_shape* s, const fl_kv_base_q* q) {
   a.Lq = s->L > q->tail ? s->L - q->tail : 0;
   a.d = s->n_heads * s->head_dim;
   a.group = q->group;
+  a.dh = s->head_dim;
+  a.L = s->L;
+  a.k_tail = q->k_tail;
+  a.v_tail = q->v_tail;
+  a.mask_words = (s->L + 31) / 32;
+  a.row_mask = nullptr;
   return a;
 }
 
@@ -211,7 +297,7 @@ int launch_quant_base(fl_ctx* ctx, const fl_shape* s, const BaseArgs& a, cudaStr
 
 template <typename T>
 int launch_dequant_base(fl_ctx* ctx, const fl_shape* s, const BaseArgs& a, cudaStream_t st) {
-  int64_t b = ((int64_t)a.Lq * (a.d / 8) + 255) / 256;
+  int64_t b = a.L;     // one CTA per row, up to 16 CTAs per SM and side; each then walks several rows
   const dim3 grid((unsigned)(b > (int64_t)ctx->sm_count * 16 ? (int64_t)ctx->sm_count * 16 : b), 2);
   if (s->bits == 8) FL_CHECK_CUDA(fl_launch(ctx, base_dequant_kernel<T, 8>, grid, dim3(256), 0, st, a));
   else if (s->bits == 4) FL_CHECK_CUDA(fl_launch(ctx, base_dequant_kernel<T, 4>, grid, dim3(256), 0, st, a));
@@ -243,29 +329,18 @@ extern "C" int fl_quant_kv_base(fl_ctx* ctx, const fl_shape* shape, const void* 
                                 : launch_quant_base<__nv_bfloat16>(ctx, shape, a, st);
 }
 
-extern "C" int fl_dequant_kv_base(fl_ctx* ctx, const fl_shape* shape, const fl_kv_base_q* base, void* k_out,
-                                  void* v_out, int32_t* status, void* stream) {
+extern "C" int fl_dequant_kv_base(fl_ctx* ctx, const fl_shape* shape, const fl_kv_base_q* base,
+                                  const uint32_t* row_mask, void* k_out, void* v_out, int32_t* status, void* stream) {
   (void)status;
   int rc = check_base(ctx, shape, base);
   if (rc != FL_OK) return rc;
   FL_REQUIRE(k_out != nullptr && v_out != nullptr && fl_aligned16(k_out) && fl_aligned16(v_out));
   BaseArgs a = base_args(shape, base);
   a.k_out = k_out; a.v_out = v_out;
+  a.row_mask = row_mask;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  const size_t row_bytes = (size_t)a.d * fl_elem_bytes(shape);
-  if (a.Lq > 0) {
-    rc = shape->dtype == FL_F32 ? launch_dequant_base<float>(ctx, shape, a, st)
+  return shape->dtype == FL_F32 ? launch_dequant_base<float>(ctx, shape, a, st)
                                 : launch_dequant_base<__nv_bfloat16>(ctx, shape, a, st);
-    if (rc != FL_OK) return rc;
-  }
-  if (a.Lq < shape->L) {
-    const size_t n = (size_t)(shape->L - a.Lq) * row_bytes;
-    FL_CHECK_CUDA(cudaMemcpyAsync(static_cast<char*>(k_out) + (size_t)a.Lq * row_bytes, base->k_tail, n,
-                                  cudaMemcpyDeviceToDevice, st));
-    FL_CHECK_CUDA(cudaMemcpyAsync(static_cast<char*>(v_out) + (size_t)a.Lq * row_bytes, base->v_tail, n,
-                                  cudaMemcpyDeviceToDevice, st));
-  }
-  return FL_OK;
 }
 
 extern "C" int fl_kv_base_q_bytes(const fl_shape* shape, int32_t group, int32_t tail, int64_t* bytes) {
@@ -279,4 +354,30 @@ extern "C" int fl_kv_base_q_bytes(const fl_shape* shape, int32_t group, int32_t 
   *bytes = 2 * Lq * (d * shape->bits / 8) + 2 * 2 * n_tg * d + 2 * 2 * Lq * (d / group) +
            2 * (shape->L - Lq) * d * fl_elem_bytes(shape);
   return FL_OK;
+}
+
+extern "C" int fl_mark_base_rows(fl_ctx* ctx, const fl_shape* shape, const int32_t* col_idx, const int32_t* col_cnt,
+                                 int32_t c, const int32_t* active_idx, int32_t n_active, uint32_t* row_mask,
+                                 int32_t* status, void* stream) {
+  FL_REQUIRE(ctx != nullptr);
+  int rc = fl_check_shape(shape);
+  if (rc != FL_OK) return rc;
+  FL_REQUIRE(row_mask != nullptr && c >= 1 && n_active >= 0 && n_active <= shape->L);
+  FL_REQUIRE(col_idx != nullptr && col_cnt != nullptr && (n_active == 0 || active_idx != nullptr));
+  const int nb = fl_n_blocks(shape), H = shape->n_heads;
+  {
+    const fl_idx_check ck[2] = {{active_idx, n_active, 0, nullptr, 0, shape->L - 1, 1},
+                                {col_idx, (int64_t)H * nb * c, c, col_cnt, 0, shape->L - 1, 1}};
+    rc = fl_debug_check(ctx, ck, 2, status, stream);
+    if (rc != FL_OK) return rc;
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int mask_words = (shape->L + 31) / 32;
+  FL_CHECK_CUDA(cudaMemsetAsync(row_mask, 0, sizeof(uint32_t) * (size_t)H * mask_words, st));
+  const int64_t total = (int64_t)H * nb * c + (int64_t)H * n_active;
+  int64_t blocks = (total + 255) / 256;
+  if (blocks > (int64_t)ctx->sm_count * 8) blocks = (int64_t)ctx->sm_count * 8;
+  FL_CHECK_CUDA(fl_launch(ctx, mark_base_rows_kernel, dim3((unsigned)blocks), dim3(256), 0, st, col_idx, col_cnt, c, nb, H,
+                          active_idx, n_active, row_mask, mask_words));
+  return fl_launch_status();
 }

@@ -80,6 +80,48 @@ def test_base_codes_metadata_and_rebuilt_rows_bit_exact(env, name):
                                                                     2 if w.dtype == "bf16" else 4)
 
 
+def test_masked_rebuild_touches_only_the_rows_the_sparse_loops_read(env):
+    B, P, ctx = env
+    w = small_bf16(L=1500, H=2, R=2)
+    x = workloads.make_layer_inputs(w, seed=19)
+    k1 = storage_round(x.K[0], w).reshape(w.L, w.d)
+    v1 = storage_round(x.V[0], w).reshape(w.L, w.d)
+    ref = fo.quantize_base(k1, v1, 4, 64, 64, storage_round=fo.round_bf16)
+    sh = P.shape_of(w)
+    q, t, Lq, n_tg = alloc_base(B, w, 4, 64, 64)
+    B.fl_quant_kv_base(ctx, sh, to_dev(k1, w), to_dev(v1, w), q)
+    # column lists with ragged counts and an active list, as a sparse loop would hand them over
+    rng = np.random.default_rng(4)
+    nb, c = (w.L + w.q_block - 1) // w.q_block, 40
+    col_idx = np.full((w.n_heads, nb, c), -1, dtype=np.int32)
+    col_cnt = np.zeros((w.n_heads, nb), dtype=np.int32)
+    sets = {}
+    for h in range(w.n_heads):
+        for b in range(nb):
+            m = int(rng.integers(0, c + 1)) if (h, b) != (0, 0) else 0
+            S = np.sort(rng.choice(min(w.L, (b + 1) * w.q_block), size=m, replace=False))
+            col_idx[h, b, :m], col_cnt[h, b], sets[(h, b)] = S, m, S
+    active = np.sort(rng.choice(w.L, size=97, replace=False)).astype(np.int32)
+    need = fo.base_rows_needed(sets, active, w.n_heads, w.L)
+    words = (w.L + 31) // 32
+    mask = torch.full((w.n_heads, words), -1, dtype=torch.int32, device="cuda:0")      # the call clears it first
+    B.fl_mark_base_rows(ctx, sh, torch.from_numpy(col_idx).cuda(), torch.from_numpy(col_cnt).cuda(), c,
+                        torch.from_numpy(active).cuda(), len(active), mask)
+    torch.cuda.synchronize()
+    bits = mask.cpu().numpy().view(np.uint32)
+    got = ((bits[:, :, None] >> np.arange(32, dtype=np.uint32)) & 1).reshape(w.n_heads, -1)[:, :w.L].astype(bool)
+    assert np.array_equal(got, need)
+    k_out = torch.full((w.L, w.n_heads, w.head_dim), 9.0, dtype=torch.bfloat16, device="cuda:0")
+    v_out = torch.full_like(k_out, 9.0)
+    B.fl_dequant_kv_base(ctx, sh, q, k_out, v_out, row_mask=mask)
+    torch.cuda.synchronize()
+    shp = (w.L, w.n_heads, w.head_dim)
+    want_k = np.where(need.T[:, :, None], ref["khat"].reshape(shp), np.float32(9.0))
+    want_v = np.where(need.T[:, :, None], ref["vhat"].reshape(shp), np.float32(9.0))
+    want_k[Lq:], want_v[Lq:] = ref["khat"].reshape(shp)[Lq:], ref["vhat"].reshape(shp)[Lq:]   # the tail is always copied
+    assert np.array_equal(to_np(k_out), want_k) and np.array_equal(to_np(v_out), want_v)
+
+
 def test_dense_and_sparse_loop_on_the_rebuilt_base(env):
     """The base is packed and rebuilt first, then loop 1 (dense) and loop 2 (sparse) both read the rebuilt rows: the
     attention of every loop sees the cache as it is stored, so the old term recomputed from the previous loop's

@@ -76,3 +76,10 @@ def test_base_bytes_by_hand():
     # the configuration of the paper's setting at scale approaches 4.5 bits per element against 16
     full = 2 * 32768 * 2048 * 2
     assert 3.3 < full / fo.base_q_bytes(32768, 2048, 4, 64, 64) < 3.6
+
+
+def test_rows_needed_by_hand():
+    sets = {(0, 0): np.array([0, 2]), (0, 1): np.array([2, 5]), (1, 0): np.array([], dtype=np.int64), (1, 1): np.array([7])}
+    need = fo.base_rows_needed(sets, [3, 6], H=2, L=8)
+    assert np.flatnonzero(need[0]).tolist() == [0, 2, 3, 5, 6]
+    assert np.flatnonzero(need[1]).tolist() == [3, 6, 7]

@@ -637,6 +637,16 @@ def run_ours(args):
     if rank == 0:
         out["breakdown_ms"] = bench.breakdown()
         out["per_loop"] = bench.per_loop
+        # the memory-bound stages: algorithmic bytes per step, time of the evented pass, achieved bandwidth
+        bd = out["breakdown_ms"]
+        stage_ms = {"select_tokens": bd.get("select_tokens", 0.0), "quant": bd.get("quant", 0.0),
+                    "select_columns": bd.get("select_columns", 0.0),
+                    "gather_scatter": bd.get("gather", 0.0) + bd.get("scatter", 0.0),
+                    "dequant_base": bd.get("dequant_base", 0.0)}
+        out["memory_bound_stages"] = {
+            k: {"bytes_per_step": v, "ms_per_step": stage_ms[k], "achieved_gbs": v / (stage_ms[k] * 1e-3) / 1e9,
+                "frac_of_hbm_peak": v / (stage_ms[k] * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+            for k, v in stage_bytes.items() if stage_ms.get(k, 0.0) > 0.0}
     if not args.no_variants and not args.no_graph:
         # stage (4) as the paper words it: the packed residual streams are read, dequantized and added inside the
         # attention kernel (no materialized rows); same step otherwise

@@ -814,9 +814,36 @@ def run_projection(args, device, rank):
         lib_gather(l); lib_qkv(l)
     def lib_o_both(l):
         lib_o(l); lib_add(l)
+    # the same with the residual codec (Eq. 8) as the epilogue of the K and V columns, against row copy + library GEMM
+    # + fl_quant_kv_residual: loop 2 of a config-3 layer (random base rows, one residual stream, materialized rows)
+    from paper_2609_29812_b200 import pipeline as P, workloads
+    wl = workloads.replace(workloads.config3(L=L, n_layers=1))
+    slot = torch.full((L,), -1, dtype=torch.int32, device=device)
+    slot[idx64] = torch.arange(n, dtype=torch.int32, device=device)
+    sel = P.TokenSelection(idx, slot, None, n)
+    states = []
+    for l in range(NL):
+        st = P.LayerState(ctx, wl, device)
+        st.k_base = torch.randn(L, wl.n_heads, wl.head_dim, device=device, generator=g).to(bf)
+        st.v_base = torch.randn(L, wl.n_heads, wl.head_dim, device=device, generator=g).to(bf)
+        st.alloc_stream(sel)
+        states.append(st)
+    sh = states[0].shape
+    q_out = torch.empty(n, d, device=device, dtype=bf)
+    qkv3 = torch.empty(3, n, d, device=device, dtype=bf)
+    w3 = [w_.view(3, d, d).transpose(1, 2) for w_ in wqkv]
+    fused_qkv_quant = lambda l: B.fl_project_qkv_quant(ctx, sh, 2, hid[l], L, idx, n, wqkv[l], q_out, None,
+                                                       states[l].store, status, stream=stream)
+    lib_qkv3 = lambda l: torch.matmul(rows.unsqueeze(0), w3[l], out=qkv3)
+    lib_quant = lambda l: B.fl_quant_kv_residual(ctx, sh, 2, qkv3[1], qkv3[2], idx, n, states[l].store, stream=stream)
+    def lib_qkv_quant(l):
+        lib_gather(l); lib_qkv3(l); lib_quant(l)
     sampler = ClockSampler(torch.device(device).index or 0)
     sampler.start()
     res = {"fused_qkv": timed(fused_qkv, reps), "fused_o": timed(fused_o, reps),
+           "fused_qkv_with_codec_epilogue": timed(fused_qkv_quant, reps),
+           "library_qkv_then_quant": timed(lib_qkv_quant, reps),
+           "library_batched_qkv_gemm_alone": timed(lib_qkv3, reps), "quant_alone": timed(lib_quant, reps),
            "same_kernel_qkv_on_compact_rows": timed(fused_qkv_compact, reps),
            "library_qkv": timed(lib_qkv_both, reps), "library_o": timed(lib_o_both, reps),
            "library_gather_alone": timed(lib_gather, reps), "library_qkv_gemm_alone": timed(lib_qkv, reps),

@@ -155,6 +155,23 @@ FL_API int fl_project_rows(fl_ctx* ctx, const void* x, int64_t x_rows, const int
                     const void* w, int32_t d_out, void* y, int64_t y_rows, const int32_t* dst_idx,
                     int32_t accumulate, int32_t* status, void* stream);
 
+/* Stacked Q/K/V projection of the active rows with the residual codec as the epilogue of its K and V columns
+ * (Section 4.4: cache update and quantization fused into the producing kernel; Appendix G: Q, K and V in one GEMM).
+ * One launch replaces fl_gather_rows + the projection GEMM + fl_quant_kv_residual:
+ *   [q | k | v] = x[active_idx[t], :] . w_qkv^T          (w_qkv: bf16 [3d, d], rows 0..d-1 -> Q, d..2d-1 -> K, 2d..3d-1 -> V)
+ *   q_out[t, :] = bf16(q);  k, v rounded to bf16 and then coded exactly as fl_quant_kv_residual codes them, against
+ *   the reconstruction of loop_r - 1 (base + earlier streams of `store`), into stream loop_r - 2 of `store`
+ *   (codes, scale, zero, and rows_prev / rows_cur when the stream lends them).
+ * x: bf16 [x_rows, d] (the hidden states); q_out: bf16 [n_active, d]; kv_out: optional bf16 [n_active, 2d] that
+ * receives the new K | V rows as the codec saw them (NULL: they are never written anywhere). The codes are those of the
+ * GEMM's own bf16 outputs: a different GEMM (other accumulation order) may round a value differently and so code it
+ * differently; given kv_out they are bit-exact against the reference codec.
+ * Errors: as fl_quant_kv_residual and fl_project_rows; FL_ERR_UNSUPPORTED unless the storage type is bf16, bits < 16,
+ * group >= 32 and d is a multiple of 256. `status` receives FL_ERR_TIMEOUT if a bounded wait ran out. */
+FL_API int fl_project_qkv_quant(fl_ctx* ctx, const fl_shape* shape, int loop_r, const void* x, int64_t x_rows,
+                         const int32_t* active_idx, int32_t n_active, const void* w_qkv, void* q_out, void* kv_out,
+                         const fl_kv_store* store, int32_t* status, void* stream);
+
 /* Stage 3 -- Eq. 8 with the quantizer of Appendix E (asymmetric, group-wise, min/max).
  * For each active row i = active_idx[t], X in {K, V}, head, group of `group` elements, in binary32:
  *   delta = X^(r)_i - Xhat^(r-1)_i            (Xhat^(r-1) rebuilt from base + streams of loops < r)

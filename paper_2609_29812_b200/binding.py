@@ -74,6 +74,7 @@ def _load() -> C.CDLL:
         "fl_gather_rows": [p, p, p, i32, i64, p, p],
         "fl_scatter_update": [p, p, p, i32, i64, p, p],
         "fl_project_rows": [p, p, i64, p, i32, i32, p, i32, p, i64, p, i32, p, p],
+        "fl_project_qkv_quant": [p, C.POINTER(FlShape), C.c_int, p, i64, p, i32, p, p, p, C.POINTER(FlKvStore), p, p],
         "fl_quant_kv_residual": [p, C.POINTER(FlShape), C.c_int, p, p, p, i32, C.POINTER(FlKvStore), p, p],
         "fl_dense_loop_attention": [p, C.POINTER(FlShape), p, p, p, p, p, p, p, p],
         "fl_select_columns": [p, C.POINTER(FlShape), p, p, p, i32, i32, p, p, p, p],
@@ -226,6 +227,14 @@ def fl_project_rows(ctx, x, x_rows, src_idx, n, d_in, w, d_out, y, y_rows, dst_i
     rc = lib.fl_project_rows(_h(ctx), _ptr(x), int(x_rows), _ptr(src_idx), int(n), int(d_in), _ptr(w), int(d_out),
                              _ptr(y), int(y_rows), _ptr(dst_idx), int(accumulate), _ptr(status), _stream(stream))
     return _check("fl_project_rows", rc, check)
+
+
+def fl_project_qkv_quant(ctx, shape, loop_r, x, x_rows, active_idx, n_active, w_qkv, q_out, kv_out, store, status=None,
+                         stream=None, check=True) -> int:
+    rc = lib.fl_project_qkv_quant(_h(ctx), C.byref(shape), int(loop_r), _ptr(x), int(x_rows), _ptr(active_idx),
+                                  int(n_active), _ptr(w_qkv), _ptr(q_out), _ptr(kv_out),
+                                  C.byref(store) if store is not None else None, _ptr(status), _stream(stream))
+    return _check("fl_project_qkv_quant", rc, check)
 
 
 def make_base_q(k_codes, k_scale, k_zero, v_codes, v_scale, v_zero, k_tail, v_tail, group, tail) -> FlKvBaseQ:

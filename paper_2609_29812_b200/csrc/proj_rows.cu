@@ -44,10 +44,125 @@ struct ProjArgs {
   const int32_t* dst_idx;   // [n] rows of Y, or null
   __nv_bfloat16* y;
   int n, d_in, d_out;
+  int y_stride, y_cols;     // row stride of y and the number of output columns that go to it
   int m_tiles, n_tiles;
   int accumulate;
   int* status;
+  // Fused residual codec (Eq. 8) of the K and V columns of a stacked Q/K/V projection: output columns
+  // [d_model, 2 d_model) are the new K rows, [2 d_model, 3 d_model) the new V rows of the active positions src_idx.
+  DevSide k, v;             // base + earlier streams (read), in loop order
+  uint8_t* k_codes; __half* k_scale; __half* k_zero;   // the stream being written
+  uint8_t* v_codes; __half* v_scale; __half* v_zero;
+  __nv_bfloat16* k_rows_prev; __nv_bfloat16* k_rows_cur;   // optional [n, d_model]: Xhat^(r-1) / Xhat^(r) of the active rows
+  __nv_bfloat16* v_rows_prev; __nv_bfloat16* v_rows_cur;
+  __nv_bfloat16* kv_out;    // optional [n, 2 d_model]: the new K | V rows themselves (bf16), as the codec saw them
+  int d_model, n_prev, group;
 };
+
+// Xhat^(r-1) of 8 consecutive elements of position pos: base plus the earlier streams in loop order (binary32)
+template <int BITS>
+__device__ __forceinline__ void chain8(const DevSide& side, int n_prev, int pos, int elem, int d, int group,
+                                       float (&xh)[8]) {
+  load8<__nv_bfloat16>(static_cast<const __nv_bfloat16*>(side.base) + (size_t)pos * d + elem, xh);
+  for (int s = 0; s < n_prev; ++s) apply_stream8<__nv_bfloat16, BITS>(side.s[s], pos, elem, d, group, xh);
+}
+
+// The codec on one row of a 256-column K or V tile, by the thread that owns the row's lane of tensor memory: every
+// group of `group` columns lies inside the thread's own 256 accumulator values, so minimum and maximum need no
+// exchange. Two passes over a group (range, then codes); the accumulator is read from tensor memory twice and the
+// previous reconstruction rebuilt twice (the second time from L1/L2). Arithmetic as in the stand-alone quantizer:
+// binary32, offset rounded down and scale rounded up to fp16, codes by round-half-even of the true quotient.
+template <int BITS>
+__device__ __forceinline__ void codec_row(const ProjArgs& a, uint32_t tmem_row, bool row_ok, int t, int pos, bool is_v,
+                                          int elem0, uint64_t* acc_free, int lane) {
+  const DevSide& side = is_v ? a.v : a.k;
+  uint8_t* codes = is_v ? a.v_codes : a.k_codes;
+  __half* scale = is_v ? a.v_scale : a.k_scale;
+  __half* zero = is_v ? a.v_zero : a.k_zero;
+  __nv_bfloat16* rows_prev = is_v ? a.v_rows_prev : a.k_rows_prev;
+  __nv_bfloat16* rows_cur = is_v ? a.v_rows_cur : a.k_rows_cur;
+  const int d = a.d_model, g = a.group, pieces = g >> 5, n_groups = 256 / g;
+  const float qmax = (float)((1 << BITS) - 1);
+  for (int gi = 0; gi < n_groups; ++gi) {
+    const int e_g = elem0 + gi * g;
+    float mn = INFINITY, mx = -INFINITY;
+#pragma unroll 1
+    for (int pc = 0; pc < pieces; ++pc) {
+      uint32_t r[32];
+      tc::tmem_ld32(tmem_row + gi * g + pc * 32, r);
+      tc::tmem_wait_ld();
+      if (row_ok) {
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {
+          float xh[8];
+          chain8<BITS>(side, a.n_prev, pos, e_g + pc * 32 + v * 8, d, g, xh);
+#pragma unroll
+          for (int u = 0; u < 8; ++u) {
+            const float xn = __bfloat162float(__float2bfloat16_rn(__uint_as_float(r[v * 8 + u])));
+            const float dl = __fsub_rn(xn, xh[u]);
+            mn = fminf(mn, dl);
+            mx = fmaxf(mx, dl);
+          }
+        }
+      }
+    }
+    const __half zh = __float2half_rd(mn);
+    const float zf = __half2float(zh);
+    const float range = __fsub_rn(mx, zf);
+    const __half sh = range == 0.f ? __float2half_rn(0.f) : __float2half_ru(__fdiv_rn(range, qmax));
+    const float sf = __half2float(sh);
+#pragma unroll 1
+    for (int pc = 0; pc < pieces; ++pc) {
+      uint32_t r[32];
+      tc::tmem_ld32(tmem_row + gi * g + pc * 32, r);
+      tc::tmem_wait_ld();
+      if (gi == n_groups - 1 && pc == pieces - 1) {
+        // last read of the accumulator: the issuer may start the tile after next
+        tc::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) tc::mbar_arrive(acc_free);
+      }
+      if (!row_ok) continue;
+      const int e_p = e_g + pc * 32;
+      uint32_t packed[8];     // 32 codes: BITS / 8 words of 32 bits each hold 32 / BITS ... filled below
+#pragma unroll
+      for (int wd = 0; wd < 8; ++wd) packed[wd] = 0u;
+#pragma unroll
+      for (int v = 0; v < 4; ++v) {
+        float xh[8], xn[8], xc[8];
+        chain8<BITS>(side, a.n_prev, pos, e_p + v * 8, d, g, xh);
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          xn[u] = __bfloat162float(__float2bfloat16_rn(__uint_as_float(r[v * 8 + u])));
+          const float dl = __fsub_rn(xn[u], xh[u]);
+          const float q = sf == 0.f ? 0.f : rintf(__fdiv_rn(__fsub_rn(dl, zf), sf));
+          xc[u] = __fadd_rn(xh[u], __fmaf_rn(q, sf, zf));
+          const int idx = v * 8 + u;                       // code index inside the piece
+          packed[(idx * BITS) >> 5] |= (uint32_t)q << ((idx * BITS) & 31);
+        }
+        if (rows_prev != nullptr) store8<__nv_bfloat16>(rows_prev + (size_t)t * d + e_p + v * 8, xh);
+        if (rows_cur != nullptr) store8<__nv_bfloat16>(rows_cur + (size_t)t * d + e_p + v * 8, xc);
+        if (a.kv_out != nullptr)
+          store8<__nv_bfloat16>(a.kv_out + (size_t)t * (2 * d) + (is_v ? d : 0) + e_p + v * 8, xn);
+      }
+      uint8_t* crow = codes + (size_t)t * (d * BITS / 8) + e_p * BITS / 8;
+      if (BITS == 8) {
+        *reinterpret_cast<uint4*>(crow) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+        *reinterpret_cast<uint4*>(crow + 16) = make_uint4(packed[4], packed[5], packed[6], packed[7]);
+      } else if (BITS == 4) {
+        *reinterpret_cast<uint4*>(crow) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+      } else {
+        *reinterpret_cast<uint2*>(crow) = make_uint2(packed[0], packed[1]);
+      }
+    }
+    if (row_ok) {
+      const int gs = 31 - __clz(g);
+      const size_t mi = (size_t)t * (d >> gs) + (e_g >> gs);
+      scale[mi] = sh;
+      zero[mi] = zh;
+    }
+  }
+}
 
 __device__ __forceinline__ void mma_ss_acc(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t hi, uint32_t idesc,
                                            uint32_t accum) {
@@ -60,7 +175,7 @@ __device__ __forceinline__ void mma_ss_acc(uint32_t d_tmem, uint32_t a_lo, uint3
       : "memory");
 }
 
-template <bool GATHER, int kBN>
+template <bool GATHER, int kBN, int CODEC>   // CODEC: 0, or the bit width of the fused residual codec (wide tiles only)
 __global__ void __launch_bounds__(kThreads, 1) proj_rows_kernel(const __grid_constant__ ProjArgs a) {
   constexpr int kBBytes = kBN * kBK * 2;
   extern __shared__ uint8_t smem_raw[];
@@ -170,8 +285,18 @@ __global__ void __launch_bounds__(kThreads, 1) proj_rows_kernel(const __grid_con
       const int buf = i & 1;
       const int m = (w / a.n_tiles) * kBM + warp * 32 + lane, n0 = (w % a.n_tiles) * kBN;
       const bool row_ok = m < a.n;
+      if (CODEC != 0 && n0 >= a.d_model) {
+        // a K or V tile of the stacked projection: the residual codec instead of a plain store
+        const bool is_v = n0 >= 2 * a.d_model;
+        const int pos = row_ok ? __ldg(a.src_idx + m) : 0;
+        if (!warp_wait(&ctl.acc_full[buf], (i >> 1) & 1, abort_flag)) break;
+        tc::tc_fence_after();
+        codec_row<CODEC == 0 ? 4 : CODEC>(a, tmem + lane_base + buf * kBN, row_ok, m, pos, is_v,
+                                          n0 - (is_v ? 2 : 1) * a.d_model, &ctl.acc_free[buf], lane);
+        continue;
+      }
       const int64_t dst_row = row_ok ? (a.dst_idx != nullptr ? (int64_t)__ldg(a.dst_idx + m) : (int64_t)m) : 0;
-      __nv_bfloat16* y_row = a.y + dst_row * a.d_out + n0;
+      __nv_bfloat16* y_row = a.y + dst_row * a.y_stride + n0;
       // the rows this tile adds into are read one piece ahead of the accumulator (the first piece before the
       // accumulator is even complete): nothing else writes them during the launch
       const bool rmw = a.accumulate != 0 && row_ok;
@@ -179,7 +304,7 @@ __global__ void __launch_bounds__(kThreads, 1) proj_rows_kernel(const __grid_con
 #pragma unroll
       for (int v = 0; v < 4; ++v) {
         old_cur[v] = make_uint4(0u, 0u, 0u, 0u);
-        if (rmw && n0 + v * 8 < a.d_out) old_cur[v] = *reinterpret_cast<const uint4*>(y_row + v * 8);
+        if (rmw && n0 + v * 8 < a.y_cols) old_cur[v] = *reinterpret_cast<const uint4*>(y_row + v * 8);
       }
       if (!warp_wait(&ctl.acc_full[buf], (i >> 1) & 1, abort_flag)) break;
       tc::tc_fence_after();
@@ -188,7 +313,7 @@ __global__ void __launch_bounds__(kThreads, 1) proj_rows_kernel(const __grid_con
 #pragma unroll
         for (int v = 0; v < 4; ++v) {
           old_nxt[v] = make_uint4(0u, 0u, 0u, 0u);
-          if (rmw && p + 1 < kBN / 32 && n0 + (p + 1) * 32 + v * 8 < a.d_out)
+          if (rmw && p + 1 < kBN / 32 && n0 + (p + 1) * 32 + v * 8 < a.y_cols)
             old_nxt[v] = *reinterpret_cast<const uint4*>(y_row + (p + 1) * 32 + v * 8);
         }
         uint32_t r[32];
@@ -203,7 +328,7 @@ __global__ void __launch_bounds__(kThreads, 1) proj_rows_kernel(const __grid_con
         if (row_ok) {
 #pragma unroll
           for (int v = 0; v < 4; ++v) {
-            if (n0 + p * 32 + v * 8 < a.d_out) {
+            if (n0 + p * 32 + v * 8 < a.y_cols) {
               float x[8], old[8];
               fl_tc::unpack8(old_cur[v], old);      // zeros unless the call accumulates
 #pragma unroll
@@ -256,7 +381,7 @@ extern "C" int fl_project_rows(fl_ctx* ctx, const void* x, int64_t x_rows, const
     const int rc = fl_debug_check(ctx, ck, 2, status, stream);
     if (rc != FL_OK) return rc;
   }
-  ProjArgs a;
+  ProjArgs a = {};
   const bool gather = src_idx != nullptr;
   a.m_tiles = (n + kBM - 1) / kBM;
   // Tile width: 256 columns keep the tensor pipe busiest per byte loaded; 128 columns when that leaves the last of the
@@ -274,6 +399,9 @@ extern "C" int fl_project_rows(fl_ctx* ctx, const void* x, int64_t x_rows, const
   a.n = n;
   a.d_in = d_in;
   a.d_out = d_out;
+  a.y_stride = d_out;
+  a.y_cols = d_out;
+  a.d_model = 0;
   a.n_tiles = (d_out + bn - 1) / bn;
   a.accumulate = accumulate;
   a.status = status;
@@ -282,7 +410,7 @@ extern "C" int fl_project_rows(fl_ctx* ctx, const void* x, int64_t x_rows, const
   cudaStream_t st = static_cast<cudaStream_t>(stream);
 #define FL_PROJ(G, BN)                                                                                              \
   do {                                                                                                              \
-    auto kern = proj_rows_kernel<G, BN>;                                                                            \
+    auto kern = proj_rows_kernel<G, BN, 0>;                                                                          \
     FL_CHECK_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kProjSmem));         \
     FL_CHECK_CUDA(fl_launch(ctx, kern, dim3(grid), dim3(kThreads), kProjSmem, st, a));                              \
   } while (0)
@@ -292,5 +420,82 @@ extern "C" int fl_project_rows(fl_ctx* ctx, const void* x, int64_t x_rows, const
     if (bn == 256) FL_PROJ(false, 256); else FL_PROJ(false, 128);
   }
 #undef FL_PROJ
+  return fl_launch_status();
+}
+
+extern "C" int fl_project_qkv_quant(fl_ctx* ctx, const fl_shape* shape, int loop_r, const void* x, int64_t x_rows,
+                                    const int32_t* active_idx, int32_t n_active, const void* w_qkv, void* q_out,
+                                    void* kv_out, const fl_kv_store* store, int32_t* status, void* stream) {
+  FL_REQUIRE(ctx != nullptr);
+  int rc = fl_check_shape(shape);
+  if (rc != FL_OK) return rc;
+  FL_REQUIRE(loop_r >= 2 && loop_r <= FL_MAX_LOOPS + 1);
+  FL_REQUIRE(n_active >= 0 && n_active <= shape->L && x_rows > 0 && x_rows <= INT32_MAX);
+  rc = fl_check_store(shape, store, loop_r - 1);
+  if (rc != FL_OK) return rc;
+  const fl_kv_stream& ks = store->k_res[loop_r - 2];
+  const fl_kv_stream& vs = store->v_res[loop_r - 2];
+  FL_REQUIRE(ks.n_rows == n_active && vs.n_rows == n_active);
+  const int d = shape->n_heads * shape->head_dim;
+  // bf16 storage, a real codec, groups that tile a 256-column output tile, Q / K / V boundaries on tile boundaries
+  if (shape->dtype != FL_BF16 || shape->bits == 16 || shape->group < 32 || d % 256 != 0) return FL_ERR_UNSUPPORTED;
+  if (n_active == 0) return FL_OK;
+  FL_REQUIRE(x != nullptr && w_qkv != nullptr && q_out != nullptr && active_idx != nullptr);
+  FL_REQUIRE(fl_aligned16(x) && fl_aligned16(w_qkv) && fl_aligned16(q_out) && fl_aligned16(kv_out));
+  FL_REQUIRE(x != q_out && w_qkv != q_out && kv_out != q_out);
+  if ((size_t)ctx->max_smem_optin < kProjSmem || ctx->encode_tiled == nullptr || ctx->tmaps == nullptr)
+    return FL_ERR_UNSUPPORTED;
+  {
+    fl_idx_check ck[1 + 2 * FL_MAX_LOOPS];
+    int nck = 0;
+    ck[nck++] = {active_idx, n_active, 0, nullptr, 0, (int32_t)(x_rows < shape->L ? x_rows : shape->L) - 1, 1};
+    for (int i = 0; i < loop_r - 2; ++i) {
+      ck[nck++] = {store->k_res[i].slot_of_pos, shape->L, 0, nullptr, -1, store->k_res[i].n_rows - 1, 0};
+      ck[nck++] = {store->v_res[i].slot_of_pos, shape->L, 0, nullptr, -1, store->v_res[i].n_rows - 1, 0};
+    }
+    rc = fl_debug_check(ctx, ck, nck, status, stream);
+    if (rc != FL_OK) return rc;
+  }
+  ProjArgs a = {};
+  if (!fl_tile_tmap(ctx, x, x_rows, d, 1, &a.x_map) || !fl_tile_tmap(ctx, w_qkv, 3 * (int64_t)d, d, 256, &a.w_map))
+    return FL_ERR_CUDA;
+  a.src_idx = active_idx;
+  a.dst_idx = nullptr;
+  a.y = static_cast<__nv_bfloat16*>(q_out);
+  a.n = n_active;
+  a.d_in = d;
+  a.d_out = 3 * d;
+  a.y_stride = d;
+  a.y_cols = d;
+  a.m_tiles = (n_active + kBM - 1) / kBM;
+  a.n_tiles = 3 * d / 256;
+  a.accumulate = 0;
+  a.status = status;
+  fl_dev_side(store, true, &a.k);
+  fl_dev_side(store, false, &a.v);
+  a.k_codes = static_cast<uint8_t*>(ks.codes); a.k_scale = reinterpret_cast<__half*>(ks.scale);
+  a.k_zero = reinterpret_cast<__half*>(ks.zero);
+  a.v_codes = static_cast<uint8_t*>(vs.codes); a.v_scale = reinterpret_cast<__half*>(vs.scale);
+  a.v_zero = reinterpret_cast<__half*>(vs.zero);
+  const bool rows = ks.rows_prev != nullptr && vs.rows_prev != nullptr;
+  a.k_rows_prev = rows ? static_cast<__nv_bfloat16*>(ks.rows_prev) : nullptr;
+  a.k_rows_cur = rows ? static_cast<__nv_bfloat16*>(ks.rows_cur) : nullptr;
+  a.v_rows_prev = rows ? static_cast<__nv_bfloat16*>(vs.rows_prev) : nullptr;
+  a.v_rows_cur = rows ? static_cast<__nv_bfloat16*>(vs.rows_cur) : nullptr;
+  a.kv_out = static_cast<__nv_bfloat16*>(kv_out);
+  a.d_model = d;
+  a.n_prev = loop_r - 2;
+  a.group = shape->group;
+  const int64_t n_work = (int64_t)a.m_tiles * a.n_tiles;
+  const int grid = (int)(n_work < ctx->sm_count ? n_work : ctx->sm_count);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+#define FL_PROJQ(BITS)                                                                                              \
+  do {                                                                                                              \
+    auto kern = proj_rows_kernel<true, 256, BITS>;                                                                  \
+    FL_CHECK_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kProjSmem));         \
+    FL_CHECK_CUDA(fl_launch(ctx, kern, dim3(grid), dim3(kThreads), kProjSmem, st, a));                              \
+  } while (0)
+  if (shape->bits == 8) FL_PROJQ(8); else if (shape->bits == 4) FL_PROJQ(4); else FL_PROJQ(2);
+#undef FL_PROJQ
   return fl_launch_status();
 }

@@ -83,6 +83,16 @@ def test_argument_validation_happens_before_any_launch(B):
     assert pr(din=100) == UNS and pr(dout=100) == UNS
     assert pr(n=0) == B.FL_OK
     assert pr() == UNS                                                   # the stand-in context has no tensor path
+    st = fake_store(B)
+    pq = lambda **kw: B.fl_project_qkv_quant(ctx, kw.get("sh", sh), kw.get("r", 2), kw.get("x", P), 1024, P,
+                                             kw.get("n", 16), P + 0x100000, kw.get("q", P + 0x200000), None,
+                                             kw.get("st", st), **call)
+    assert pq(r=1) == INV and pq(r=3) == INV and pq(n=17) == INV and pq(st=None) == INV and pq(x=None) == INV
+    assert pq(q=None) == INV and pq(x=P + 4) == INV
+    assert pq(sh=good_shape(B, dtype=B.FL_F32)) == UNS and pq(sh=good_shape(B, bits=16)) == UNS
+    assert pq(sh=good_shape(B, n_heads=1)) == UNS                                               # d = 128
+    assert pq(n=0, st=fake_store(B, n_rows=0)) == B.FL_OK
+    assert pq() == UNS                                                   # the stand-in context has no tensor path
     # quantizer
     st = fake_store(B)
     assert B.fl_quant_kv_residual(ctx, sh, 1, P, P, P, 16, st, **call) == INV                  # loop_r < 2

@@ -106,3 +106,80 @@ def test_project_rows_benchmark_shape_sampled(env):
     check(B, ctx, x, w, y, src, None, n, 0, rows=rows)
     x, w, y, _, dst = make(11, n, L, n, d, d, False, True)
     check(B, ctx, x, w, y, None, dst, n, 1, rows=rows)
+
+
+# ---- the stacked Q/K/V projection with the residual codec as its epilogue ---------------------------------------
+from paper_2609_29812_b200 import workloads            # noqa: E402
+from helpers import to_dev, to_np                       # noqa: E402
+from test_gpu_parity import small_bf16                  # noqa: E402
+
+
+@pytest.mark.parametrize("bits,group,H,n_loops", [(4, 128, 2, 3), (8, 64, 2, 2), (2, 32, 4, 2)])
+def test_projection_with_codec_epilogue(env, bits, group, H, n_loops):
+    """Loops 2..n_loops of one small layer through fl_project_qkv_quant.  Q and the new K | V rows against the oracle's
+    fp64 projection; codes, scales, offsets and the materialized rows bit for bit against the oracle's residual codec
+    applied to the kernel's own bf16 K | V rows (the reading: the codes are those of the GEMM's own outputs); and every
+    output bit for bit against the unfused calls (fl_project_rows, then fl_quant_kv_residual)."""
+    from paper_2609_29812_b200 import pipeline as P
+    B, ctx = env
+    w = small_bf16(L=700, H=H, R=n_loops, bits=bits, group=group)
+    L, d = w.L, w.d
+    rng = np.random.default_rng(31)
+    hid = [round_to_bf16(rng.standard_normal((L, d)).astype(np.float32)) for _ in range(n_loops)]
+    wqkv = round_to_bf16((rng.standard_normal((3 * d, d)) / np.sqrt(d)).astype(np.float32))
+    k1 = round_to_bf16(rng.standard_normal((L, d)).astype(np.float32))
+    v1 = round_to_bf16(rng.standard_normal((L, d)).astype(np.float32))
+    shp = (L, w.n_heads, w.head_dim)
+    st, st_ref = P.LayerState(ctx, w), P.LayerState(ctx, w)
+    for s_ in (st, st_ref):
+        s_.k_base, s_.v_base = to_dev(k1.reshape(shp), w), to_dev(v1.reshape(shp), w)
+    wd = dev(wqkv, torch.bfloat16)
+    khat, vhat = k1.reshape(shp).copy(), v1.reshape(shp).copy()
+    act = np.arange(L)
+    for r in range(2, n_loops + 1):
+        act = np.sort(rng.choice(act, size=max(40, len(act) // 3), replace=False))     # nested, ragged against 128
+        n = len(act)
+        sel = P.TokenSelection(torch.from_numpy(act.astype(np.int32)).cuda(),
+                               torch.from_numpy(fo.slot_map(act, L)).cuda(), None, n)
+        hd = dev(hid[r - 1], torch.bfloat16)
+        st.alloc_stream(sel)
+        q_out = torch.full((n, d), 5.0, dtype=torch.bfloat16, device="cuda:0")
+        kv_out = torch.full((n, 2 * d), 5.0, dtype=torch.bfloat16, device="cuda:0")
+        status = torch.zeros(1, dtype=torch.int32, device="cuda:0")
+        B.fl_project_qkv_quant(ctx, st.shape, r, hd, L, sel.active_idx, n, wd, q_out, kv_out, st.store, status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        rows_prev = [to_np(st.k_streams[-1]["rows_prev"]).copy(), to_np(st.v_streams[-1]["rows_prev"]).copy()]
+        rows_cur = [to_np(st.k_streams[-1]["rows_cur"]).copy(), to_np(st.v_streams[-1]["rows_cur"]).copy()]
+        # (1) the projection itself
+        ref = fo.project_rows(hid[r - 1], act, wqkv, np.zeros((n, 3 * d)), None, False)
+        mag = np.abs(hid[r - 1][act].astype(np.float64)) @ np.abs(wqkv.astype(np.float64)).T
+        got = np.concatenate([to_np(q_out), to_np(kv_out)], axis=1).astype(np.float64)
+        assert np.max(np.abs(got - ref) / (2.0 ** -8 * np.abs(ref) + d * 2.0 ** -23 * mag + 1e-30)) <= 1.0
+        # (2) the codec, on the kernel's own K | V rows
+        kv = to_np(kv_out)
+        for side, (streams, hat, new) in enumerate(((st.k_streams, khat, kv[:, :d]), (st.v_streams, vhat, kv[:, d:]))):
+            hat_new, pay = fo.residual_update(new.reshape(n, w.n_heads, w.head_dim), hat, act, bits, group)
+            got_s = streams[-1]
+            assert np.array_equal(got_s["codes"].cpu().numpy().reshape(n, -1), pay["packed"].reshape(n, -1)), (r, side)
+            assert np.array_equal(got_s["scale"].cpu().numpy().view(np.uint16).reshape(-1), pay["scale"].view(np.uint16).reshape(-1))
+            assert np.array_equal(got_s["zero"].cpu().numpy().view(np.uint16).reshape(-1), pay["zero"].view(np.uint16).reshape(-1))
+            assert np.array_equal(rows_prev[side].reshape(n, -1), fo.round_bf16(hat[act]).reshape(n, -1))
+            assert np.array_equal(rows_cur[side].reshape(n, -1), fo.round_bf16(hat_new[act]).reshape(n, -1))
+            if side == 0:
+                khat = hat_new
+            else:
+                vhat = hat_new
+        # (3) the unfused calls on a second store
+        st_ref.alloc_stream(sel)
+        qkv = torch.empty(n, 3 * d, dtype=torch.bfloat16, device="cuda:0")
+        B.fl_project_rows(ctx, hd, L, sel.active_idx, n, d, wd, 3 * d, qkv, n, None, 0, status)
+        k_new, v_new = qkv[:, d:2 * d].contiguous(), qkv[:, 2 * d:].contiguous()
+        B.fl_quant_kv_residual(ctx, st_ref.shape, r, k_new, v_new, sel.active_idx, n, st_ref.store)
+        torch.cuda.synchronize()
+        assert torch.equal(qkv[:, :d], q_out) and torch.equal(qkv[:, d:], kv_out)
+        for a_, b_ in ((st.k_streams[-1], st_ref.k_streams[-1]), (st.v_streams[-1], st_ref.v_streams[-1])):
+            for key in ("codes", "scale", "zero"):
+                assert torch.equal(a_[key], b_[key]), (r, key)
+        assert np.array_equal(to_np(st_ref.k_streams[-1]["rows_cur"]), rows_cur[0])
+        assert np.array_equal(to_np(st_ref.v_streams[-1]["rows_prev"]), rows_prev[1])

@@ -235,7 +235,8 @@ class Bench:
                 for r in range(2, self.R + 1):
                     sel = self.sels[r - 2]
                     st.rows[r] = gen.rows(r, sel.active_idx)
-                    st.alloc_stream(sel)
+                    # loops that reuse the carried old term read only the rows after the loop's residual
+                    st.alloc_stream(sel, rows="cur" if (self.economy and r > 2) else True)
                 # the same store without the transient rows: the attention kernel then rebuilds every
                 # residual-carrying column itself (dequantize-and-add inside the kernel)
                 strip = lambda streams: [{k: v for k, v in s_.items() if not k.startswith("rows_")} for s_ in streams]

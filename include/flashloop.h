@@ -81,12 +81,15 @@ typedef struct {
  *                    value = code * scale + zero (one binary32 rounding).
  *   bits == 16     : codes [n_rows, H, dh] in storage type holds the loop's rows themselves;
  *                    scale and zero are ignored (may be NULL).
- * rows_prev / rows_cur (optional; both NULL or both set, for the K and the V stream of a loop alike; bf16
- * storage only, ignored otherwise): [n_rows, H, dh] storage type, 16-byte aligned. A transient workspace, not
+ * rows_prev / rows_cur (optional, for the K and the V stream of a loop alike; rows_cur may be set without
+ * rows_prev, not the reverse; bf16 storage only, ignored otherwise): [n_rows, H, dh] storage type, 16-byte aligned. A transient workspace, not
  * part of the cache: fl_quant_kv_residual of loop r, which has both values in registers, leaves there the
  * reconstructed rows of the stream's tokens before and after the loop's residual, Xhat^(r-1) and Xhat^(r)
  * (Eq. 4 / Eq. 8 chain in binary32, rounded once to the storage type), and fl_loop_attention of the same loop
  * gathers the selected columns that are active in loop r from them instead of dequantizing those columns again.
+ * A call that reuses the carried old term (fl_attn_carry.reuse) reads rows_cur only, so a loop that is known to
+ * reuse may lend rows_cur alone and save the quantizer the other write; a recomputing call that finds rows_cur
+ * alone rebuilds the columns itself, as if neither were there.
  * The buffers may be reused for the next loop or layer once that attention call has been issued on the stream.
  * This is a choice of this implementation; the paper reconstructs inside its attention kernel. */
 typedef struct {

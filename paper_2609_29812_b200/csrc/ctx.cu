@@ -93,6 +93,8 @@ extern "C" int fl_create(fl_ctx** out, int device) {
   c->fused_attn = (fused != nullptr && fused[0] == '1') ? 1 : 0;
   const char* two_pass = std::getenv("FL_TWO_PASS");
   c->two_pass = (two_pass != nullptr && two_pass[0] == '1') ? 1 : 0;
+  const char* qn = std::getenv("FL_QUANT_NARROW");
+  c->quant_narrow = (qn != nullptr && qn[0] == '1') ? 1 : 0;
   c->dbg_flag = nullptr;
   c->encode_tiled = nullptr;
   {
@@ -154,7 +156,7 @@ int fl_check_store(const fl_shape* s, const fl_kv_store* st, int n_streams_neede
       const fl_kv_stream& r = side == 0 ? st->k_res[i] : st->v_res[i];
       if (r.n_rows < 0 || r.n_rows > s->L) return FL_ERR_INVALID_ARG;
       if (r.slot_of_pos == nullptr) return FL_ERR_INVALID_ARG;
-      if ((r.rows_prev == nullptr) != (r.rows_cur == nullptr)) return FL_ERR_INVALID_ARG;
+      if (r.rows_prev != nullptr && r.rows_cur == nullptr) return FL_ERR_INVALID_ARG;   // rows_cur alone is fine
       if (!fl_aligned16(r.rows_prev) || !fl_aligned16(r.rows_cur)) return FL_ERR_INVALID_ARG;
       if (r.n_rows > 0) {
         if (r.codes == nullptr || !fl_aligned16(r.codes)) return FL_ERR_INVALID_ARG;
@@ -166,6 +168,7 @@ int fl_check_store(const fl_shape* s, const fl_kv_store* st, int n_streams_neede
     }
     if (st->k_res[i].n_rows != st->v_res[i].n_rows) return FL_ERR_INVALID_ARG;
     if ((st->k_res[i].rows_prev == nullptr) != (st->v_res[i].rows_prev == nullptr)) return FL_ERR_INVALID_ARG;
+    if ((st->k_res[i].rows_cur == nullptr) != (st->v_res[i].rows_cur == nullptr)) return FL_ERR_INVALID_ARG;
   }
   return FL_OK;
 }

@@ -15,6 +15,7 @@ struct fl_ctx {
   int force_simt;  // environment FL_FORCE_SIMT=1 at fl_create: keep attention on the binary32 SIMT kernels
   int fused_attn;  // environment FL_FUSED_ATTN=1 at fl_create: calls with a carried old term keep the fused kernel
   int two_pass;    // environment FL_TWO_PASS=1 at fl_create: recomputing calls with carried buffers run as two launches
+  int quant_narrow;  // environment FL_QUANT_NARROW=1 at fl_create: the quantizer keeps 8 elements per thread
   void* encode_tiled;       // cuTensorMapEncodeTiled, resolved through cudaGetDriverEntryPoint (may be null)
   struct fl_tmap_cache* tmaps;  // tensor maps, keyed by (base pointer, rows, row elements, box rows)
   int pdl;                  // launch the hot-path kernels with programmatic stream serialization (FL_NO_PDL=1: off)

@@ -657,15 +657,16 @@ int launch_mode(fl_ctx* ctx, int bits, dim3 grid, const StArgs& a, cudaStream_t 
 
 }  // namespace
 
-// Whether the single-term kernels can take the call: the loop's materialized rows must be there (all four buffers).
+// Whether the single-term kernels can take the call: the loop's materialized rows must be there (the rows after the
+// loop's residual for the new-term pass; those before it as well when the old-term pass runs).
 bool fl_loop_attn_stream_covers(const fl_ctx* ctx, const fl_shape* s, int loop_r, int n_active,
-                                const fl_kv_store* store, int c) {
+                                const fl_kv_store* store, int c, bool old_pass) {
   if (s->dtype != FL_BF16 || s->head_dim != kDH || c > kMaxCols) return false;
   if ((size_t)ctx->max_smem_optin < kStSmemBytes || ctx->encode_tiled == nullptr || ctx->tmaps == nullptr) return false;
   const fl_kv_stream& ks = store->k_res[loop_r - 2];
   const fl_kv_stream& vs = store->v_res[loop_r - 2];
-  return ks.rows_prev != nullptr && ks.rows_cur != nullptr && vs.rows_prev != nullptr && vs.rows_cur != nullptr &&
-         ks.n_rows == n_active && n_active > 0;
+  if (old_pass && (ks.rows_prev == nullptr || vs.rows_prev == nullptr)) return false;
+  return ks.rows_cur != nullptr && vs.rows_cur != nullptr && ks.n_rows == n_active && n_active > 0;
 }
 
 // Position-indexed loop attention with the carried old term, as one or two single-term launches:
@@ -675,7 +676,7 @@ int fl_launch_loop_attn_stream(fl_ctx* ctx, const fl_shape* s, int loop_r, const
                                const int32_t* col_idx, const int32_t* col_cnt, int c, const float* lse_in,
                                float* lse_out, const void* o_store_in, void* o_store_out, const fl_attn_carry* carry,
                                int32_t* status, cudaStream_t st) {
-  if (!fl_loop_attn_stream_covers(ctx, s, loop_r, n_active, store, c)) return FL_ERR_UNSUPPORTED;
+  if (!fl_loop_attn_stream_covers(ctx, s, loop_r, n_active, store, c, carry->reuse == 0)) return FL_ERR_UNSUPPORTED;
   StArgs a{};
   const int64_t d_row = (int64_t)s->n_heads * s->head_dim;
   const fl_kv_stream& ks = store->k_res[loop_r - 2];

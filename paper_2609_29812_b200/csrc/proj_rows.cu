@@ -477,11 +477,10 @@ extern "C" int fl_project_qkv_quant(fl_ctx* ctx, const fl_shape* shape, int loop
   a.k_zero = reinterpret_cast<__half*>(ks.zero);
   a.v_codes = static_cast<uint8_t*>(vs.codes); a.v_scale = reinterpret_cast<__half*>(vs.scale);
   a.v_zero = reinterpret_cast<__half*>(vs.zero);
-  const bool rows = ks.rows_prev != nullptr && vs.rows_prev != nullptr;
-  a.k_rows_prev = rows ? static_cast<__nv_bfloat16*>(ks.rows_prev) : nullptr;
-  a.k_rows_cur = rows ? static_cast<__nv_bfloat16*>(ks.rows_cur) : nullptr;
-  a.v_rows_prev = rows ? static_cast<__nv_bfloat16*>(vs.rows_prev) : nullptr;
-  a.v_rows_cur = rows ? static_cast<__nv_bfloat16*>(vs.rows_cur) : nullptr;
+  a.k_rows_prev = static_cast<__nv_bfloat16*>(ks.rows_prev);   // each written when it is there
+  a.k_rows_cur = static_cast<__nv_bfloat16*>(ks.rows_cur);
+  a.v_rows_prev = static_cast<__nv_bfloat16*>(vs.rows_prev);
+  a.v_rows_cur = static_cast<__nv_bfloat16*>(vs.rows_cur);
   a.kv_out = static_cast<__nv_bfloat16*>(kv_out);
   a.d_model = d;
   a.n_prev = loop_r - 2;

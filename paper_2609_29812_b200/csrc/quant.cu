@@ -228,6 +228,241 @@ __global__ void __launch_bounds__(256, 4) quant_residual_pipelined_kernel(const 
   }
 }
 
+// ------------------------------------------------------------------------------------------------------------
+// The same pipeline with SIXTEEN consecutive elements per thread (two 16-byte loads per operand): the per-thread
+// work that does not depend on the element count (addresses, slot lookups, metadata, the sub-warp reduction, the
+// pipeline's bookkeeping) is paid once per 16 elements, and a group of 128 spans 8 lanes (three shuffle rounds).
+// bf16 rows whose width is a multiple of 512 (whole warps per row), groups of at least 16, at most three earlier
+// streams. Arithmetic identical to encode8, element by element.
+// ------------------------------------------------------------------------------------------------------------
+template <int BITS>
+struct Pay16 {
+  uint4 raw;      // BITS 8: 16 bytes; 4: x, y; 2: x
+  __half sc, zr;
+};
+template <int BITS>
+__device__ __forceinline__ void pay16_load(const DevStream& st, int slot, int elem, int d, int group, Pay16<BITS>& p) {
+  const uint8_t* row = st.codes + (size_t)slot * (d * BITS / 8);
+  if (BITS == 8) {
+    p.raw = __ldg(reinterpret_cast<const uint4*>(row + elem));
+  } else if (BITS == 4) {
+    const uint2 t = __ldg(reinterpret_cast<const uint2*>(row + elem / 2));
+    p.raw.x = t.x; p.raw.y = t.y;
+  } else {
+    p.raw.x = __ldg(reinterpret_cast<const uint32_t*>(row + elem / 4));
+  }
+  const int gs = 31 - __clz(group);
+  const size_t gi = (size_t)slot * (d >> gs) + (elem >> gs);
+  p.sc = __ldg(st.scale + gi);
+  p.zr = __ldg(st.zero + gi);
+}
+template <int BITS>
+__device__ __forceinline__ void pay16_apply(const Pay16<BITS>& p, float (&x)[16]) {
+  const float sc = __half2float(p.sc), zr = __half2float(p.zr);
+  const uint32_t w[4] = {p.raw.x, p.raw.y, p.raw.z, p.raw.w};
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+    uint32_t c;
+    if (BITS == 8) c = (w[i >> 2] >> (8 * (i & 3))) & 0xFFu;
+    else if (BITS == 4) c = (w[i >> 3] >> (4 * (i & 7))) & 0xFu;
+    else c = (w[0] >> (2 * i)) & 0x3u;
+    const float cf = __fsub_rn(__uint_as_float(0x4B000000u | c), 8388608.f);   // exact: 2^23 + c
+    x[i] = __fadd_rn(x[i], __fmaf_rn(cf, sc, zr));
+  }
+}
+__device__ __forceinline__ void unpack16(const uint4& lo, const uint4& hi, float (&x)[16]) {
+  const __nv_bfloat162* a = reinterpret_cast<const __nv_bfloat162*>(&lo);
+  const __nv_bfloat162* b = reinterpret_cast<const __nv_bfloat162*>(&hi);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float2 fa = __bfloat1622float2(a[i]), fb = __bfloat1622float2(b[i]);
+    x[2 * i] = fa.x; x[2 * i + 1] = fa.y;
+    x[8 + 2 * i] = fb.x; x[8 + 2 * i + 1] = fb.y;
+  }
+}
+__device__ __forceinline__ void store16(__nv_bfloat16* p, const float (&x)[16]) {
+  uint4 lo, hi;
+  __nv_bfloat162* a = reinterpret_cast<__nv_bfloat162*>(&lo);
+  __nv_bfloat162* b = reinterpret_cast<__nv_bfloat162*>(&hi);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    a[i] = __floats2bfloat162_rn(x[2 * i], x[2 * i + 1]);
+    b[i] = __floats2bfloat162_rn(x[8 + 2 * i], x[8 + 2 * i + 1]);
+  }
+  reinterpret_cast<uint4*>(p)[0] = lo;
+  reinterpret_cast<uint4*>(p)[1] = hi;
+}
+
+template <int BITS>
+__device__ __forceinline__ void encode16(const QuantArgs& a, bool is_v, int t, int elem, int lanes_per_group,
+                                         float (&xn)[16], float (&xh)[16]) {
+  using T = __nv_bfloat16;
+  uint8_t* codes = is_v ? a.v_codes : a.k_codes;
+  __half* scale = is_v ? a.v_scale : a.k_scale;
+  __half* zero = is_v ? a.v_zero : a.k_zero;
+  T* rows_prev = static_cast<T*>(is_v ? a.v_rows_prev : a.k_rows_prev);
+  T* rows_cur = static_cast<T*>(is_v ? a.v_rows_cur : a.k_rows_cur);
+  const size_t row_off = (size_t)t * a.d + elem;
+  if (rows_prev != nullptr) store16(rows_prev + row_off, xh);
+  float dl[16];
+#pragma unroll
+  for (int i = 0; i < 16; ++i) dl[i] = __fsub_rn(xn[i], xh[i]);
+  float mn = dl[0], mx = dl[0];
+#pragma unroll
+  for (int i = 1; i < 16; ++i) { mn = fminf(mn, dl[i]); mx = fmaxf(mx, dl[i]); }
+  for (int o = 1; o < lanes_per_group; o <<= 1) {
+    mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+  }
+  const __half zh = __float2half_rd(mn);
+  const float zf = __half2float(zh);
+  const float range = __fsub_rn(mx, zf);
+  const float qmax = (float)((1 << BITS) - 1);
+  const __half sh = range == 0.f ? __float2half_rn(0.f) : __float2half_ru(__fdiv_rn(range, qmax));
+  const float sf = __half2float(sh);
+  float q[16];
+  if (sf != 0.f) {
+    // reciprocal estimate of the quotient, exact divisions only where its rounding could differ (see encode8)
+    const float inv = __frcp_rn(sf);
+    bool ambiguous = false;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      const float est = __fmul_rn(__fsub_rn(dl[i], zf), inv);
+      q[i] = __fsub_rn(__fadd_rn(est, 12582912.f), 12582912.f);
+      ambiguous |= 0.5f - fabsf(est - q[i]) < 1e-4f;
+    }
+    if (__any_sync(__activemask(), ambiguous)) {
+#pragma unroll
+      for (int i = 0; i < 16; ++i) q[i] = rintf(__fdiv_rn(__fsub_rn(dl[i], zf), sf));
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < 16; ++i) q[i] = 0.f;
+  }
+  if (rows_cur != nullptr) {
+#pragma unroll
+    for (int i = 0; i < 16; ++i) xh[i] = __fadd_rn(xh[i], __fmaf_rn(q[i], sf, zf));
+    store16(rows_cur + row_off, xh);
+  }
+  // packing by exact binary32 arithmetic (sums below 2^24), the integer read from the low mantissa bits of value + 2^23
+  uint8_t* row = codes + (size_t)t * (a.d * BITS / 8);
+  if constexpr (BITS == 8) {
+    uint32_t w[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+      w[i] = __float_as_uint(__fadd_rn(__fmaf_rn(q[2 * i + 1], 256.f, q[2 * i]), 8388608.f)) & 0xFFFFu;
+    *reinterpret_cast<uint4*>(row + elem) = make_uint4(w[0] | (w[1] << 16), w[2] | (w[3] << 16), w[4] | (w[5] << 16),
+                                                       w[6] | (w[7] << 16));
+  } else {
+    const float r1 = (float)(1 << BITS), r2 = r1 * r1, r3 = r2 * r1;
+    const uint32_t quad_mask = (1u << (4 * BITS)) - 1u;
+    uint32_t quad[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float v = __fmaf_rn(q[4 * j + 3], r3, __fmaf_rn(q[4 * j + 2], r2, __fmaf_rn(q[4 * j + 1], r1, q[4 * j])));
+      quad[j] = __float_as_uint(__fadd_rn(v, 8388608.f)) & quad_mask;
+    }
+    if (BITS == 4)
+      *reinterpret_cast<uint2*>(row + elem / 2) = make_uint2(quad[0] | (quad[1] << 16), quad[2] | (quad[3] << 16));
+    else
+      *reinterpret_cast<uint32_t*>(row + elem / 4) = quad[0] | (quad[1] << 8) | (quad[2] << 16) | (quad[3] << 24);
+  }
+  if (((elem >> 4) & (lanes_per_group - 1)) == 0) {
+    const int gs = 31 - __clz(a.group);
+    const size_t gi = (size_t)t * (a.d >> gs) + (elem >> gs);
+    scale[gi] = sh;
+    zero[gi] = zh;
+  }
+}
+
+template <int BITS, int NP>
+__global__ void __launch_bounds__(256) quant_residual_wide_kernel(const __grid_constant__ QuantArgs a, int n) {
+  using T = __nv_bfloat16;
+  fl_grid_wait();
+  fl_grid_release();
+  const bool is_v = blockIdx.y != 0;
+  const DevSide& side = is_v ? a.v : a.k;
+  const int elem = threadIdx.x * 16, G = gridDim.x;
+  const int lanes_per_group = a.group >> 4;
+  const T* x_new = static_cast<const T*>(is_v ? a.v_new : a.k_new) + elem;
+  const T* base = static_cast<const T*>(side.base) + elem;
+  int t = blockIdx.x;
+  if (t >= n) return;
+  constexpr int NPA = NP > 0 ? NP : 1;
+  int pos = __ldg(a.active_idx + t);
+  int pos1 = t + G < n ? __ldg(a.active_idx + t + G) : 0;
+  int pos2 = t + 2 * G < n ? __ldg(a.active_idx + t + 2 * G) : 0;
+  const uint4* px = reinterpret_cast<const uint4*>(x_new + (size_t)t * a.d);
+  const uint4* ph = reinterpret_cast<const uint4*>(base + (size_t)pos * a.d);
+  uint4 rx0 = __ldg(px), rx1 = __ldg(px + 1), rh0 = __ldg(ph), rh1 = __ldg(ph + 1);
+  int sl[NPA], sl_n[NPA];
+  Pay16<BITS> pl[NPA];
+#pragma unroll
+  for (int s = 0; s < NP; ++s) {
+    sl[s] = __ldg(side.s[s].slot + pos);
+    sl_n[s] = t + G < n ? __ldg(side.s[s].slot + pos1) : -1;
+  }
+#pragma unroll
+  for (int s = 0; s < NP; ++s)
+    if (sl[s] >= 0) pay16_load<BITS>(side.s[s], sl[s], elem, a.d, a.group, pl[s]);
+  for (;;) {
+    const int t1 = t + G;
+    const bool has1 = t1 < n;
+    uint4 nx0 = rx0, nx1 = rx1, nh0 = rh0, nh1 = rh1;
+    Pay16<BITS> pl_n[NPA];
+    int sl_nn[NPA];
+    int pos3 = 0;
+    if (has1) {
+      const uint4* qx = reinterpret_cast<const uint4*>(x_new + (size_t)t1 * a.d);
+      const uint4* qh = reinterpret_cast<const uint4*>(base + (size_t)pos1 * a.d);
+      nx0 = __ldg(qx); nx1 = __ldg(qx + 1); nh0 = __ldg(qh); nh1 = __ldg(qh + 1);
+#pragma unroll
+      for (int s = 0; s < NP; ++s) {
+        if (sl_n[s] >= 0) pay16_load<BITS>(side.s[s], sl_n[s], elem, a.d, a.group, pl_n[s]);
+        sl_nn[s] = t + 2 * G < n ? __ldg(side.s[s].slot + pos2) : -1;
+      }
+      if (t + 3 * G < n) pos3 = __ldg(a.active_idx + t + 3 * G);
+    }
+    float xn[16], xh[16];
+    unpack16(rx0, rx1, xn);
+    unpack16(rh0, rh1, xh);
+#pragma unroll
+    for (int s = 0; s < NP; ++s)
+      if (sl[s] >= 0) pay16_apply<BITS>(pl[s], xh);
+    if (lanes_per_group == 8) encode16<BITS>(a, is_v, t, elem, 8, xn, xh);
+    else encode16<BITS>(a, is_v, t, elem, lanes_per_group, xn, xh);
+    if (!has1) break;
+    t = t1;
+    rx0 = nx0; rx1 = nx1; rh0 = nh0; rh1 = nh1;
+    pos1 = pos2; pos2 = pos3;
+#pragma unroll
+    for (int s = 0; s < NP; ++s) { sl[s] = sl_n[s]; sl_n[s] = sl_nn[s]; pl[s] = pl_n[s]; }
+  }
+}
+
+template <int BITS, int NP>
+int launch_quant_wide_np(const fl_ctx* ctx, const QuantArgs& a, int n_active, cudaStream_t st) {
+  auto kern = quant_residual_wide_kernel<BITS, NP>;
+  const int threads = a.d / 16;
+  int per_sm = 0;
+  FL_CHECK_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, threads, 0));
+  if (per_sm < 1) per_sm = 1;
+  const int resident = ctx->sm_count * per_sm / 2;
+  const int gx = n_active < resident ? n_active : (resident < 1 ? 1 : resident);
+  FL_CHECK_CUDA(fl_launch(ctx, kern, dim3(gx, 2), dim3(threads), 0, st, a, n_active));
+  return fl_launch_status();
+}
+
+template <int BITS>
+int launch_quant_wide(const fl_ctx* ctx, const QuantArgs& a, int n_active, cudaStream_t st) {
+  switch (a.n_prev) {
+    case 0: return launch_quant_wide_np<BITS, 0>(ctx, a, n_active, st);
+    case 1: return launch_quant_wide_np<BITS, 1>(ctx, a, n_active, st);
+    case 2: return launch_quant_wide_np<BITS, 2>(ctx, a, n_active, st);
+    default: return launch_quant_wide_np<BITS, 3>(ctx, a, n_active, st);
+  }
+}
+
 template <int BITS, int NP>
 int launch_quant_pipelined_np(const fl_ctx* ctx, const QuantArgs& a, int n_active, cudaStream_t st) {
   auto kern = quant_residual_pipelined_kernel<BITS, NP>;
@@ -253,6 +488,14 @@ int launch_quant_pipelined(const fl_ctx* ctx, const QuantArgs& a, int n_active, 
 
 template <typename T>
 int launch_quant(const fl_ctx* ctx, const fl_shape* s, const QuantArgs& a, int n_active, cudaStream_t st) {
+  if (sizeof(T) == 2 && a.d % 512 == 0 && a.d <= 4096 && a.n_prev <= 3 && s->bits != 16 && a.group >= 16 &&
+      !ctx->quant_narrow) {
+    switch (s->bits) {
+      case 2: return launch_quant_wide<2>(ctx, a, n_active, st);
+      case 4: return launch_quant_wide<4>(ctx, a, n_active, st);
+      default: return launch_quant_wide<8>(ctx, a, n_active, st);
+    }
+  }
   if (sizeof(T) == 2 && a.d <= 2048 && a.n_prev <= 3 && s->bits != 16) {
     switch (s->bits) {
       case 2: return launch_quant_pipelined<2>(ctx, a, n_active, st);
@@ -312,7 +555,7 @@ extern "C" int fl_quant_kv_residual(fl_ctx* ctx, const fl_shape* shape, int loop
   a.k_zero = reinterpret_cast<__half*>(ks.zero);
   a.v_codes = static_cast<uint8_t*>(vs.codes); a.v_scale = reinterpret_cast<__half*>(vs.scale);
   a.v_zero = reinterpret_cast<__half*>(vs.zero);
-  const bool rows = shape->dtype == FL_BF16 && ks.rows_prev != nullptr && vs.rows_prev != nullptr;
+  const bool rows = shape->dtype == FL_BF16;   // each buffer is written when it is there (rows_cur may come alone)
   a.k_rows_prev = rows ? ks.rows_prev : nullptr; a.k_rows_cur = rows ? ks.rows_cur : nullptr;
   a.v_rows_prev = rows ? vs.rows_prev : nullptr; a.v_rows_cur = rows ? vs.rows_cur : nullptr;
   a.n_prev = loop_r - 2; a.d = d; a.group = shape->group;

@@ -145,7 +145,8 @@ class LayerState:
     def alloc_stream(self, sel: TokenSelection, rows: bool = True):
         """Adds the residual stream of the next loop.  rows: also lend it the transient workspace for the loop's
         materialized rows (bf16 storage only), which the quantization kernel fills and the attention kernel of the
-        same loop gathers from; the workspace is shared by every LayerState of the device."""
+        same loop gathers from; the workspace is shared by every LayerState of the device.  rows="cur": only the
+        rows after the loop's residual (all a call that reuses the carried old term reads)."""
         w, n = self.w, sel.n
         d = w.d
         ws = rows_workspace(self.dev, n, d) if rows and self.dt == torch.bfloat16 and n > 0 else None
@@ -153,7 +154,9 @@ class LayerState:
         def one(side):
             st = {"slot_of_pos": sel.slot_of_pos, "n_rows": n}
             if ws is not None:
-                st["rows_prev"], st["rows_cur"] = ws[side][0][:n], ws[side][1][:n]
+                st["rows_cur"] = ws[side][1][:n]
+                if rows != "cur":    # rows="cur": a loop that reuses the carried old term reads nothing else
+                    st["rows_prev"] = ws[side][0][:n]
             if self.bits == 16:
                 st.update(codes=torch.empty(max(n, 1), d, dtype=self.dt, device=self.dev), scale=None, zero=None)
             else:

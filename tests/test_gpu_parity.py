@@ -533,3 +533,37 @@ def test_column_selection_exact_on_long_problems(env):
                 k = min(c, n)
                 assert cnt[h, b] == k and np.all(idx[h, b, k:] == -1)
                 assert np.array_equal(idx[h, b, :k], cand[fo.topk_ascending(cs[h, b, :n], k)]), (c, h, b)
+
+
+@pytest.mark.parametrize("bits,group", [(4, 128), (4, 64), (8, 32), (2, 16), (2, 128)])
+def test_quantizer_wide_rows_bit_exact(env, bits, group):
+    """Rows of 512 elements (4 heads): the quantizer's 16-elements-per-thread kernel, five loops (up to three earlier
+    streams in the chain, then the general kernel), codes, metadata and materialized rows against the oracle's codec
+    alone (no attention: the oracle's residual_update chained by hand)."""
+    B, P, ctx = env
+    w = dataclasses.replace(small_bf16(L=700, H=4, R=4, bits=bits, group=group), n_loops=6,
+                            changed_fracs=(0.3, 0.2, 0.15, 0.1, 0.08))
+    x = workloads.make_layer_inputs(w, seed=23)
+    st = P.LayerState(ctx, w)
+    st.k_base, st.v_base = to_dev(x.K[0], w), to_dev(x.V[0], w)
+    hats = [np.asarray(storage_round(x.K[0], w), dtype=np.float32), np.asarray(storage_round(x.V[0], w), dtype=np.float32)]
+    rng = np.random.default_rng(5)
+    act = np.arange(w.L)
+    for r in range(2, w.n_loops + 1):
+        act = np.sort(rng.choice(act, size=max(33, int(len(act) * 0.6)), replace=False))     # nested, odd counts
+        sel = P.TokenSelection(torch.from_numpy(act.astype(np.int32)).cuda(),
+                               torch.from_numpy(fo.slot_map(act, w.L)).cuda(), None, len(act))
+        st.alloc_stream(sel)
+        new = [storage_round(x.K[r - 1][act], w), storage_round(x.V[r - 1][act], w)]
+        st.quantize(r, to_dev(new[0], w), to_dev(new[1], w), sel)
+        for side, streams in enumerate((st.k_streams, st.v_streams)):
+            hat_new, pay = fo.residual_update(new[side], hats[side], act, bits, group)
+            got = streams[-1]
+            n = len(act)
+            assert np.array_equal(to_np(got["codes"]).reshape(n, w.n_heads, -1), pay["packed"]), (r, side)
+            assert np.array_equal(to_np(got["scale"]).view(np.uint16).reshape(pay["scale"].shape), pay["scale"].view(np.uint16))
+            assert np.array_equal(to_np(got["zero"]).view(np.uint16).reshape(pay["zero"].shape), pay["zero"].view(np.uint16))
+            for name, want in (("rows_prev", hats[side]), ("rows_cur", hat_new)):
+                got_rows = to_np(got[name]).astype(np.float32).reshape(n, w.n_heads, -1)
+                assert np.array_equal(got_rows.view(np.uint32), fo.round_bf16(want[act]).view(np.uint32)), (r, side, name)
+            hats[side] = hat_new

@@ -52,7 +52,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
     headers.append(os.path.join(ROOT, "include", "flashloop.h"))
     stamp = os.path.join(PKG, "libflashloop.stamp")
     digest = _digest(srcs + headers)
-    if not force and os.path.exists(LIB_PATH) and os.path.exists(stamp) and open(stamp).read() == digest:
+    built = all(os.path.exists(p) for p in (LIB_PATH, DEBUG_LIB_PATH, SELFTEST_LIB_PATH))
+    if not force and built and os.path.exists(stamp) and open(stamp).read() == digest:
         return LIB_PATH
     os.makedirs(OBJ_DIR, exist_ok=True)
     nvcc = _nvcc()

@@ -26,6 +26,8 @@ def child(mode, lib):
 def test_checked_build_agrees_and_refuses_damaged_indices():
     if not torch.cuda.is_available():
         pytest.skip("no CUDA device")
+    from paper_2609_29812_b200 import build
+    build.build()                      # no-op when the three libraries are there and current
     normal = child("run", "libflashloop.so")
     checked = child("run", "libflashloop_debug.so")
     assert len(normal) == 2 and normal == checked

@@ -520,10 +520,11 @@ struct SampledSmem {
 
 // `rank`-th largest (1-based) of the keys the threads hold (KPT per thread, `valid` marks the real ones), by four
 // 8-bit radix passes with warp-aggregated shared-memory histograms. Returns the key; *rank_in_eq = how many of the
-// keys equal to it belong to the `rank` largest, *n_eq = how many keys equal it. All kSelThreads threads call it.
+// keys equal to it belong to the `rank` largest, *n_eq = how many keys equal it. Only the first kpt_used slots of a
+// thread are looked at (the same number in every thread). All kSelThreads threads call it.
 template <int KPT>
-__device__ uint32_t block_kth_largest(const uint32_t (&key)[KPT], const bool (&valid)[KPT], uint32_t rank, SampledSmem& sm,
-                                      uint32_t* rank_in_eq, uint32_t* n_eq) {
+__device__ uint32_t block_kth_largest(const uint32_t (&key)[KPT], const bool (&valid)[KPT], int kpt_used, uint32_t rank,
+                                      SampledSmem& sm, uint32_t* rank_in_eq, uint32_t* n_eq) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   uint32_t prefix = 0;
   for (int shift = 24; shift >= 0; shift -= 8) {
@@ -532,6 +533,7 @@ __device__ uint32_t block_kth_largest(const uint32_t (&key)[KPT], const bool (&v
     const uint32_t hi_mask = shift == 24 ? 0u : (0xFFFFFFFFu << (shift + 8));
 #pragma unroll
     for (int q = 0; q < KPT; ++q) {
+      if (q >= kpt_used) break;               // CTA-uniform: the slots beyond it hold no key in any thread
       const bool on = valid[q] && (key[q] & hi_mask) == prefix;
       const uint32_t digit = (key[q] >> shift) & 0xFFu;
       const uint32_t active = __ballot_sync(0xffffffffu, on);
@@ -618,7 +620,7 @@ __global__ void __launch_bounds__(kSelThreads, 2) column_select_sampled_kernel(c
     uint32_t r_s = (uint32_t)((target * kSample + n - 1) / n);
     r_s = min(max(r_s, 1u), (uint32_t)kSample);
     uint32_t dummy0, dummy1;
-    thr_lo = block_kth_largest<1>(skey, sval, r_s, sm, &dummy0, &dummy1);
+    thr_lo = block_kth_largest<1>(skey, sval, 1, r_s, sm, &dummy0, &dummy1);
   }
   if (tid == 0) { sm.n_cand = 0; sm.n_tie = 0; }
   const int n_words = (n + 31) >> 5;
@@ -681,13 +683,15 @@ __global__ void __launch_bounds__(kSelThreads, 2) column_select_sampled_kernel(c
       key[q] = valid[q] ? cand_key[u] : 0u;
     }
     uint32_t n_eq;
-    thr = block_kth_largest<KPT>(key, valid, (uint32_t)k, sm, &take_eq, &n_eq);
+    const int kpt_used = (int)((n_cand + kSelThreads - 1) / kSelThreads);
+    thr = block_kth_largest<KPT>(key, valid, kpt_used, (uint32_t)k, sm, &take_eq, &n_eq);
     // ties with the threshold: all of them, or the take_eq lowest positions
     const bool rank_ties = take_eq < n_eq;
     if (rank_ties && n_eq > (uint32_t)kTieCap) fallback = true;            // CTA-uniform (n_eq is)
     if (!fallback) {
 #pragma unroll
       for (int q = 0; q < KPT; ++q) {
+        if (q >= kpt_used) break;
         if (!valid[q]) continue;
         const int idx = cand_idx[q * kSelThreads + tid];
         if (key[q] > thr || (key[q] == thr && !rank_ties)) atomicOr(&bitmap[idx >> 5], 1u << (idx & 31));

@@ -72,6 +72,8 @@ def parse_args():
                     help="keep every layer's loop-1 K/V packed (Appendix E: int4, keys per channel, values per token, "
                          "groups of 64, last 64 positions unquantized) and rebuild one layer's rows into a transient "
                          "buffer before each layer's work in each loop (fl_dequant_kv_base, inside the timed step)")
+    ap.add_argument("--no-overlap", action="store_true",
+                    help="issue the column selections in the main stream's order instead of on a second stream")
     ap.add_argument("--no-economy", action="store_true", help="recompute the old term in every loop")
     ap.add_argument("--no-variants", action="store_true", help="skip the in-kernel dequantization variant")
     ap.add_argument("--layers", type=int, default=0, help="override the number of layers (development)")
@@ -170,6 +172,9 @@ class Bench:
         self.base_group, self.base_tail = 64, 64
         self.stream = torch.cuda.Stream(device=device)
         self.sp = int(self.stream.cuda_stream)
+        self.side = torch.cuda.Stream(device=device)      # column selections of the step (see run_step)
+        self.sp2 = int(self.side.cuda_stream)
+        self.overlap_select = not bool(getattr(args, "no_overlap", False))
         self.keep = []           # keeps tensors and host structs alive
         self.attn_flops_min, self.attn_flops_exec, self.attn_bytes = {}, {}, {}   # per loop r: lists over layers
         self.setup_ms = {}
@@ -408,11 +413,34 @@ class Bench:
         return self.plans[key]
 
     def run_step(self, rows=True, attn_events=None):
-        """Issue one step on self.stream.  attn_events: list to which (loop, start, end) events are appended."""
+        """Issue one step on self.stream.  attn_events: list to which (loop, start, end) events are appended.
+        Column selection depends on nothing inside the step (its scores come from the source loop), so unless
+        --no-overlap is given every layer's selection is issued on a second stream when the step starts and the
+        layer's first consumer (the attention call of loop 2, or the row marking of the packed base) waits for it:
+        the selections then run in the SM slots the attention launches leave idle."""
         torch = self.torch
         calls = self.plan(rows)[0]
         bad = 0
-        for tag, fn, a, r in calls:
+        overlap = self.overlap_select and attn_events is None
+        sel_events = {}
+        if overlap:
+            start = torch.cuda.Event()
+            start.record(self.stream)
+            self.side.wait_event(start)          # the previous step's readers of the column lists are done
+            for i, (tag, fn, a, r) in enumerate(calls):
+                if tag == "select_columns":
+                    bad |= fn(*(a[:-1] + (self.sp2,)))
+                    ev = torch.cuda.Event()
+                    ev.record(self.side)
+                    sel_events[i] = ev
+        pending = None
+        for i, (tag, fn, a, r) in enumerate(calls):
+            if overlap and tag == "select_columns":
+                pending = sel_events[i]
+                continue
+            if pending is not None and tag in ("attention", "dequant_base"):
+                self.stream.wait_event(pending)
+                pending = None
             if attn_events is not None and tag == "attention":
                 e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
                 e0.record(self.stream)
@@ -621,6 +649,9 @@ def run_ours(args):
                       "base": ("int4 per-channel K / per-token V, groups of 64, last 64 positions bf16; one layer's rows "
                                "rebuilt into a transient buffer per layer and loop inside the step"
                                if bench.int4_base else "bf16 rows resident"),
+                      "column_selection": ("every layer's selection issued on a second stream at the start of the step, "
+                                           "joined before its first consumer" if bench.overlap_select
+                                           else "in the main stream's order"),
                       "old_term": ("recomputed in loop 2, carried (background rows + mass) in later loops"
                                    if bench.economy else "recomputed in every loop"),
                       "parallelism": "replicas only" if world > 1 else "single GPU",

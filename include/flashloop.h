@@ -383,7 +383,8 @@ FL_API int fl_kv_base_q_bytes(const fl_shape* shape, int32_t group, int32_t tail
 /* The checked build (libflashloop_debug.so, compiled with -DFL_DEBUG_BOUNDS) validates, before every launch, the
  * index arrays the call is about to trust: row lists (range, strictly ascending), column lists against their counts
  * (range, ascending, counts within [0, c]), candidate lists, and the slot maps of the residual streams the call reads
- * (each value -1 or a row of its stream). A small kernel reads the arrays (never what they point to), the host waits for
+ * (each value -1 or a row of its stream), and fl_select_tokens its two hidden-state matrices (every value finite). A small
+ * kernel reads the arrays (never what they point to), the host waits for
  * its verdict, and on a violation the call returns FL_ERR_INVALID_ARG, writes that code to `status` when one was given
  * (also in the calls whose normal build never writes it) and launches nothing else. Nothing traps. The wait makes the
  * checked build slow and unusable inside a stream capture: it is for tests and debugging. Returns 1 in the checked

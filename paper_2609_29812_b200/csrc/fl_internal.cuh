@@ -40,6 +40,8 @@ struct fl_idx_check {
 // must then launch nothing. Synchronises the stream in the checked build.
 int fl_debug_check(fl_ctx* ctx, const fl_idx_check* checks, int n_checks, int32_t* status, void* stream);
 int fl_debug_init(fl_ctx* ctx);   // allocates the validator's device word (checked build); FL_OK or FL_ERR_CUDA
+// n values of the storage type `dtype` must be finite; same contract as fl_debug_check.
+int fl_debug_check_finite(fl_ctx* ctx, const void* x, int64_t n, int dtype, int32_t* status, void* stream);
 // The index inputs of an attention call: the active list, the column lists with their counts (n_segments lists of c
 // entries) and the slot maps of the first n_streams residual streams.
 int fl_debug_check_attn(fl_ctx* ctx, const fl_shape* s, int n_streams, const int32_t* active_idx, int32_t n_active,

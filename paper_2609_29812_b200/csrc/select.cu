@@ -782,6 +782,10 @@ extern "C" int fl_select_tokens(fl_ctx* ctx, const fl_shape* shape, int loop_r, 
     const fl_idx_check ck = {cand, n_cand, 0, nullptr, 0, shape->L - 1, 1};
     rc = fl_debug_check(ctx, &ck, 1, status, stream);
     if (rc != FL_OK) return rc;
+    rc = fl_debug_check_finite(ctx, h_prev, (int64_t)shape->L * d, shape->dtype, status, stream);
+    if (rc != FL_OK) return rc;
+    rc = fl_debug_check_finite(ctx, h_cur, (int64_t)shape->L * d, shape->dtype, status, stream);
+    if (rc != FL_OK) return rc;
   }
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int warps = 8;

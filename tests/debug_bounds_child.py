@@ -81,6 +81,19 @@ def main():
             for a, b in zip(before, untouched):
                 assert torch.equal(a, b), (name, what, "an output was written")
 
+        # 0. a hidden state that is not finite: the token selection must refuse
+        g_prev, g_cur = to_dev(x.G[0], w), to_dev(x.G[1], w)
+        g_bad = g_cur.clone(); g_bad[7, 3] = float("nan")
+        sc = torch.full((L,), 5.0, device="cuda:0")
+        ai = torch.full((w.k_tokens,), -9, dtype=torch.int32, device="cuda:0")
+        sp = torch.full((L,), -9, dtype=torch.int32, device="cuda:0")
+        expect_refusal("hidden state with a NaN",
+                       lambda: B.fl_select_tokens(ctx, st.shape, 2, g_prev, g_bad, None, L, w.k_tokens, sc, ai, sp, status,
+                                                  check=False), [sc, ai, sp])
+        g_bad = g_prev.clone(); g_bad[L - 1, 0] = float("inf")
+        expect_refusal("hidden state with an infinity",
+                       lambda: B.fl_select_tokens(ctx, st.shape, 2, g_bad, g_cur, None, L, w.k_tokens, sc, ai, sp, status,
+                                                  check=False), [sc, ai, sp])
         # 1. an active list that leaves the sequence / is not ascending: the quantizer must refuse
         st.alloc_stream(sel, rows=True)
         ks, vs = st.k_streams[0], st.v_streams[0]

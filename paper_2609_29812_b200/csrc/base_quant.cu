@@ -144,7 +144,7 @@ __global__ void __launch_bounds__(256) base_dequant_kernel(const __grid_constant
   const __half* scale = is_v ? a.v_scale : a.k_scale;
   const __half* zero = is_v ? a.v_zero : a.k_zero;
   T* out = static_cast<T*>(is_v ? a.v_out : a.k_out);
-  constexpr int U = 4;
+  constexpr int U = 4;      // rows whose loads are in flight together
   // the unquantized tail rows, copied as they are (always: they are few)
   {
     const T* tail = static_cast<const T*>(is_v ? a.v_tail : a.k_tail);
@@ -153,65 +153,79 @@ __global__ void __launch_bounds__(256) base_dequant_kernel(const __grid_constant
     uint4* dst = reinterpret_cast<uint4*>(out + (size_t)a.Lq * a.d);
     for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n_vec; i += gridDim.x * blockDim.x) dst[i] = __ldg(src + i);
   }
-  // a CTA walks rows blockIdx.x, blockIdx.x + gridDim.x, ...; its threads cover a row in steps of blockDim.x vectors
-  for (int v0 = threadIdx.x; v0 < per_row; v0 += blockDim.x)
-  for (int t0 = blockIdx.x; t0 < a.Lq; t0 += U * gridDim.x) {
-    int t[U], elem[U];
-    bool on[U];
-    uint32_t raw[U][2];
-    uint4 sraw[U], zraw[U];
-    const int head = (v0 * 8) / a.dh;
-#pragma unroll
-    for (int u = 0; u < U; ++u) {
-      t[u] = t0 + u * gridDim.x;
-      elem[u] = v0 * 8;
-      on[u] = t[u] < a.Lq;
-      if (on[u] && a.row_mask != nullptr)
-        on[u] = (__ldg(a.row_mask + (size_t)head * a.mask_words + (t[u] >> 5)) >> (t[u] & 31)) & 1u;
-    }
-#pragma unroll
-    for (int u = 0; u < U; ++u) {
-      if (!on[u]) continue;
-      const uint8_t* row = codes + (size_t)t[u] * (a.d * BITS / 8);
-      if (BITS == 8) {
-        const uint2 r2 = __ldg(reinterpret_cast<const uint2*>(row + elem[u]));
-        raw[u][0] = r2.x; raw[u][1] = r2.y;
-      } else if (BITS == 4) {
-        raw[u][0] = __ldg(reinterpret_cast<const uint32_t*>(row + elem[u] / 2));
-      } else {
-        raw[u][0] = __ldg(reinterpret_cast<const uint16_t*>(row + elem[u] / 4));
+  // A CTA owns a run of consecutive rows and its threads the same 8 channels of each. Per batch of four rows a thread
+  // makes two trips to memory: its head's mask bits (two words), then the codes (and the values' metadata) of every
+  // wanted row at once. The keys' scales and offsets (per channel and token group) are read and converted once per
+  // token group, not once per row. The code becomes a float by arithmetic (2^23 + c is exact), not by a conversion:
+  // conversions run on a narrow pipe.
+  const int rows_per_cta = (a.Lq + gridDim.x - 1) / gridDim.x;
+  const int r_lo = blockIdx.x * rows_per_cta, r_hi = min(a.Lq, r_lo + rows_per_cta);
+  for (int v0 = threadIdx.x; v0 < per_row; v0 += blockDim.x) {
+    const int elem = v0 * 8;
+    const int head = elem / a.dh;
+    int tg_cached = -1;
+    float ksc[8], kzr[8];
+    for (int t0 = r_lo; t0 < r_hi; t0 += U) {
+      uint32_t want = (1u << U) - 1u;                          // bit u: row t0 + u is rebuilt
+      if (a.row_mask != nullptr) {
+        const uint32_t* mrow = a.row_mask + (size_t)head * a.mask_words;
+        const int w = t0 >> 5;
+        const uint32_t lo = __ldg(mrow + w), hi = w + 1 < a.mask_words ? __ldg(mrow + w + 1) : 0u;
+        want = __funnelshift_r(lo, hi, t0 & 31) & ((1u << U) - 1u);
       }
-      if (is_v) {
-        const size_t gi = (size_t)t[u] * (a.d >> gs) + (elem[u] >> gs);
-        sraw[u].x = __half_as_ushort(__ldg(scale + gi));
-        zraw[u].x = __half_as_ushort(__ldg(zero + gi));
-      } else {
-        const size_t mi = (size_t)(t[u] >> gs) * a.d + elem[u];
-        sraw[u] = __ldg(reinterpret_cast<const uint4*>(scale + mi));
-        zraw[u] = __ldg(reinterpret_cast<const uint4*>(zero + mi));
-      }
-    }
+      if (r_hi - t0 < U) want &= (1u << (r_hi - t0)) - 1u;
+      if (want == 0u) continue;
+      uint32_t raw[U][BITS == 8 ? 2 : 1];
+      __half vsh[U], vzh[U];
 #pragma unroll
-    for (int u = 0; u < U; ++u) {
-      if (!on[u]) continue;
-      float x[8];
-#pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        uint32_t c;
-        if (BITS == 8) c = (raw[u][e >> 2] >> (8 * (e & 3))) & 0xFFu;
-        else if (BITS == 4) c = (raw[u][0] >> (4 * e)) & 0xFu;
-        else c = (raw[u][0] >> (2 * e)) & 0x3u;
-        float sc, zr;
-        if (is_v) {
-          sc = __half2float(__ushort_as_half((unsigned short)sraw[u].x));
-          zr = __half2float(__ushort_as_half((unsigned short)zraw[u].x));
+      for (int u = 0; u < U; ++u) {
+        if (!((want >> u) & 1u)) continue;
+        const int t = t0 + u;
+        const uint8_t* row = codes + (size_t)t * (a.d * BITS / 8);
+        if (BITS == 8) {
+          const uint2 r2 = __ldg(reinterpret_cast<const uint2*>(row + elem));
+          raw[u][0] = r2.x; raw[u][BITS == 8 ? 1 : 0] = r2.y;
+        } else if (BITS == 4) {
+          raw[u][0] = __ldg(reinterpret_cast<const uint32_t*>(row + elem / 2));
         } else {
-          sc = __half2float(reinterpret_cast<const __half*>(&sraw[u])[e]);
-          zr = __half2float(reinterpret_cast<const __half*>(&zraw[u])[e]);
+          raw[u][0] = __ldg(reinterpret_cast<const uint16_t*>(row + elem / 4));
         }
-        x[e] = __fmaf_rn((float)c, sc, zr);
+        if (is_v) {
+          const size_t gi = (size_t)t * (a.d >> gs) + (elem >> gs);
+          vsh[u] = __ldg(scale + gi);
+          vzh[u] = __ldg(zero + gi);
+        }
       }
-      store8<T>(out + (size_t)t[u] * a.d + elem[u], x);
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        if (!((want >> u) & 1u)) continue;
+        const int t = t0 + u;
+        float x[8];
+        if (!is_v) {
+          if ((t >> gs) != tg_cached) {      // the same for every thread of the CTA
+            tg_cached = t >> gs;
+            const size_t mi = (size_t)tg_cached * a.d + elem;
+            const uint4 sraw = __ldg(reinterpret_cast<const uint4*>(scale + mi));
+            const uint4 zraw = __ldg(reinterpret_cast<const uint4*>(zero + mi));
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+              ksc[e] = __half2float(reinterpret_cast<const __half*>(&sraw)[e]);
+              kzr[e] = __half2float(reinterpret_cast<const __half*>(&zraw)[e]);
+            }
+          }
+        }
+        const float vsc = is_v ? __half2float(vsh[u]) : 0.f, vzr = is_v ? __half2float(vzh[u]) : 0.f;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          uint32_t c;
+          if (BITS == 8) c = (raw[u][BITS == 8 ? (e >> 2) : 0] >> (8 * (e & 3))) & 0xFFu;
+          else if (BITS == 4) c = (raw[u][0] >> (4 * e)) & 0xFu;
+          else c = (raw[u][0] >> (2 * e)) & 0x3u;
+          const float cf = __fsub_rn(__uint_as_float(0x4B000000u | c), 8388608.f);
+          x[e] = is_v ? __fmaf_rn(cf, vsc, vzr) : __fmaf_rn(cf, ksc[e], kzr[e]);
+        }
+        store8<T>(out + (size_t)t * a.d + elem, x);
+      }
     }
   }
 }

@@ -156,3 +156,46 @@ def test_config2_full_size_chained_on_gpu_against_the_full_oracle():
     assert_attn_close(to_np(st.o_store), ref["loops"][-1]["O_full"], "config 2 chained final O store",
                       carried=w.n_loops - 1)
     ctx.close()
+
+
+def test_packed_base_at_bench_size_sampled_against_oracle():
+    """The packed loop-1 base at the benchmark's size (L = 32768, d = 2048, int4, groups of 64, tail 64): sampled token
+    groups of the keys and sampled rows of the values bit for bit against the oracle (groups are independent, so the
+    oracle packs just the sampled slices), the rebuilt rows of the same samples, and the tail."""
+    torch = pytest.importorskip("torch")
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2609_29812_b200 import binding as B, pipeline as P
+    w = workloads.config3(n_layers=1)
+    L, d, g, tail, bits = w.L, w.d, 64, 64, 4
+    Lq, n_tg = L - tail, (L - tail + g - 1) // g
+    gen = torch.Generator(device="cuda:0"); gen.manual_seed(11)
+    scale_c = 10.0 ** (torch.rand(d, device="cuda:0", generator=gen) * 3 - 2)              # channels of mixed magnitude
+    k = (torch.randn(L, d, device="cuda:0", generator=gen) * scale_c).to(torch.bfloat16)
+    v = (torch.randn(L, d, device="cuda:0", generator=gen) * (10.0 ** (torch.rand(L, 1, device="cuda:0", generator=gen) * 3 - 2))
+         ).to(torch.bfloat16)
+    u8 = lambda *s: torch.empty(s, dtype=torch.uint8, device="cuda:0")
+    f16 = lambda *s: torch.empty(s, dtype=torch.float16, device="cuda:0")
+    t = [u8(Lq, d // 2), f16(n_tg, d), f16(n_tg, d), u8(Lq, d // 2), f16(Lq, d // g), f16(Lq, d // g),
+         torch.empty(tail, d, dtype=torch.bfloat16, device="cuda:0"), torch.empty(tail, d, dtype=torch.bfloat16, device="cuda:0")]
+    with B.Context(0) as ctx:
+        sh = P.shape_of(w)
+        q = B.make_base_q(*t, g, tail)
+        B.fl_quant_kv_base(ctx, sh, k, v, q)
+        k_out, v_out = torch.empty_like(k), torch.empty_like(v)
+        B.fl_dequant_kv_base(ctx, sh, q, k_out, v_out)
+        torch.cuda.synchronize()
+        assert B.fl_kv_base_q_bytes(sh, g, tail) == fo.base_q_bytes(L, d, bits, g, tail)
+    rng = np.random.default_rng(3)
+    for tg in [0, n_tg - 1] + rng.choice(n_tg, size=4, replace=False).tolist():        # the last group is 0 .. 63 rows short
+        lo, hi = tg * g, min(Lq, (tg + 1) * g)
+        ks = to_np(k[lo:hi]); vs = to_np(v[lo:hi])
+        ref = fo.quantize_base(ks, vs, bits, g, 0, storage_round=fo.round_bf16)
+        assert np.array_equal(t[0][lo:hi].cpu().numpy(), fo.pack_codes(ref["k_codes"], bits)), tg
+        assert np.array_equal(t[1][tg].cpu().numpy().view(np.uint16), ref["k_scale"][0].view(np.uint16)), tg
+        assert np.array_equal(t[2][tg].cpu().numpy().view(np.uint16), ref["k_zero"][0].view(np.uint16)), tg
+        assert np.array_equal(t[3][lo:hi].cpu().numpy(), fo.pack_codes(ref["v_codes"], bits)), tg
+        assert np.array_equal(t[4][lo:hi].cpu().numpy().view(np.uint16), ref["v_scale"].view(np.uint16)), tg
+        assert np.array_equal(t[5][lo:hi].cpu().numpy().view(np.uint16), ref["v_zero"].view(np.uint16)), tg
+        assert np.array_equal(to_np(k_out[lo:hi]), ref["khat"]) and np.array_equal(to_np(v_out[lo:hi]), ref["vhat"]), tg
+    assert torch.equal(k_out[Lq:], k[Lq:]) and torch.equal(v_out[Lq:], v[Lq:]) and torch.equal(t[6], k[Lq:])

@@ -138,6 +138,38 @@ class LayerState:
                             new_idx, new_cnt)
         self.col_idx, self.col_cnt, self.c = new_idx, new_cnt, c_next
 
+    # ---- packed loop-1 base (Appendix E) ------------------------------------------------------
+    def pack_base(self, k, v, group: int = 64, tail: int = 64):
+        """Packs the loop-1 K and V of the layer (keys per channel over `group` positions, values per token over
+        `group` channels, the last `tail` positions unquantized) and keeps only the packed form; returns its bytes."""
+        w, L, d = self.w, self.w.L, self.w.d
+        Lq = max(0, L - tail)
+        n_tg = (Lq + group - 1) // group
+        u8 = lambda *s_: torch.empty(s_, dtype=torch.uint8, device=self.dev)
+        f16 = lambda *s_: torch.empty(s_, dtype=torch.float16, device=self.dev)
+        self.base_tensors = [u8(max(Lq, 1), d * self.bits // 8), f16(max(n_tg, 1), d), f16(max(n_tg, 1), d),
+                             u8(max(Lq, 1), d * self.bits // 8), f16(max(Lq, 1), d // group), f16(max(Lq, 1), d // group),
+                             torch.empty(max(L - Lq, 1), d, dtype=self.dt, device=self.dev),
+                             torch.empty(max(L - Lq, 1), d, dtype=self.dt, device=self.dev)]
+        self.base_q = B.make_base_q(*self.base_tensors, group, tail)
+        B.fl_quant_kv_base(self.ctx, self.shape, k, v, self.base_q)
+        return B.fl_kv_base_q_bytes(self.shape, group, tail)
+
+    def rebuild_base(self, k_out, v_out, sel: Optional["TokenSelection"] = None):
+        """Rebuilds the packed base into k_out, v_out ([L, H, dh], e.g. a buffer shared by all layers) and makes them
+        the layer's base.  With a token selection (and the layer's column lists) only the rows the sparse loops read."""
+        mask = None
+        if sel is not None and self.col_idx is not None:
+            words = (self.w.L + 31) // 32
+            if getattr(self, "row_mask", None) is None:
+                self.row_mask = torch.empty(self.w.n_heads, words, dtype=torch.int32, device=self.dev)
+            B.fl_mark_base_rows(self.ctx, self.shape, self.col_idx, self.col_cnt, self.c, sel.active_idx, sel.n,
+                                self.row_mask)
+            mask = self.row_mask
+        B.fl_dequant_kv_base(self.ctx, self.shape, self.base_q, k_out, v_out, row_mask=mask)
+        self.k_base, self.v_base = k_out, v_out
+        self._rebuild_store()
+
     # ---- loop r >= 2 --------------------------------------------------------------------------
     def _rebuild_store(self):
         self.store = B.make_store(self.k_base, self.v_base, self.k_streams, self.v_streams)

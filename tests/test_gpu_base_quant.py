@@ -137,15 +137,17 @@ def test_dense_and_sparse_loop_on_the_rebuilt_base(env):
     ref = orc.run(x.G, x.Q, [qb["khat"].reshape(shp), x.K[1]], [qb["vhat"].reshape(shp), x.V[1]], [w.k_tokens],
                   [w.col_budget])
     st = P.LayerState(ctx, w)
-    q, t, Lq, n_tg = alloc_base(B, w, 4, 64, 64)
-    B.fl_quant_kv_base(ctx, st.shape, to_dev(k1, w), to_dev(v1, w), q)
+    assert st.pack_base(to_dev(k1, w), to_dev(v1, w), 64, 64) == fo.base_q_bytes(w.L, w.d, 4, 64, 64)
     k_re = torch.empty(shp, dtype=torch.bfloat16, device="cuda:0")
     v_re = torch.empty_like(k_re)
-    B.fl_dequant_kv_base(ctx, st.shape, q, k_re, v_re)
+    st.rebuild_base(k_re, v_re)                    # every row: the dense loop reads all of them
     st.dense_loop(to_dev(x.Q[0], w), k_re, v_re)
     st.select_columns_dense()
     sel = oracle_selection(P, w, ref, 2)
     act = ref["active"][0]
+    # before the sparse loop only the rows it reads are rebuilt, into a buffer that holds nothing else
+    k_tr, v_tr = torch.full_like(k_re, float("nan")), torch.full_like(v_re, float("nan"))
+    st.rebuild_base(k_tr, v_tr, sel)
     o_rows, _ = st.sparse_loop(2, to_dev(x.Q[1][act], w), to_dev(x.K[1][act], w), to_dev(x.V[1][act], w), sel,
                                indexed=True)
     st.check_status()
